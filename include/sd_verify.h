@@ -1,0 +1,170 @@
+/*
+ * sd_verify.h -- C ABI of the verify-and-feedback step of speculative decoding
+ * with an online-learned draft model (OnlineSpec, Algorithm 1).
+ *
+ * One call processes one decoding round for a batch of B sequences, each with k
+ * draft tokens and a vocabulary of V entries:
+ *
+ *   p_{b,i} = softmax(T[b,i,:] / tau), i = 0..k   ("predicted distribution" of the
+ *   q_{b,i} = softmax(D[b,i,:] / tau), i = 0..k-1   target / draft, Algorithm 1 inputs)
+ *   accept draft token i  iff  u[b,i] < min(1, p_{b,i}(x_{b,i}) / q_{b,i}(x_{b,i}))
+ *                                        (Algorithm 1, "Determine the accepted token length";
+ *                                         the accept-iff form is restated in the proof of Lemma 1)
+ *   n_b = index of the first rejected draft token, k if none
+ *   y_b ~ max(0, p_{b,n_b} - q_{b,n_b}) normalised   if n_b < k
+ *   y_b ~ p_{b,k}                                    if n_b = k
+ *                                        (Algorithm 1, "Verify and update the draft sequence");
+ *         drawn by inverse CDF in ascending vocabulary order with u[b,k]:
+ *         y_b = min{ v : sum_{w<=v} r_w > u[b,k] * sum_w r_w }
+ *   loss[b,i]   = KL(p_{b,i} || q_{b,i})                 (Eq. "kl_divergence" in the proof of
+ *                 Lemma 1: the excess of the cross-entropy loss of Assumption 1 over its optimum)
+ *   grad[b,i,v] = d loss[b,i] / d D[b,i,v] = (q_{b,i,v} - p_{b,i,v}) / tau
+ *                                        (the feedback gradient "nabla f_t" of Sec. 3.1,
+ *                                         taken w.r.t. the raw draft logits)
+ *   acc_prob[b,i] = sum_v min(p, q) = 1 - TV(p, q)       (Eq. 1 and the proof of Lemma 1)
+ *
+ * Conventions common to every entry point
+ *   - Unless an argument is documented as HOST, every pointer is a DEVICE pointer owned by the
+ *     caller.  The library never frees or reallocates caller memory.
+ *   - Tensors are dense, row-major, contiguous.  Logit rows may start at any element-aligned
+ *     address; rows whose byte length and base address are multiples of 16 take the fast
+ *     (bulk-copy, cluster) path, everything else takes a slower generic path with the same
+ *     results.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = the legacy default
+ *     stream).  The call does not synchronise; outputs are valid once the stream reaches the
+ *     end of the enqueued work.
+ *   - Return value: SD_OK, or a negative SD_ERR_* code for an error the host can detect; in that
+ *     case nothing has been enqueued.  Problems only visible in the data on the device (a token
+ *     outside [0,V), a row without a finite positive softmax denominator, a rejection whose
+ *     residual is numerically zero) never trap: they set bits in out_status[b] and the affected
+ *     outputs are memory-safe but otherwise unspecified.
+ *   - dtype: SD_DTYPE_F32 (float) or SD_DTYPE_BF16 (bfloat16 bit patterns in uint16_t) for both
+ *     logit tensors and for out_grad_draft.  Arithmetic is fp32 per element with fp64 row
+ *     scalars in both cases.
+ *   - Calls that share a workspace must not overlap on the GPU.
+ */
+#ifndef SD_VERIFY_H
+#define SD_VERIFY_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SD_VERSION 100 /* major*10000 + minor*100 + patch */
+
+/* dtype codes */
+#define SD_DTYPE_F32 0
+#define SD_DTYPE_BF16 1
+
+/* return codes */
+#define SD_OK 0
+#define SD_ERR_NULL (-1)        /* a required pointer is NULL */
+#define SD_ERR_SHAPE (-2)       /* B, k or V < 1, k > SD_MAX_K, or B*(k+1)*V overflows 2^62 */
+#define SD_ERR_TEMPERATURE (-3) /* temperature is not a finite number > 0 */
+#define SD_ERR_WORKSPACE (-4)   /* workspace NULL, misaligned (256 B) or too small */
+#define SD_ERR_DTYPE (-5)       /* unknown dtype code */
+#define SD_ERR_CUDA (-6)        /* a CUDA runtime call failed; text via sd_last_cuda_error() */
+#define SD_ERR_NO_DEVICE (-7)   /* no sm_100 device is current */
+#define SD_ERR_ALIGN (-8)       /* a pointer is not aligned to its element type */
+
+#define SD_MAX_K 64 /* largest number of draft tokens per sequence */
+
+/* bits of out_status[b] */
+#define SD_STATUS_BAD_TOKEN 1u      /* some draft token of the sequence is outside [0,V): treated as rejected */
+#define SD_STATUS_BAD_ROW 2u        /* a softmax denominator of the sequence is not finite and positive */
+#define SD_STATUS_ZERO_RESIDUAL 4u  /* rejection with sum max(0,p-q) == 0: token drawn from p instead */
+
+/*
+ * sd_verify_feedback / sd_verify_feedback_bf16 -- the whole step (Algorithm 1 from "Determine
+ * the accepted token length" to "Receive interactive feedback") for fp32 / bf16 logits.
+ *
+ *   target_logits  [B, k+1, V]  in   row i < k pairs with draft row i; row k is the bonus row
+ *   draft_logits   [B, k,   V]  in
+ *   draft_tokens   [B, k]       in   int32, x[b,i] in [0,V)
+ *   uniforms       [B, k+1]     in   fp32 in [0,1): u[b,0..k-1] drive the k accept tests,
+ *                                    u[b,k] drives the residual / bonus draw
+ *   temperature                 in   tau > 0, applied to both models' logits
+ *   out_accept_len [B]          out  int32 n_b in [0,k]
+ *   out_tokens     [B, k+1]     out  int32: x[b,0..n_b-1], then y_b at index n_b, then -1 padding
+ *   out_loss       [B, k]       out  fp32 KL(p||q) per position; may be NULL together with
+ *                                    out_grad_draft (verify-only mode)
+ *   out_grad_draft [B, k, V]    out  (q-p)/tau, same dtype as the logits (bf16: round to nearest
+ *                                    even); may be NULL (no gradient is written)
+ *   stream                      in   cudaStream_t
+ *
+ * Scratch memory comes from a per-device buffer the library keeps and grows on demand
+ * (cudaMalloc on the first call and whenever a larger problem arrives; that growth synchronises
+ * the device).  Use sd_verify_feedback_ex to supply the scratch memory yourself.
+ */
+int sd_verify_feedback(const float* target_logits, const float* draft_logits,
+                       const int32_t* draft_tokens, const float* uniforms, float temperature,
+                       int B, int k, int V, int32_t* out_accept_len, int32_t* out_tokens,
+                       float* out_loss, float* out_grad_draft, void* stream);
+
+int sd_verify_feedback_bf16(const uint16_t* target_logits, const uint16_t* draft_logits,
+                            const int32_t* draft_tokens, const float* uniforms, float temperature,
+                            int B, int k, int V, int32_t* out_accept_len, int32_t* out_tokens,
+                            float* out_loss, uint16_t* out_grad_draft, void* stream);
+
+/*
+ * sd_verify_feedback_ex -- same computation with every option exposed.
+ *
+ *   dtype            SD_DTYPE_F32 or SD_DTYPE_BF16; target_logits, draft_logits and out_grad_draft
+ *                    are of that type
+ *   workspace        device scratch of at least sd_workspace_bytes(B,k,V,dtype) bytes, aligned to
+ *                    256 bytes; contents need not be initialised and are undefined afterwards
+ *   out_acc_prob     [B,k] fp32 sum_v min(p,q) per position (Eq. 1), or NULL
+ *   out_status       [B] uint32 SD_STATUS_* bits, or NULL
+ */
+int sd_verify_feedback_ex(const void* target_logits, const void* draft_logits,
+                          const int32_t* draft_tokens, const float* uniforms, float temperature,
+                          int B, int k, int V, int dtype, int32_t* out_accept_len,
+                          int32_t* out_tokens, float* out_loss, void* out_grad_draft,
+                          float* out_acc_prob, uint32_t* out_status, void* workspace,
+                          size_t workspace_bytes, void* stream);
+
+/* Bytes of scratch sd_verify_feedback_ex needs for this shape; 0 if the shape is invalid. */
+size_t sd_workspace_bytes(int B, int k, int V, int dtype);
+
+/*
+ * sd_verify_feedback_host -- the same step for callers whose tensors live in HOST memory.
+ * Every pointer is a HOST pointer (pinned memory gives asynchronous copies, pageable memory
+ * works too).  The call copies the inputs to device buffers the library keeps per device
+ * (grown on demand), runs the step in slices of sequences so that copies in both directions
+ * overlap the kernels, copies every requested output back and returns after all of it has
+ * completed.  out_loss, out_grad_draft, out_acc_prob and out_status may be NULL.
+ */
+int sd_verify_feedback_host(const void* target_logits, const void* draft_logits,
+                            const int32_t* draft_tokens, const float* uniforms, float temperature,
+                            int B, int k, int V, int dtype, int32_t* out_accept_len,
+                            int32_t* out_tokens, float* out_loss, void* out_grad_draft,
+                            float* out_acc_prob, uint32_t* out_status);
+
+/*
+ * sd_launch_info -- HOST out-parameters describing how the last successful device call on this
+ * thread was launched: path (0 = generic, 1 = cluster fast path), cluster size, threads per
+ * block, dynamic shared memory per block, blocks launched, kernels launched.  Any pointer may
+ * be NULL.  Diagnostic only.
+ */
+void sd_launch_info(int* path, int* cluster_size, int* threads, int* smem_bytes, int* blocks,
+                    int* kernels);
+
+/* Release the per-device scratch and staging buffers the library keeps (synchronises). */
+void sd_release_cached_buffers(void);
+
+/* Text for a return code; never NULL. */
+const char* sd_strerror(int code);
+
+/* Text of the CUDA error behind the last SD_ERR_CUDA on this thread ("" if none). */
+const char* sd_last_cuda_error(void);
+
+/* SD_VERSION of the loaded library. */
+int sd_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SD_VERIFY_H */

@@ -1,0 +1,258 @@
+/*
+ * sd_oracle.c -- TEST INFRASTRUCTURE, not part of the product.
+ *
+ * A plain, slow CPU statement of the verify-and-feedback step of speculative decoding with an
+ * online-learned draft (OnlineSpec, Algorithm 1), in double precision, with sequential sums in
+ * vocabulary order.  Only the tests, the smoke check and the benchmark's CPU-baseline leg may
+ * call it.  It shares no code with the CUDA path.
+ *
+ * Every function below is pinned by tests that do not use this file to produce their expected
+ * values (closed forms, brute-force enumeration, finite differences, library routines).
+ *
+ * Readings taken where the paper is silent (each also listed in the design notes):
+ *   - accept iff u < min(1, p/q) (strict), uniforms are fp32 in [0,1);
+ *   - the (k+1)-th uniform of a sequence draws the residual / bonus token by inverse CDF in
+ *     ascending vocabulary order with a strict ">" (first v whose running sum exceeds u*R);
+ *   - the loss reported per position is KL(p||q), the excess of the cross-entropy of
+ *     Assumption 1 over its optimum; the gradient is with respect to the raw draft logits of the
+ *     sum over positions: (q - p)/tau;
+ *   - all k positions of a sequence produce a loss and a gradient, accepted or not.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define SD_ORACLE_F32 0
+#define SD_ORACLE_BF16 1
+
+#define ST_BAD_TOKEN 1u
+#define ST_BAD_ROW 2u
+#define ST_ZERO_RESIDUAL 4u
+
+/* A logit as a double; a bf16 value is the upper half of the fp32 with the same value. */
+static double logit_at(const void* base, int dtype, size_t idx) {
+    if (dtype == SD_ORACLE_F32) return (double)((const float*)base)[idx];
+    uint32_t bits = ((uint32_t)((const uint16_t*)base)[idx]) << 16;
+    float f;
+    memcpy(&f, &bits, sizeof f);
+    return (double)f;
+}
+
+/*
+ * Temperature softmax of one row ("predicted distribution", inputs of Algorithm 1):
+ * m = max_v z_v, e_v = exp((z_v - m)/tau), S = sum_v e_v, prob_v = e_v / S.
+ * Also returns log-probabilities (z_v - m)/tau - log S, which stay finite where prob underflows.
+ */
+static void softmax_row(const void* base, int dtype, size_t off, int V, double tau, double* prob,
+                        double* logprob, double* S_out) {
+    double m = -INFINITY;
+    for (int v = 0; v < V; ++v) {
+        double z = logit_at(base, dtype, off + (size_t)v);
+        if (z > m) m = z;
+    }
+    double S = 0.0;
+    for (int v = 0; v < V; ++v) {
+        double z = logit_at(base, dtype, off + (size_t)v);
+        double e = exp((z - m) / tau);
+        prob[v] = e;
+        S += e;
+    }
+    double logS = log(S);
+    for (int v = 0; v < V; ++v) {
+        double z = logit_at(base, dtype, off + (size_t)v);
+        prob[v] = prob[v] / S;
+        logprob[v] = (z - m) / tau - logS;
+    }
+    *S_out = S;
+}
+
+/* One sequence: Algorithm 1 from the rejection test to the feedback loss. */
+static void one_sequence(const void* T, const void* D, int dtype, const int32_t* x, const float* u,
+                         double tau, int k, int V, int32_t* accept_len, int32_t* tokens,
+                         double* loss, double* grad, double* acc_prob, double* ratio,
+                         uint8_t* accept_band, double* cdf_margin, uint32_t* status, double* p,
+                         double* logp, double* q, double* logq, double* r) {
+    uint32_t st = 0;
+    /* Step 1: p_i for i = 0..k and q_i for i = 0..k-1. */
+    for (int i = 0; i <= k; ++i) {
+        double S;
+        softmax_row(T, dtype, (size_t)i * V, V, tau, p + (size_t)i * V, logp + (size_t)i * V, &S);
+        if (!(S > 0.0) || !isfinite(S)) st |= ST_BAD_ROW;
+    }
+    for (int i = 0; i < k; ++i) {
+        double S;
+        softmax_row(D, dtype, (size_t)i * V, V, tau, q + (size_t)i * V, logq + (size_t)i * V, &S);
+        if (!(S > 0.0) || !isfinite(S)) st |= ST_BAD_ROW;
+    }
+
+    /* Step 2: rejection tests in order; n = index of the first rejected draft token. */
+    int n = k;
+    for (int i = 0; i < k; ++i) {
+        double rho;
+        int32_t xi = x[i];
+        if (xi < 0 || xi >= V) {
+            st |= ST_BAD_TOKEN;
+            rho = 0.0;
+        } else {
+            double px = p[(size_t)i * V + xi], qx = q[(size_t)i * V + xi];
+            if (qx > 0.0) rho = px / qx;
+            else rho = (px > 0.0) ? INFINITY : 0.0;
+        }
+        if (ratio) ratio[i] = rho;
+        double thr = rho < 1.0 ? rho : 1.0;
+        int accepted = ((double)u[i] < thr);
+        /* the band flag only counts for tests that are reached: none yet rejected (n == k here) */
+        if (accept_band) accept_band[i] = (n == k) && (fabs((double)u[i] - rho) < 1e-6);
+        if (!accepted && n == k) n = i;
+    }
+
+    /* Step 3: the distribution the extra token is drawn from. */
+    double R = 0.0;
+    if (n < k) {
+        for (int v = 0; v < V; ++v) {
+            double d = p[(size_t)n * V + v] - q[(size_t)n * V + v];
+            r[v] = d > 0.0 ? d : 0.0;
+            R += r[v];
+        }
+        if (!(R > 0.0)) { /* cannot happen in exact arithmetic: fall back to p_n */
+            st |= ST_ZERO_RESIDUAL;
+            R = 0.0;
+            for (int v = 0; v < V; ++v) {
+                r[v] = p[(size_t)n * V + v];
+                R += r[v];
+            }
+        }
+    } else {
+        for (int v = 0; v < V; ++v) {
+            r[v] = p[(size_t)k * V + v];
+            R += r[v];
+        }
+    }
+
+    /* Step 4: inverse CDF in vocabulary order with the (k+1)-th uniform. */
+    double t = (double)u[k] * R;
+    double c = 0.0, c_before = 0.0;
+    int y = -1;
+    for (int v = 0; v < V; ++v) {
+        double c_next = c + r[v];
+        if (c_next > t) {
+            y = v;
+            c_before = c;
+            c = c_next;
+            break;
+        }
+        c = c_next;
+    }
+    if (y < 0) { /* rounding pushed t to the total: last token with mass */
+        for (int v = V - 1; v >= 0; --v)
+            if (r[v] > 0.0) {
+                y = v;
+                break;
+            }
+        if (y < 0) y = 0;
+        if (cdf_margin) *cdf_margin = 0.0;
+    } else if (cdf_margin) {
+        double lo = t - c_before, hi = c - t;
+        *cdf_margin = (lo < hi ? lo : hi) / R;
+    }
+
+    /* Step 5: emitted tokens. */
+    *accept_len = n;
+    for (int i = 0; i <= k; ++i) tokens[i] = (i < n) ? x[i] : (i == n ? y : -1);
+
+    /* Step 6: feedback loss KL(p||q) and its gradient w.r.t. the draft logits. */
+    for (int i = 0; i < k; ++i) {
+        const double* pi = p + (size_t)i * V;
+        const double* qi = q + (size_t)i * V;
+        const double* lpi = logp + (size_t)i * V;
+        const double* lqi = logq + (size_t)i * V;
+        double kl = 0.0, acc = 0.0;
+        for (int v = 0; v < V; ++v) {
+            if (pi[v] > 0.0) kl += pi[v] * (lpi[v] - lqi[v]);
+            acc += pi[v] < qi[v] ? pi[v] : qi[v];
+            if (grad) grad[(size_t)i * V + v] = (qi[v] - pi[v]) / tau;
+        }
+        if (loss) loss[i] = kl;
+        if (acc_prob) acc_prob[i] = acc;
+    }
+    if (status) *status = st;
+}
+
+/*
+ * sd_oracle -- the whole step for B sequences.  All pointers are host pointers.
+ *   T [B,k+1,V], D [B,k,V] in `dtype`; x [B,k] int32; u [B,k+1] fp32; tau > 0.
+ *   out_accept_len [B], out_tokens [B,k+1] (-1 padded) are required; the rest may be NULL:
+ *   out_loss [B,k], out_grad [B,k,V], out_acc_prob [B,k], out_ratio [B,k] (p(x)/q(x)),
+ *   out_accept_band [B,k] (1 where a reached test has |u - p/q| < 1e-6),
+ *   out_cdf_margin [B] (distance of u*R to the nearer edge of the chosen CDF interval, over R),
+ *   out_status [B].
+ *   nthreads: sequences are independent; > 1 spreads them over OpenMP threads when built with
+ *   OpenMP (the arithmetic of a sequence does not change).  Returns 0, or -1 on a bad argument
+ *   or allocation failure.
+ */
+int sd_oracle(const void* T, const void* D, int dtype, const int32_t* x, const float* u,
+              double tau, int B, int k, int V, int32_t* out_accept_len, int32_t* out_tokens,
+              double* out_loss, double* out_grad, double* out_acc_prob, double* out_ratio,
+              uint8_t* out_accept_band, double* out_cdf_margin, uint32_t* out_status,
+              int nthreads) {
+    if (!T || !D || !x || !u || !out_accept_len || !out_tokens) return -1;
+    if (B < 1 || k < 1 || V < 1 || !(tau > 0.0) || !isfinite(tau)) return -1;
+    if (dtype != SD_ORACLE_F32 && dtype != SD_ORACLE_BF16) return -1;
+    size_t esz = dtype == SD_ORACLE_F32 ? 4 : 2;
+    int failed = 0;
+#ifdef _OPENMP
+    if (nthreads < 1) nthreads = 1;
+#pragma omp parallel num_threads(nthreads)
+#endif
+    {
+        size_t rows = (size_t)(k + 1) * V;
+        double* p = (double*)malloc(rows * sizeof(double));
+        double* logp = (double*)malloc(rows * sizeof(double));
+        double* q = (double*)malloc((size_t)k * V * sizeof(double));
+        double* logq = (double*)malloc((size_t)k * V * sizeof(double));
+        double* r = (double*)malloc((size_t)V * sizeof(double));
+        if (!p || !logp || !q || !logq || !r) {
+#ifdef _OPENMP
+#pragma omp atomic write
+#endif
+            failed = 1;
+        } else {
+#ifdef _OPENMP
+#pragma omp for schedule(dynamic, 1)
+#endif
+            for (int b = 0; b < B; ++b) {
+                const char* Tb = (const char*)T + (size_t)b * (k + 1) * V * esz;
+                const char* Db = (const char*)D + (size_t)b * k * V * esz;
+                one_sequence(Tb, Db, dtype, x + (size_t)b * k, u + (size_t)b * (k + 1), tau, k, V,
+                             out_accept_len + b, out_tokens + (size_t)b * (k + 1),
+                             out_loss ? out_loss + (size_t)b * k : NULL,
+                             out_grad ? out_grad + (size_t)b * k * V : NULL,
+                             out_acc_prob ? out_acc_prob + (size_t)b * k : NULL,
+                             out_ratio ? out_ratio + (size_t)b * k : NULL,
+                             out_accept_band ? out_accept_band + (size_t)b * k : NULL,
+                             out_cdf_margin ? out_cdf_margin + b : NULL,
+                             out_status ? out_status + b : NULL, p, logp, q, logq, r);
+            }
+        }
+        free(p);
+        free(logp);
+        free(q);
+        free(logq);
+        free(r);
+    }
+    (void)nthreads;
+    return failed ? -1 : 0;
+}
+
+/* Threads the build can use: 1 without OpenMP. */
+int sd_oracle_max_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

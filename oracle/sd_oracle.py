@@ -1,0 +1,105 @@
+"""TEST INFRASTRUCTURE: ctypes front end of the CPU oracle in ``sd_oracle.c``.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import this module.
+It compiles ``sd_oracle.c`` with gcc on first use (``build()``), loads it and exposes
+``verify_feedback`` which takes and returns numpy arrays.  Nothing here touches CUDA and nothing
+here is imported by the product package.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "sd_oracle.c")
+_LIB = os.path.join(_HERE, "libsd_oracle.so")
+_lib = None
+
+F32 = 0
+BF16 = 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle into a shared object next to its source; returns the path."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-shared", "-fPIC", "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        P = ctypes.c_void_p
+        lib.sd_oracle.restype = ctypes.c_int
+        lib.sd_oracle.argtypes = [P, P, ctypes.c_int, P, P, ctypes.c_double, ctypes.c_int,
+                                  ctypes.c_int, ctypes.c_int, P, P, P, P, P, P, P, P, P,
+                                  ctypes.c_int]
+        lib.sd_oracle_max_threads.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def max_threads() -> int:
+    return int(_load().sd_oracle_max_threads())
+
+
+@dataclass
+class OracleResult:
+    accept_len: np.ndarray          # [B] int32
+    tokens: np.ndarray              # [B,k+1] int32, -1 padded
+    loss: Optional[np.ndarray]      # [B,k] float64  KL(p||q)
+    grad: Optional[np.ndarray]      # [B,k,V] float64 (q-p)/tau
+    acc_prob: np.ndarray            # [B,k] float64 sum min(p,q)
+    ratio: np.ndarray               # [B,k] float64 p(x)/q(x)
+    accept_band: np.ndarray         # [B,k] uint8: reached test with |u - p/q| < 1e-6
+    cdf_margin: np.ndarray          # [B] float64
+    status: np.ndarray              # [B] uint32
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def verify_feedback(target_logits: np.ndarray, draft_logits: np.ndarray, draft_tokens: np.ndarray,
+                    uniforms: np.ndarray, temperature: float, *, want_grad: bool = True,
+                    want_loss: bool = True, nthreads: int = 1) -> OracleResult:
+    """Run the oracle.  Logits are float32 arrays, or uint16 arrays holding bf16 bit patterns."""
+    T = np.ascontiguousarray(target_logits)
+    D = np.ascontiguousarray(draft_logits)
+    if T.dtype == np.float32 and D.dtype == np.float32:
+        dtype = F32
+    elif T.dtype == np.uint16 and D.dtype == np.uint16:
+        dtype = BF16
+    else:
+        raise TypeError("logits must both be float32 or both be uint16 (bf16 bits)")
+    if T.ndim != 3 or D.ndim != 3:
+        raise ValueError("logits must be [B,k+1,V] and [B,k,V]")
+    B, k1, V = T.shape
+    k = k1 - 1
+    if D.shape != (B, k, V):
+        raise ValueError(f"draft logits {D.shape} do not match target logits {T.shape}")
+    x = np.ascontiguousarray(draft_tokens, dtype=np.int32)
+    u = np.ascontiguousarray(uniforms, dtype=np.float32)
+    if x.shape != (B, k) or u.shape != (B, k + 1):
+        raise ValueError("draft_tokens must be [B,k] and uniforms [B,k+1]")
+    res = OracleResult(
+        accept_len=np.empty(B, np.int32), tokens=np.empty((B, k + 1), np.int32),
+        loss=np.empty((B, k), np.float64) if want_loss else None,
+        grad=np.empty((B, k, V), np.float64) if want_grad else None,
+        acc_prob=np.empty((B, k), np.float64), ratio=np.empty((B, k), np.float64),
+        accept_band=np.empty((B, k), np.uint8), cdf_margin=np.empty(B, np.float64),
+        status=np.empty(B, np.uint32))
+    rc = _load().sd_oracle(_ptr(T), _ptr(D), dtype, _ptr(x), _ptr(u), float(temperature), B, k, V,
+                           _ptr(res.accept_len), _ptr(res.tokens), _ptr(res.loss), _ptr(res.grad),
+                           _ptr(res.acc_prob), _ptr(res.ratio), _ptr(res.accept_band),
+                           _ptr(res.cdf_margin), _ptr(res.status), int(nthreads))
+    if rc != 0:
+        raise RuntimeError(f"sd_oracle failed with code {rc}")
+    return res
