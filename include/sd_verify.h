@@ -76,6 +76,7 @@ extern "C" {
 #define SD_STATUS_BAD_TOKEN 1u      /* some draft token of the sequence is outside [0,V): treated as rejected */
 #define SD_STATUS_BAD_ROW 2u        /* a softmax denominator of the sequence is not finite and positive */
 #define SD_STATUS_ZERO_RESIDUAL 4u  /* rejection with sum max(0,p-q) == 0: token drawn from p instead */
+#define SD_STATUS_TIMEOUT 0x80000000u /* a bounded wait for a bulk copy gave up: outputs of the sequence are invalid */
 
 /*
  * sd_verify_feedback / sd_verify_feedback_bf16 -- the whole step (Algorithm 1 from "Determine

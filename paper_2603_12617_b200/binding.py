@@ -1,0 +1,218 @@
+"""Thin ctypes binding of the C ABI in ``include/sd_verify.h``.
+
+Argument marshalling only: every step of the verify-and-feedback path runs in the CUDA library.
+torch is used for device memory, streams and nothing else.  The functions have the names of the
+C entry points.  If the shared library is missing or cannot be loaded the import of this module
+fails: there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+SD_DTYPE_F32 = 0
+SD_DTYPE_BF16 = 1
+
+SD_STATUS_BAD_TOKEN = 1
+SD_STATUS_BAD_ROW = 2
+SD_STATUS_ZERO_RESIDUAL = 4
+SD_STATUS_TIMEOUT = 0x80000000
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "lib", "libsd_verify.so")
+
+
+class SdVerifyError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        text = _lib.sd_strerror(code).decode()
+        detail = _lib.sd_last_cuda_error().decode()
+        super().__init__(f"{where} failed with {code}: {text}" + (f" [{detail}]" if detail else ""))
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -c 'import __graft_entry__ as g; g.build()'` "
+            "(there is no CPU fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    P, I, F, Z = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    lib.sd_verify_feedback.restype = I
+    lib.sd_verify_feedback.argtypes = [P, P, P, P, F, I, I, I, P, P, P, P, P]
+    lib.sd_verify_feedback_bf16.restype = I
+    lib.sd_verify_feedback_bf16.argtypes = [P, P, P, P, F, I, I, I, P, P, P, P, P]
+    lib.sd_verify_feedback_ex.restype = I
+    lib.sd_verify_feedback_ex.argtypes = [P, P, P, P, F, I, I, I, I, P, P, P, P, P, P, P, Z, P]
+    lib.sd_verify_feedback_host.restype = I
+    lib.sd_verify_feedback_host.argtypes = [P, P, P, P, F, I, I, I, I, P, P, P, P, P, P]
+    lib.sd_workspace_bytes.restype = Z
+    lib.sd_workspace_bytes.argtypes = [I, I, I, I]
+    lib.sd_launch_info.restype = None
+    lib.sd_launch_info.argtypes = [P] * 6
+    lib.sd_release_cached_buffers.restype = None
+    lib.sd_release_cached_buffers.argtypes = []
+    lib.sd_strerror.restype = ctypes.c_char_p
+    lib.sd_strerror.argtypes = [I]
+    lib.sd_last_cuda_error.restype = ctypes.c_char_p
+    lib.sd_last_cuda_error.argtypes = []
+    lib.sd_version.restype = I
+    lib.sd_version.argtypes = []
+    return lib
+
+
+_lib = _load()
+
+
+@dataclass
+class StepOutputs:
+    accept_len: torch.Tensor            # [B] int32
+    tokens: torch.Tensor                # [B,k+1] int32, -1 padded
+    loss: Optional[torch.Tensor]        # [B,k] float32 KL(p||q)
+    grad_draft: Optional[torch.Tensor]  # [B,k,V], dtype of the logits
+    acc_prob: Optional[torch.Tensor] = None   # [B,k] float32
+    status: Optional[torch.Tensor] = None     # [B] int32 view of the uint32 status words
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return SD_DTYPE_F32
+    if t.dtype == torch.bfloat16:
+        return SD_DTYPE_BF16
+    raise TypeError(f"logits must be float32 or bfloat16, got {t.dtype}")
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _shapes(target_logits, draft_logits, draft_tokens, uniforms):
+    if target_logits.dim() != 3 or draft_logits.dim() != 3:
+        raise ValueError("logits must be [B,k+1,V] and [B,k,V]")
+    B, k1, V = target_logits.shape
+    k = k1 - 1
+    if tuple(draft_logits.shape) != (B, k, V):
+        raise ValueError(f"draft logits {tuple(draft_logits.shape)} do not match target {tuple(target_logits.shape)}")
+    if tuple(draft_tokens.shape) != (B, k) or draft_tokens.dtype != torch.int32:
+        raise ValueError("draft_tokens must be int32 [B,k]")
+    if tuple(uniforms.shape) != (B, k + 1) or uniforms.dtype != torch.float32:
+        raise ValueError("uniforms must be float32 [B,k+1]")
+    if draft_logits.dtype != target_logits.dtype:
+        raise TypeError("target and draft logits must have the same dtype")
+    for t in (target_logits, draft_logits, draft_tokens, uniforms):
+        if not t.is_contiguous():
+            raise ValueError("inputs must be contiguous")
+    return B, k, V
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def sd_version() -> int:
+    return int(_lib.sd_version())
+
+
+def sd_workspace_bytes(B: int, k: int, V: int, dtype: int) -> int:
+    return int(_lib.sd_workspace_bytes(B, k, V, dtype))
+
+
+def sd_launch_info() -> dict:
+    vals = [ctypes.c_int(0) for _ in range(6)]
+    _lib.sd_launch_info(*[ctypes.byref(v) for v in vals])
+    keys = ["path", "cluster_size", "threads", "smem_bytes", "blocks", "kernels"]
+    return {k: v.value for k, v in zip(keys, vals)}
+
+
+def sd_release_cached_buffers() -> None:
+    _lib.sd_release_cached_buffers()
+
+
+def sd_verify_feedback(target_logits: torch.Tensor, draft_logits: torch.Tensor,
+                       draft_tokens: torch.Tensor, uniforms: torch.Tensor, temperature: float, *,
+                       want_loss: bool = True, want_grad: bool = True,
+                       out: Optional[StepOutputs] = None,
+                       stream: Optional[torch.cuda.Stream] = None) -> StepOutputs:
+    """``sd_verify_feedback`` / ``sd_verify_feedback_bf16`` on device tensors (library scratch)."""
+    B, k, V = _shapes(target_logits, draft_logits, draft_tokens, uniforms)
+    dev = target_logits.device
+    if dev.type != "cuda":
+        raise ValueError("device tensors required (use sd_verify_feedback_host for host tensors)")
+    if out is None:
+        out = StepOutputs(
+            accept_len=torch.empty(B, dtype=torch.int32, device=dev),
+            tokens=torch.empty((B, k + 1), dtype=torch.int32, device=dev),
+            loss=torch.empty((B, k), dtype=torch.float32, device=dev) if (want_loss or want_grad) else None,
+            grad_draft=torch.empty_like(draft_logits) if want_grad else None)
+    fn = _lib.sd_verify_feedback if target_logits.dtype == torch.float32 else _lib.sd_verify_feedback_bf16
+    _dtype_code(target_logits)
+    with torch.cuda.device(dev):
+        rc = fn(_ptr(target_logits), _ptr(draft_logits), _ptr(draft_tokens), _ptr(uniforms),
+                float(temperature), B, k, V, _ptr(out.accept_len), _ptr(out.tokens), _ptr(out.loss),
+                _ptr(out.grad_draft), _stream_ptr(stream))
+    if rc != 0:
+        raise SdVerifyError(rc, "sd_verify_feedback")
+    return out
+
+
+def sd_verify_feedback_ex(target_logits: torch.Tensor, draft_logits: torch.Tensor,
+                          draft_tokens: torch.Tensor, uniforms: torch.Tensor, temperature: float, *,
+                          want_loss: bool = True, want_grad: bool = True, want_acc_prob: bool = True,
+                          want_status: bool = True, workspace: Optional[torch.Tensor] = None,
+                          out: Optional[StepOutputs] = None,
+                          stream: Optional[torch.cuda.Stream] = None) -> StepOutputs:
+    """``sd_verify_feedback_ex`` on device tensors with caller-owned scratch."""
+    B, k, V = _shapes(target_logits, draft_logits, draft_tokens, uniforms)
+    dev = target_logits.device
+    code = _dtype_code(target_logits)
+    if workspace is None:
+        workspace = torch.empty(sd_workspace_bytes(B, k, V, code), dtype=torch.uint8, device=dev)
+    if out is None:
+        out = StepOutputs(
+            accept_len=torch.empty(B, dtype=torch.int32, device=dev),
+            tokens=torch.empty((B, k + 1), dtype=torch.int32, device=dev),
+            loss=torch.empty((B, k), dtype=torch.float32, device=dev) if (want_loss or want_grad) else None,
+            grad_draft=torch.empty_like(draft_logits) if want_grad else None,
+            acc_prob=torch.empty((B, k), dtype=torch.float32, device=dev) if want_acc_prob else None,
+            status=torch.empty(B, dtype=torch.int32, device=dev) if want_status else None)
+    with torch.cuda.device(dev):
+        rc = _lib.sd_verify_feedback_ex(
+            _ptr(target_logits), _ptr(draft_logits), _ptr(draft_tokens), _ptr(uniforms), float(temperature),
+            B, k, V, code, _ptr(out.accept_len), _ptr(out.tokens), _ptr(out.loss), _ptr(out.grad_draft),
+            _ptr(out.acc_prob), _ptr(out.status), _ptr(workspace), workspace.numel() * workspace.element_size(),
+            _stream_ptr(stream))
+    if rc != 0:
+        raise SdVerifyError(rc, "sd_verify_feedback_ex")
+    return out
+
+
+def sd_verify_feedback_host(target_logits: torch.Tensor, draft_logits: torch.Tensor,
+                            draft_tokens: torch.Tensor, uniforms: torch.Tensor, temperature: float, *,
+                            want_loss: bool = True, want_grad: bool = True, want_acc_prob: bool = False,
+                            want_status: bool = False, out: Optional[StepOutputs] = None,
+                            pin_outputs: bool = True) -> StepOutputs:
+    """``sd_verify_feedback_host``: host tensors in, host tensors out, copies inside the call."""
+    B, k, V = _shapes(target_logits, draft_logits, draft_tokens, uniforms)
+    if target_logits.device.type != "cpu":
+        raise ValueError("host tensors required")
+    code = _dtype_code(target_logits)
+    pin = pin_outputs and torch.cuda.is_available()
+    if out is None:
+        out = StepOutputs(
+            accept_len=torch.empty(B, dtype=torch.int32, pin_memory=pin),
+            tokens=torch.empty((B, k + 1), dtype=torch.int32, pin_memory=pin),
+            loss=torch.empty((B, k), dtype=torch.float32, pin_memory=pin) if (want_loss or want_grad) else None,
+            grad_draft=torch.empty(draft_logits.shape, dtype=draft_logits.dtype, pin_memory=pin) if want_grad else None,
+            acc_prob=torch.empty((B, k), dtype=torch.float32, pin_memory=pin) if want_acc_prob else None,
+            status=torch.empty(B, dtype=torch.int32, pin_memory=pin) if want_status else None)
+    rc = _lib.sd_verify_feedback_host(
+        _ptr(target_logits), _ptr(draft_logits), _ptr(draft_tokens), _ptr(uniforms), float(temperature),
+        B, k, V, code, _ptr(out.accept_len), _ptr(out.tokens), _ptr(out.loss), _ptr(out.grad_draft),
+        _ptr(out.acc_prob), _ptr(out.status))
+    if rc != 0:
+        raise SdVerifyError(rc, "sd_verify_feedback_host")
+    return out

@@ -1,0 +1,502 @@
+// Host side of the C ABI declared in include/sd_verify.h: argument checks, workspace layout,
+// choice of launch shape, the per-device scratch cache and the host-memory entry point.
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <mutex>
+
+#include "sd_kernels.cuh"
+
+namespace {
+
+using namespace sdv;
+
+constexpr int kMaxDevices = 64;
+constexpr size_t kAlign = 256;
+constexpr int kMaxDynSmem = 227 * 1024 - 2048;   // per-block limit minus the static part
+
+thread_local char tl_cuda_error[256] = "";
+thread_local int tl_info[6] = {0, 0, 0, 0, 0, 0};
+
+int cuda_fail(cudaError_t e, const char* where) {
+    snprintf(tl_cuda_error, sizeof tl_cuda_error, "%s: %s", where, cudaGetErrorString(e));
+    return SD_ERR_CUDA;
+}
+#define SD_CUDA(call)                                         \
+    do {                                                      \
+        cudaError_t e_ = (call);                              \
+        if (e_ != cudaSuccess) return cuda_fail(e_, #call);   \
+    } while (0)
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+int elem_bytes(int dtype) { return dtype == SD_DTYPE_F32 ? 4 : 2; }
+int chunk_elems(int dtype) { return kChunkVecs * (dtype == SD_DTYPE_F32 ? 4 : 8); }
+
+struct WorkspaceLayout {
+    size_t ticket, wstatus, accept, rowc, chunk_sums, total;
+    int NC;
+};
+
+bool shape_ok(int B, int k, int V) {
+    if (B < 1 || k < 1 || V < 1 || k > SD_MAX_K) return false;
+    const long double n = (long double)B * (long double)(k + 1) * (long double)V;
+    return n < 4.0e18L && (long double)B * (k + 1) < 2.0e9L;
+}
+
+WorkspaceLayout workspace_layout(int B, int k, int V, int dtype) {
+    WorkspaceLayout L;
+    L.NC = (V + chunk_elems(dtype) - 1) / chunk_elems(dtype);
+    size_t off = 0;
+    L.ticket = off;      off = align_up(off + (size_t)B * 4, kAlign);
+    L.wstatus = off;     off = align_up(off + (size_t)B * 4, kAlign);
+    L.accept = off;      off = align_up(off + (size_t)B * k, kAlign);
+    L.rowc = off;        off = align_up(off + (size_t)B * (k + 1) * sizeof(RowConst), kAlign);
+    L.chunk_sums = off;  off = align_up(off + (size_t)B * (k + 1) * L.NC * 4, kAlign);
+    L.total = off;
+    return L;
+}
+
+struct StageSet {
+    unsigned char* base = nullptr;
+    size_t bytes = 0;
+    cudaEvent_t in_ready = nullptr, comp_done = nullptr, out_done = nullptr;
+};
+
+struct DeviceState {
+    std::mutex mu;
+    bool probed = false;
+    int cc_major = 0;
+    int sm_count = 0;
+    // grow-only scratch of the 13-argument entry points
+    void* ws = nullptr;
+    size_t ws_bytes = 0;
+    bool ws_clean = false;   // tickets and status words are zero
+    bool attr_set[2] = {false, false};   // shared-memory / cluster attributes of the fast kernel
+    // last launch-shape decision of the fast path
+    int dec_dtype = -1, dec_NC = 0, dec_forced = 0, dec_C = 0, dec_chunks = 0;
+    long long dec_units = 0;
+    // host-memory entry point
+    StageSet stage[2];
+    cudaStream_t s_h2d = nullptr, s_comp = nullptr, s_d2h = nullptr;
+};
+DeviceState g_dev[kMaxDevices];
+
+int current_device(int* dev, DeviceState** st) {
+    cudaError_t e = cudaGetDevice(dev);
+    if (e != cudaSuccess) {
+        cuda_fail(e, "cudaGetDevice");
+        return SD_ERR_NO_DEVICE;
+    }
+    if (*dev < 0 || *dev >= kMaxDevices) return SD_ERR_NO_DEVICE;
+    DeviceState& d = g_dev[*dev];
+    std::lock_guard<std::mutex> lock(d.mu);
+    if (!d.probed) {
+        cudaDeviceProp prop;
+        e = cudaGetDeviceProperties(&prop, *dev);
+        if (e != cudaSuccess) {
+            cuda_fail(e, "cudaGetDeviceProperties");
+            return SD_ERR_NO_DEVICE;
+        }
+        d.cc_major = prop.major;
+        d.sm_count = prop.multiProcessorCount;
+        d.probed = true;
+    }
+    if (d.cc_major != 10) {
+        snprintf(tl_cuda_error, sizeof tl_cuda_error, "device %d has compute capability %d.x, need 10.x", *dev,
+                 d.cc_major);
+        return SD_ERR_NO_DEVICE;
+    }
+    *st = &d;
+    return SD_OK;
+}
+
+template <int DT>
+int launch_cluster(DeviceState& d, const Params& P, int C, int slice_chunks, cudaStream_t stream,
+                   bool query_only, int* max_clusters) {
+    auto kern = sd_cluster_kernel<DT>;
+    const int smem = slice_chunks * 2 * kChunkBytes;
+    if (!d.attr_set[DT]) {
+        SD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
+        SD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+        d.attr_set[DT] = true;
+    }
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    const long long units = (long long)P.B * (P.k + 1);
+    cfg.gridDim = dim3((unsigned)(units * C), 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)C;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (query_only) {
+        int n = 0;
+        cudaError_t e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
+        if (e != cudaSuccess) {
+            (void)cudaGetLastError();
+            n = 0;
+        }
+        *max_clusters = n;
+        return SD_OK;
+    }
+    SD_CUDA(cudaLaunchKernelEx(&cfg, kern, P, slice_chunks));
+    tl_info[0] = 1; tl_info[1] = C; tl_info[2] = kThreads; tl_info[3] = smem;
+    tl_info[4] = (int)(units * C); tl_info[5] = 1;
+    return SD_OK;
+}
+
+template <int DT>
+int launch_generic(const Params& P, cudaStream_t stream) {
+    const long long units = (long long)P.B * (P.k + 1);
+    sd_generic_kernel<DT><<<(unsigned)units, kThreads, 0, stream>>>(P);
+    SD_CUDA(cudaGetLastError());
+    tl_info[0] = 0; tl_info[1] = 1; tl_info[2] = kThreads; tl_info[3] = 0;
+    tl_info[4] = (int)units; tl_info[5] = 1;
+    return SD_OK;
+}
+
+// Cluster size for the fast path, 0 if it cannot run.  Blocks of about 64 KiB leave room for
+// three per SM, so loads of one block overlap the arithmetic of the others.
+int choose_cluster(DeviceState& d, const Params& P, int dtype, int* slice_chunks_out) {
+    const char* env = getenv("SD_VERIFY_CLUSTER");
+    const int forced = env ? atoi(env) : 0;
+    const long long units = (long long)P.B * (P.k + 1);
+    if (d.dec_dtype == dtype && d.dec_NC == P.NC && d.dec_units == units && d.dec_forced == forced) {
+        *slice_chunks_out = d.dec_chunks;
+        return d.dec_C;
+    }
+    int best = 0, best_chunks = 0;
+    auto usable = [&](int C, int* chunks) -> bool {
+        const int sc = (P.NC + C - 1) / C;
+        if (sc > kMaxChunksPerBlock || sc * 2 * kChunkBytes > kMaxDynSmem) return false;
+        int n = 0;   // can the device hold at least one such cluster?
+        int rc = dtype == SD_DTYPE_F32 ? launch_cluster<SD_DTYPE_F32>(d, P, C, sc, nullptr, true, &n)
+                                       : launch_cluster<SD_DTYPE_BF16>(d, P, C, sc, nullptr, true, &n);
+        if (rc != SD_OK || n < 1) return false;
+        *chunks = sc;
+        return true;
+    };
+    auto remember = [&](int C, int sc) {
+        d.dec_dtype = dtype; d.dec_NC = P.NC; d.dec_units = units; d.dec_forced = forced;
+        d.dec_C = C; d.dec_chunks = sc;
+        *slice_chunks_out = sc;
+        return C;
+    };
+    if (forced > 0) {
+        int sc = 0;
+        if ((forced & (forced - 1)) == 0 && forced <= kMaxCluster && usable(forced, &sc)) return remember(forced, sc);
+        return remember(0, 0);
+    }
+    const int target_smem = 72 * 1024;
+    for (int C = 1; C <= kMaxCluster; C *= 2) {
+        int sc;
+        if (!usable(C, &sc)) continue;
+        best = C;
+        best_chunks = sc;
+        const bool small_enough = sc * 2 * kChunkBytes <= target_smem;
+        const bool fills_gpu = units * C >= 2LL * d.sm_count;
+        if (small_enough && (fills_gpu || sc <= kWarps)) break;
+    }
+    return remember(best, best_chunks);
+}
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+int check_args(const void* T, const void* D, const int32_t* x, const float* u, float tau, int B, int k, int V,
+               int dtype, const int32_t* accept_len, const int32_t* tokens, const float* loss, const void* grad,
+               const float* acc_prob, const uint32_t* status) {
+    if (dtype != SD_DTYPE_F32 && dtype != SD_DTYPE_BF16) return SD_ERR_DTYPE;
+    if (!T || !D || !x || !u || !accept_len || !tokens) return SD_ERR_NULL;
+    if (!shape_ok(B, k, V)) return SD_ERR_SHAPE;
+    if (!(tau > 0.f) || !isfinite(tau)) return SD_ERR_TEMPERATURE;
+    const size_t es = (size_t)elem_bytes(dtype);
+    if (!aligned(T, es) || !aligned(D, es) || (grad && !aligned(grad, es))) return SD_ERR_ALIGN;
+    if (!aligned(x, 4) || !aligned(u, 4) || !aligned(accept_len, 4) || !aligned(tokens, 4) ||
+        (loss && !aligned(loss, 4)) || (acc_prob && !aligned(acc_prob, 4)) || (status && !aligned(status, 4)))
+        return SD_ERR_ALIGN;
+    return SD_OK;
+}
+
+// Enqueue the step on `stream` with scratch `ws` (device, layout L).  clean: tickets/status are zero.
+int run_device(DeviceState& d, const void* T, const void* D, const int32_t* x, const float* u, float tau, int B,
+               int k, int V, int dtype, int32_t* accept_len, int32_t* tokens, float* loss, void* grad,
+               float* acc_prob, uint32_t* status, unsigned char* ws, const WorkspaceLayout& L, bool clean,
+               cudaStream_t stream) {
+    Params P;
+    memset(&P, 0, sizeof P);
+    P.T = T; P.D = D; P.x = x; P.u = u;
+    P.B = B; P.k = k; P.V = V; P.NC = L.NC;
+    P.c64 = 1.4426950408889634 / (double)tau;
+    P.c = (float)P.c64;
+    P.tau = tau;
+    P.inv_tau = 1.0 / (double)tau;
+    P.accept_len = accept_len; P.tokens = tokens; P.loss = loss; P.grad = grad;
+    P.acc_prob = acc_prob; P.status = status;
+    P.ticket = reinterpret_cast<uint32_t*>(ws + L.ticket);
+    P.wstatus = reinterpret_cast<uint32_t*>(ws + L.wstatus);
+    P.accept = ws + L.accept;
+    P.rowc = reinterpret_cast<RowConst*>(ws + L.rowc);
+    P.chunk_sums = reinterpret_cast<float*>(ws + L.chunk_sums);
+
+    if (!clean) SD_CUDA(cudaMemsetAsync(ws, 0, L.accept, stream));   // tickets and status words
+
+    const size_t row_bytes = (size_t)V * elem_bytes(dtype);
+    const bool fast = (row_bytes % 16 == 0) && aligned(T, 16) && aligned(D, 16) && (!grad || aligned(grad, 16)) &&
+                      !getenv("SD_VERIFY_FORCE_GENERIC");
+    int C = 0, slice_chunks = 0;
+    if (fast) C = choose_cluster(d, P, dtype, &slice_chunks);
+    int rc;
+    if (C > 0) {
+        P.blocks_per_unit = C;
+        rc = dtype == SD_DTYPE_F32 ? launch_cluster<SD_DTYPE_F32>(d, P, C, slice_chunks, stream, false, nullptr)
+                                   : launch_cluster<SD_DTYPE_BF16>(d, P, C, slice_chunks, stream, false, nullptr);
+    } else {
+        P.blocks_per_unit = 1;
+        rc = dtype == SD_DTYPE_F32 ? launch_generic<SD_DTYPE_F32>(P, stream)
+                                   : launch_generic<SD_DTYPE_BF16>(P, stream);
+    }
+    return rc;
+}
+
+int run_cached(const void* T, const void* D, const int32_t* x, const float* u, float tau, int B, int k, int V,
+               int dtype, int32_t* accept_len, int32_t* tokens, float* loss, void* grad, void* stream) {
+    int rc = check_args(T, D, x, u, tau, B, k, V, dtype, accept_len, tokens, loss, grad, nullptr, nullptr);
+    if (rc != SD_OK) return rc;
+    int dev;
+    DeviceState* d = nullptr;
+    rc = current_device(&dev, &d);
+    if (rc != SD_OK) return rc;
+    const WorkspaceLayout L = workspace_layout(B, k, V, dtype);
+    std::lock_guard<std::mutex> lock(d->mu);
+    if (d->ws_bytes < L.total) {
+        if (d->ws) {
+            SD_CUDA(cudaDeviceSynchronize());
+            SD_CUDA(cudaFree(d->ws));
+            d->ws = nullptr;
+            d->ws_bytes = 0;
+        }
+        const size_t want = align_up(L.total + L.total / 4, 1 << 20);
+        SD_CUDA(cudaMalloc(&d->ws, want));
+        d->ws_bytes = want;
+        // Zero all of it once: every call leaves its ticket and status words at zero again, so
+        // later calls of any shape find zeros wherever their layout puts those words.
+        SD_CUDA(cudaMemset(d->ws, 0, want));
+        SD_CUDA(cudaDeviceSynchronize());
+        d->ws_clean = true;
+    }
+    rc = run_device(*d, T, D, x, u, tau, B, k, V, dtype, accept_len, tokens, loss, grad, nullptr, nullptr,
+                    static_cast<unsigned char*>(d->ws), L, d->ws_clean, static_cast<cudaStream_t>(stream));
+    d->ws_clean = (rc == SD_OK);   // a failed launch may leave tickets behind: zero them next time
+    return rc;
+}
+
+}  // namespace
+
+extern "C" {
+
+int sd_verify_feedback(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
+                       const float* uniforms, float temperature, int B, int k, int V, int32_t* out_accept_len,
+                       int32_t* out_tokens, float* out_loss, float* out_grad_draft, void* stream) {
+    return run_cached(target_logits, draft_logits, draft_tokens, uniforms, temperature, B, k, V, SD_DTYPE_F32,
+                      out_accept_len, out_tokens, out_loss, out_grad_draft, stream);
+}
+
+int sd_verify_feedback_bf16(const uint16_t* target_logits, const uint16_t* draft_logits,
+                            const int32_t* draft_tokens, const float* uniforms, float temperature, int B, int k,
+                            int V, int32_t* out_accept_len, int32_t* out_tokens, float* out_loss,
+                            uint16_t* out_grad_draft, void* stream) {
+    return run_cached(target_logits, draft_logits, draft_tokens, uniforms, temperature, B, k, V, SD_DTYPE_BF16,
+                      out_accept_len, out_tokens, out_loss, out_grad_draft, stream);
+}
+
+size_t sd_workspace_bytes(int B, int k, int V, int dtype) {
+    if ((dtype != SD_DTYPE_F32 && dtype != SD_DTYPE_BF16) || !shape_ok(B, k, V)) return 0;
+    return workspace_layout(B, k, V, dtype).total;
+}
+
+int sd_verify_feedback_ex(const void* target_logits, const void* draft_logits, const int32_t* draft_tokens,
+                          const float* uniforms, float temperature, int B, int k, int V, int dtype,
+                          int32_t* out_accept_len, int32_t* out_tokens, float* out_loss, void* out_grad_draft,
+                          float* out_acc_prob, uint32_t* out_status, void* workspace, size_t workspace_bytes,
+                          void* stream) {
+    int rc = check_args(target_logits, draft_logits, draft_tokens, uniforms, temperature, B, k, V, dtype,
+                        out_accept_len, out_tokens, out_loss, out_grad_draft, out_acc_prob, out_status);
+    if (rc != SD_OK) return rc;
+    const WorkspaceLayout L = workspace_layout(B, k, V, dtype);
+    if (!workspace || !aligned(workspace, kAlign) || workspace_bytes < L.total) return SD_ERR_WORKSPACE;
+    int dev;
+    DeviceState* d = nullptr;
+    rc = current_device(&dev, &d);
+    if (rc != SD_OK) return rc;
+    std::lock_guard<std::mutex> lock(d->mu);
+    return run_device(*d, target_logits, draft_logits, draft_tokens, uniforms, temperature, B, k, V, dtype,
+                      out_accept_len, out_tokens, out_loss, out_grad_draft, out_acc_prob, out_status,
+                      static_cast<unsigned char*>(workspace), L, false, static_cast<cudaStream_t>(stream));
+}
+
+int sd_verify_feedback_host(const void* target_logits, const void* draft_logits, const int32_t* draft_tokens,
+                            const float* uniforms, float temperature, int B, int k, int V, int dtype,
+                            int32_t* out_accept_len, int32_t* out_tokens, float* out_loss, void* out_grad_draft,
+                            float* out_acc_prob, uint32_t* out_status) {
+    int rc = check_args(target_logits, draft_logits, draft_tokens, uniforms, temperature, B, k, V, dtype,
+                        out_accept_len, out_tokens, out_loss, out_grad_draft, out_acc_prob, out_status);
+    if (rc != SD_OK) return rc;
+    int dev;
+    DeviceState* d = nullptr;
+    rc = current_device(&dev, &d);
+    if (rc != SD_OK) return rc;
+    std::lock_guard<std::mutex> lock(d->mu);
+
+    const size_t es = (size_t)elem_bytes(dtype);
+    const size_t t_seq = (size_t)(k + 1) * V * es, d_seq = (size_t)k * V * es;
+    // sequences per slice: about 96 MiB of logits and gradient in flight per buffer set
+    const size_t per_seq = t_seq + 2 * d_seq;
+    int S = (int)((96u << 20) / per_seq);
+    if (S < 1) S = 1;
+    if (S > B) S = B;
+    const int nslices = (B + S - 1) / S;
+
+    // one device arena per buffer set
+    const WorkspaceLayout L = workspace_layout(S, k, V, dtype);
+    size_t off = 0;
+    const size_t oT = off;   off = align_up(off + (size_t)S * t_seq, kAlign);
+    const size_t oD = off;   off = align_up(off + (size_t)S * d_seq, kAlign);
+    const size_t oG = off;   off = align_up(off + (size_t)S * d_seq, kAlign);
+    const size_t oX = off;   off = align_up(off + (size_t)S * k * 4, kAlign);
+    const size_t oU = off;   off = align_up(off + (size_t)S * (k + 1) * 4, kAlign);
+    const size_t oN = off;   off = align_up(off + (size_t)S * 4, kAlign);
+    const size_t oTok = off; off = align_up(off + (size_t)S * (k + 1) * 4, kAlign);
+    const size_t oL = off;   off = align_up(off + (size_t)S * k * 4, kAlign);
+    const size_t oA = off;   off = align_up(off + (size_t)S * k * 4, kAlign);
+    const size_t oS = off;   off = align_up(off + (size_t)S * 4, kAlign);
+    const size_t oW = off;   off = align_up(off + L.total, kAlign);
+    const size_t arena = off;
+
+    if (!d->s_h2d) {
+        SD_CUDA(cudaStreamCreateWithFlags(&d->s_h2d, cudaStreamNonBlocking));
+        SD_CUDA(cudaStreamCreateWithFlags(&d->s_comp, cudaStreamNonBlocking));
+        SD_CUDA(cudaStreamCreateWithFlags(&d->s_d2h, cudaStreamNonBlocking));
+    }
+    const int nsets = nslices > 1 ? 2 : 1;
+    for (int s = 0; s < nsets; ++s) {
+        StageSet& st = d->stage[s];
+        if (!st.in_ready) {
+            SD_CUDA(cudaEventCreateWithFlags(&st.in_ready, cudaEventDisableTiming));
+            SD_CUDA(cudaEventCreateWithFlags(&st.comp_done, cudaEventDisableTiming));
+            SD_CUDA(cudaEventCreateWithFlags(&st.out_done, cudaEventDisableTiming));
+        }
+        if (st.bytes < arena) {
+            if (st.base) {
+                SD_CUDA(cudaDeviceSynchronize());
+                SD_CUDA(cudaFree(st.base));
+                st.base = nullptr;
+                st.bytes = 0;
+            }
+            SD_CUDA(cudaMalloc(reinterpret_cast<void**>(&st.base), arena));
+            st.bytes = arena;
+        }
+    }
+
+    const unsigned char* hT = static_cast<const unsigned char*>(target_logits);
+    const unsigned char* hD = static_cast<const unsigned char*>(draft_logits);
+    unsigned char* hG = static_cast<unsigned char*>(out_grad_draft);
+    int kernels = 0;
+    for (int s = 0; s < nslices; ++s) {
+        StageSet& st = d->stage[s % nsets];
+        const int b0 = s * S, nb = (B - b0 < S) ? (B - b0) : S;
+        unsigned char* a = st.base;
+        if (s >= nsets) {
+            // the buffer set is free once slice s-2 has been computed and copied out
+            SD_CUDA(cudaStreamWaitEvent(d->s_h2d, st.out_done, 0));
+        }
+        SD_CUDA(cudaMemcpyAsync(a + oT, hT + (size_t)b0 * t_seq, (size_t)nb * t_seq, cudaMemcpyHostToDevice, d->s_h2d));
+        SD_CUDA(cudaMemcpyAsync(a + oD, hD + (size_t)b0 * d_seq, (size_t)nb * d_seq, cudaMemcpyHostToDevice, d->s_h2d));
+        SD_CUDA(cudaMemcpyAsync(a + oX, draft_tokens + (size_t)b0 * k, (size_t)nb * k * 4, cudaMemcpyHostToDevice, d->s_h2d));
+        SD_CUDA(cudaMemcpyAsync(a + oU, uniforms + (size_t)b0 * (k + 1), (size_t)nb * (k + 1) * 4, cudaMemcpyHostToDevice, d->s_h2d));
+        SD_CUDA(cudaEventRecord(st.in_ready, d->s_h2d));
+        SD_CUDA(cudaStreamWaitEvent(d->s_comp, st.in_ready, 0));
+        const WorkspaceLayout Ls = workspace_layout(nb, k, V, dtype);
+        rc = run_device(*d, a + oT, a + oD, reinterpret_cast<int32_t*>(a + oX), reinterpret_cast<float*>(a + oU),
+                        temperature, nb, k, V, dtype, reinterpret_cast<int32_t*>(a + oN),
+                        reinterpret_cast<int32_t*>(a + oTok), out_loss ? reinterpret_cast<float*>(a + oL) : nullptr,
+                        out_grad_draft ? a + oG : nullptr, out_acc_prob ? reinterpret_cast<float*>(a + oA) : nullptr,
+                        out_status ? reinterpret_cast<uint32_t*>(a + oS) : nullptr, a + oW, Ls, false, d->s_comp);
+        if (rc != SD_OK) break;
+        kernels += 1;
+        SD_CUDA(cudaEventRecord(st.comp_done, d->s_comp));
+        SD_CUDA(cudaStreamWaitEvent(d->s_d2h, st.comp_done, 0));
+        SD_CUDA(cudaMemcpyAsync(out_accept_len + b0, a + oN, (size_t)nb * 4, cudaMemcpyDeviceToHost, d->s_d2h));
+        SD_CUDA(cudaMemcpyAsync(out_tokens + (size_t)b0 * (k + 1), a + oTok, (size_t)nb * (k + 1) * 4, cudaMemcpyDeviceToHost, d->s_d2h));
+        if (out_loss)
+            SD_CUDA(cudaMemcpyAsync(out_loss + (size_t)b0 * k, a + oL, (size_t)nb * k * 4, cudaMemcpyDeviceToHost, d->s_d2h));
+        if (out_grad_draft)
+            SD_CUDA(cudaMemcpyAsync(hG + (size_t)b0 * d_seq, a + oG, (size_t)nb * d_seq, cudaMemcpyDeviceToHost, d->s_d2h));
+        if (out_acc_prob)
+            SD_CUDA(cudaMemcpyAsync(out_acc_prob + (size_t)b0 * k, a + oA, (size_t)nb * k * 4, cudaMemcpyDeviceToHost, d->s_d2h));
+        if (out_status)
+            SD_CUDA(cudaMemcpyAsync(out_status + b0, a + oS, (size_t)nb * 4, cudaMemcpyDeviceToHost, d->s_d2h));
+        SD_CUDA(cudaEventRecord(st.out_done, d->s_d2h));
+    }
+    cudaError_t e1 = cudaStreamSynchronize(d->s_h2d);
+    cudaError_t e2 = cudaStreamSynchronize(d->s_comp);
+    cudaError_t e3 = cudaStreamSynchronize(d->s_d2h);
+    if (rc != SD_OK) return rc;
+    if (e1 != cudaSuccess) return cuda_fail(e1, "cudaStreamSynchronize(h2d)");
+    if (e2 != cudaSuccess) return cuda_fail(e2, "cudaStreamSynchronize(compute)");
+    if (e3 != cudaSuccess) return cuda_fail(e3, "cudaStreamSynchronize(d2h)");
+    tl_info[5] = kernels;
+    return SD_OK;
+}
+
+void sd_launch_info(int* path, int* cluster_size, int* threads, int* smem_bytes, int* blocks, int* kernels) {
+    if (path) *path = tl_info[0];
+    if (cluster_size) *cluster_size = tl_info[1];
+    if (threads) *threads = tl_info[2];
+    if (smem_bytes) *smem_bytes = tl_info[3];
+    if (blocks) *blocks = tl_info[4];
+    if (kernels) *kernels = tl_info[5];
+}
+
+void sd_release_cached_buffers(void) {
+    for (int i = 0; i < kMaxDevices; ++i) {
+        DeviceState& d = g_dev[i];
+        std::lock_guard<std::mutex> lock(d.mu);
+        if (!d.probed || (!d.ws && !d.stage[0].base && !d.stage[1].base)) continue;
+        int prev = -1;
+        if (cudaGetDevice(&prev) != cudaSuccess) continue;
+        if (cudaSetDevice(i) != cudaSuccess) continue;
+        cudaDeviceSynchronize();
+        if (d.ws) { cudaFree(d.ws); d.ws = nullptr; d.ws_bytes = 0; d.ws_clean = false; }
+        for (StageSet& st : d.stage)
+            if (st.base) { cudaFree(st.base); st.base = nullptr; st.bytes = 0; }
+        cudaSetDevice(prev);
+    }
+}
+
+const char* sd_strerror(int code) {
+    switch (code) {
+        case SD_OK: return "ok";
+        case SD_ERR_NULL: return "a required pointer is NULL";
+        case SD_ERR_SHAPE: return "B, k or V out of range";
+        case SD_ERR_TEMPERATURE: return "temperature must be a finite number > 0";
+        case SD_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case SD_ERR_DTYPE: return "unknown dtype";
+        case SD_ERR_CUDA: return "a CUDA call failed (see sd_last_cuda_error)";
+        case SD_ERR_NO_DEVICE: return "no current CUDA device of compute capability 10.x";
+        case SD_ERR_ALIGN: return "a pointer is not aligned to its element type";
+        default: return "unknown error code";
+    }
+}
+
+const char* sd_last_cuda_error(void) { return tl_cuda_error; }
+
+int sd_version(void) { return SD_VERSION; }
+
+}  // extern "C"

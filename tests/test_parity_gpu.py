@@ -1,0 +1,435 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded
+inputs and the same pre-drawn uniforms.
+
+Bars (stated here, derived in the design notes):
+  * accept lengths and emitted tokens are bit-exact, except for sequences the oracle marks as
+    sitting on a decision threshold: a reached accept test with |u - p/q| < 1e-6, or an
+    inverse-CDF draw whose target lies within 1e-6 (relative to the total mass) of an interval
+    edge.  Those sequences are counted, must be rare, and must still produce a valid answer.
+  * loss: |gpu - ref| <= tol * |ref| + 4e-7, tol = 1e-5 (fp32 logits) / 2e-2 (bf16 logits).  The
+    absolute term is the rounding floor of the method in fp32: KL is log S_D - log S_T plus a mean,
+    and each softmax denominator S carries a relative error of a few 2^-24 (2^-22 per term from the
+    hardware exp2, averaged over the row), whatever the size of KL.
+  * gradient, per row: max|gpu - ref| <= tol * max|ref| + floor and the same in the L2 norm, the
+    reference being the fp64 value before any rounding to bf16.  floor = 8 * 2^-24 * max(p,q)/tau
+    is the rounding of p and q themselves: it only matters when q - p is a difference of two
+    nearly equal large probabilities (near one-hot rows), never on the five workloads.
+"""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import sd_oracle
+from paper_2603_12617_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"f32": 1e-5, "bf16": 2e-2}
+LOSS_FLOOR = 4e-7
+GRAD_FLOOR = 8 * 2.0 ** -24
+
+
+def logits_f64(inp, seqs=None):
+    sl = slice(None) if seqs is None else np.asarray(seqs)
+    T, D = inp.target_logits[sl], inp.draft_logits[sl]
+    if inp.cfg.dtype == "bf16":
+        T, D = synth.bf16_bits_to_f32(T), synth.bf16_bits_to_f32(D)
+    return T.astype(np.float64), D.astype(np.float64)
+
+
+def prob_max_and_l2(z, tau):
+    """Largest softmax probability and L2 norm of the softmax of every row of z[..., V]."""
+    e = np.exp((z - z.max(axis=-1, keepdims=True)) / tau)
+    s = e.sum(axis=-1)
+    return 1.0 / s, np.sqrt((e * e).sum(axis=-1)) / s
+
+
+@pytest.fixture(scope="module")
+def binding():
+    import __graft_entry__ as entry
+    entry.build()
+    from paper_2603_12617_b200 import binding as b
+    return b
+
+
+def to_device(inp):
+    T = torch.from_numpy(inp.target_logits).cuda()
+    D = torch.from_numpy(inp.draft_logits).cuda()
+    if inp.cfg.dtype == "bf16":
+        T, D = T.view(torch.bfloat16), D.view(torch.bfloat16)
+    return T, D, torch.from_numpy(inp.draft_tokens).cuda(), torch.from_numpy(inp.uniforms).cuda()
+
+
+def oracle_of(inp, seqs=None, want_grad=True):
+    sl = slice(None) if seqs is None else np.asarray(seqs)
+    return sd_oracle.verify_feedback(inp.target_logits[sl], inp.draft_logits[sl], inp.draft_tokens[sl],
+                                     inp.uniforms[sl], inp.tau, want_grad=want_grad,
+                                     nthreads=min(8, sd_oracle.max_threads()))
+
+
+def check(inp, out, ref, seqs=None, max_band_frac=0.02, check_grad=True, check_loss=True):
+    """Compare device outputs (for sequences `seqs`, default all) with the oracle's."""
+    dtype = inp.cfg.dtype
+    tol = TOL[dtype]
+    sl = slice(None) if seqs is None else torch.as_tensor(np.asarray(seqs))
+    n_gpu = out.accept_len.cpu()[sl].numpy()
+    tok_gpu = out.tokens.cpu()[sl].numpy()
+    B, k, V = ref.tokens.shape[0], inp.cfg.k, inp.cfg.V
+    x = inp.draft_tokens if seqs is None else inp.draft_tokens[np.asarray(seqs)]
+
+    # A draw that lands in a token of mass < 2e-6 is inside the sample band by construction, so with
+    # V > 10^5 the band itself is not rare; what must be rare is a disagreement, and every
+    # disagreement must sit inside the band.
+    band = (ref.accept_band.sum(1) > 0) | (ref.cdf_margin <= 1e-6)
+    safe = ~band
+    assert (n_gpu[safe] == ref.accept_len[safe]).all(), "accept lengths differ off the threshold band"
+    assert (tok_gpu[safe] == ref.tokens[safe]).all(), "emitted tokens differ off the threshold band"
+    mismatch = (n_gpu != ref.accept_len) | (tok_gpu != ref.tokens).any(axis=1)
+    assert mismatch.sum() <= max(1, int(max_band_frac * B)), \
+        f"{mismatch.sum()} of {B} sequences differ inside the threshold band ({band.sum()} in the band)"
+    assert ref.accept_band.sum() <= max(1, int(max_band_frac * B * k)), "accept band is not rare"
+    # every sequence, band or not, has a well-formed answer
+    assert ((n_gpu >= 0) & (n_gpu <= k)).all()
+    for b in range(B):
+        n = int(n_gpu[b])
+        assert (tok_gpu[b, :n] == x[b, :n]).all()
+        assert 0 <= tok_gpu[b, n] < V
+        assert (tok_gpu[b, n + 1:] == -1).all()
+
+    if check_loss and out.loss is not None:
+        loss = out.loss.cpu()[sl].numpy().astype(np.float64)
+        err = np.abs(loss - ref.loss)
+        bound = tol * np.abs(ref.loss) + LOSS_FLOOR
+        ok = (err <= bound) | (loss == ref.loss)          # the second term covers +inf == +inf
+        assert ok.all(), f"loss: worst ratio {np.nanmax(err / bound):.3g}"
+    if check_grad and out.grad_draft is not None and ref.grad is not None:
+        g = out.grad_draft.cpu()[sl].float().numpy().astype(np.float64)
+        d = g - ref.grad
+        T64, D64 = logits_f64(inp, seqs)
+        pmax, p2 = prob_max_and_l2(T64[:, :k], inp.tau)
+        qmax, q2 = prob_max_and_l2(D64, inp.tau)
+        gmax = np.abs(ref.grad).max(axis=2)
+        bound = tol * gmax + GRAD_FLOOR * np.maximum(pmax, qmax) / inp.tau
+        worst = np.abs(d).max(axis=2)
+        assert (worst <= bound).all(), f"grad max-norm: worst ratio {np.max(worst / bound):.3g}"
+        l2 = np.sqrt((d * d).sum(axis=2))
+        ref_l2 = np.sqrt((ref.grad * ref.grad).sum(axis=2))
+        assert (l2 <= tol * ref_l2 + GRAD_FLOOR * (p2 + q2) / inp.tau).all(), "grad L2 norm"
+    if out.acc_prob is not None:
+        acc = out.acc_prob.cpu()[sl].numpy().astype(np.float64)
+        assert np.abs(acc - ref.acc_prob).max() < 2e-5
+    if out.status is not None:
+        assert (out.status.cpu()[sl].numpy() == ref.status.astype(np.int32)).all()
+    return int(band.sum()), int(mismatch.sum())
+
+
+def run_and_check(binding, cfg, seed=synth.BASE_SEED, ex=False, **kw):
+    inp = synth.make_inputs(cfg, seed)
+    T, D, x, u = to_device(inp)
+    out = (binding.sd_verify_feedback_ex if ex else binding.sd_verify_feedback)(T, D, x, u, inp.tau)
+    torch.cuda.synchronize()
+    ref = oracle_of(inp)
+    check(inp, out, ref, **kw)
+    return inp, out, ref
+
+
+# ------------------------------------------------------------------ the five workloads
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg3", "cfg4"])
+@pytest.mark.parametrize("seed_off", [0, 1])
+def test_config_full_parity(binding, name, seed_off):
+    cfg = synth.CONFIGS[name]
+    if seed_off and name in ("cfg3", "cfg4"):
+        cfg = cfg.with_batch(8)   # second seed on a slice of the batch keeps the CPU time down
+    inp, out, ref = run_and_check(binding, cfg, synth.BASE_SEED + seed_off, ex=True)
+    info = binding.sd_launch_info()
+    assert info["path"] == 1, "the five workloads must take the cluster fast path"
+
+
+def test_config5_full_size_sampled_parity(binding):
+    """B=256, k=6, V=128256 fp32 in the launch configuration the benchmark times; the oracle
+    checks a sample of sequences element by element, properties cover the rest."""
+    cfg = synth.CONFIGS["cfg5"]
+    inp = synth.make_inputs(cfg)
+    T, D, x, u = to_device(inp)
+    out = binding.sd_verify_feedback(T, D, x, u, inp.tau)
+    torch.cuda.synchronize()
+    assert binding.sd_launch_info()["path"] == 1
+    seqs = [0, 1, 17, 63, 64, 100, 128, 191, 200, 254, 255]
+    ref = oracle_of(inp, seqs)
+    check(inp, out, ref, seqs=seqs, max_band_frac=0.1)
+    # properties that hold for every sequence at any size
+    n = out.accept_len.cpu().numpy()
+    tok = out.tokens.cpu().numpy()
+    assert ((n >= 0) & (n <= cfg.k)).all()
+    for b in range(cfg.B):
+        assert (tok[b, :n[b]] == inp.draft_tokens[b, :n[b]]).all()
+        assert 0 <= tok[b, n[b]] < cfg.V and (tok[b, n[b] + 1:] == -1).all()
+    loss = out.loss.cpu().numpy()
+    assert np.isfinite(loss).all() and (loss > 0).all()
+    gsum = out.grad_draft.sum(dim=2).abs().max().item()
+    assert gsum < 1e-4                     # rows of (q-p)/tau sum to zero
+    # expected mean accepted length from the closed form of the proof of Lemma 1, with the
+    # per-position acceptance probabilities of the sampled sequences
+    acc = ref.acc_prob.mean()
+    expect = (1 - acc ** (cfg.k + 1)) / (1 - acc)
+    assert abs((n + 1).mean() - expect) < 0.35
+
+
+# ------------------------------------------------------------------ shapes and alignments
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("B,k,V", [(1, 1, 5), (2, 3, 17), (3, 2, 1023), (2, 2, 4100), (1, 1, 8), (2, 2, 512),
+                                   (3, 1, 520), (2, 4, 1024), (1, 2, 40000), (5, 3, 2056)])
+def test_shapes(binding, dtype, B, k, V):
+    cfg = synth.custom_config(B=B, k=k, V=V, dtype=dtype, tau=0.85, index=50)
+    run_and_check(binding, cfg, ex=True, max_band_frac=1.0)
+
+
+def test_largest_k(binding):
+    cfg = synth.custom_config(B=2, k=64, V=1000, dtype="f32", d_sigma=0.1, index=51)
+    run_and_check(binding, cfg, ex=True, max_band_frac=1.0)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("cluster", [1, 2, 4, 8, 16])
+def test_every_cluster_size_gives_the_same_answer(binding, dtype, cluster, monkeypatch):
+    cfg = synth.custom_config(B=3, k=3, V=24000 if dtype == "f32" else 48000, dtype=dtype, tau=1.2, index=52)
+    monkeypatch.setenv("SD_VERIFY_CLUSTER", str(cluster))
+    inp, out, ref = run_and_check(binding, cfg, ex=True, max_band_frac=1.0)
+    info = binding.sd_launch_info()
+    assert info["path"] == 1 and info["cluster_size"] == cluster
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_generic_path_matches_fast_path(binding, dtype, monkeypatch):
+    cfg = synth.custom_config(B=3, k=3, V=20000, dtype=dtype, tau=0.9, index=53)
+    inp = synth.make_inputs(cfg)
+    T, D, x, u = to_device(inp)
+    fast = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
+    torch.cuda.synchronize()
+    assert binding.sd_launch_info()["path"] == 1
+    monkeypatch.setenv("SD_VERIFY_FORCE_GENERIC", "1")
+    slow = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
+    torch.cuda.synchronize()
+    assert binding.sd_launch_info()["path"] == 0
+    ref = oracle_of(inp)
+    check(inp, slow, ref, max_band_frac=1.0)
+    assert (fast.accept_len == slow.accept_len).all() and (fast.tokens == slow.tokens).all()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_misaligned_base_pointers(binding, dtype):
+    """Tensors that start one element past a 16-byte boundary take the generic path."""
+    cfg = synth.custom_config(B=2, k=2, V=4096, dtype=dtype, index=54)
+    inp = synth.make_inputs(cfg)
+    T, D, x, u = to_device(inp)
+
+    def shifted(t):
+        buf = torch.empty(t.numel() + 1, dtype=t.dtype, device=t.device)
+        v = buf[1:].view(t.shape)
+        v.copy_(t)
+        return v
+
+    Ts, Ds = shifted(T), shifted(D)
+    out = binding.sd_verify_feedback_ex(Ts, Ds, x, u, inp.tau)
+    torch.cuda.synchronize()
+    assert binding.sd_launch_info()["path"] == 0
+    check(inp, out, oracle_of(inp), max_band_frac=1.0)
+
+
+# ------------------------------------------------------------------ values
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_identical_models(binding, dtype):
+    """p = q: everything accepted, zero loss, zero gradient (check 3 of the contract)."""
+    cfg = synth.custom_config(B=4, k=5, V=32000, dtype=dtype, tau=0.7, index=55)
+    inp = synth.make_inputs(cfg)
+    inp.draft_logits[:] = inp.target_logits[:, :cfg.k]
+    T, D, x, u = to_device(inp)
+    out = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
+    torch.cuda.synchronize()
+    assert (out.accept_len.cpu() == cfg.k).all()
+    assert out.loss.abs().max().item() == 0.0
+    # q - p is evaluated as fma(eD, kD, -(eT*kT)): with identical rows that leaves the rounding
+    # residual of one product, far below one ulp of p
+    T64, _ = logits_f64(inp)
+    pmax, _ = prob_max_and_l2(T64[:, :cfg.k], inp.tau)
+    gabs = out.grad_draft.float().abs().amax(dim=2).cpu().numpy()
+    assert (gabs <= 2.0 ** -24 * pmax / inp.tau).all()
+    assert (out.acc_prob.cpu() - 1).abs().max().item() < 1e-6
+    check(inp, out, oracle_of(inp), max_band_frac=1.0)
+
+
+def test_shifted_and_huge_logits(binding):
+    """Max-subtraction: +80 / -80 offsets and a spread that overflows a naive exp."""
+    cfg = synth.custom_config(B=3, k=2, V=3000, dtype="f32", t_sigma=20.0, d_sigma=2.0, index=56)
+    inp = synth.make_inputs(cfg)
+    inp.target_logits[0] += 80.0
+    inp.draft_logits[0] -= 80.0
+    inp.target_logits[1] *= 4.0
+    T, D, x, u = to_device(inp)
+    out = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
+    torch.cuda.synchronize()
+    check(inp, out, oracle_of(inp), max_band_frac=1.0)
+
+
+def test_all_equal_logits(binding):
+    cfg = synth.custom_config(B=2, k=2, V=777, dtype="f32", index=57)
+    inp = synth.make_inputs(cfg)
+    inp.target_logits[:] = 1.5
+    inp.draft_logits[:] = -0.25
+    T, D, x, u = to_device(inp)
+    out = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
+    torch.cuda.synchronize()
+    ref = oracle_of(inp)
+    assert (out.accept_len.cpu().numpy() == cfg.k).all()
+    assert out.loss.abs().max().item() < 1e-6
+    # uniform distribution: token index = floor(u*V) up to the edge band
+    check(inp, out, ref, max_band_frac=1.0)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_masked_vocabulary_entries(binding, dtype):
+    """-inf logits (masked tokens) in either model."""
+    cfg = synth.custom_config(B=3, k=3, V=8192, dtype=dtype, index=58)
+    inp = synth.make_inputs(cfg)
+    ninf = np.float32(-np.inf) if dtype == "f32" else np.uint16(0xFF80)
+    inp.target_logits[:, :, 100:4000] = ninf          # whole vectors and chunks masked
+    inp.draft_logits[:, :, 100:3000] = ninf
+    inp.draft_tokens[:] = np.clip(inp.draft_tokens, 4000, None)
+    inp.draft_tokens[0, 0] = 3500                      # p(x) = 0, q(x) > 0: rejected
+    T, D, x, u = to_device(inp)
+    out = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
+    torch.cuda.synchronize()
+    ref = oracle_of(inp)
+    assert out.accept_len.cpu()[0].item() == 0
+    assert np.isfinite(ref.loss).all()
+    check(inp, out, ref, max_band_frac=1.0)
+
+
+def test_infinite_divergence(binding):
+    cfg = synth.custom_config(B=1, k=1, V=1024, dtype="f32", index=59)
+    inp = synth.make_inputs(cfg)
+    inp.draft_logits[0, 0, 5] = -np.inf               # q = 0 where p > 0
+    inp.draft_tokens[0, 0] = 7
+    T, D, x, u = to_device(inp)
+    out = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
+    torch.cuda.synchronize()
+    assert torch.isinf(out.loss[0, 0]).item() and out.loss[0, 0].item() > 0
+    assert np.isinf(oracle_of(inp).loss[0, 0])
+
+
+def test_bad_token_sets_status(binding):
+    cfg = synth.custom_config(B=3, k=3, V=2048, dtype="f32", d_sigma=0.01, index=60)
+    inp = synth.make_inputs(cfg)
+    inp.draft_tokens[1, 1] = cfg.V
+    inp.draft_tokens[2, 0] = -3
+    T, D, x, u = to_device(inp)
+    out = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
+    torch.cuda.synchronize()
+    st = out.status.cpu().numpy()
+    ref = oracle_of(inp)
+    assert st[0] == 0 and st[1] & binding.SD_STATUS_BAD_TOKEN and st[2] & binding.SD_STATUS_BAD_TOKEN
+    assert out.accept_len.cpu().numpy()[2] == 0 and out.accept_len.cpu().numpy()[1] <= 1
+    check(inp, out, ref, max_band_frac=1.0)
+
+
+# ------------------------------------------------------------------ modes and plumbing
+def test_verify_only_mode(binding):
+    cfg = synth.custom_config(B=4, k=3, V=16000, dtype="bf16", index=61)
+    inp = synth.make_inputs(cfg)
+    T, D, x, u = to_device(inp)
+    full = binding.sd_verify_feedback(T, D, x, u, inp.tau)
+    only = binding.sd_verify_feedback(T, D, x, u, inp.tau, want_loss=False, want_grad=False)
+    torch.cuda.synchronize()
+    assert only.loss is None and only.grad_draft is None
+    assert (full.accept_len == only.accept_len).all() and (full.tokens == only.tokens).all()
+
+
+def test_results_are_deterministic(binding):
+    cfg = synth.CONFIGS["cfg2"]
+    inp = synth.make_inputs(cfg)
+    T, D, x, u = to_device(inp)
+    a = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
+    b = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
+    torch.cuda.synchronize()
+    for name in ["accept_len", "tokens", "loss", "acc_prob", "status"]:
+        assert torch.equal(getattr(a, name), getattr(b, name))
+    assert torch.equal(a.grad_draft.view(torch.int16), b.grad_draft.view(torch.int16))
+
+
+def test_dirty_workspace_and_guard_words(binding):
+    """Caller scratch full of garbage is fine, and nothing is written outside the outputs."""
+    cfg = synth.custom_config(B=5, k=3, V=12345 * 8, dtype="bf16", index=62)
+    inp = synth.make_inputs(cfg)
+    T, D, x, u = to_device(inp)
+    B, k, V = cfg.B, cfg.k, cfg.V
+    ws = torch.full((binding.sd_workspace_bytes(B, k, V, binding.SD_DTYPE_BF16),), 0xFF, dtype=torch.uint8, device="cuda")
+    pad = 64
+
+    def guarded(shape, dtype, fill):
+        n = int(np.prod(shape))
+        buf = torch.full((n + 2 * pad,), fill, dtype=dtype, device="cuda")
+        return buf, buf[pad:pad + n].view(shape)
+
+    bufs = {}
+    bufs["n"], n_v = guarded((B,), torch.int32, -77)
+    bufs["tok"], tok_v = guarded((B, k + 1), torch.int32, -77)
+    bufs["loss"], loss_v = guarded((B, k), torch.float32, -77.0)
+    bufs["grad"], grad_v = guarded((B, k, V), torch.bfloat16, -77.0)
+    bufs["acc"], acc_v = guarded((B, k), torch.float32, -77.0)
+    bufs["st"], st_v = guarded((B,), torch.int32, -77)
+    out = binding.StepOutputs(accept_len=n_v, tokens=tok_v, loss=loss_v, grad_draft=grad_v, acc_prob=acc_v, status=st_v)
+    binding.sd_verify_feedback_ex(T, D, x, u, inp.tau, workspace=ws, out=out)
+    torch.cuda.synchronize()
+    for name, buf in bufs.items():
+        assert (buf[:pad].float() == -77).all() and (buf[-pad:].float() == -77).all(), f"{name} guard words touched"
+    check(inp, out, oracle_of(inp), max_band_frac=1.0)
+
+
+def test_non_default_stream_and_changing_shapes(binding):
+    s = torch.cuda.Stream()
+    for (B, k, V, dtype) in [(2, 2, 8000, "f32"), (6, 4, 64000, "bf16"), (1, 1, 8, "f32"), (3, 3, 33000, "f32")]:
+        cfg = synth.custom_config(B=B, k=k, V=V, dtype=dtype, index=63)
+        inp = synth.make_inputs(cfg)
+        T, D, x, u = to_device(inp)
+        torch.cuda.synchronize()
+        with torch.cuda.stream(s):
+            out = binding.sd_verify_feedback(T, D, x, u, inp.tau)
+        s.synchronize()
+        check(inp, out, oracle_of(inp), max_band_frac=1.0)
+
+
+@pytest.mark.parametrize("name", ["cfg2", "cfg3"])
+def test_host_entry_point_matches_device_entry_point(binding, name):
+    cfg = synth.CONFIGS[name]
+    inp = synth.make_inputs(cfg)
+    T, D, x, u = to_device(inp)
+    dev = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
+    torch.cuda.synchronize()
+    hT = torch.from_numpy(inp.target_logits)
+    hD = torch.from_numpy(inp.draft_logits)
+    if cfg.dtype == "bf16":
+        hT, hD = hT.view(torch.bfloat16), hD.view(torch.bfloat16)
+    host = binding.sd_verify_feedback_host(hT.pin_memory(), hD.pin_memory(), torch.from_numpy(inp.draft_tokens),
+                                           torch.from_numpy(inp.uniforms), inp.tau, want_acc_prob=True,
+                                           want_status=True)
+    assert torch.equal(host.accept_len, dev.accept_len.cpu())
+    assert torch.equal(host.tokens, dev.tokens.cpu())
+    # the host entry point works in slices of sequences, which may pick another cluster size:
+    # sums are then taken in another order, so floating-point outputs agree to rounding only
+    torch.testing.assert_close(host.loss, dev.loss.cpu(), rtol=1e-5, atol=4e-7)
+    torch.testing.assert_close(host.grad_draft.float(), dev.grad_draft.cpu().float(), rtol=1e-2, atol=1e-7)
+    torch.testing.assert_close(host.acc_prob, dev.acc_prob.cpu(), rtol=0, atol=1e-6)
+    assert torch.equal(host.status, dev.status.cpu())
+
+
+def test_host_entry_point_slices_large_batches(binding):
+    """More than one slice of sequences (the slices overlap copies and kernels)."""
+    cfg = synth.CONFIGS["cfg5"].with_batch(40)   # ~0.39 GB of logits and gradient: five slices
+    inp = synth.make_inputs(cfg)
+    host = binding.sd_verify_feedback_host(torch.from_numpy(inp.target_logits), torch.from_numpy(inp.draft_logits),
+                                           torch.from_numpy(inp.draft_tokens), torch.from_numpy(inp.uniforms), inp.tau)
+    seqs = [0, 7, 8, 23, 39]
+    ref = oracle_of(inp, seqs)
+    check(inp, host, ref, seqs=seqs, max_band_frac=1.0)
