@@ -206,58 +206,82 @@ struct LaneStats {
     }
 };
 
-// Merge of two partial statistics in fp64 (symmetric: merge(a,b) and merge(b,a) give the same bits).
-__device__ __forceinline__ PartialStats merge_two(const PartialStats& a, const PartialStats& b, float c) {
-    PartialStats r;
-    r.mT = fmaxf(a.mT, b.mT);
-    r.mD = fmaxf(a.mD, b.mD);
-    const double RT = (double)__fmul_rn(r.mT, c), RD = (double)__fmul_rn(r.mD, c);
-    double sTa = 0.0, sTb = 0.0, wa = 0.0, wb = 0.0, sDa = 0.0, sDb = 0.0;
-    if (a.sT > 0.0) {
-        const double f = (a.mT == r.mT) ? 1.0 : exp2((double)__fmul_rn(a.mT, c) - RT);
-        sTa = a.sT * f;
-        wa = (a.w - a.sT * (((double)r.mT - (double)a.mT) - ((double)r.mD - (double)a.mD))) * f;
-    }
-    if (b.sT > 0.0) {
-        const double f = (b.mT == r.mT) ? 1.0 : exp2((double)__fmul_rn(b.mT, c) - RT);
-        sTb = b.sT * f;
-        wb = (b.w - b.sT * (((double)r.mT - (double)b.mT) - ((double)r.mD - (double)b.mD))) * f;
-    }
-    if (a.sD > 0.0) sDa = a.sD * ((a.mD == r.mD) ? 1.0 : exp2((double)__fmul_rn(a.mD, c) - RD));
-    if (b.sD > 0.0) sDb = b.sD * ((b.mD == r.mD) ? 1.0 : exp2((double)__fmul_rn(b.mD, c) - RD));
-    r.sT = sTa + sTb;
-    r.w = wa + wb;
-    r.sD = sDa + sDb;
-    return r;
-}
-
 __device__ __forceinline__ double shfl_xor_f64(double v, int off) {
     return __shfl_xor_sync(0xffffffffu, v, off);
 }
-
-// Butterfly reduction of the lane statistics in fp64; every lane ends with the warp's statistics.
-__device__ __forceinline__ PartialStats warp_reduce_stats(const LaneStats& s, float c) {
-    PartialStats a;
-    a.mT = s.mT; a.mD = s.mD; a.sT = (double)s.sT; a.sD = (double)s.sD; a.w = (double)s.w;
+__device__ __forceinline__ float warp_max_f32(float v) {
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        PartialStats b;
-        b.mT = __shfl_xor_sync(0xffffffffu, a.mT, off);
-        b.mD = __shfl_xor_sync(0xffffffffu, a.mD, off);
-        b.sT = shfl_xor_f64(a.sT, off);
-        b.sD = shfl_xor_f64(a.sD, off);
-        b.w = shfl_xor_f64(a.w, off);
-        // order the operands by lane so both partners evaluate the same expression
-        const bool low = (threadIdx.x & off) == 0;
-        a = low ? merge_two(a, b, c) : merge_two(b, a, c);
-    }
-    return a;
+    for (int off = 16; off > 0; off >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, off));
+    return v;
 }
 
-// fp64 merge of `n` partial statistics in index order.
-__device__ inline PartialStats merge_partials(const PartialStats* p, int n, float c) {
-    PartialStats r = p[0];
-    for (int j = 1; j < n; ++j) r = merge_two(r, p[j], c);
+// Shared scratch of the block-level reduction of the statistics.
+struct StatScratch {
+    float wmaxT[kWarps], wmaxD[kWarps];
+    double wsT[kWarps], wsD[kWarps], ww[kWarps];
+};
+
+// Statistics of everything the block has seen, in every thread.  All threads must call.
+// Lanes are first brought to the block's maxima (one fp32 rescale each), then summed in fp64 in
+// a fixed order, so the result does not depend on scheduling and costs no serial fp64 exp.
+__device__ inline PartialStats block_reduce_stats(const LaneStats& ls, float c, StatScratch& sc) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const float wmT = warp_max_f32(ls.mT), wmD = warp_max_f32(ls.mD);
+    if (lane == 0) { sc.wmaxT[warp] = wmT; sc.wmaxD[warp] = wmD; }
+    __syncthreads();
+    float bmT = sc.wmaxT[0], bmD = sc.wmaxD[0];
+#pragma unroll
+    for (int w = 1; w < kWarps; ++w) { bmT = fmaxf(bmT, sc.wmaxT[w]); bmD = fmaxf(bmD, sc.wmaxD[w]); }
+    float sT = 0.f, wv = 0.f, sD = 0.f;
+    if (ls.sT > 0.f) {
+        const float f = (ls.mT == bmT) ? 1.f : ex2f(neg_ref(bmT, c) - ls.negRT);
+        sT = ls.sT * f;
+        wv = (ls.w - ls.sT * ((bmT - ls.mT) - (bmD - ls.mD))) * f;
+    }
+    if (ls.sD > 0.f) sD = ls.sD * ((ls.mD == bmD) ? 1.f : ex2f(neg_ref(bmD, c) - ls.negRD));
+    double dT = (double)sT, dW = (double)wv, dD = (double)sD;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        dT += shfl_xor_f64(dT, off);
+        dW += shfl_xor_f64(dW, off);
+        dD += shfl_xor_f64(dD, off);
+    }
+    if (lane == 0) { sc.wsT[warp] = dT; sc.ww[warp] = dW; sc.wsD[warp] = dD; }
+    __syncthreads();
+    PartialStats r;
+    r.mT = bmT; r.mD = bmD;
+    r.sT = r.sD = r.w = 0.0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) { r.sT += sc.wsT[w]; r.w += sc.ww[w]; r.sD += sc.wsD[w]; }
+    return r;
+}
+
+// Merge of the block statistics of a cluster by one full warp: lane j takes block j, one fp64
+// exp2 per lane in parallel, then a butterfly sum.  Every lane returns the row statistics.
+__device__ inline PartialStats warp_merge_partials(const PartialStats* p, int n, float c) {
+    const int lane = threadIdx.x & 31;
+    PartialStats m;
+    m.mT = m.mD = -3.402823466e+38f;
+    m.sT = m.sD = m.w = 0.0;
+    if (lane < n) m = p[lane];
+    PartialStats r;
+    r.mT = warp_max_f32(m.mT);
+    r.mD = warp_max_f32(m.mD);
+    double sT = 0.0, wv = 0.0, sD = 0.0;
+    if (m.sT > 0.0) {
+        const double f = (m.mT == r.mT) ? 1.0 : exp2((double)__fmul_rn(m.mT, c) - (double)__fmul_rn(r.mT, c));
+        sT = m.sT * f;
+        wv = (m.w - m.sT * (((double)r.mT - (double)m.mT) - ((double)r.mD - (double)m.mD))) * f;
+    }
+    if (m.sD > 0.0)
+        sD = m.sD * ((m.mD == r.mD) ? 1.0 : exp2((double)__fmul_rn(m.mD, c) - (double)__fmul_rn(r.mD, c)));
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        sT += shfl_xor_f64(sT, off);
+        wv += shfl_xor_f64(wv, off);
+        sD += shfl_xor_f64(sD, off);
+    }
+    r.sT = sT; r.w = wv; r.sD = sD;
     return r;
 }
 
@@ -305,20 +329,43 @@ __device__ inline double block_exclusive_scan(double v, double* scratch, double*
 }
 
 // ------------------------------------------------------------------------------------------
-// End of a (sequence, row) unit: what one thread does once the row statistics are known.
-// Writes the row constants, the loss and the accept flag; returns the constants.
-template <int DT>
-__device__ inline RowConst finish_row(const Params& P, int b, int i, const PartialStats& st,
-                                      bool write_out) {
-    const bool bonus = (i == P.k);
-    const int unit = b * (P.k + 1) + i;
+// Constants of a finished row for the second sweep and the inverse-CDF search.
+__device__ __forceinline__ RowConst row_constants(const Params& P, bool bonus, const PartialStats& st) {
     RowConst rc;
     rc.negRT = neg_ref(st.mT, P.c);
     rc.negRD = bonus ? 0.f : neg_ref(st.mD, P.c);
     rc.kT = (float)((bonus ? 1.0 : P.inv_tau) / st.sT);
     rc.kD = bonus ? 0.f : (float)(P.inv_tau / st.sD);
-    if (!write_out) return rc;
+    return rc;
+}
 
+// What the accept test of one pair row needs from global memory; loaded early by the thread that
+// will finish the row so that the latency is off the critical path.
+struct AcceptOperands {
+    int32_t x;
+    float u, tx, dx;
+    bool valid;
+};
+template <int DT>
+__device__ __forceinline__ AcceptOperands load_accept_operands(const Params& P, int b, int i) {
+    AcceptOperands a;
+    a.x = P.x[b * P.k + i];
+    a.u = P.u[b * (P.k + 1) + i];
+    a.valid = (a.x >= 0 && a.x < P.V);
+    a.tx = a.dx = 0.f;
+    if (a.valid) {
+        a.tx = Elem<DT>::load(P.T, (size_t)(b * (P.k + 1) + i) * P.V + a.x);
+        a.dx = Elem<DT>::load(P.D, (size_t)(b * P.k + i) * P.V + a.x);
+    }
+    return a;
+}
+
+// End of a (sequence, row) unit, by one thread: row constants to the workspace, the KL loss and
+// the rejection test of the row's draft token.
+__device__ inline void finish_row(const Params& P, int b, int i, const PartialStats& st, const RowConst& rc,
+                                  const AcceptOperands& op) {
+    const bool bonus = (i == P.k);
+    const int unit = b * (P.k + 1) + i;
     uint32_t flags = 0;
     const bool okT = (st.sT > 0.0) && isfinite(st.sT);
     const bool okD = bonus || ((st.sD > 0.0) && isfinite(st.sD));
@@ -337,13 +384,11 @@ __device__ inline RowConst finish_row(const Params& P, int b, int i, const Parti
             P.loss[b * P.k + i] = (float)kl;
         }
         // rejection test for draft token x[b,i] with ratio p(x)/q(x) in fp64
-        const int32_t xi = P.x[b * P.k + i];
         bool acc = false;
-        if (xi < 0 || xi >= P.V) {
+        if (!op.valid) {
             flags |= SD_STATUS_BAD_TOKEN;
         } else if (okT && okD) {
-            const double tx = (double)Elem<DT>::load(P.T, (size_t)unit * P.V + xi);
-            const double dx = (double)Elem<DT>::load(P.D, (size_t)(b * P.k + i) * P.V + xi);
+            const double tx = (double)op.tx, dx = (double)op.dx;
             double rho;
             if (dx == -INFINITY) {
                 rho = (tx == -INFINITY) ? 0.0 : INFINITY;
@@ -353,12 +398,11 @@ __device__ inline RowConst finish_row(const Params& P, int b, int i, const Parti
                 rho = exp2(l2p - l2q);
             }
             const double thr = rho < 1.0 ? rho : 1.0;
-            acc = (double)P.u[b * (P.k + 1) + i] < thr;
+            acc = (double)op.u < thr;
         }
         P.accept[b * P.k + i] = acc ? 1 : 0;
     }
     if (flags) atomicOr(&P.wstatus[b], flags);
-    return rc;
 }
 
 // ------------------------------------------------------------------------------------------

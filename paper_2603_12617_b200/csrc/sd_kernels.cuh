@@ -77,7 +77,7 @@ __device__ __forceinline__ void block_chunks(int NC, int C, int rank, int& c0, i
 
 struct ClusterShared {
     uint64_t bar[kMaxPieces];
-    PartialStats warp_part[kWarps];
+    StatScratch stat;
     PartialStats xchg[kMaxCluster];   // written by every block of the cluster (distributed shared memory)
     RowConst rc;
     ResolveScratch rs;
@@ -129,6 +129,10 @@ __global__ void __launch_bounds__(kThreads) sd_cluster_kernel(const Params P, co
                           &sh.bar[p]);
         }
     }
+    // the thread that will report the row fetches what the accept test needs while the copies fly
+    AcceptOperands aop;
+    aop.valid = false;
+    if (rank == 0 && tid == 0 && !bonus) aop = load_accept_operands<DT>(P, b, i);
     __syncthreads();          // barriers are initialised before anyone polls them
     cluster.barrier_arrive(); // matched by the wait before the first remote store: every block of
                               // the cluster must be running before its shared memory is written
@@ -156,27 +160,21 @@ __global__ void __launch_bounds__(kThreads) sd_cluster_kernel(const Params P, co
             }
         }
     }
-    {
-        const PartialStats wp = warp_reduce_stats(ls, P.c);
-        if (lane == 0) sh.warp_part[warp] = wp;
-    }
     if (timed_out && lane == 0) atomicOr(&P.wstatus[b], kStatusTimeout);
-    __syncthreads();
+    const PartialStats mine = block_reduce_stats(ls, P.c, sh.stat);   // same in every thread
 
     // -- block statistics to every block of the cluster
     cluster.barrier_wait();
-    if (warp == 0) {
-        PartialStats mine = merge_partials(sh.warp_part, kWarps, P.c);   // same in every lane
-        if (lane < C) {
-            PartialStats* remote = cluster.map_shared_rank(&sh.xchg[rank], lane);
-            *remote = mine;
-        }
-    }
+    if (warp == 0 && lane < C) *cluster.map_shared_rank(&sh.xchg[rank], lane) = mine;
     cluster.sync();   // all partials of the row are now in this block's shared memory
 
-    if (tid == 0) {
-        const PartialStats row = merge_partials(sh.xchg, C, P.c);
-        sh.rc = finish_row<DT>(P, b, i, row, rank == 0);
+    if (warp == 0) {
+        const PartialStats row = warp_merge_partials(sh.xchg, C, P.c);
+        const RowConst rcw = row_constants(P, bonus, row);
+        if (lane == 0) sh.rc = rcw;
+        __syncwarp();
+        // one thread of the cluster reports the row: loss, accept flag, constants for the resolver
+        if (rank == 0 && lane == 0) finish_row(P, b, i, row, rcw, aop);
     }
     __syncthreads();
     const RowConst rc = sh.rc;
@@ -222,7 +220,7 @@ __global__ void __launch_bounds__(kThreads) sd_cluster_kernel(const Params P, co
 
 // ---- generic path --------------------------------------------------------------------------
 struct GenericShared {
-    PartialStats warp_part[kWarps];
+    StatScratch stat;
     RowConst rc;
     ResolveScratch rs;
 };
@@ -260,13 +258,15 @@ __global__ void __launch_bounds__(kThreads) sd_generic_kernel(const Params P) {
         }
     }
     {
-        const PartialStats wp = warp_reduce_stats(ls, P.c);
-        if (lane == 0) sh.warp_part[warp] = wp;
-    }
-    __syncthreads();
-    if (tid == 0) {
-        const PartialStats row = merge_partials(sh.warp_part, kWarps, P.c);
-        sh.rc = finish_row<DT>(P, b, i, row, true);
+        const PartialStats row = block_reduce_stats(ls, P.c, sh.stat);
+        if (tid == 0) {
+            const RowConst rcw = row_constants(P, bonus, row);
+            sh.rc = rcw;
+            AcceptOperands aop;
+            aop.valid = false;
+            if (!bonus) aop = load_accept_operands<DT>(P, b, i);
+            finish_row(P, b, i, row, rcw, aop);
+        }
     }
     __syncthreads();
     const RowConst rc = sh.rc;
