@@ -15,7 +15,10 @@ using namespace sdv;
 
 constexpr int kMaxDevices = 64;
 constexpr size_t kAlign = 256;
-constexpr int kMaxDynSmem = 227 * 1024 - 2048;   // per-block limit minus the static part
+constexpr int kRingStages = 12;                   // 12 x 16 KiB + control block < 227 KiB per block
+constexpr int kStreamSmem = kRingStages * kStageBytes + (int)sizeof(StreamShared);
+static_assert(kRingStages <= kMaxStages, "ring larger than the control block allows");
+static_assert(kStreamSmem <= 227 * 1024, "ring does not fit the shared memory of a block");
 
 thread_local char tl_cuda_error[256] = "";
 thread_local int tl_info[6] = {0, 0, 0, 0, 0, 0};
@@ -32,11 +35,11 @@ int cuda_fail(cudaError_t e, const char* where) {
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 int elem_bytes(int dtype) { return dtype == SD_DTYPE_F32 ? 4 : 2; }
-int chunk_elems(int dtype) { return kChunkVecs * (dtype == SD_DTYPE_F32 ? 4 : 8); }
+int vec_elems(int dtype) { return 16 / elem_bytes(dtype); }
 
 struct WorkspaceLayout {
-    size_t ticket, wstatus, accept, rowc, chunk_sums, total;
-    int NC;
+    size_t ticket, wstatus, sticky, accept, rowc, region_sums, total;
+    int NRmax;   // room for region sums per row: enough for either path at any cluster size
 };
 
 bool shape_ok(int B, int k, int V) {
@@ -47,13 +50,16 @@ bool shape_ok(int B, int k, int V) {
 
 WorkspaceLayout workspace_layout(int B, int k, int V, int dtype) {
     WorkspaceLayout L;
-    L.NC = (V + chunk_elems(dtype) - 1) / chunk_elems(dtype);
+    (void)dtype;
+    const int generic_regions = (V + kGenericRegionElems - 1) / kGenericRegionElems;
+    L.NRmax = generic_regions > kMaxCluster * kConsumerWarps ? generic_regions : kMaxCluster * kConsumerWarps;
     size_t off = 0;
     L.ticket = off;      off = align_up(off + (size_t)B * 4, kAlign);
     L.wstatus = off;     off = align_up(off + (size_t)B * 4, kAlign);
+    L.sticky = off;      off = align_up(off + 4, kAlign);
     L.accept = off;      off = align_up(off + (size_t)B * k, kAlign);
     L.rowc = off;        off = align_up(off + (size_t)B * (k + 1) * sizeof(RowConst), kAlign);
-    L.chunk_sums = off;  off = align_up(off + (size_t)B * (k + 1) * L.NC * 4, kAlign);
+    L.region_sums = off; off = align_up(off + (size_t)B * (k + 1) * L.NRmax * 4, kAlign);
     L.total = off;
     return L;
 }
@@ -74,8 +80,9 @@ struct DeviceState {
     size_t ws_bytes = 0;
     bool ws_clean = false;   // tickets and status words are zero
     bool attr_set[2] = {false, false};   // shared-memory / cluster attributes of the fast kernel
+    int max_clusters[2][5] = {{-1, -1, -1, -1, -1}, {-1, -1, -1, -1, -1}};   // resident clusters of 1,2,4,8,16 blocks
     // last launch-shape decision of the fast path
-    int dec_dtype = -1, dec_NC = 0, dec_forced = 0, dec_C = 0, dec_chunks = 0;
+    int dec_dtype = -1, dec_V = 0, dec_forced = 0, dec_C = 0, dec_G = 0, dec_lag = 0, dec_per = 0;
     long long dec_units = 0;
     // host-memory entry point
     StageSet stage[2];
@@ -112,22 +119,22 @@ int current_device(int* dev, DeviceState** st) {
     return SD_OK;
 }
 
+// Launches the fast path with G clusters of C blocks, or (query_only) asks how many such
+// clusters the device can hold at once.
 template <int DT>
-int launch_cluster(DeviceState& d, const Params& P, int C, int slice_chunks, cudaStream_t stream,
-                   bool query_only, int* max_clusters) {
-    auto kern = sd_cluster_kernel<DT>;
-    const int smem = slice_chunks * 2 * kChunkBytes;
+int launch_stream(DeviceState& d, const Params& P, int C, int G, int lag, cudaStream_t stream, bool query_only,
+                  int* max_clusters) {
+    auto kern = sd_stream_kernel<DT>;
     if (!d.attr_set[DT]) {
-        SD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem));
+        SD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmem));
         SD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
         d.attr_set[DT] = true;
     }
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
-    const long long units = (long long)P.B * (P.k + 1);
-    cfg.gridDim = dim3((unsigned)(units * C), 1, 1);
-    cfg.blockDim = dim3(kThreads, 1, 1);
-    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.gridDim = dim3((unsigned)(G * C), 1, 1);
+    cfg.blockDim = dim3(kStreamThreads, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)kStreamSmem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -146,65 +153,70 @@ int launch_cluster(DeviceState& d, const Params& P, int C, int slice_chunks, cud
         *max_clusters = n;
         return SD_OK;
     }
-    SD_CUDA(cudaLaunchKernelEx(&cfg, kern, P, slice_chunks));
-    tl_info[0] = 1; tl_info[1] = C; tl_info[2] = kThreads; tl_info[3] = smem;
-    tl_info[4] = (int)(units * C); tl_info[5] = 1;
+    SD_CUDA(cudaLaunchKernelEx(&cfg, kern, P, (int)kRingStages, lag));
+    tl_info[0] = 1; tl_info[1] = C; tl_info[2] = kStreamThreads; tl_info[3] = kStreamSmem;
+    tl_info[4] = G * C; tl_info[5] = 1;
     return SD_OK;
 }
 
 template <int DT>
 int launch_generic(const Params& P, cudaStream_t stream) {
     const long long units = (long long)P.B * (P.k + 1);
-    sd_generic_kernel<DT><<<(unsigned)units, kThreads, 0, stream>>>(P);
+    sd_generic_kernel<DT><<<(unsigned)units, kGenericThreads, 0, stream>>>(P);
     SD_CUDA(cudaGetLastError());
-    tl_info[0] = 0; tl_info[1] = 1; tl_info[2] = kThreads; tl_info[3] = 0;
+    tl_info[0] = 0; tl_info[1] = 1; tl_info[2] = kGenericThreads; tl_info[3] = 0;
     tl_info[4] = (int)units; tl_info[5] = 1;
     return SD_OK;
 }
 
-// Cluster size for the fast path, 0 if it cannot run.  Blocks of about 64 KiB leave room for
-// three per SM, so loads of one block overlap the arithmetic of the others.
-int choose_cluster(DeviceState& d, const Params& P, int dtype, int* slice_chunks_out) {
+// Launch shape of the fast path: cluster size C (0 if the fast path cannot run), number of
+// clusters G, vectors per sampling region, and whether sweep 2 may lag one unit behind sweep 1.
+//
+// With C blocks of 16 consumer warps a row of NV vectors is cut into regions of
+// per = 32*ceil(NV/(C*512)) vectors; a block's slice is then m = per/32 stages, which must fit the
+// ring, and two slices must fit for the lag.  Among the cluster sizes that qualify, take the one
+// that keeps most blocks busy (resident clusters, but no more clusters than units), prefer the
+// lag, then the smaller cluster.
+int choose_stream(DeviceState& d, int V, long long units, int dtype, int* G_out, int* per_out, int* lag_out) {
     const char* env = getenv("SD_VERIFY_CLUSTER");
     const int forced = env ? atoi(env) : 0;
-    const long long units = (long long)P.B * (P.k + 1);
-    if (d.dec_dtype == dtype && d.dec_NC == P.NC && d.dec_units == units && d.dec_forced == forced) {
-        *slice_chunks_out = d.dec_chunks;
+    if (d.dec_dtype == dtype && d.dec_V == V && d.dec_units == units && d.dec_forced == forced) {
+        *G_out = d.dec_G;
+        *per_out = d.dec_per;
+        *lag_out = d.dec_lag;
         return d.dec_C;
     }
-    int best = 0, best_chunks = 0;
-    auto usable = [&](int C, int* chunks) -> bool {
-        const int sc = (P.NC + C - 1) / C;
-        if (sc > kMaxChunksPerBlock || sc * 2 * kChunkBytes > kMaxDynSmem) return false;
-        int n = 0;   // can the device hold at least one such cluster?
-        int rc = dtype == SD_DTYPE_F32 ? launch_cluster<SD_DTYPE_F32>(d, P, C, sc, nullptr, true, &n)
-                                       : launch_cluster<SD_DTYPE_BF16>(d, P, C, sc, nullptr, true, &n);
-        if (rc != SD_OK || n < 1) return false;
-        *chunks = sc;
-        return true;
-    };
-    auto remember = [&](int C, int sc) {
-        d.dec_dtype = dtype; d.dec_NC = P.NC; d.dec_units = units; d.dec_forced = forced;
-        d.dec_C = C; d.dec_chunks = sc;
-        *slice_chunks_out = sc;
-        return C;
-    };
-    if (forced > 0) {
-        int sc = 0;
-        if ((forced & (forced - 1)) == 0 && forced <= kMaxCluster && usable(forced, &sc)) return remember(forced, sc);
-        return remember(0, 0);
+    const int NV = V / vec_elems(dtype);
+    int best_C = 0, best_G = 0, best_lag = 0, best_per = 0;
+    long long best_busy = -1;
+    Params dummy;
+    memset(&dummy, 0, sizeof dummy);
+    for (int ci = 0, C = 1; C <= kMaxCluster; ++ci, C *= 2) {
+        if (forced > 0 && C != forced) continue;
+        const int slice = C * kConsumerWarps * 32;
+        const int m = (NV + slice - 1) / slice;
+        if (m > kRingStages) continue;
+        if (d.max_clusters[dtype][ci] < 0) {
+            int n = 0;
+            int rc = dtype == SD_DTYPE_F32 ? launch_stream<SD_DTYPE_F32>(d, dummy, C, 1, 0, nullptr, true, &n)
+                                           : launch_stream<SD_DTYPE_BF16>(d, dummy, C, 1, 0, nullptr, true, &n);
+            d.max_clusters[dtype][ci] = (rc == SD_OK) ? n : 0;
+        }
+        const int resident = d.max_clusters[dtype][ci];
+        if (resident < 1) continue;
+        const int G = (int)(units < resident ? units : resident);
+        const int lag = (2 * m <= kRingStages) ? 1 : 0;
+        const int used = (NV + kConsumerWarps * 32 * m - 1) / (kConsumerWarps * 32 * m);   // blocks with work
+        const long long busy = (long long)G * used;
+        const bool better = busy > best_busy || (busy == best_busy && lag > best_lag);
+        if (better) { best_C = C; best_G = G; best_lag = lag; best_per = 32 * m; best_busy = busy; }
     }
-    const int target_smem = 72 * 1024;
-    for (int C = 1; C <= kMaxCluster; C *= 2) {
-        int sc;
-        if (!usable(C, &sc)) continue;
-        best = C;
-        best_chunks = sc;
-        const bool small_enough = sc * 2 * kChunkBytes <= target_smem;
-        const bool fills_gpu = units * C >= 2LL * d.sm_count;
-        if (small_enough && (fills_gpu || sc <= kWarps)) break;
-    }
-    return remember(best, best_chunks);
+    d.dec_dtype = dtype; d.dec_V = V; d.dec_units = units; d.dec_forced = forced;
+    d.dec_C = best_C; d.dec_G = best_G; d.dec_lag = best_lag; d.dec_per = best_per;
+    *G_out = best_G;
+    *per_out = best_per;
+    *lag_out = best_lag;
+    return best_C;
 }
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
@@ -232,33 +244,37 @@ int run_device(DeviceState& d, const void* T, const void* D, const int32_t* x, c
     Params P;
     memset(&P, 0, sizeof P);
     P.T = T; P.D = D; P.x = x; P.u = u;
-    P.B = B; P.k = k; P.V = V; P.NC = L.NC;
-    P.c64 = 1.4426950408889634 / (double)tau;
-    P.c = (float)P.c64;
+    P.B = B; P.k = k; P.V = V;
+    P.c = (float)(1.4426950408889634 / (double)tau);
     P.tau = tau;
     P.inv_tau = 1.0 / (double)tau;
     P.accept_len = accept_len; P.tokens = tokens; P.loss = loss; P.grad = grad;
     P.acc_prob = acc_prob; P.status = status;
     P.ticket = reinterpret_cast<uint32_t*>(ws + L.ticket);
     P.wstatus = reinterpret_cast<uint32_t*>(ws + L.wstatus);
+    P.sticky = reinterpret_cast<uint32_t*>(ws + L.sticky);
     P.accept = ws + L.accept;
     P.rowc = reinterpret_cast<RowConst*>(ws + L.rowc);
-    P.chunk_sums = reinterpret_cast<float*>(ws + L.chunk_sums);
+    P.region_sums = reinterpret_cast<float*>(ws + L.region_sums);
 
-    if (!clean) SD_CUDA(cudaMemsetAsync(ws, 0, L.accept, stream));   // tickets and status words
+    if (!clean) SD_CUDA(cudaMemsetAsync(ws, 0, L.accept, stream));   // tickets, status words, sticky flag
 
     const size_t row_bytes = (size_t)V * elem_bytes(dtype);
     const bool fast = (row_bytes % 16 == 0) && aligned(T, 16) && aligned(D, 16) && (!grad || aligned(grad, 16)) &&
                       !getenv("SD_VERIFY_FORCE_GENERIC");
-    int C = 0, slice_chunks = 0;
-    if (fast) C = choose_cluster(d, P, dtype, &slice_chunks);
+    int C = 0, G = 0, lag = 0, per = 0;
+    if (fast) C = choose_stream(d, V, (long long)B * (k + 1), dtype, &G, &per, &lag);
     int rc;
     if (C > 0) {
         P.blocks_per_unit = C;
-        rc = dtype == SD_DTYPE_F32 ? launch_cluster<SD_DTYPE_F32>(d, P, C, slice_chunks, stream, false, nullptr)
-                                   : launch_cluster<SD_DTYPE_BF16>(d, P, C, slice_chunks, stream, false, nullptr);
+        P.RE = per * vec_elems(dtype);
+        P.NR = (V + P.RE - 1) / P.RE;
+        rc = dtype == SD_DTYPE_F32 ? launch_stream<SD_DTYPE_F32>(d, P, C, G, lag, stream, false, nullptr)
+                                   : launch_stream<SD_DTYPE_BF16>(d, P, C, G, lag, stream, false, nullptr);
     } else {
         P.blocks_per_unit = 1;
+        P.RE = kGenericRegionElems;
+        P.NR = (V + P.RE - 1) / P.RE;
         rc = dtype == SD_DTYPE_F32 ? launch_generic<SD_DTYPE_F32>(P, stream)
                                    : launch_generic<SD_DTYPE_BF16>(P, stream);
     }

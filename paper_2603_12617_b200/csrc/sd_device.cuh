@@ -1,14 +1,17 @@
 // Device-side building blocks of the verify-and-feedback kernels (sm_100a).
 //
 // Arithmetic contract shared by every kernel in this library, so that a value recomputed later
-// (the in-chunk inverse-CDF search) is bit-identical to the value summed earlier:
+// (the inverse-CDF search inside a sampling region) is bit-identical to the value summed earlier:
 //   c      = fp32(log2(e)/tau)
-//   e_v    = ex2.approx.ftz( fma(z_v, c, -R) ),  R = fl(m*c), m = row maximum
+//   a_v    = fma(z_v, c, -R),  R an INTEGER >= max_v z_v*c  (the reference of the exponentials)
+//   e_v    = ex2.approx.ftz(a_v)
 //   g_v    = fma(eD_v, kD, -(eT_v*kT)),          kX = fp32((1/tau)/S_X)       [ = (q-p)/tau ]
 //   r_v    = max(0, -g_v)                                                      [ = max(0,p-q)/tau ]
 //   bonus row: r_v = eT_v * kT with kT = fp32(1/S_T)                           [ = p ]
-// Row scalars (S, the KL accumulator, log-sum-exp, the accept ratio, CDF prefixes) are combined
-// in fp64 in a fixed order, so results do not depend on scheduling.
+// Because references are integers, sums taken under different references (by different warps or
+// blocks) are brought together by exact multiplications with powers of two: no exponential is
+// evaluated outside the elementwise sweeps.  Partial sums are combined in fp64 in a fixed order,
+// so results do not depend on scheduling.
 #pragma once
 
 #include <cooperative_groups.h>
@@ -22,16 +25,11 @@ namespace sdv {
 
 namespace cg = cooperative_groups;
 
-constexpr int kWarps = 8;
-constexpr int kThreads = kWarps * 32;
-constexpr int kChunkVecs = 128;                  // 16-byte vectors of one row in a sampling chunk
-constexpr int kChunkBytes = kChunkVecs * 16;     // 2 KiB of one row
-constexpr int kPieceChunks = 4;                  // sampling chunks fetched by one bulk copy
-constexpr int kMaxPieces = 16;                   // bulk copies (per row) a block may issue
-constexpr int kMaxChunksPerBlock = kMaxPieces * kPieceChunks;
 constexpr int kMaxCluster = 16;
-constexpr uint32_t kStatusTimeout = 0x80000000u; // internal: a bounded wait gave up
-constexpr uint32_t kWaitLimit = 1u << 22;        // polls of an mbarrier before giving up
+constexpr int kGenericRegionElems = 512;         // sampling region of the generic path
+constexpr uint32_t kStatusTimeout = 0x80000000u; // a bounded wait gave up
+constexpr uint32_t kWaitLimit = 1u << 21;        // polls of an mbarrier before giving up
+constexpr long long kWaitCycles = 2000000000ll;  // ... or about a second of waiting
 
 // Constants a finished row leaves behind for the inverse-CDF search.
 struct __align__(16) RowConst {
@@ -41,12 +39,13 @@ struct __align__(16) RowConst {
     float kD;     // pair row: (1/tau)/S_D ; bonus row: 0
 };
 
-// Softmax statistics of a slice of one row pair.
-struct PartialStats {
-    float mT, mD;      // slice maxima (raw logits); -FLT_MAX for an empty slice
-    double sT, sD;     // sum of ex2(fma(z,c,-fl(m*c)))
-    double w;          // sum of eT*((t-mT)-(d-mD)), same reference as sT
+// Softmax statistics of a part of one row pair, relative to integer references RT and RD.
+struct __align__(8) PartialStats {
+    float RT, RD;      // references of the exponentials (integer values)
+    double sT, sD;     // sum of eT = 2^aT, aT = t*c - RT; sum of eD likewise
+    double w;          // sum of eT*(aT - aD)
 };
+constexpr float kEmptyRef = -1073741824.f;       // reference of a part without a finite entry (-2^30)
 
 struct Params {
     const void* T;           // [B,k+1,V]
@@ -54,10 +53,10 @@ struct Params {
     const int32_t* x;        // [B,k]
     const float* u;          // [B,k+1]
     int B, k, V;
-    int NC;                  // sampling chunks per row
+    int RE;                  // vocabulary entries per sampling region (a multiple of 32)
+    int NR;                  // sampling regions per row: ceil(V / RE)
     float c;                 // fp32(log2e/tau)
     float tau;
-    double c64;              // log2e/tau
     double inv_tau;
     // outputs
     int32_t* accept_len;     // [B]
@@ -69,9 +68,10 @@ struct Params {
     // workspace
     uint32_t* ticket;        // [B] zero on entry; reset to zero by the resolver
     uint32_t* wstatus;       // [B] zero on entry; reset to zero by the resolver
+    uint32_t* sticky;        // [1] zero on entry; set (and left set) when a bounded wait gave up
     uint8_t* accept;         // [B*k]
     RowConst* rowc;          // [B*(k+1)]
-    float* chunk_sums;       // [B*(k+1)*NC]
+    float* region_sums;      // [B*(k+1)*NR] mass of each sampling region of each row
     int blocks_per_unit;     // blocks that take a ticket per (sequence, row)
 };
 
@@ -129,7 +129,11 @@ __device__ __forceinline__ float ex2f(float a) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(a));
     return r;
 }
-__device__ __forceinline__ float neg_ref(float m, float c) { return -__fmul_rn(m, c); }
+// Integer reference for exponentials of logits whose maximum is m: ceil(m*c), kept inside
+// [-2^30, 2^30] so that it converts to int and differences of references are exact.
+__device__ __forceinline__ float ref_of(float m, float c) {
+    return fminf(fmaxf(ceilf(__fmul_rn(fmaxf(m, -1e30f), c)), kEmptyRef), 1073741824.f);
+}
 __device__ __forceinline__ float exp_term(float z, float c, float negR) {
     return ex2f(__fmaf_rn(z, c, negR));
 }
@@ -143,69 +147,59 @@ __device__ __forceinline__ float grad_elem(float t, float d, float c, const RowC
 __device__ __forceinline__ float prob_elem(float t, float c, const RowConst& rc) {
     return __fmul_rn(exp_term(t, c, rc.negRT), rc.kT);
 }
+// 2^d as a double for an integer-valued d <= 0; 0 when the result would not be a normal number.
+__device__ __forceinline__ double pow2_neg(float d) {
+    const int e = (int)fmaxf(d, -2000.f);
+    return e < -1022 ? 0.0 : __hiloint2double((1023 + e) << 20, 0);
+}
 
-// Per-lane running softmax statistics of a row pair; every lane keeps its own reference.
-struct LaneStats {
-    float mT, negRT, sT, w;
-    float mD, negRD, sD;
-    __device__ __forceinline__ void init(float c) {
-        mT = mD = -3.402823466e+38f;
-        negRT = negRD = fminf(neg_ref(mT, c), 3.402823466e+38f);   // finite, so masked (-inf) entries give 0
-        sT = sD = w = 0.f;
-    }
-    // The KL accumulator w = sum eT*((t-mT)-(d-mD)) is kept relative to both running maxima, so a
-    // constant offset between the two models' logits cancels exactly instead of in the last bits.
-    // Both maxima move in one step: with identical rows the correction (dT - dD) is exactly zero.
+// Sum of VEC values as a balanced tree (short dependency chains, fixed order).
+template <int VEC>
+__device__ __forceinline__ float tree_sum(const float (&v)[VEC]) {
+    if constexpr (VEC == 1) return v[0];
+    else if constexpr (VEC == 4) return (v[0] + v[1]) + (v[2] + v[3]);
+    else return ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
+}
+template <int VEC>
+__device__ __forceinline__ float tree_max(const float (&v)[VEC]) {
+    if constexpr (VEC == 1) return v[0];
+    else if constexpr (VEC == 4) return fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3]));
+    else return fmaxf(fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3])), fmaxf(fmaxf(v[4], v[5]), fmaxf(v[6], v[7])));
+}
+
+// Softmax sums of one lane relative to integer references that the lane's whole warp shares:
+//   sT = sum eT, sD = sum eD, w = sum eT*(aT - aD)    with a = fma(z, c, -R), e = ex2(a).
+// aT - aD is log2(p/q) up to the two row constants, so w/sT leads to KL(p||q); each a is relative
+// to its own row's reference, so an offset between the two models' logits drops out.
+struct LaneSums {
+    float sT, sD, w;
+    __device__ __forceinline__ void init() { sT = sD = w = 0.f; }
     template <int VEC>
-    __device__ __forceinline__ void add_pair(const float (&t)[VEC], const float (&d)[VEC], float c) {
-        float vmT = t[0], vmD = d[0];
-#pragma unroll
-        for (int e = 1; e < VEC; ++e) {
-            vmT = fmaxf(vmT, t[e]);
-            vmD = fmaxf(vmD, d[e]);
-        }
-        if (vmT > mT || vmD > mD) {
-            const float nT = fmaxf(mT, vmT), nD = fmaxf(mD, vmD);
-            const float nrT = (nT > mT) ? neg_ref(nT, c) : negRT;
-            const float nrD = (nD > mD) ? neg_ref(nD, c) : negRD;
-            const float fT = (nT > mT) ? ex2f(nrT - negRT) : 1.f;
-            const float fD = (nD > mD) ? ex2f(nrD - negRD) : 1.f;
-            w = (sT > 0.f) ? (w - sT * ((nT - mT) - (nD - mD))) * fT : 0.f;
-            sT *= fT;
-            sD *= fD;
-            mT = nT; negRT = nrT;
-            mD = nD; negRD = nrD;
-        }
+    __device__ __forceinline__ void add_pair(const float (&t)[VEC], const float (&d)[VEC], float c, float negRT,
+                                             float negRD) {
+        float eT[VEC], eD[VEC], pw[VEC];
 #pragma unroll
         for (int e = 0; e < VEC; ++e) {
-            float eT = exp_term(t[e], c, negRT);
-            float eD = exp_term(d[e], c, negRD);
-            sT += eT;
-            sD += eD;
-            float diff = (t[e] - mT) - (d[e] - mD);
-            w = (eT > 0.f) ? __fmaf_rn(eT, diff, w) : w;   // masked target entries (p = 0) add nothing
+            const float aT = __fmaf_rn(t[e], c, negRT), aD = __fmaf_rn(d[e], c, negRD);
+            eT[e] = ex2f(aT);
+            eD[e] = ex2f(aD);
+            pw[e] = (eT[e] > 0.f) ? eT[e] * (aT - aD) : 0.f;   // masked target entries (p = 0) add nothing
         }
+        sT += tree_sum<VEC>(eT);
+        sD += tree_sum<VEC>(eD);
+        w += tree_sum<VEC>(pw);
     }
     template <int VEC>
-    __device__ __forceinline__ void add_target(const float (&t)[VEC], float c) {
-        float vm = t[0];
+    __device__ __forceinline__ void add_bonus(const float (&t)[VEC], float c, float negRT) {
+        float eT[VEC];
 #pragma unroll
-        for (int e = 1; e < VEC; ++e) vm = fmaxf(vm, t[e]);
-        if (vm > mT) {
-            float nr = neg_ref(vm, c);
-            sT *= ex2f(nr - negRT);
-            mT = vm;
-            negRT = nr;
-        }
-    }
-    template <int VEC>
-    __device__ __forceinline__ void add_bonus(const float (&t)[VEC], float c) {
-        add_target<VEC>(t, c);
-#pragma unroll
-        for (int e = 0; e < VEC; ++e) sT += exp_term(t[e], c, negRT);
+        for (int e = 0; e < VEC; ++e) eT[e] = exp_term(t[e], c, negRT);
+        sT += tree_sum<VEC>(eT);
     }
 };
 
+// ------------------------------------------------------------------------------------------
+// warp-wide helpers (all 32 lanes of the warp must call them)
 __device__ __forceinline__ double shfl_xor_f64(double v, int off) {
     return __shfl_xor_sync(0xffffffffu, v, off);
 }
@@ -214,126 +208,79 @@ __device__ __forceinline__ float warp_max_f32(float v) {
     for (int off = 16; off > 0; off >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, off));
     return v;
 }
-
-// Shared scratch of the block-level reduction of the statistics.
-struct StatScratch {
-    float wmaxT[kWarps], wmaxD[kWarps];
-    double wsT[kWarps], wsD[kWarps], ww[kWarps];
-};
-
-// Statistics of everything the block has seen, in every thread.  All threads must call.
-// Lanes are first brought to the block's maxima (one fp32 rescale each), then summed in fp64 in
-// a fixed order, so the result does not depend on scheduling and costs no serial fp64 exp.
-__device__ inline PartialStats block_reduce_stats(const LaneStats& ls, float c, StatScratch& sc) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const float wmT = warp_max_f32(ls.mT), wmD = warp_max_f32(ls.mD);
-    if (lane == 0) { sc.wmaxT[warp] = wmT; sc.wmaxD[warp] = wmD; }
-    __syncthreads();
-    float bmT = sc.wmaxT[0], bmD = sc.wmaxD[0];
+// Largest of the lanes' integer-valued references (one redux instruction).
+__device__ __forceinline__ float warp_max_ref(float R) {
+    return (float)__reduce_max_sync(0xffffffffu, (int)R);
+}
+__device__ __forceinline__ double warp_sum(double v) {
 #pragma unroll
-    for (int w = 1; w < kWarps; ++w) { bmT = fmaxf(bmT, sc.wmaxT[w]); bmD = fmaxf(bmD, sc.wmaxD[w]); }
-    float sT = 0.f, wv = 0.f, sD = 0.f;
-    if (ls.sT > 0.f) {
-        const float f = (ls.mT == bmT) ? 1.f : ex2f(neg_ref(bmT, c) - ls.negRT);
-        sT = ls.sT * f;
-        wv = (ls.w - ls.sT * ((bmT - ls.mT) - (bmD - ls.mD))) * f;
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    return v;
+}
+// Inclusive prefix sum over the lanes of a warp.
+__device__ __forceinline__ double warp_inclusive_scan(double v) {
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        double o = __shfl_up_sync(0xffffffffu, v, off);
+        if (lane >= off) v += o;
     }
-    if (ls.sD > 0.f) sD = ls.sD * ((ls.mD == bmD) ? 1.f : ex2f(neg_ref(bmD, c) - ls.negRD));
-    double dT = (double)sT, dW = (double)wv, dD = (double)sD;
+    return v;
+}
+
+// A partial rescaled from its own references to (RT, RD); exact, because references are integers.
+__device__ __forceinline__ PartialStats rescaled(const PartialStats& m, float RT, float RD) {
+    PartialStats r;
+    r.RT = RT; r.RD = RD;
+    const double f = pow2_neg(m.RT - RT), g = pow2_neg(m.RD - RD);
+    r.sT = m.sT * f;
+    r.sD = m.sD * g;
+    r.w = (m.sT > 0.0 && f > 0.0) ? (m.w - m.sT * (double)((RT - m.RT) - (RD - m.RD))) * f : 0.0;
+    return r;
+}
+__device__ __forceinline__ PartialStats empty_partial() {
+    PartialStats m;
+    m.RT = m.RD = kEmptyRef;
+    m.sT = m.sD = m.w = 0.0;
+    return m;
+}
+
+// Merge of up to 16 partials in shared memory by every calling lane on its own, in index order:
+// no lane talks to another, and all lanes get the same bits.
+__device__ __forceinline__ PartialStats merge_partials_serial(const PartialStats* p, int n) {
+    float RT = kEmptyRef, RD = kEmptyRef;
+    for (int i = 0; i < n; ++i) { RT = fmaxf(RT, p[i].RT); RD = fmaxf(RD, p[i].RD); }
+    PartialStats r;
+    r.RT = RT; r.RD = RD;
+    r.sT = r.sD = r.w = 0.0;
+    for (int i = 0; i < n; ++i) {
+        const PartialStats q = rescaled(p[i], RT, RD);
+        r.sT += q.sT; r.sD += q.sD; r.w += q.w;
+    }
+    return r;
+}
+
+// Sums of the lanes of a warp that share the references (RT, RD), as one partial in every lane.
+__device__ __forceinline__ PartialStats warp_sum_lanes(const LaneSums& ls, float RT, float RD) {
+    double dT = (double)ls.sT, dW = (double)ls.w, dD = (double)ls.sD;
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
         dT += shfl_xor_f64(dT, off);
         dW += shfl_xor_f64(dW, off);
         dD += shfl_xor_f64(dD, off);
     }
-    if (lane == 0) { sc.wsT[warp] = dT; sc.ww[warp] = dW; sc.wsD[warp] = dD; }
-    __syncthreads();
     PartialStats r;
-    r.mT = bmT; r.mD = bmD;
-    r.sT = r.sD = r.w = 0.0;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) { r.sT += sc.wsT[w]; r.w += sc.ww[w]; r.sD += sc.wsD[w]; }
+    r.RT = RT; r.RD = RD;
+    r.sT = dT; r.sD = dD; r.w = dW;
     return r;
-}
-
-// Merge of the block statistics of a cluster by one full warp: lane j takes block j, one fp64
-// exp2 per lane in parallel, then a butterfly sum.  Every lane returns the row statistics.
-__device__ inline PartialStats warp_merge_partials(const PartialStats* p, int n, float c) {
-    const int lane = threadIdx.x & 31;
-    PartialStats m;
-    m.mT = m.mD = -3.402823466e+38f;
-    m.sT = m.sD = m.w = 0.0;
-    if (lane < n) m = p[lane];
-    PartialStats r;
-    r.mT = warp_max_f32(m.mT);
-    r.mD = warp_max_f32(m.mD);
-    double sT = 0.0, wv = 0.0, sD = 0.0;
-    if (m.sT > 0.0) {
-        const double f = (m.mT == r.mT) ? 1.0 : exp2((double)__fmul_rn(m.mT, c) - (double)__fmul_rn(r.mT, c));
-        sT = m.sT * f;
-        wv = (m.w - m.sT * (((double)r.mT - (double)m.mT) - ((double)r.mD - (double)m.mD))) * f;
-    }
-    if (m.sD > 0.0)
-        sD = m.sD * ((m.mD == r.mD) ? 1.0 : exp2((double)__fmul_rn(m.mD, c) - (double)__fmul_rn(r.mD, c)));
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        sT += shfl_xor_f64(sT, off);
-        wv += shfl_xor_f64(wv, off);
-        sD += shfl_xor_f64(sD, off);
-    }
-    r.sT = sT; r.w = wv; r.sD = sD;
-    return r;
-}
-
-// ------------------------------------------------------------------------------------------
-// block-wide helpers (all threads of the block must call them)
-__device__ __forceinline__ double warp_sum(double v) {
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-    return v;
-}
-
-// Sum over the block in a fixed order; result in every thread.  scratch: kWarps doubles.
-__device__ inline double block_sum(double v, double* scratch) {
-    v = warp_sum(v);
-    __syncthreads();
-    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
-    __syncthreads();
-    double t = 0.0;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) t += scratch[w];
-    return t;
-}
-
-// Exclusive prefix sum over the block in thread order; `total` receives the block sum.
-__device__ inline double block_exclusive_scan(double v, double* scratch, double* total) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    double incl = v;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        double o = __shfl_up_sync(0xffffffffu, incl, off);
-        if (lane >= off) incl += o;
-    }
-    __syncthreads();
-    if (lane == 31) scratch[warp] = incl;
-    __syncthreads();
-    double base = 0.0, tot = 0.0;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
-        double s = scratch[w];
-        if (w < warp) base += s;
-        tot += s;
-    }
-    *total = tot;
-    return base + incl - v;
 }
 
 // ------------------------------------------------------------------------------------------
 // Constants of a finished row for the second sweep and the inverse-CDF search.
 __device__ __forceinline__ RowConst row_constants(const Params& P, bool bonus, const PartialStats& st) {
     RowConst rc;
-    rc.negRT = neg_ref(st.mT, P.c);
-    rc.negRD = bonus ? 0.f : neg_ref(st.mD, P.c);
+    rc.negRT = -st.RT;
+    rc.negRD = bonus ? 0.f : -st.RD;
     rc.kT = (float)((bonus ? 1.0 : P.inv_tau) / st.sT);
     rc.kD = bonus ? 0.f : (float)(P.inv_tau / st.sD);
     return rc;
@@ -372,15 +319,11 @@ __device__ inline void finish_row(const Params& P, int b, int i, const PartialSt
     if (!okT || !okD) flags |= SD_STATUS_BAD_ROW;
     P.rowc[unit] = rc;
     if (!bonus) {
-        // log2 of the softmax denominators at temperature tau, reference = the row maximum:
-        // the elementwise reference fl(m*c) differs from m*c by eps, which is known exactly.
-        const double epsT = (double)st.mT * (double)P.c - (double)__fmul_rn(st.mT, P.c);
-        const double epsD = (double)st.mD * (double)P.c - (double)__fmul_rn(st.mD, P.c);
-        const double l2ST = log2(st.sT) - epsT;   // log2 sum_v 2^((t_v - mT) c)
-        const double l2SD = log2(st.sD) - epsD;
+        // log2 p_v = aT_v - log2 S_T and log2 q_v = aD_v - log2 S_D, so
+        // KL(p||q) = ln2 * [ E_p(aT - aD) - log2 S_T + log2 S_D ]
+        const double l2ST = log2(st.sT), l2SD = log2(st.sD);
         if (P.loss) {
-            // KL(p||q) = ln2 * [ c * E_p((t-mT)-(d-mD)) - log2 S_T + log2 S_D ], S relative to the maxima
-            const double kl = 0.6931471805599453 * (P.c64 * (st.w / st.sT) - l2ST + l2SD);
+            const double kl = 0.6931471805599453 * (st.w / st.sT - l2ST + l2SD);
             P.loss[b * P.k + i] = (float)kl;
         }
         // rejection test for draft token x[b,i] with ratio p(x)/q(x) in fp64
@@ -393,8 +336,8 @@ __device__ inline void finish_row(const Params& P, int b, int i, const PartialSt
             if (dx == -INFINITY) {
                 rho = (tx == -INFINITY) ? 0.0 : INFINITY;
             } else {
-                const double l2p = (tx - (double)st.mT) * P.c64 - l2ST;
-                const double l2q = (dx - (double)st.mD) * P.c64 - l2SD;
+                const double l2p = (tx * (double)P.c - (double)st.RT) - l2ST;
+                const double l2q = (dx * (double)P.c - (double)st.RD) - l2SD;
                 rho = exp2(l2p - l2q);
             }
             const double thr = rho < 1.0 ? rho : 1.0;
@@ -406,8 +349,9 @@ __device__ inline void finish_row(const Params& P, int b, int i, const PartialSt
 }
 
 // ------------------------------------------------------------------------------------------
-// Last block of a sequence: accept length, emitted tokens, the residual / bonus draw.
-// Reads what other blocks wrote (after their fence + ticket), so those loads bypass L1.
+// Resolution of a sequence by one warp, once every (row, slice) of the sequence has been
+// processed: accept length, emitted tokens, the residual / bonus draw.  It reads what other
+// blocks wrote (after their fence + ticket), so those loads bypass L1.
 
 // Unnormalised mass of vocabulary entry v in the distribution the extra token is drawn from.
 //   mode 0: pair row, max(0,p-q)/tau     mode 1: bonus row, p     mode 2: pair row, p/tau
@@ -421,118 +365,111 @@ __device__ __forceinline__ float mass_elem(const Params& P, const RowConst& rc, 
     return fmaxf(-grad_elem(t, d, P.c, rc), 0.f);
 }
 
-struct ResolveScratch {
-    double red[kWarps];
-    int found;
-    int n;
-    int ticket_last;
-};
-
-// Inverse-CDF search inside one sampling chunk.  prefix = mass before the chunk, t = target.
-// last_with_mass: ignore t and return the last entry of the chunk that has mass.
-// Returns the vocabulary index, or -1 if the chunk has no qualifying entry.
+// Inverse-CDF search inside one sampling region.  prefix = mass before the region, t = target.
+// last_with_mass: ignore t and return the last entry of the region that has mass.
+// Every lane takes a contiguous run of RE/32 entries and visits it twice (sum, then search), so
+// nothing is kept per entry.  Returns (in every lane) the vocabulary index, or -1 if the region
+// has no qualifying entry.
 template <int DT>
-__device__ int search_chunk(const Params& P, const RowConst& rc, int mode, size_t offT, size_t offD,
-                            int chunk, double prefix, double t, bool last_with_mass,
-                            ResolveScratch& S, double* chunk_total) {
-    constexpr int CE = kChunkVecs * Elem<DT>::VEC;
-    constexpr int PER = CE / kThreads;            // contiguous entries per thread
-    const int tid = threadIdx.x;
-    const int v0 = chunk * CE + tid * PER;
-    float r[PER];
+__device__ int search_region(const Params& P, const RowConst& rc, int mode, size_t offT, size_t offD,
+                             int region, double prefix, double t, bool last_with_mass, double* region_total) {
+    const int lane = threadIdx.x & 31;
+    const int per = P.RE / 32;                    // contiguous entries per lane
+    const int v0 = region * P.RE + lane * per;
     double loc = 0.0;
-#pragma unroll
-    for (int e = 0; e < PER; ++e) {
-        r[e] = mass_elem<DT>(P, rc, mode, offT, offD, v0 + e);
-        loc += (double)r[e];
-    }
-    double run = prefix + block_exclusive_scan(loc, S.red, chunk_total);
-    if (tid == 0) S.found = last_with_mass ? -1 : 0x7fffffff;
-    __syncthreads();
+    for (int e = 0; e < per; ++e) loc += (double)mass_elem<DT>(P, rc, mode, offT, offD, v0 + e);
+    const double incl = warp_inclusive_scan(loc);
+    *region_total = __shfl_sync(0xffffffffu, incl, 31);
+    int cand = last_with_mass ? -1 : 0x7fffffff;
     if (!last_with_mass) {
-#pragma unroll
-        for (int e = 0; e < PER; ++e) {
-            run += (double)r[e];
-            if (run > t && r[e] > 0.f) { atomicMin(&S.found, v0 + e); break; }
+        double run = prefix + (incl - loc);
+        if (run + loc > t) {                      // the crossing can only be in a lane whose run reaches t
+            for (int e = 0; e < per; ++e) {
+                const float r = mass_elem<DT>(P, rc, mode, offT, offD, v0 + e);
+                run += (double)r;
+                if (run > t && r > 0.f) { cand = v0 + e; break; }
+            }
         }
-    } else {
 #pragma unroll
-        for (int e = 0; e < PER; ++e)
-            if (r[e] > 0.f) atomicMax(&S.found, v0 + e);
+        for (int off = 16; off > 0; off >>= 1) cand = min(cand, __shfl_xor_sync(0xffffffffu, cand, off));
+        return cand == 0x7fffffff ? -1 : cand;
     }
-    __syncthreads();
-    const int y = S.found;
-    __syncthreads();
-    return y == 0x7fffffff ? -1 : y;
+    if (loc > 0.0)
+        for (int e = 0; e < per; ++e)
+            if (mass_elem<DT>(P, rc, mode, offT, offD, v0 + e) > 0.f) cand = v0 + e;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) cand = max(cand, __shfl_xor_sync(0xffffffffu, cand, off));
+    return cand;
 }
 
-// Draw from a row without chunk sums (two sweeps over the row by one block).  Only used when a
+// Draw from a row without region sums (two sweeps over the row by one warp).  Only used when a
 // rejection leaves no residual mass in fp32, which exact arithmetic rules out.
 template <int DT>
 __device__ int draw_row_slow(const Params& P, const RowConst& rc, int mode, size_t offT,
-                             size_t offD, double u, ResolveScratch& S) {
-    double total = 0.0, ctot;
-    for (int j = 0; j < P.NC; ++j) {
-        search_chunk<DT>(P, rc, mode, offT, offD, j, 0.0, 0.0, true, S, &ctot);
-        total += ctot;
+                             size_t offD, double u) {
+    double total = 0.0, rtot;
+    for (int j = 0; j < P.NR; ++j) {
+        search_region<DT>(P, rc, mode, offT, offD, j, 0.0, 0.0, true, &rtot);
+        total += rtot;
     }
     if (!(total > 0.0) || !isfinite(total)) return 0;
     const double t = u * total;
     double prefix = 0.0;
     int last_mass = -1;
-    for (int j = 0; j < P.NC; ++j) {
-        const int y = search_chunk<DT>(P, rc, mode, offT, offD, j, prefix, t, false, S, &ctot);
+    for (int j = 0; j < P.NR; ++j) {
+        const int y = search_region<DT>(P, rc, mode, offT, offD, j, prefix, t, false, &rtot);
         if (y >= 0) return y;
-        if (ctot > 0.0) last_mass = j;
-        prefix += ctot;
+        if (rtot > 0.0) last_mass = j;
+        prefix += rtot;
     }
     if (last_mass < 0) return 0;
-    const int y = search_chunk<DT>(P, rc, mode, offT, offD, last_mass, 0.0, 0.0, true, S, &ctot);
+    const int y = search_region<DT>(P, rc, mode, offT, offD, last_mass, 0.0, 0.0, true, &rtot);
     return y < 0 ? 0 : y;
 }
 
 template <int DT>
-__device__ void resolve_sequence(const Params& P, int b, ResolveScratch& S) {
-    const int tid = threadIdx.x;
-    const int k = P.k, NC = P.NC;
+__device__ void resolve_sequence(const Params& P, int b) {
+    const int lane = threadIdx.x & 31;
+    const int k = P.k, NR = P.NR;
 
-    if (tid == 0) {
-        int n = k;
-        for (int i = 0; i < k; ++i)
-            if (__ldcg(P.accept + b * k + i) == 0) { n = i; break; }
-        S.n = n;
+    // accept length: first rejected position
+    int n = k;
+    for (int i0 = 0; i0 < k; i0 += 32) {
+        const int i = i0 + lane;
+        const bool rej = (i < k) && (__ldcg(P.accept + b * k + i) == 0);
+        const unsigned m = __ballot_sync(0xffffffffu, rej);
+        if (m) { n = i0 + __ffs(m) - 1; break; }
     }
-    __syncthreads();
-    const int n = S.n;
     uint32_t flags = 0;
 
     // diagnostic: acceptance probability 1 - sum max(0,p-q) per position (Eq. 1)
     if (P.acc_prob) {
         for (int i = 0; i < k; ++i) {
-            const float* csi = P.chunk_sums + (size_t)(b * (k + 1) + i) * NC;
+            const float* rsi = P.region_sums + (size_t)(b * (k + 1) + i) * NR;
             double part = 0.0;
-            for (int j = tid; j < NC; j += kThreads) part += (double)__ldcg(csi + j);
-            const double R = block_sum(part, S.red) * (double)P.tau;
-            if (tid == 0) P.acc_prob[b * k + i] = (float)(1.0 - R);
+            for (int j = lane; j < NR; j += 32) part += (double)__ldcg(rsi + j);
+            const double R = warp_sum(part) * (double)P.tau;
+            if (lane == 0) P.acc_prob[b * k + i] = (float)(1.0 - R);
         }
     }
 
     const bool bonus = (n == k);
     const int unit = b * (k + 1) + n;
-    const float* cs = P.chunk_sums + (size_t)unit * NC;
+    const float* rs = P.region_sums + (size_t)unit * NR;
     const float4 rcv = __ldcg(reinterpret_cast<const float4*>(P.rowc + unit));
     const RowConst rc{rcv.x, rcv.y, rcv.z, rcv.w};
     const size_t offT = (size_t)unit * P.V;
     const size_t offD = (size_t)(b * k + (bonus ? 0 : n)) * P.V;
     const double uk = (double)P.u[b * (k + 1) + k];
 
-    // prefix over the chunk sums: each thread owns a contiguous run of chunks
-    const int per = (NC + kThreads - 1) / kThreads;
-    const int j0 = min(NC, tid * per), j1 = min(NC, j0 + per);
+    // prefix over the region sums: each lane owns a contiguous run of regions
+    const int per = (NR + 31) / 32;
+    const int j0 = min(NR, lane * per), j1 = min(NR, j0 + per);
     double mine = 0.0;
-    for (int j = j0; j < j1; ++j) mine += (double)__ldcg(cs + j);
-    double total;
-    const double before = block_exclusive_scan(mine, S.red, &total);
+    for (int j = j0; j < j1; ++j) mine += (double)__ldcg(rs + j);
+    const double incl = warp_inclusive_scan(mine);
+    const double before = incl - mine;
+    const double total = __shfl_sync(0xffffffffu, incl, 31);
     const double t = uk * total;
 
     int y = 0;
@@ -541,70 +478,70 @@ __device__ void resolve_sequence(const Params& P, int b, ResolveScratch& S) {
             flags |= SD_STATUS_BAD_ROW;
         } else {
             flags |= SD_STATUS_ZERO_RESIDUAL;   // draw from p_n instead
-            y = draw_row_slow<DT>(P, rc, 2, offT, offD, uk, S);
+            y = draw_row_slow<DT>(P, rc, 2, offT, offD, uk);
         }
     } else {
-        if (tid == 0) S.found = 0x7fffffff;
-        __syncthreads();
+        // first region whose running sum exceeds t, and the mass before it
+        int cand = 0x7fffffff;
+        double cand_prefix = 0.0;
         {
             double run = before;
             for (int j = j0; j < j1; ++j) {
-                run += (double)__ldcg(cs + j);
-                if (run > t) { atomicMin(&S.found, j); break; }
+                const double next = run + (double)__ldcg(rs + j);
+                if (next > t) { cand = j; cand_prefix = run; break; }
+                run = next;
             }
         }
-        __syncthreads();
-        int chunk = S.found;
-        __syncthreads();
+        const unsigned has = __ballot_sync(0xffffffffu, cand != 0x7fffffff);
+        int region = -1;
+        double prefix = 0.0;
         bool past_end = false;
-        if (chunk == 0x7fffffff) {
-            // rounding pushed u*R to the total: last chunk that holds mass
+        if (has) {
+            const int owner = __ffs(has) - 1;
+            region = __shfl_sync(0xffffffffu, cand, owner);
+            prefix = __shfl_sync(0xffffffffu, cand_prefix, owner);
+        } else {
+            // rounding pushed u*R to the total: last region that holds mass
             past_end = true;
-            if (tid == 0) S.found = -1;
-            __syncthreads();
+            int lastr = -1;
             for (int j = j0; j < j1; ++j)
-                if (__ldcg(cs + j) > 0.f) atomicMax(&S.found, j);
-            __syncthreads();
-            chunk = S.found;
-            __syncthreads();
+                if (__ldcg(rs + j) > 0.f) lastr = j;
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) lastr = max(lastr, __shfl_xor_sync(0xffffffffu, lastr, off));
+            region = lastr;
         }
-        if (chunk >= 0) {
-            double pre_part = 0.0;
-            for (int j = tid; j < chunk; j += kThreads) pre_part += (double)__ldcg(cs + j);
-            const double prefix = block_sum(pre_part, S.red);
-            double ctot;
-            y = search_chunk<DT>(P, rc, bonus ? 1 : 0, offT, offD, chunk, prefix, t, past_end, S, &ctot);
-            // chunk sum and re-summed entries may disagree in the last bits: last entry with mass
-            if (y < 0) y = search_chunk<DT>(P, rc, bonus ? 1 : 0, offT, offD, chunk, 0.0, 0.0, true, S, &ctot);
+        if (region >= 0) {
+            double rtot;
+            y = search_region<DT>(P, rc, bonus ? 1 : 0, offT, offD, region, prefix, t, past_end, &rtot);
+            // region sum and re-summed entries may disagree in the last bits: last entry with mass
+            if (y < 0) y = search_region<DT>(P, rc, bonus ? 1 : 0, offT, offD, region, 0.0, 0.0, true, &rtot);
             if (y < 0) y = 0;
         }
     }
 
-    if (tid == 0) {
+    if (lane == 0) {
         P.accept_len[b] = n;
-        const uint32_t st = __ldcg(P.wstatus + b) | flags;
+        uint32_t st = __ldcg(P.wstatus + b) | flags;
+        if (__ldcg(P.sticky) != 0) st |= kStatusTimeout;
         if (P.status) P.status[b] = st;
         // leave the workspace ready for the next call
         P.wstatus[b] = 0;
         P.ticket[b] = 0;
     }
-    for (int i = tid; i <= k; i += kThreads)
+    for (int i = lane; i <= k; i += 32)
         P.tokens[b * (k + 1) + i] = (i < n) ? P.x[b * k + i] : (i == n ? y : -1);
 }
 
-// Take a ticket for sequence b; true in every thread of the block that arrives last.
-__device__ inline bool take_ticket(const Params& P, int b, int* flag_smem) {
+// Tickets of one block for sequence b: `n` of the (k+1) * blocks_per_unit tickets of the
+// sequence at once, by one thread, after everything the tickets stand for has been ordered before
+// this thread.  True if these were the last tickets of the sequence.
+__device__ __forceinline__ bool take_tickets(const Params& P, int b, uint32_t n) {
     __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        __threadfence();
-        const uint32_t total = (uint32_t)(P.k + 1) * (uint32_t)P.blocks_per_unit;
-        const uint32_t old = atomicAdd(P.ticket + b, 1u);
-        *flag_smem = (old == total - 1);
-        __threadfence();
-    }
-    __syncthreads();
-    return *flag_smem != 0;
+    const uint32_t total = (uint32_t)(P.k + 1) * (uint32_t)P.blocks_per_unit;
+    const uint32_t old = atomicAdd(P.ticket + b, n);
+    const bool last = (old + n == total);
+    if (last) __threadfence();
+    return last;
 }
 
 }  // namespace sdv

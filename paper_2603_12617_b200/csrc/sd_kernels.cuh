@@ -1,23 +1,54 @@
 // The two kernels of the verify-and-feedback step.
 //
-//   sd_cluster_kernel  fast path.  One thread-block cluster per (sequence, row) unit; each block
-//                      owns a contiguous slice of the vocabulary, pulls it into shared memory once
-//                      with bulk asynchronous copies (cp.async.bulk + mbarrier), computes the
-//                      softmax statistics from shared memory, exchanges them through distributed
-//                      shared memory, and makes the second sweep (gradient, residual chunk sums)
-//                      over the copy that is still resident.  HBM sees each logit once.
-//   sd_generic_kernel  any V and any alignment.  One block per unit, two sweeps over global
-//                      memory with element loads.  Same arithmetic, same workspace, same resolver.
+//   sd_stream_kernel   fast path.  A persistent kernel of thread-block clusters.  A cluster takes a
+//                      contiguous range of (sequence, row) units, one after the other; each block
+//                      of the cluster owns a contiguous slice of the vocabulary.  Inside a block
+//                      the warps are specialised:
+//                        producer   one thread streams the block's slices of successive units into
+//                                   a ring of shared-memory stages with bulk asynchronous copies
+//                                   (cp.async.bulk + mbarrier), running ahead as far as the ring
+//                                   allows, so HBM never waits for arithmetic;
+//                        consumers  sweep 1 over a slice (maxima, then softmax sums relative to
+//                                   integer references), later sweep 2 over the same stages, still
+//                                   resident (gradient out, residual mass per lane), then hand the
+//                                   stages back;
+//                        statistics adds up the consumers' sums, exchanges the block's partial
+//                                   with the other blocks of the cluster through distributed
+//                                   shared memory (remote stores + remote mbarrier arrivals, no
+//                                   cluster-wide barrier) and publishes the row constants;
+//                        resolver   turns the lanes' residual masses into region sums, reports
+//                                   rows (loss, rejection test), takes the sequence's tickets when
+//                                   the block leaves a sequence and, if they were the last ones,
+//                                   draws the extra token.
+//                      Sweep 2 of a unit runs one unit behind sweep 1 when the ring holds two
+//                      slices, which hides the exchange.  HBM sees each logit once.
+//   sd_generic_kernel  any V and any alignment.  One block per unit, sweeps over global memory
+//                      with element loads.  Same arithmetic, same workspace, same resolver.
 //
 // A unit is row i of sequence b: i < k pairs target row i with draft row i (Algorithm 1's
 // rejection test, the KL loss of Eq. "kl_divergence" and its gradient); i == k is the bonus row.
-// The block that takes the last ticket of a sequence resolves it (accept length, emitted tokens,
-// inverse-CDF draw); nobody waits for anybody.
+// Every wait is bounded; nobody waits for another cluster.
 #pragma once
 
 #include "sd_device.cuh"
 
 namespace sdv {
+
+// ---- geometry of the fast path -------------------------------------------------------------
+// A row is cut into sampling regions of `per` 16-byte vectors (per = 32*m).  Block r of a
+// cluster owns the 16 regions [16r, 16r+16) of every row it works on, one per consumer warp;
+// the block's slice is streamed through the ring in stages of 512 vectors (8 KiB) per row, so
+// a full slice is m stages and group g of 32 vectors of the slice lies in stage g/16.
+constexpr int kConsumerWarps = 16;
+constexpr int kStageVecs = 512;                               // vectors of one row in a stage
+constexpr int kStageRowBytes = kStageVecs * 16;               // 8 KiB of one row
+constexpr int kStageBytes = 2 * kStageRowBytes;               // target part + draft part
+constexpr int kMaxStages = 12;
+constexpr int kDoneDepth = 4;                                 // units the resolver may lag behind
+constexpr int kProducerWarp = 0, kStatsWarp = 1, kResolverWarp = 2, kFirstConsumerWarp = 3;
+constexpr int kStreamThreads = (kFirstConsumerWarp + kConsumerWarps) * 32;
+constexpr int kGenericWarps = 8;
+constexpr int kGenericThreads = kGenericWarps * 32;
 
 // ---- PTX wrappers --------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -30,22 +61,68 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
                  : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// Arrival on the barrier at the same shared-memory offset in block `rank` of the cluster; orders
+// this thread's earlier (remote) stores before it at cluster scope.
+__device__ __forceinline__ void mbar_arrive_remote(uint64_t* bar, uint32_t rank) {
+    asm volatile(
+        "{\n\t.reg .b32 ra;\n\t"
+        "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
+        "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}" ::"r"(smem_u32(bar)),
+        "r"(rank)
+        : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.acquire.cta.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(smem_u32(bar)), "r"(parity)
         : "memory");
     return ok != 0;
 }
-// Bounded wait: false if the copy did not land within kWaitLimit polls.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
-    for (uint32_t it = 0; it < kWaitLimit; ++it)
-        if (mbar_try_wait(bar, parity)) return true;
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait of one thread.  It gives up after kWaitLimit polls or kWaitCycles clock cycles,
+// whichever comes first, or as soon as another thread of the block has given up (*abort != 0);
+// the caller then leaves its loop and the kernel returns.  A failed poll is followed by a short
+// sleep, so that waiting warps leave the issue slots and the shared-memory pipe to working ones.
+template <bool CLUSTER>
+__device__ __forceinline__ bool mbar_wait_thread(uint64_t* bar, uint32_t parity, volatile int* abort) {
+    long long t0 = 0;
+    for (uint32_t it = 0; it < kWaitLimit; ++it) {
+        if (CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 63u) {
+            if (*abort) return false;
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitCycles) break;
+        }
+    }
+    *abort = 1;
     return false;
+}
+// The same for a whole warp (all 32 lanes call it): every lane observes the barrier itself (a
+// warp whose lanes part ways at a wait is slow to get back together), and all lanes get the same
+// answer.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
+    return __all_sync(0xffffffffu, mbar_wait_thread<false>(bar, parity, abort) ? 1 : 0) != 0;
+}
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, volatile int* abort) {
+    return __all_sync(0xffffffffu, mbar_wait_thread<true>(bar, parity, abort) ? 1 : 0) != 0;
 }
 // 1-D bulk copy global -> shared of this block, completion counted on `bar`.
 // Both addresses 16-byte aligned, bytes a multiple of 16.
@@ -68,168 +145,368 @@ __device__ __forceinline__ void store_streaming(void* p, const uint4& v) {
                  : "memory");
 }
 
-// Chunks [c0, c0+nc) of the row that block `rank` of `C` owns.
-__device__ __forceinline__ void block_chunks(int NC, int C, int rank, int& c0, int& nc) {
-    const int base = NC / C, rem = NC % C;
-    nc = base + (rank < rem ? 1 : 0);
-    c0 = rank * base + min(rank, rem);
-}
-
-struct ClusterShared {
-    uint64_t bar[kMaxPieces];
-    StatScratch stat;
-    PartialStats xchg[kMaxCluster];   // written by every block of the cluster (distributed shared memory)
-    RowConst rc;
-    ResolveScratch rs;
+// Control block of the fast path; lives in dynamic shared memory after the ring.
+struct StreamShared {
+    uint64_t full[kMaxStages];          // stage filled by the bulk copies        (1 arrival + bytes)
+    uint64_t empty[kMaxStages];         // stage handed back after sweep 2        (consumer warps)
+    uint64_t s1_done[2];                // consumers' sums of a unit posted       (consumer warps)
+    uint64_t xchg_bar[2];               // partials of every block have arrived   (cluster size, remote)
+    uint64_t rc_ready[2];               // row constants published                (1)
+    uint64_t s2_done[kDoneDepth];       // unit finished in this block            (consumer warps + 1)
+    uint64_t res_free[kDoneDepth];      // resolver is done with the unit         (1)
+    float lane_sums[2][3][kConsumerWarps][33];        // sT, sD, w of every consumer lane (33: no bank conflicts)
+    float warp_ref[2][kConsumerWarps][2];             // RT, RD each consumer warp used
+    float lane_mass[kDoneDepth][kConsumerWarps][33];  // residual / bonus mass of every consumer lane
+    PartialStats wpart[kConsumerWarps]; // the consumer warps' partials of the unit being merged
+    PartialStats xchg[2][kMaxCluster];  // written by every block of the cluster (distributed shared memory)
+    PartialStats row[kDoneDepth];       // statistics of the whole row, for the row report
+    RowConst rc[2];
+    RowConst rc_done[kDoneDepth];       // the same, kept for the row report
+    int abort;                          // a bounded wait gave up somewhere in this block
 };
 
+// Position of a stage in the ring: slot index and the parity of its current use.
+struct RingPos {
+    int slot;
+    uint32_t phase;
+    __device__ __forceinline__ void advance(int n, int R) {
+        slot += n;
+        if (slot >= R) { slot -= R; phase ^= 1u; }
+    }
+    __device__ __forceinline__ RingPos plus(int n, int R) const {
+        RingPos r = *this;
+        r.advance(n, R);
+        return r;
+    }
+};
+
+// Units [u0, u0+n) of cluster `cid` of `G`: contiguous, sizes differ by at most one.
+__device__ __host__ __forceinline__ void cluster_units(int units, int G, int cid, int& u0, int& n) {
+    const int base = units / G, rem = units % G;
+    n = base + (cid < rem ? 1 : 0);
+    u0 = cid * base + (cid < rem ? cid : rem);
+}
+
 // ---- fast path -----------------------------------------------------------------------------
+// R: stages of the ring (every slice has at most R stages).  lag: 1 if sweep 2 runs one unit
+// behind sweep 1 (needs a ring of at least two slices), else 0.
 template <int DT>
-__global__ void __launch_bounds__(kThreads) sd_cluster_kernel(const Params P, const int slice_chunks) {
+__global__ void __launch_bounds__(kStreamThreads, 1)
+sd_stream_kernel(const __grid_constant__ Params P, const int R, const int lag) {
     using E = Elem<DT>;
+    using ET = typename E::type;
     constexpr int VEC = E::VEC;
-    constexpr int CE = kChunkVecs * VEC;
     extern __shared__ __align__(128) unsigned char dyn_smem[];
-    __shared__ ClusterShared sh;
+    unsigned char* ring = dyn_smem;
+    StreamShared& sh = *reinterpret_cast<StreamShared*>(dyn_smem + (size_t)R * kStageBytes);
 
     cg::cluster_group cluster = cg::this_cluster();
     const int C = (int)cluster.num_blocks();
     const int rank = (int)cluster.block_rank();
-    const int unit = blockIdx.x / C;
-    const int b = unit / (P.k + 1), i = unit % (P.k + 1);
-    const bool bonus = (i == P.k);
+    const int G = (int)gridDim.x / C;             // clusters in the grid
+    const int cid = (int)blockIdx.x / C;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int K1 = P.k + 1;
+    int u0, nu;
+    cluster_units(P.B * K1, G, cid, u0, nu);      // this cluster works on units u0 .. u0+nu-1
 
-    int c0, nc;
-    block_chunks(P.NC, C, rank, c0, nc);
-    const int npieces = (nc + kPieceChunks - 1) / kPieceChunks;
+    const int per = P.RE / VEC;                   // vectors per sampling region
+    const int m = per >> 5;                       // groups of 32 vectors per region = stages per full slice
+    const int NV = P.V / VEC;                     // vectors per row
+    const int vb0 = rank * kConsumerWarps * per;  // first vector of this block's slice
+    const int nvb = max(0, min(NV - vb0, kConsumerWarps * per));
+    const int ns = (nvb + kStageVecs - 1) / kStageVecs;
+    volatile int* abort = &sh.abort;
 
-    uint4* sT = reinterpret_cast<uint4*>(dyn_smem);
-    uint4* sD = reinterpret_cast<uint4*>(dyn_smem + (size_t)slice_chunks * kChunkBytes);
-    const typename E::type* Trow = reinterpret_cast<const typename E::type*>(P.T) + (size_t)unit * P.V;
-    const typename E::type* Drow =
-        reinterpret_cast<const typename E::type*>(P.D) + (size_t)(b * P.k + (bonus ? 0 : i)) * P.V;
-
-    // -- issue every bulk copy of this block's slice up front
     if (tid == 0) {
-        for (int p = 0; p < npieces; ++p) mbar_init(&sh.bar[p], 1);
+        for (int s = 0; s < R; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], kConsumerWarps); }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&sh.s1_done[s], kConsumerWarps);
+            mbar_init(&sh.xchg_bar[s], (uint32_t)C);
+            mbar_init(&sh.rc_ready[s], 1);
+        }
+        for (int s = 0; s < kDoneDepth; ++s) {
+            mbar_init(&sh.s2_done[s], kConsumerWarps + 1);
+            mbar_init(&sh.res_free[s], 1);
+        }
+        sh.abort = 0;
         fence_barrier_init();
         fence_proxy_async();
-        for (int p = 0; p < npieces; ++p) {
-            const int q0 = p * kPieceChunks;
-            const int nch = min(kPieceChunks, nc - q0);
-            const int e0 = (c0 + q0) * CE;
-            const int elems = min(nch * CE, P.V - e0);
-            const uint32_t bytes = (uint32_t)elems * (uint32_t)sizeof(typename E::type);
-            mbar_expect_tx(&sh.bar[p], bonus ? bytes : 2u * bytes);
-            bulk_load(reinterpret_cast<unsigned char*>(sT) + (size_t)q0 * kChunkBytes, Trow + e0, bytes,
-                      &sh.bar[p]);
-            if (!bonus)
-                bulk_load(reinterpret_cast<unsigned char*>(sD) + (size_t)q0 * kChunkBytes, Drow + e0, bytes,
-                          &sh.bar[p]);
-        }
     }
-    // the thread that will report the row fetches what the accept test needs while the copies fly
-    AcceptOperands aop;
-    aop.valid = false;
-    if (rank == 0 && tid == 0 && !bonus) aop = load_accept_operands<DT>(P, b, i);
-    __syncthreads();          // barriers are initialised before anyone polls them
-    cluster.barrier_arrive(); // matched by the wait before the first remote store: every block of
-                              // the cluster must be running before its shared memory is written
+    // every block of the cluster has initialised its barriers before anyone arrives on them
+    cluster.sync();
 
-    // -- sweep 1 (shared memory): online softmax statistics, one reference per lane
-    LaneStats ls;
-    ls.init(P.c);
-    bool timed_out = false;
-    for (int q = warp; q < nc; q += kWarps) {
-        if (!mbar_wait_bounded(&sh.bar[q / kPieceChunks], 0)) { timed_out = true; break; }
-        const int ebase = (c0 + q) * CE;
-#pragma unroll
-        for (int j = 0; j < kChunkVecs / 32; ++j) {
-            const int vi = j * 32 + lane;
-            if (ebase + vi * VEC < P.V) {
-                float t[VEC];
-                E::unpack(sT[q * kChunkVecs + vi], t);
-                if (!bonus) {
-                    float d[VEC];
-                    E::unpack(sD[q * kChunkVecs + vi], d);
-                    ls.template add_pair<VEC>(t, d, P.c);
-                } else {
-                    ls.template add_bonus<VEC>(t, P.c);
+    if (warp == kProducerWarp) {
+        // ---- producer: one thread keeps the ring full
+        if (lane == 0) {
+            RingPos pos{0, 0};
+            int n_issued = 0;
+            bool ok = true;
+            for (int j = 0; j < nu && ok; ++j) {
+                const int unit = u0 + j;
+                const int b = unit / K1, i = unit - b * K1;
+                const bool bonus = (i == P.k);
+                const ET* Trow = reinterpret_cast<const ET*>(P.T) + (size_t)unit * P.V + (size_t)vb0 * VEC;
+                const ET* Drow = reinterpret_cast<const ET*>(P.D) + (size_t)(b * P.k + (bonus ? 0 : i)) * P.V +
+                                 (size_t)vb0 * VEC;
+                for (int s = 0; s < ns; ++s) {
+                    if (!mbar_wait_thread<false>(&sh.empty[pos.slot], pos.phase ^ 1u, abort)) { ok = false; break; }
+                    const int v0 = s * kStageVecs;
+                    const uint32_t bytes = (uint32_t)min(kStageVecs, nvb - v0) * 16u;
+                    unsigned char* dst = ring + (size_t)pos.slot * kStageBytes;
+                    mbar_expect_tx(&sh.full[pos.slot], bonus ? bytes : 2u * bytes);
+                    bulk_load(dst, Trow + (size_t)v0 * VEC, bytes, &sh.full[pos.slot]);
+                    if (!bonus) bulk_load(dst + kStageRowBytes, Drow + (size_t)v0 * VEC, bytes, &sh.full[pos.slot]);
+                    ++n_issued;
+                    pos.advance(1, R);
+                }
+            }
+            if (!ok || *abort) {
+                // giving up: no copy may still be in flight when the block returns
+                for (int s = 0; s < R && s < n_issued; ++s) {
+                    const uint32_t last_phase = (uint32_t)((n_issued - 1 - s) / R) & 1u;   // of the slot's last use
+                    for (uint32_t it = 0; it < kWaitLimit && !mbar_try_wait(&sh.full[s], last_phase); ++it) {}
                 }
             }
         }
-    }
-    if (timed_out && lane == 0) atomicOr(&P.wstatus[b], kStatusTimeout);
-    const PartialStats mine = block_reduce_stats(ls, P.c, sh.stat);   // same in every thread
-
-    // -- block statistics to every block of the cluster
-    cluster.barrier_wait();
-    if (warp == 0 && lane < C) *cluster.map_shared_rank(&sh.xchg[rank], lane) = mine;
-    cluster.sync();   // all partials of the row are now in this block's shared memory
-
-    if (warp == 0) {
-        const PartialStats row = warp_merge_partials(sh.xchg, C, P.c);
-        const RowConst rcw = row_constants(P, bonus, row);
-        if (lane == 0) sh.rc = rcw;
-        __syncwarp();
-        // one thread of the cluster reports the row: loss, accept flag, constants for the resolver
-        if (rank == 0 && lane == 0) finish_row(P, b, i, row, rcw, aop);
-    }
-    __syncthreads();
-    const RowConst rc = sh.rc;
-
-    // -- sweep 2 (shared memory): gradient out, residual / bonus mass per sampling chunk
-    typename E::type* Grow =
-        P.grad ? reinterpret_cast<typename E::type*>(P.grad) + (size_t)(b * P.k + (bonus ? 0 : i)) * P.V
-               : nullptr;
-    float* csum = P.chunk_sums + (size_t)unit * P.NC;
-    for (int q = warp; q < nc; q += kWarps) {
-        const int ebase = (c0 + q) * CE;
-        float mass = 0.f;
+    } else if (warp == kStatsWarp) {
+        // ---- statistics: block partial -> cluster exchange -> row constants
+        for (int j = 0; j < nu; ++j) {
+            const int unit = u0 + j;
+            const bool bonus = (unit % K1 == P.k);
+            const int par = j & 1;
+            const uint32_t ph = (uint32_t)(j >> 1) & 1u;
+            const int dslot = j % kDoneDepth;
+            if (!mbar_wait(&sh.s1_done[par], ph, abort)) break;
+            // lane l adds up half of the lanes of consumer warp l%16 (they share that warp's
+            // references) in fp64; the 32 halves then meet in shared memory
+            {
+                const int w = lane & 15, h0 = (lane >> 4) * 16;
+                double sT = 0.0, sD = 0.0, wv = 0.0;
 #pragma unroll
-        for (int j = 0; j < kChunkVecs / 32; ++j) {
-            const int vi = j * 32 + lane;
-            const int e = ebase + vi * VEC;
-            if (e < P.V) {
-                float t[VEC];
-                E::unpack(sT[q * kChunkVecs + vi], t);
-                if (!bonus) {
-                    float d[VEC], g[VEC];
-                    E::unpack(sD[q * kChunkVecs + vi], d);
+                for (int l = 0; l < 16; ++l) {
+                    sT += (double)sh.lane_sums[par][0][w][h0 + l];
+                    sD += (double)sh.lane_sums[par][1][w][h0 + l];
+                    wv += (double)sh.lane_sums[par][2][w][h0 + l];
+                }
+                sT += shfl_xor_f64(sT, 16);
+                sD += shfl_xor_f64(sD, 16);
+                wv += shfl_xor_f64(wv, 16);
+                if (lane < kConsumerWarps) {
+                    PartialStats wp;
+                    wp.RT = sh.warp_ref[par][w][0];
+                    wp.RD = sh.warp_ref[par][w][1];
+                    wp.sT = sT; wp.sD = sD; wp.w = wv;
+                    sh.wpart[lane] = wp;
+                }
+            }
+            __syncwarp();
+            const PartialStats mine = merge_partials_serial(sh.wpart, kConsumerWarps);
+            __syncwarp();
+            if (lane < C) {
+                *cluster.map_shared_rank(&sh.xchg[par][rank], lane) = mine;
+                mbar_arrive_remote(&sh.xchg_bar[par], (uint32_t)lane);
+            }
+            if (!mbar_wait_cluster(&sh.xchg_bar[par], ph, abort)) break;
+            const PartialStats row = merge_partials_serial(sh.xchg[par], C);
+            const RowConst rcw = row_constants(P, bonus, row);
+            if (lane == 0) {
+                sh.rc[par] = rcw;
+                mbar_arrive(&sh.rc_ready[par]);
+                // for the row report by the resolver: wait until it is done with the slot's last use
+                bool ok = true;
+                if (j >= kDoneDepth)
+                    ok = mbar_wait_thread<false>(&sh.res_free[dslot], (uint32_t)(j / kDoneDepth - 1) & 1u, abort);
+                if (ok) {
+                    sh.row[dslot] = row;
+                    sh.rc_done[dslot] = rcw;
+                    mbar_arrive(&sh.s2_done[dslot]);
+                }
+            }
+            if (__any_sync(0xffffffffu, *abort)) break;
+        }
+    } else if (warp == kResolverWarp) {
+        // ---- resolver: region sums, row reports, tickets; the sequence's last tickets draw the token
+        int seg = 0;                               // units of the current sequence finished so far
+        for (int j = 0; j < nu; ++j) {
+            const int unit = u0 + j;
+            const int b = unit / K1, i = unit - b * K1;
+            const bool bonus = (i == P.k);
+            const int dslot = j % kDoneDepth;
+            const bool reports = (j % C == rank);   // the blocks of the cluster take turns
+            AcceptOperands aop;
+            aop.valid = false;
+            if (reports && lane == 0 && !bonus) aop = load_accept_operands<DT>(P, b, i);
+            if (!mbar_wait(&sh.s2_done[dslot], (uint32_t)(j / kDoneDepth) & 1u, abort)) break;
+            // mass of this block's 16 regions of the row: lane l adds up half of warp l%16's lanes
+            {
+                const int w = lane & 15, h0 = (lane >> 4) * 16;
+                float ms = 0.f;
 #pragma unroll
-                    for (int z = 0; z < VEC; ++z) {
-                        g[z] = grad_elem(t[z], d[z], P.c, rc);
-                        mass += fmaxf(-g[z], 0.f);
+                for (int l = 0; l < 16; ++l) ms += sh.lane_mass[dslot][w][h0 + l];
+                ms += __shfl_xor_sync(0xffffffffu, ms, 16);
+                const int region = rank * kConsumerWarps + w;
+                if (lane < kConsumerWarps && region < P.NR) P.region_sums[(size_t)unit * P.NR + region] = ms;
+            }
+            if (reports && lane == 0) finish_row(P, b, i, sh.row[dslot], sh.rc_done[dslot], aop);
+            __syncwarp();
+            ++seg;
+            const bool leaves = (i == P.k) || (j == nu - 1);   // last unit of the sequence in this cluster
+            if (leaves) {
+                int last = 0;
+                if (lane == 0) last = take_tickets(P, b, (uint32_t)seg) ? 1 : 0;
+                last = __shfl_sync(0xffffffffu, last, 0);
+                if (last) resolve_sequence<DT>(P, b);
+                seg = 0;
+                __syncwarp();
+            }
+            if (lane == 0) mbar_arrive(&sh.res_free[dslot]);
+        }
+    } else {
+        // ---- consumers: warp cw owns region 16*rank + cw of every row, m groups of 32 vectors
+        const int cw = warp - kFirstConsumerWarp;
+        const int g0 = cw * m;                                   // first group of the region in the slice
+        const int ng = max(0, min(m, (nvb - g0 * 32 + 31) / 32));   // groups of the region that exist
+        RingPos p1{0, 0}, p2{0, 0};                              // stage 0 of the unit in sweep 1 / sweep 2
+        bool ok = true;
+        for (int j = 0; j < nu + lag && ok; ++j) {
+            if (j < nu) {
+                // sweep 1 of unit j.  Pass A: the region's maxima; pass B: sums relative to them.
+                const bool bonus = ((u0 + j) % K1 == P.k);
+                float mT = -3.402823466e+38f, mD = -3.402823466e+38f;
+                int waited = -1;
+                for (int t = 0; t < ng; ++t) {
+                    const int g = g0 + t, st = g >> 4;
+                    const RingPos rp = p1.plus(st, R);
+                    if (st > waited) {
+                        if (!mbar_wait(&sh.full[rp.slot], rp.phase, abort)) { ok = false; break; }
+                        waited = st;
                     }
-                    if (Grow) store_streaming(Grow + e, E::pack(g));
-                } else {
-#pragma unroll
-                    for (int z = 0; z < VEC; ++z) mass += prob_elem(t[z], P.c, rc);
+                    const int vi = (g & 15) * 32 + lane;
+                    if (g * 32 + lane < nvb) {
+                        const uint4* sT = reinterpret_cast<const uint4*>(ring + (size_t)rp.slot * kStageBytes);
+                        float tv[VEC];
+                        E::unpack(sT[vi], tv);
+                        mT = fmaxf(mT, tree_max<VEC>(tv));
+                        if (!bonus) {
+                            float dv[VEC];
+                            E::unpack(sT[kStageVecs + vi], dv);
+                            mD = fmaxf(mD, tree_max<VEC>(dv));
+                        }
+                    }
                 }
+                if (!ok) break;
+                const float RT = warp_max_ref(ref_of(mT, P.c));
+                const float RD = bonus ? kEmptyRef : warp_max_ref(ref_of(mD, P.c));
+                LaneSums ls;
+                ls.init();
+                for (int t = 0; t < ng; ++t) {
+                    const int g = g0 + t;
+                    const RingPos rp = p1.plus(g >> 4, R);
+                    const int vi = (g & 15) * 32 + lane;
+                    if (g * 32 + lane < nvb) {
+                        const uint4* sT = reinterpret_cast<const uint4*>(ring + (size_t)rp.slot * kStageBytes);
+                        float tv[VEC];
+                        E::unpack(sT[vi], tv);
+                        if (!bonus) {
+                            float dv[VEC];
+                            E::unpack(sT[kStageVecs + vi], dv);
+                            ls.template add_pair<VEC>(tv, dv, P.c, -RT, -RD);
+                        } else {
+                            ls.template add_bonus<VEC>(tv, P.c, -RT);
+                        }
+                    }
+                }
+                const int par = j & 1;
+                sh.lane_sums[par][0][cw][lane] = ls.sT;
+                sh.lane_sums[par][1][cw][lane] = ls.sD;
+                sh.lane_sums[par][2][cw][lane] = ls.w;
+                if (lane == 0) { sh.warp_ref[par][cw][0] = RT; sh.warp_ref[par][cw][1] = RD; }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.s1_done[par]);
+                p1.advance(ns, R);
+            }
+            if (j >= lag) {
+                // sweep 2 of unit j-lag over the stages that are still resident
+                const int jj = j - lag;
+                const int unit = u0 + jj;
+                const int b = unit / K1, i = unit - b * K1;
+                const bool bonus = (i == P.k);
+                const int dslot = jj % kDoneDepth;
+                if (!mbar_wait(&sh.rc_ready[jj & 1], (uint32_t)(jj >> 1) & 1u, abort)) { ok = false; break; }
+                const RowConst rc = sh.rc[jj & 1];
+                ET* Grow = (P.grad && !bonus)
+                               ? reinterpret_cast<ET*>(P.grad) + (size_t)(b * P.k + i) * P.V + (size_t)vb0 * VEC
+                               : nullptr;
+                float mass = 0.f;
+                int arrived = 0;      // stages of the unit this warp has handed back
+                for (int t = 0; t < ng; ++t) {
+                    const int g = g0 + t, st = g >> 4;
+                    if (arrived < st) {
+                        __syncwarp();
+                        if (lane == 0)
+                            for (int s = arrived; s < st; ++s) mbar_arrive(&sh.empty[p2.plus(s, R).slot]);
+                        arrived = st;
+                    }
+                    const RingPos rp = p2.plus(st, R);
+                    const int vi = (g & 15) * 32 + lane;
+                    if (g * 32 + lane < nvb) {
+                        const uint4* sT = reinterpret_cast<const uint4*>(ring + (size_t)rp.slot * kStageBytes);
+                        float tv[VEC], r[VEC];
+                        E::unpack(sT[vi], tv);
+                        if (!bonus) {
+                            float dv[VEC], gv[VEC];
+                            E::unpack(sT[kStageVecs + vi], dv);
+#pragma unroll
+                            for (int z = 0; z < VEC; ++z) {
+                                gv[z] = grad_elem(tv[z], dv[z], P.c, rc);
+                                r[z] = fmaxf(-gv[z], 0.f);
+                            }
+                            if (Grow) store_streaming(Grow + (size_t)(g * 32 + lane) * VEC, E::pack(gv));
+                        } else {
+#pragma unroll
+                            for (int z = 0; z < VEC; ++z) r[z] = prob_elem(tv[z], P.c, rc);
+                        }
+                        mass += tree_sum<VEC>(r);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0)
+                    for (int s = arrived; s < ns; ++s) mbar_arrive(&sh.empty[p2.plus(s, R).slot]);
+                // the resolver must be done with the slot's last use before the masses are replaced
+                if (jj >= kDoneDepth &&
+                    !mbar_wait(&sh.res_free[dslot], (uint32_t)(jj / kDoneDepth - 1) & 1u, abort)) { ok = false; break; }
+                sh.lane_mass[dslot][cw][lane] = mass;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.s2_done[dslot]);
+                p2.advance(ns, R);
             }
         }
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) mass += __shfl_xor_sync(0xffffffffu, mass, off);
-        if (lane == 0) csum[c0 + q] = mass;
     }
 
-    // -- last block of the sequence resolves it
-    if (take_ticket(P, b, &sh.rs.ticket_last)) resolve_sequence<DT>(P, b, sh.rs);
+    __syncthreads();
+    if (sh.abort) {
+        // a wait gave up: say so in every sequence this cluster has a unit of, and in every
+        // sequence resolved from now on
+        if (tid == 0) atomicExch(P.sticky, 1u);
+        if (P.status)
+            for (int j = tid; j < nu; j += kStreamThreads) atomicOr(P.status + (u0 + j) / K1, kStatusTimeout);
+    }
+    // no block leaves while another may still write to its shared memory
+    cluster.sync();
 }
 
 // ---- generic path --------------------------------------------------------------------------
 struct GenericShared {
-    StatScratch stat;
+    float wmax[2][kGenericWarps];
+    PartialStats warp_part[kGenericWarps];
     RowConst rc;
-    ResolveScratch rs;
+    int last;
 };
 
 template <int DT>
-__global__ void __launch_bounds__(kThreads) sd_generic_kernel(const Params P) {
+__global__ void __launch_bounds__(kGenericThreads) sd_generic_kernel(const __grid_constant__ Params P) {
     using E = Elem<DT>;
-    constexpr int VEC = E::VEC;
-    constexpr int CE = kChunkVecs * VEC;
     __shared__ GenericShared sh;
 
     const int unit = blockIdx.x;
@@ -239,27 +516,38 @@ __global__ void __launch_bounds__(kThreads) sd_generic_kernel(const Params P) {
     const size_t offT = (size_t)unit * P.V;
     const size_t offD = (size_t)(b * P.k + (bonus ? 0 : i)) * P.V;
 
-    // sweep 1: statistics; lanes take consecutive elements
-    LaneStats ls;
-    ls.init(P.c);
-    for (int q = warp; q < P.NC; q += kWarps) {
-        const int ebase = q * CE;
-        for (int j = lane; j < CE; j += 32) {
-            const int v = ebase + j;
-            if (v < P.V) {
-                float t[1] = {E::load(P.T, offT + v)};
-                if (!bonus) {
-                    float d[1] = {E::load(P.D, offD + v)};
-                    ls.template add_pair<1>(t, d, P.c);
-                } else {
-                    ls.template add_bonus<1>(t, P.c);
-                }
-            }
+    // sweep 0: the row maxima give the references of every exponential
+    float mT = -3.402823466e+38f, mD = -3.402823466e+38f;
+    for (int v = tid; v < P.V; v += kGenericThreads) {
+        mT = fmaxf(mT, E::load(P.T, offT + v));
+        if (!bonus) mD = fmaxf(mD, E::load(P.D, offD + v));
+    }
+    mT = warp_max_f32(mT);
+    mD = warp_max_f32(mD);
+    if (lane == 0) { sh.wmax[0][warp] = mT; sh.wmax[1][warp] = mD; }
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < kGenericWarps; ++w) { mT = fmaxf(mT, sh.wmax[0][w]); mD = fmaxf(mD, sh.wmax[1][w]); }
+    const float RT = ref_of(mT, P.c), RD = bonus ? kEmptyRef : ref_of(mD, P.c);
+
+    // sweep 1: softmax sums
+    LaneSums ls;
+    ls.init();
+    for (int v = tid; v < P.V; v += kGenericThreads) {
+        float t[1] = {E::load(P.T, offT + v)};
+        if (!bonus) {
+            float d[1] = {E::load(P.D, offD + v)};
+            ls.template add_pair<1>(t, d, P.c, -RT, -RD);
+        } else {
+            ls.template add_bonus<1>(t, P.c, -RT);
         }
     }
     {
-        const PartialStats row = block_reduce_stats(ls, P.c, sh.stat);
+        const PartialStats part = warp_sum_lanes(ls, RT, RD);
+        if (lane == 0) sh.warp_part[warp] = part;
+        __syncthreads();
         if (tid == 0) {
+            const PartialStats row = merge_partials_serial(sh.warp_part, kGenericWarps);
             const RowConst rcw = row_constants(P, bonus, row);
             sh.rc = rcw;
             AcceptOperands aop;
@@ -271,12 +559,12 @@ __global__ void __launch_bounds__(kThreads) sd_generic_kernel(const Params P) {
     __syncthreads();
     const RowConst rc = sh.rc;
 
-    // sweep 2: gradient and chunk sums
-    float* csum = P.chunk_sums + (size_t)unit * P.NC;
-    for (int q = warp; q < P.NC; q += kWarps) {
-        const int ebase = q * CE;
+    // sweep 2: gradient and region sums, one sampling region per warp at a time
+    float* rsum = P.region_sums + (size_t)unit * P.NR;
+    for (int q = warp; q < P.NR; q += kGenericWarps) {
+        const int ebase = q * P.RE;
         float mass = 0.f;
-        for (int j = lane; j < CE; j += 32) {
+        for (int j = lane; j < P.RE; j += 32) {
             const int v = ebase + j;
             if (v < P.V) {
                 const float t = E::load(P.T, offT + v);
@@ -292,10 +580,14 @@ __global__ void __launch_bounds__(kThreads) sd_generic_kernel(const Params P) {
         }
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) mass += __shfl_xor_sync(0xffffffffu, mass, off);
-        if (lane == 0) csum[q] = mass;
+        if (lane == 0) rsum[q] = mass;
     }
 
-    if (take_ticket(P, b, &sh.rs.ticket_last)) resolve_sequence<DT>(P, b, sh.rs);
+    // the block that takes the sequence's last ticket resolves it
+    __syncthreads();
+    if (tid == 0) sh.last = take_tickets(P, b, 1u) ? 1 : 0;
+    __syncthreads();
+    if (sh.last && warp == 0) resolve_sequence<DT>(P, b);
 }
 
 }  // namespace sdv
