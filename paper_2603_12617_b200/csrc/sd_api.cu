@@ -15,10 +15,9 @@ using namespace sdv;
 
 constexpr int kMaxDevices = 64;
 constexpr size_t kAlign = 256;
-constexpr int kRingStages = 12;                   // 12 x 16 KiB + control block < 227 KiB per block
-constexpr int kStreamSmem = kRingStages * kStageBytes + (int)sizeof(StreamShared);
-static_assert(kRingStages <= kMaxStages, "ring larger than the control block allows");
+constexpr int kStreamSmem = kRingSlots * kStageBytes + (int)sizeof(StreamShared);
 static_assert(kStreamSmem <= 227 * 1024, "ring does not fit the shared memory of a block");
+constexpr double kL2BudgetMiB = 48.0;             // slices in flight between their two passes should fit this
 
 thread_local char tl_cuda_error[256] = "";
 thread_local int tl_info[6] = {0, 0, 0, 0, 0, 0};
@@ -84,6 +83,7 @@ struct DeviceState {
     // last launch-shape decision of the fast path
     int dec_dtype = -1, dec_V = 0, dec_forced = 0, dec_C = 0, dec_G = 0, dec_lag = 0, dec_per = 0;
     long long dec_units = 0;
+    double dec_l2 = 0.0;
     // host-memory entry point
     StageSet stage[2];
     cudaStream_t s_h2d = nullptr, s_comp = nullptr, s_d2h = nullptr;
@@ -153,7 +153,7 @@ int launch_stream(DeviceState& d, const Params& P, int C, int G, int lag, cudaSt
         *max_clusters = n;
         return SD_OK;
     }
-    SD_CUDA(cudaLaunchKernelEx(&cfg, kern, P, (int)kRingStages, lag));
+    SD_CUDA(cudaLaunchKernelEx(&cfg, kern, P, lag));
     tl_info[0] = 1; tl_info[1] = C; tl_info[2] = kStreamThreads; tl_info[3] = kStreamSmem;
     tl_info[4] = G * C; tl_info[5] = 1;
     return SD_OK;
@@ -170,32 +170,40 @@ int launch_generic(const Params& P, cudaStream_t stream) {
 }
 
 // Launch shape of the fast path: cluster size C (0 if the fast path cannot run), number of
-// clusters G, vectors per sampling region, and whether sweep 2 may lag one unit behind sweep 1.
+// clusters G, vectors per sampling region, and whether pass 2 of a unit is scheduled after pass 1
+// of the next one.
 //
 // With C blocks of 16 consumer warps a row of NV vectors is cut into regions of
-// per = 32*ceil(NV/(C*512)) vectors; a block's slice is then m = per/32 stages, which must fit the
-// ring, and two slices must fit for the lag.  Among the cluster sizes that qualify, take the one
-// that keeps most blocks busy (resident clusters, but no more clusters than units), prefer the
-// lag, then the smaller cluster.
+// per = 32*max(4, ceil(NV/(C*512))) vectors.  A block's slice lives in L2 between its two passes,
+// so the row pairs all resident clusters have in flight (two each, with the lag) should fit a
+// part of L2.  Among the cluster sizes that qualify, take the one that keeps most blocks busy
+// (resident clusters, but no more clusters than units), then the smaller cluster: larger slices
+// spread the per-unit costs (exchange, row report) over more bytes.  If none qualifies, the
+// largest cluster.
 int choose_stream(DeviceState& d, int V, long long units, int dtype, int* G_out, int* per_out, int* lag_out) {
     const char* env = getenv("SD_VERIFY_CLUSTER");
     const int forced = env ? atoi(env) : 0;
-    if (d.dec_dtype == dtype && d.dec_V == V && d.dec_units == units && d.dec_forced == forced) {
+    const char* env_l2 = getenv("SD_VERIFY_L2_MIB");
+    const double l2_budget = (env_l2 ? atof(env_l2) : kL2BudgetMiB) * 1048576.0;
+    if (d.dec_dtype == dtype && d.dec_V == V && d.dec_units == units && d.dec_forced == forced &&
+        d.dec_l2 == l2_budget) {
         *G_out = d.dec_G;
         *per_out = d.dec_per;
         *lag_out = d.dec_lag;
         return d.dec_C;
     }
     const int NV = V / vec_elems(dtype);
-    int best_C = 0, best_G = 0, best_lag = 0, best_per = 0;
+    const int lag = 1;
+    int best_C = 0, best_G = 0, best_per = 0;
     long long best_busy = -1;
+    bool best_fits = false;
     Params dummy;
     memset(&dummy, 0, sizeof dummy);
     for (int ci = 0, C = 1; C <= kMaxCluster; ++ci, C *= 2) {
         if (forced > 0 && C != forced) continue;
         const int slice = C * kConsumerWarps * 32;
-        const int m = (NV + slice - 1) / slice;
-        if (m > kRingStages) continue;
+        int m = (NV + slice - 1) / slice;
+        if (m < kStageGroups) m = kStageGroups;
         if (d.max_clusters[dtype][ci] < 0) {
             int n = 0;
             int rc = dtype == SD_DTYPE_F32 ? launch_stream<SD_DTYPE_F32>(d, dummy, C, 1, 0, nullptr, true, &n)
@@ -205,17 +213,20 @@ int choose_stream(DeviceState& d, int V, long long units, int dtype, int* G_out,
         const int resident = d.max_clusters[dtype][ci];
         if (resident < 1) continue;
         const int G = (int)(units < resident ? units : resident);
-        const int lag = (2 * m <= kRingStages) ? 1 : 0;
         const int used = (NV + kConsumerWarps * 32 * m - 1) / (kConsumerWarps * 32 * m);   // blocks with work
-        const long long busy = (long long)G * used;
-        const bool better = busy > best_busy || (busy == best_busy && lag > best_lag);
-        if (better) { best_C = C; best_G = G; best_lag = lag; best_per = 32 * m; best_busy = busy; }
+        const long long busy = (long long)G * (used < C ? used : C);
+        const double in_flight = (double)G * (double)NV * 16.0 * 2.0 * (1 + lag);
+        const bool fits = in_flight <= l2_budget;
+        // a shape that fits L2 beats one that does not; then more busy blocks; then the smaller cluster
+        const bool better = best_C == 0 || (fits && !best_fits) || (fits == best_fits && busy > best_busy) ||
+                            (!fits && !best_fits);
+        if (better) { best_C = C; best_G = G; best_per = 32 * m; best_busy = busy; best_fits = fits; }
     }
-    d.dec_dtype = dtype; d.dec_V = V; d.dec_units = units; d.dec_forced = forced;
-    d.dec_C = best_C; d.dec_G = best_G; d.dec_lag = best_lag; d.dec_per = best_per;
+    d.dec_dtype = dtype; d.dec_V = V; d.dec_units = units; d.dec_forced = forced; d.dec_l2 = l2_budget;
+    d.dec_C = best_C; d.dec_G = best_G; d.dec_lag = lag; d.dec_per = best_per;
     *G_out = best_G;
     *per_out = best_per;
-    *lag_out = best_lag;
+    *lag_out = lag;
     return best_C;
 }
 

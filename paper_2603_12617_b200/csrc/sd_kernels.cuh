@@ -2,16 +2,18 @@
 //
 //   sd_stream_kernel   fast path.  A persistent kernel of thread-block clusters.  A cluster takes a
 //                      contiguous range of (sequence, row) units, one after the other; each block
-//                      of the cluster owns a contiguous slice of the vocabulary.  Inside a block
-//                      the warps are specialised:
-//                        producer   one thread streams the block's slices of successive units into
-//                                   a ring of shared-memory stages with bulk asynchronous copies
-//                                   (cp.async.bulk + mbarrier), running ahead as far as the ring
-//                                   allows, so HBM never waits for arithmetic;
-//                        consumers  sweep 1 over a slice (maxima, then softmax sums relative to
-//                                   integer references), later sweep 2 over the same stages, still
-//                                   resident (gradient out, residual mass per lane), then hand the
-//                                   stages back;
+//                      of the cluster owns a contiguous slice of the vocabulary, and each of its
+//                      16 consumer warps a contiguous part of that slice (a sampling region).
+//                      A slice is streamed through a ring of small shared-memory stages twice:
+//                      pass 1 (maxima, then softmax sums relative to integer references) reads it
+//                      from HBM, pass 2 (gradient out, residual mass) reads it again a few
+//                      microseconds later, when it is still in L2, so HBM sees each logit once.
+//                      Inside a block the warps are specialised:
+//                        producer   its lanes issue the bulk asynchronous copies (cp.async.bulk +
+//                                   mbarrier) of both passes in consumption order, running ahead
+//                                   as far as the ring allows, so memory never waits for arithmetic;
+//                        consumers  each works through the stages of its own region and hands
+//                                   them back; warps meet only once per unit and pass;
 //                        statistics adds up the consumers' sums, exchanges the block's partial
 //                                   with the other blocks of the cluster through distributed
 //                                   shared memory (remote stores + remote mbarrier arrivals, no
@@ -20,8 +22,8 @@
 //                                   rows (loss, rejection test), takes the sequence's tickets when
 //                                   the block leaves a sequence and, if they were the last ones,
 //                                   draws the extra token.
-//                      Sweep 2 of a unit runs one unit behind sweep 1 when the ring holds two
-//                      slices, which hides the exchange.  HBM sees each logit once.
+//                      Pass 2 of a unit is scheduled after pass 1 of the next unit (lag 1), which
+//                      hides the exchange.
 //   sd_generic_kernel  any V and any alignment.  One block per unit, sweeps over global memory
 //                      with element loads.  Same arithmetic, same workspace, same resolver.
 //
@@ -35,15 +37,16 @@
 namespace sdv {
 
 // ---- geometry of the fast path -------------------------------------------------------------
-// A row is cut into sampling regions of `per` 16-byte vectors (per = 32*m).  Block r of a
-// cluster owns the 16 regions [16r, 16r+16) of every row it works on, one per consumer warp;
-// the block's slice is streamed through the ring in stages of 512 vectors (8 KiB) per row, so
-// a full slice is m stages and group g of 32 vectors of the slice lies in stage g/16.
+// A row is cut into sampling regions of `per` 16-byte vectors (per = 32*m, m >= 4).  Block r of
+// a cluster owns the 16 regions [16r, 16r+16) of every row it works on, one per consumer warp.
+// The block's slice is streamed in stages of 128 vectors (2 KiB) per row, so group g of 32 vectors
+// of the slice lies in stage g/4, and a stage is used by one consumer warp or by two neighbours.
 constexpr int kConsumerWarps = 16;
-constexpr int kStageVecs = 512;                               // vectors of one row in a stage
-constexpr int kStageRowBytes = kStageVecs * 16;               // 8 KiB of one row
+constexpr int kStageGroups = 4;                               // groups of 32 vectors in a stage
+constexpr int kStageVecs = 32 * kStageGroups;                 // vectors of one row in a stage
+constexpr int kStageRowBytes = kStageVecs * 16;               // 2 KiB of one row
 constexpr int kStageBytes = 2 * kStageRowBytes;               // target part + draft part
-constexpr int kMaxStages = 12;
+constexpr int kRingSlots = 48;                                // 192 KiB
 constexpr int kDoneDepth = 4;                                 // units the resolver may lag behind
 constexpr int kProducerWarp = 0, kStatsWarp = 1, kResolverWarp = 2, kFirstConsumerWarp = 3;
 constexpr int kStreamThreads = (kFirstConsumerWarp + kConsumerWarps) * 32;
@@ -63,6 +66,17 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 }
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_n(uint64_t* bar, uint32_t n) {
+    asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(n) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_acquire_shared(const uint32_t* p) {
+    uint32_t v;
+    asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_shared(uint32_t* p, uint32_t v) {
+    asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
 }
 // Arrival on the barrier at the same shared-memory offset in block `rank` of the cluster; orders
 // this thread's earlier (remote) stores before it at cluster scope.
@@ -124,15 +138,26 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
 __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, volatile int* abort) {
     return __all_sync(0xffffffffu, mbar_wait_thread<true>(bar, parity, abort) ? 1 : 0) != 0;
 }
-// 1-D bulk copy global -> shared of this block, completion counted on `bar`.
-// Both addresses 16-byte aligned, bytes a multiple of 16.
+// 1-D bulk copy global -> shared of this block, completion counted on `bar`, with an L2 eviction
+// policy.  Both addresses 16-byte aligned, bytes a multiple of 16.
 __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, uint32_t bytes,
-                                          uint64_t* bar) {
+                                          uint64_t* bar, uint64_t policy) {
     asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
             smem_u32(dst_smem)),
-        "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar))
+        "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
         : "memory");
+}
+// L2 policies: keep (a line that will be read again shortly) and drop (a line nobody reads again).
+__device__ __forceinline__ uint64_t policy_keep() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t policy_drop() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
 }
 __device__ __forceinline__ void fence_barrier_init() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -147,8 +172,9 @@ __device__ __forceinline__ void store_streaming(void* p, const uint4& v) {
 
 // Control block of the fast path; lives in dynamic shared memory after the ring.
 struct StreamShared {
-    uint64_t full[kMaxStages];          // stage filled by the bulk copies        (1 arrival + bytes)
-    uint64_t empty[kMaxStages];         // stage handed back after sweep 2        (consumer warps)
+    uint64_t full[kRingSlots];          // stage filled by the bulk copies        (1 arrival + bytes)
+    uint64_t empty[kRingSlots];         // stage handed back                      (2: its one or two users)
+    uint32_t issued[kRingSlots];        // uses of the slot whose copies have been issued so far
     uint64_t s1_done[2];                // consumers' sums of a unit posted       (consumer warps)
     uint64_t xchg_bar[2];               // partials of every block have arrived   (cluster size, remote)
     uint64_t rc_ready[2];               // row constants published                (1)
@@ -165,21 +191,6 @@ struct StreamShared {
     int abort;                          // a bounded wait gave up somewhere in this block
 };
 
-// Position of a stage in the ring: slot index and the parity of its current use.
-struct RingPos {
-    int slot;
-    uint32_t phase;
-    __device__ __forceinline__ void advance(int n, int R) {
-        slot += n;
-        if (slot >= R) { slot -= R; phase ^= 1u; }
-    }
-    __device__ __forceinline__ RingPos plus(int n, int R) const {
-        RingPos r = *this;
-        r.advance(n, R);
-        return r;
-    }
-};
-
 // Units [u0, u0+n) of cluster `cid` of `G`: contiguous, sizes differ by at most one.
 __device__ __host__ __forceinline__ void cluster_units(int units, int G, int cid, int& u0, int& n) {
     const int base = units / G, rem = units % G;
@@ -187,15 +198,32 @@ __device__ __host__ __forceinline__ void cluster_units(int units, int G, int cid
     u0 = cid * base + (cid < rem ? cid : rem);
 }
 
+// The passes of a block in the order in which it streams them: with lag 1,
+// S1(0) S1(1) S2(0) S1(2) S2(1) ... S1(n-1) S2(n-2) S2(n-1); with lag 0, S1(0) S2(0) S1(1) ...
+struct PassOrder {
+    int nu, lag;
+    __device__ __forceinline__ int count() const { return 2 * nu; }
+    __device__ __forceinline__ int index_s1(int j) const { return lag ? (j == 0 ? 0 : 2 * j - 1) : 2 * j; }
+    __device__ __forceinline__ int index_s2(int j) const { return lag ? (j == nu - 1 ? 2 * nu - 1 : 2 * j + 2) : 2 * j + 1; }
+    // unit and kind (0 = pass 1, 1 = pass 2) of pass p
+    __device__ __forceinline__ void decode(int p, int& j, int& kind) const {
+        if (!lag) { j = p >> 1; kind = p & 1; return; }
+        if (p == 0) { j = 0; kind = 0; }
+        else if (p == 2 * nu - 1) { j = nu - 1; kind = 1; }
+        else if (p & 1) { j = (p + 1) >> 1; kind = 0; }
+        else { j = (p >> 1) - 1; kind = 1; }
+    }
+};
+
 // ---- fast path -----------------------------------------------------------------------------
-// R: stages of the ring (every slice has at most R stages).  lag: 1 if sweep 2 runs one unit
-// behind sweep 1 (needs a ring of at least two slices), else 0.
+// lag: 1 if pass 2 of a unit is scheduled after pass 1 of the next unit, else 0.
 template <int DT>
 __global__ void __launch_bounds__(kStreamThreads, 1)
-sd_stream_kernel(const __grid_constant__ Params P, const int R, const int lag) {
+sd_stream_kernel(const __grid_constant__ Params P, const int lag) {
     using E = Elem<DT>;
     using ET = typename E::type;
     constexpr int VEC = E::VEC;
+    constexpr int R = kRingSlots;
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     unsigned char* ring = dyn_smem;
     StreamShared& sh = *reinterpret_cast<StreamShared*>(dyn_smem + (size_t)R * kStageBytes);
@@ -211,15 +239,17 @@ sd_stream_kernel(const __grid_constant__ Params P, const int R, const int lag) {
     cluster_units(P.B * K1, G, cid, u0, nu);      // this cluster works on units u0 .. u0+nu-1
 
     const int per = P.RE / VEC;                   // vectors per sampling region
-    const int m = per >> 5;                       // groups of 32 vectors per region = stages per full slice
+    const int m = per >> 5;                       // groups of 32 vectors per region
     const int NV = P.V / VEC;                     // vectors per row
     const int vb0 = rank * kConsumerWarps * per;  // first vector of this block's slice
     const int nvb = max(0, min(NV - vb0, kConsumerWarps * per));
-    const int ns = (nvb + kStageVecs - 1) / kStageVecs;
+    const int ns = (nvb + kStageVecs - 1) / kStageVecs;   // stages of a pass
+    const int tg = (nvb + 31) >> 5;                       // groups of the slice
+    const PassOrder order{nu, lag};
     volatile int* abort = &sh.abort;
 
     if (tid == 0) {
-        for (int s = 0; s < R; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], kConsumerWarps); }
+        for (int s = 0; s < R; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 2); sh.issued[s] = 0; }
         for (int s = 0; s < 2; ++s) {
             mbar_init(&sh.s1_done[s], kConsumerWarps);
             mbar_init(&sh.xchg_bar[s], (uint32_t)C);
@@ -237,35 +267,48 @@ sd_stream_kernel(const __grid_constant__ Params P, const int R, const int lag) {
     cluster.sync();
 
     if (warp == kProducerWarp) {
-        // ---- producer: one thread keeps the ring full
-        if (lane == 0) {
-            RingPos pos{0, 0};
-            int n_issued = 0;
-            bool ok = true;
-            for (int j = 0; j < nu && ok; ++j) {
-                const int unit = u0 + j;
-                const int b = unit / K1, i = unit - b * K1;
-                const bool bonus = (i == P.k);
-                const ET* Trow = reinterpret_cast<const ET*>(P.T) + (size_t)unit * P.V + (size_t)vb0 * VEC;
-                const ET* Drow = reinterpret_cast<const ET*>(P.D) + (size_t)(b * P.k + (bonus ? 0 : i)) * P.V +
-                                 (size_t)vb0 * VEC;
-                for (int s = 0; s < ns; ++s) {
-                    if (!mbar_wait_thread<false>(&sh.empty[pos.slot], pos.phase ^ 1u, abort)) { ok = false; break; }
-                    const int v0 = s * kStageVecs;
-                    const uint32_t bytes = (uint32_t)min(kStageVecs, nvb - v0) * 16u;
-                    unsigned char* dst = ring + (size_t)pos.slot * kStageBytes;
-                    mbar_expect_tx(&sh.full[pos.slot], bonus ? bytes : 2u * bytes);
-                    bulk_load(dst, Trow + (size_t)v0 * VEC, bytes, &sh.full[pos.slot]);
-                    if (!bonus) bulk_load(dst + kStageRowBytes, Drow + (size_t)v0 * VEC, bytes, &sh.full[pos.slot]);
-                    ++n_issued;
-                    pos.advance(1, R);
-                }
+        // ---- producer: lane l issues the copies of the stages that go to ring slots l and l+32,
+        // in the order of their sequence numbers q (stage s of pass p has q = p*ns + s, slot q % R)
+        const uint64_t keep = policy_keep(), drop = policy_drop();
+        const long long total = (long long)order.count() * ns;   // stages this block streams
+        bool ok = true;
+        long long q_last = -1;
+        long long qa = lane, qb = (lane + 32 < R) ? (long long)(lane + 32) : total;
+        while (ok) {
+            const long long q = qa < qb ? qa : qb;
+            if (q >= total) break;
+            if (q == qa) qa += R; else qb += R;
+            const int slot = (int)(q % R);
+            const uint32_t use = (uint32_t)(q / R);
+            const int p = (int)(q / ns), s = (int)(q - (long long)p * ns);
+            int j, kind;
+            order.decode(p, j, kind);
+            const int unit = u0 + j;
+            const int b = unit / K1, i = unit - b * K1;
+            const bool bonus = (i == P.k);
+            if (use > 0 && !mbar_wait_thread<false>(&sh.empty[slot], (use - 1) & 1u, abort)) { ok = false; break; }
+            const int v0 = s * kStageVecs;
+            const uint32_t bytes = (uint32_t)min(kStageVecs, nvb - v0) * 16u;
+            const ET* Tsrc = reinterpret_cast<const ET*>(P.T) + (size_t)unit * P.V + (size_t)(vb0 + v0) * VEC;
+            unsigned char* dst = ring + (size_t)slot * kStageBytes;
+            const uint64_t pol = kind == 0 ? keep : drop;
+            mbar_expect_tx(&sh.full[slot], bonus ? bytes : 2u * bytes);
+            bulk_load(dst, Tsrc, bytes, &sh.full[slot], pol);
+            if (!bonus) {
+                const ET* Dsrc = reinterpret_cast<const ET*>(P.D) + (size_t)(b * P.k + i) * P.V + (size_t)(vb0 + v0) * VEC;
+                bulk_load(dst + kStageRowBytes, Dsrc, bytes, &sh.full[slot], pol);
             }
-            if (!ok || *abort) {
-                // giving up: no copy may still be in flight when the block returns
-                for (int s = 0; s < R && s < n_issued; ++s) {
-                    const uint32_t last_phase = (uint32_t)((n_issued - 1 - s) / R) & 1u;   // of the slot's last use
-                    for (uint32_t it = 0; it < kWaitLimit && !mbar_try_wait(&sh.full[s], last_phase); ++it) {}
+            st_release_shared(&sh.issued[slot], use + 1u);
+            q_last = q;
+        }
+        if (__any_sync(0xffffffffu, !ok || *abort)) {
+            // giving up: no copy may still be in flight when the block returns
+            for (int slot = lane; slot < R; slot += 32) {
+                long long q = -1;                       // last use this lane issued into the slot
+                for (long long t = slot; t <= q_last; t += R) q = t;
+                if (q >= 0) {
+                    const uint32_t par = (uint32_t)(q / R) & 1u;
+                    for (uint32_t it = 0; it < kWaitLimit && !mbar_try_wait(&sh.full[slot], par); ++it) {}
                 }
             }
         }
@@ -279,7 +322,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int R, const int lag) {
             const int dslot = j % kDoneDepth;
             if (!mbar_wait(&sh.s1_done[par], ph, abort)) break;
             // lane l adds up half of the lanes of consumer warp l%16 (they share that warp's
-            // references) in fp64; the 32 halves then meet in shared memory
+            // references) in fp64; the 16 warp partials then meet in shared memory
             {
                 const int w = lane & 15, h0 = (lane >> 4) * 16;
                 double sT = 0.0, sD = 0.0, wv = 0.0;
@@ -363,28 +406,67 @@ sd_stream_kernel(const __grid_constant__ Params P, const int R, const int lag) {
             if (lane == 0) mbar_arrive(&sh.res_free[dslot]);
         }
     } else {
-        // ---- consumers: warp cw owns region 16*rank + cw of every row, m groups of 32 vectors
+        // ---- consumers: warp cw owns region 16*rank + cw of every row: groups [g0, g0+ng) of the slice
         const int cw = warp - kFirstConsumerWarp;
-        const int g0 = cw * m;                                   // first group of the region in the slice
-        const int ng = max(0, min(m, (nvb - g0 * 32 + 31) / 32));   // groups of the region that exist
-        RingPos p1{0, 0}, p2{0, 0};                              // stage 0 of the unit in sweep 1 / sweep 2
+        const int g0 = cw * m;
+        const int ng = max(0, min(m, tg - g0));
+        const int s_first = g0 / kStageGroups, s_last = (g0 + ng - 1) / kStageGroups;   // stages of the region
+        // a stage shared with the neighbouring warp is handed back by both, each counting once
+        const uint32_t w_first = (g0 % kStageGroups != 0) ? 1u : 2u;
+        const uint32_t w_last = ((g0 + ng) % kStageGroups != 0 && g0 + ng < tg) ? 1u : 2u;
+        auto slot_of = [&](int p, int s, uint32_t& use) -> int {
+            const long long q = (long long)p * ns + s;
+            use = (uint32_t)(q / R);
+            return (int)(q % R);
+        };
+        // Wait for use `use` of a slot.  Consumer warps run up to two passes apart, more than the
+        // ring holds, so the parity of the barrier alone could be taken for that of an older use:
+        // first wait until the copies of this very use have been issued (which happens only after
+        // the previous use was handed back), then for them to land.
+        auto wait_stage = [&](int slot, uint32_t use) -> bool {
+            bool seen = false;
+            long long t0 = 0;
+            for (uint32_t it = 0; it < kWaitLimit; ++it) {
+                if (ld_acquire_shared(&sh.issued[slot]) > use) { seen = true; break; }
+                if ((it & 63u) == 63u) {
+                    if (*abort) break;
+                    const long long now = clock64();
+                    if (t0 == 0) t0 = now;
+                    else if (now - t0 > kWaitCycles) break;
+                }
+            }
+            if (!seen) *abort = 1;
+            if (!__all_sync(0xffffffffu, seen ? 1 : 0)) return false;
+            return mbar_wait(&sh.full[slot], use & 1u, abort);
+        };
+        auto release = [&](int p, int s) {
+            uint32_t use;
+            const int slot = slot_of(p, s, use);
+            uint32_t n = 2u;
+            if (s == s_first && s == s_last) n = (w_first == 1u || w_last == 1u) ? 1u : 2u;
+            else if (s == s_first) n = w_first;
+            else if (s == s_last) n = w_last;
+            mbar_arrive_n(&sh.empty[slot], n);
+        };
         bool ok = true;
         for (int j = 0; j < nu + lag && ok; ++j) {
             if (j < nu) {
-                // sweep 1 of unit j.  Pass A: the region's maxima; pass B: sums relative to them.
+                // pass 1 of unit j.  Sweep A: the region's maxima; sweep B: sums relative to them.
                 const bool bonus = ((u0 + j) % K1 == P.k);
+                const int p = order.index_s1(j);
                 float mT = -3.402823466e+38f, mD = -3.402823466e+38f;
                 int waited = -1;
                 for (int t = 0; t < ng; ++t) {
-                    const int g = g0 + t, st = g >> 4;
-                    const RingPos rp = p1.plus(st, R);
+                    const int g = g0 + t, st = g / kStageGroups;
+                    uint32_t use;
+                    const int slot = slot_of(p, st, use);
                     if (st > waited) {
-                        if (!mbar_wait(&sh.full[rp.slot], rp.phase, abort)) { ok = false; break; }
+                        if (!wait_stage(slot, use)) { ok = false; break; }
                         waited = st;
                     }
-                    const int vi = (g & 15) * 32 + lane;
+                    const int vi = (g % kStageGroups) * 32 + lane;
                     if (g * 32 + lane < nvb) {
-                        const uint4* sT = reinterpret_cast<const uint4*>(ring + (size_t)rp.slot * kStageBytes);
+                        const uint4* sT = reinterpret_cast<const uint4*>(ring + (size_t)slot * kStageBytes);
                         float tv[VEC];
                         E::unpack(sT[vi], tv);
                         mT = fmaxf(mT, tree_max<VEC>(tv));
@@ -402,10 +484,11 @@ sd_stream_kernel(const __grid_constant__ Params P, const int R, const int lag) {
                 ls.init();
                 for (int t = 0; t < ng; ++t) {
                     const int g = g0 + t;
-                    const RingPos rp = p1.plus(g >> 4, R);
-                    const int vi = (g & 15) * 32 + lane;
+                    uint32_t use;
+                    const int slot = slot_of(p, g / kStageGroups, use);
+                    const int vi = (g % kStageGroups) * 32 + lane;
                     if (g * 32 + lane < nvb) {
-                        const uint4* sT = reinterpret_cast<const uint4*>(ring + (size_t)rp.slot * kStageBytes);
+                        const uint4* sT = reinterpret_cast<const uint4*>(ring + (size_t)slot * kStageBytes);
                         float tv[VEC];
                         E::unpack(sT[vi], tv);
                         if (!bonus) {
@@ -417,41 +500,48 @@ sd_stream_kernel(const __grid_constant__ Params P, const int R, const int lag) {
                         }
                     }
                 }
-                const int par = j & 1;
-                sh.lane_sums[par][0][cw][lane] = ls.sT;
-                sh.lane_sums[par][1][cw][lane] = ls.sD;
-                sh.lane_sums[par][2][cw][lane] = ls.w;
-                if (lane == 0) { sh.warp_ref[par][cw][0] = RT; sh.warp_ref[par][cw][1] = RD; }
+                const int parj = j & 1;
+                sh.lane_sums[parj][0][cw][lane] = ls.sT;
+                sh.lane_sums[parj][1][cw][lane] = ls.sD;
+                sh.lane_sums[parj][2][cw][lane] = ls.w;
+                if (lane == 0) { sh.warp_ref[parj][cw][0] = RT; sh.warp_ref[parj][cw][1] = RD; }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sh.s1_done[par]);
-                p1.advance(ns, R);
+                if (lane == 0) {
+                    if (ng > 0)
+                        for (int s = s_first; s <= s_last; ++s) release(p, s);
+                    mbar_arrive(&sh.s1_done[parj]);
+                }
             }
             if (j >= lag) {
-                // sweep 2 of unit j-lag over the stages that are still resident
+                // pass 2 of unit j-lag
                 const int jj = j - lag;
                 const int unit = u0 + jj;
                 const int b = unit / K1, i = unit - b * K1;
                 const bool bonus = (i == P.k);
                 const int dslot = jj % kDoneDepth;
+                const int p = order.index_s2(jj);
                 if (!mbar_wait(&sh.rc_ready[jj & 1], (uint32_t)(jj >> 1) & 1u, abort)) { ok = false; break; }
                 const RowConst rc = sh.rc[jj & 1];
                 ET* Grow = (P.grad && !bonus)
                                ? reinterpret_cast<ET*>(P.grad) + (size_t)(b * P.k + i) * P.V + (size_t)vb0 * VEC
                                : nullptr;
                 float mass = 0.f;
-                int arrived = 0;      // stages of the unit this warp has handed back
+                int cur = -1;         // stage being worked on
                 for (int t = 0; t < ng; ++t) {
-                    const int g = g0 + t, st = g >> 4;
-                    if (arrived < st) {
-                        __syncwarp();
-                        if (lane == 0)
-                            for (int s = arrived; s < st; ++s) mbar_arrive(&sh.empty[p2.plus(s, R).slot]);
-                        arrived = st;
+                    const int g = g0 + t, st = g / kStageGroups;
+                    uint32_t use;
+                    const int slot = slot_of(p, st, use);
+                    if (st != cur) {
+                        if (cur >= 0) {
+                            __syncwarp();
+                            if (lane == 0) release(p, cur);
+                        }
+                        if (!wait_stage(slot, use)) { ok = false; break; }
+                        cur = st;
                     }
-                    const RingPos rp = p2.plus(st, R);
-                    const int vi = (g & 15) * 32 + lane;
+                    const int vi = (g % kStageGroups) * 32 + lane;
                     if (g * 32 + lane < nvb) {
-                        const uint4* sT = reinterpret_cast<const uint4*>(ring + (size_t)rp.slot * kStageBytes);
+                        const uint4* sT = reinterpret_cast<const uint4*>(ring + (size_t)slot * kStageBytes);
                         float tv[VEC], r[VEC];
                         E::unpack(sT[vi], tv);
                         if (!bonus) {
@@ -470,16 +560,15 @@ sd_stream_kernel(const __grid_constant__ Params P, const int R, const int lag) {
                         mass += tree_sum<VEC>(r);
                     }
                 }
+                if (!ok) break;
                 __syncwarp();
-                if (lane == 0)
-                    for (int s = arrived; s < ns; ++s) mbar_arrive(&sh.empty[p2.plus(s, R).slot]);
+                if (lane == 0 && cur >= 0) release(p, cur);
                 // the resolver must be done with the slot's last use before the masses are replaced
                 if (jj >= kDoneDepth &&
                     !mbar_wait(&sh.res_free[dslot], (uint32_t)(jj / kDoneDepth - 1) & 1u, abort)) { ok = false; break; }
                 sh.lane_mass[dslot][cw][lane] = mass;
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.s2_done[dslot]);
-                p2.advance(ns, R);
             }
         }
     }
