@@ -173,13 +173,12 @@ int launch_generic(const Params& P, cudaStream_t stream) {
 // clusters G, vectors per sampling region, and whether pass 2 of a unit is scheduled after pass 1
 // of the next one.
 //
-// With C blocks of 16 consumer warps a row of NV vectors is cut into regions of
-// per = 32*max(4, ceil(NV/(C*512))) vectors.  A block's slice lives in L2 between its two passes,
-// so the row pairs all resident clusters have in flight (two each, with the lag) should fit a
-// part of L2.  Among the cluster sizes that qualify, take the one that keeps most blocks busy
-// (resident clusters, but no more clusters than units), then the smaller cluster: larger slices
-// spread the per-unit costs (exchange, row report) over more bytes.  If none qualifies, the
-// largest cluster.
+// A row is cut into stages of 128 vectors and block r of a cluster of C takes every C-th share of
+// them.  A block's slice lives in L2 between its two passes, so the row pairs all resident
+// clusters have in flight (two each, with the lag) should fit a part of L2.  Among the cluster
+// sizes that qualify, take the one that keeps most blocks busy (resident clusters, but no more
+// clusters than units), then the smaller cluster: larger slices spread the per-unit costs
+// (exchange, row report) over more bytes.  If none qualifies, the largest cluster.
 int choose_stream(DeviceState& d, int V, long long units, int dtype, int* G_out, int* per_out, int* lag_out) {
     const char* env = getenv("SD_VERIFY_CLUSTER");
     const int forced = env ? atoi(env) : 0;
@@ -201,9 +200,8 @@ int choose_stream(DeviceState& d, int V, long long units, int dtype, int* G_out,
     memset(&dummy, 0, sizeof dummy);
     for (int ci = 0, C = 1; C <= kMaxCluster; ++ci, C *= 2) {
         if (forced > 0 && C != forced) continue;
-        const int slice = C * kConsumerWarps * 32;
-        int m = (NV + slice - 1) / slice;
-        if (m < kStageGroups) m = kStageGroups;
+        const int stages_row = (NV + kStageVecs - 1) / kStageVecs;
+        const int stages_blk = (stages_row + C - 1) / C;
         if (d.max_clusters[dtype][ci] < 0) {
             int n = 0;
             int rc = dtype == SD_DTYPE_F32 ? launch_stream<SD_DTYPE_F32>(d, dummy, C, 1, 0, nullptr, true, &n)
@@ -213,14 +211,14 @@ int choose_stream(DeviceState& d, int V, long long units, int dtype, int* G_out,
         const int resident = d.max_clusters[dtype][ci];
         if (resident < 1) continue;
         const int G = (int)(units < resident ? units : resident);
-        const int used = (NV + kConsumerWarps * 32 * m - 1) / (kConsumerWarps * 32 * m);   // blocks with work
+        const int used = (stages_row + stages_blk - 1) / stages_blk;   // blocks with work
         const long long busy = (long long)G * (used < C ? used : C);
         const double in_flight = (double)G * (double)NV * 16.0 * 2.0 * (1 + lag);
         const bool fits = in_flight <= l2_budget;
         // a shape that fits L2 beats one that does not; then more busy blocks; then the smaller cluster
         const bool better = best_C == 0 || (fits && !best_fits) || (fits == best_fits && busy > best_busy) ||
                             (!fits && !best_fits);
-        if (better) { best_C = C; best_G = G; best_per = 32 * m; best_busy = busy; best_fits = fits; }
+        if (better) { best_C = C; best_G = G; best_per = kStageVecs; best_busy = busy; best_fits = fits; }
     }
     d.dec_dtype = dtype; d.dec_V = V; d.dec_units = units; d.dec_forced = forced; d.dec_l2 = l2_budget;
     d.dec_C = best_C; d.dec_G = best_G; d.dec_lag = lag; d.dec_per = best_per;

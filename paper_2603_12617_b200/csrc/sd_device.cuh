@@ -153,6 +153,12 @@ __device__ __forceinline__ double pow2_neg(float d) {
     return e < -1022 ? 0.0 : __hiloint2double((1023 + e) << 20, 0);
 }
 
+// The same as a float; 0 below the normal range.
+__device__ __forceinline__ float pow2_neg_f32(float d) {
+    const int e = (int)fmaxf(d, -200.f);
+    return e < -126 ? 0.f : __int_as_float((127 + e) << 23);
+}
+
 // Sum of VEC values as a balanced tree (short dependency chains, fixed order).
 template <int VEC>
 __device__ __forceinline__ float tree_sum(const float (&v)[VEC]) {
@@ -174,6 +180,13 @@ __device__ __forceinline__ float tree_max(const float (&v)[VEC]) {
 struct LaneSums {
     float sT, sD, w;
     __device__ __forceinline__ void init() { sT = sD = w = 0.f; }
+    // Move the sums to references larger by dT >= 0 and dD >= 0 (integers): exact.
+    __device__ __forceinline__ void rescale(float dT, float dD) {
+        const float f = pow2_neg_f32(-dT), g = pow2_neg_f32(-dD);
+        w = (sT > 0.f) ? (w - sT * (dT - dD)) * f : 0.f;
+        sT *= f;
+        sD *= g;
+    }
     template <int VEC>
     __device__ __forceinline__ void add_pair(const float (&t)[VEC], const float (&d)[VEC], float c, float negRT,
                                              float negRD) {

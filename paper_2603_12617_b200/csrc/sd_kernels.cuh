@@ -2,24 +2,22 @@
 //
 //   sd_stream_kernel   fast path.  A persistent kernel of thread-block clusters.  A cluster takes a
 //                      contiguous range of (sequence, row) units, one after the other; each block
-//                      of the cluster owns a contiguous slice of the vocabulary, and each of its
-//                      16 consumer warps a contiguous part of that slice (a sampling region).
+//                      of the cluster owns a contiguous slice of the vocabulary, cut into stages
+//                      of 2 KiB per row that its 16 consumer warps take in turn.
 //                      A slice is streamed through a ring of small shared-memory stages twice:
 //                      pass 1 (maxima, then softmax sums relative to integer references) reads it
 //                      from HBM, pass 2 (gradient out, residual mass) reads it again a few
 //                      microseconds later, when it is still in L2, so HBM sees each logit once.
 //                      Inside a block the warps are specialised:
-//                        producer   its lanes issue the bulk asynchronous copies (cp.async.bulk +
-//                                   mbarrier) of both passes in consumption order, running ahead
-//                                   as far as the ring allows, so memory never waits for arithmetic;
-//                        consumers  each works through the stages of its own region and hands
-//                                   them back; warps meet only once per unit and pass;
+//                        consumers  each works through its own stages, which it fetches itself into
+//                                   a private ring of three slots with bulk asynchronous copies
+//                                   (cp.async.bulk + mbarrier), always three stages ahead, across
+//                                   passes and units; warps meet only once per unit and pass;
 //                        statistics adds up the consumers' sums, exchanges the block's partial
 //                                   with the other blocks of the cluster through distributed
 //                                   shared memory (remote stores + remote mbarrier arrivals, no
 //                                   cluster-wide barrier) and publishes the row constants;
-//                        resolver   turns the lanes' residual masses into region sums, reports
-//                                   rows (loss, rejection test), takes the sequence's tickets when
+//                        resolver   reports rows (loss, rejection test), takes the sequence's tickets when
 //                                   the block leaves a sequence and, if they were the last ones,
 //                                   draws the extra token.
 //                      Pass 2 of a unit is scheduled after pass 1 of the next unit (lag 1), which
@@ -37,18 +35,19 @@
 namespace sdv {
 
 // ---- geometry of the fast path -------------------------------------------------------------
-// A row is cut into sampling regions of `per` 16-byte vectors (per = 32*m, m >= 4).  Block r of
-// a cluster owns the 16 regions [16r, 16r+16) of every row it works on, one per consumer warp.
-// The block's slice is streamed in stages of 128 vectors (2 KiB) per row, so group g of 32 vectors
-// of the slice lies in stage g/4, and a stage is used by one consumer warp or by two neighbours.
+// A row is cut into stages of 128 16-byte vectors (2 KiB); a stage is also a sampling region.
+// Block r of a cluster of C owns the stages [r*S, (r+1)*S) of every row it works on, S =
+// ceil(stages per row / C); stage s of the slice belongs to consumer warp s % 16, so sixteen
+// consecutive stages are worked on at the same time.  Every consumer warp has a ring of its own.
 constexpr int kConsumerWarps = 16;
 constexpr int kStageGroups = 4;                               // groups of 32 vectors in a stage
 constexpr int kStageVecs = 32 * kStageGroups;                 // vectors of one row in a stage
 constexpr int kStageRowBytes = kStageVecs * 16;               // 2 KiB of one row
 constexpr int kStageBytes = 2 * kStageRowBytes;               // target part + draft part
-constexpr int kRingSlots = 48;                                // 192 KiB
+constexpr int kWarpSlots = 3;                                 // stages a consumer warp has in flight or in use
+constexpr int kRingSlots = kConsumerWarps * kWarpSlots;       // 48 slots, 192 KiB
 constexpr int kDoneDepth = 4;                                 // units the resolver may lag behind
-constexpr int kProducerWarp = 0, kStatsWarp = 1, kResolverWarp = 2, kFirstConsumerWarp = 3;
+constexpr int kStatsWarp = 0, kResolverWarp = 1, kFirstConsumerWarp = 2;
 constexpr int kStreamThreads = (kFirstConsumerWarp + kConsumerWarps) * 32;
 constexpr int kGenericWarps = 8;
 constexpr int kGenericThreads = kGenericWarps * 32;
@@ -66,17 +65,6 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 }
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_n(uint64_t* bar, uint32_t n) {
-    asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(n) : "memory");
-}
-__device__ __forceinline__ uint32_t ld_acquire_shared(const uint32_t* p) {
-    uint32_t v;
-    asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
-    return v;
-}
-__device__ __forceinline__ void st_release_shared(uint32_t* p, uint32_t v) {
-    asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
 }
 // Arrival on the barrier at the same shared-memory offset in block `rank` of the cluster; orders
 // this thread's earlier (remote) stores before it at cluster scope.
@@ -148,15 +136,15 @@ __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, 
         "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
         : "memory");
 }
-// L2 policies: keep (a line that will be read again shortly) and drop (a line nobody reads again).
+// L2 policies: keep (a line that will be read again shortly) and the default.
 __device__ __forceinline__ uint64_t policy_keep() {
     uint64_t p;
     asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
     return p;
 }
-__device__ __forceinline__ uint64_t policy_drop() {
+__device__ __forceinline__ uint64_t policy_normal() {
     uint64_t p;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
     return p;
 }
 __device__ __forceinline__ void fence_barrier_init() {
@@ -173,8 +161,6 @@ __device__ __forceinline__ void store_streaming(void* p, const uint4& v) {
 // Control block of the fast path; lives in dynamic shared memory after the ring.
 struct StreamShared {
     uint64_t full[kRingSlots];          // stage filled by the bulk copies        (1 arrival + bytes)
-    uint64_t empty[kRingSlots];         // stage handed back                      (2: its one or two users)
-    uint32_t issued[kRingSlots];        // uses of the slot whose copies have been issued so far
     uint64_t s1_done[2];                // consumers' sums of a unit posted       (consumer warps)
     uint64_t xchg_bar[2];               // partials of every block have arrived   (cluster size, remote)
     uint64_t rc_ready[2];               // row constants published                (1)
@@ -182,7 +168,6 @@ struct StreamShared {
     uint64_t res_free[kDoneDepth];      // resolver is done with the unit         (1)
     float lane_sums[2][3][kConsumerWarps][33];        // sT, sD, w of every consumer lane (33: no bank conflicts)
     float warp_ref[2][kConsumerWarps][2];             // RT, RD each consumer warp used
-    float lane_mass[kDoneDepth][kConsumerWarps][33];  // residual / bonus mass of every consumer lane
     PartialStats wpart[kConsumerWarps]; // the consumer warps' partials of the unit being merged
     PartialStats xchg[2][kMaxCluster];  // written by every block of the cluster (distributed shared memory)
     PartialStats row[kDoneDepth];       // statistics of the whole row, for the row report
@@ -238,18 +223,18 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag) {
     int u0, nu;
     cluster_units(P.B * K1, G, cid, u0, nu);      // this cluster works on units u0 .. u0+nu-1
 
-    const int per = P.RE / VEC;                   // vectors per sampling region
-    const int m = per >> 5;                       // groups of 32 vectors per region
     const int NV = P.V / VEC;                     // vectors per row
-    const int vb0 = rank * kConsumerWarps * per;  // first vector of this block's slice
-    const int nvb = max(0, min(NV - vb0, kConsumerWarps * per));
-    const int ns = (nvb + kStageVecs - 1) / kStageVecs;   // stages of a pass
-    const int tg = (nvb + 31) >> 5;                       // groups of the slice
+    const int stages_row = (NV + kStageVecs - 1) / kStageVecs;   // = sampling regions per row
+    const int stages_blk = (stages_row + C - 1) / C;
+    const int s0 = rank * stages_blk;             // first stage (region) of this block's slice
+    const int ns = max(0, min(stages_row - s0, stages_blk));     // stages of a pass
+    const int vb0 = s0 * kStageVecs;              // first vector of the slice
+    const int nvb = max(0, min(NV - vb0, ns * kStageVecs));
     const PassOrder order{nu, lag};
     volatile int* abort = &sh.abort;
 
     if (tid == 0) {
-        for (int s = 0; s < R; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 2); sh.issued[s] = 0; }
+        for (int s = 0; s < R; ++s) mbar_init(&sh.full[s], 1);
         for (int s = 0; s < 2; ++s) {
             mbar_init(&sh.s1_done[s], kConsumerWarps);
             mbar_init(&sh.xchg_bar[s], (uint32_t)C);
@@ -266,53 +251,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag) {
     // every block of the cluster has initialised its barriers before anyone arrives on them
     cluster.sync();
 
-    if (warp == kProducerWarp) {
-        // ---- producer: lane l issues the copies of the stages that go to ring slots l and l+32,
-        // in the order of their sequence numbers q (stage s of pass p has q = p*ns + s, slot q % R)
-        const uint64_t keep = policy_keep(), drop = policy_drop();
-        const long long total = (long long)order.count() * ns;   // stages this block streams
-        bool ok = true;
-        long long q_last = -1;
-        long long qa = lane, qb = (lane + 32 < R) ? (long long)(lane + 32) : total;
-        while (ok) {
-            const long long q = qa < qb ? qa : qb;
-            if (q >= total) break;
-            if (q == qa) qa += R; else qb += R;
-            const int slot = (int)(q % R);
-            const uint32_t use = (uint32_t)(q / R);
-            const int p = (int)(q / ns), s = (int)(q - (long long)p * ns);
-            int j, kind;
-            order.decode(p, j, kind);
-            const int unit = u0 + j;
-            const int b = unit / K1, i = unit - b * K1;
-            const bool bonus = (i == P.k);
-            if (use > 0 && !mbar_wait_thread<false>(&sh.empty[slot], (use - 1) & 1u, abort)) { ok = false; break; }
-            const int v0 = s * kStageVecs;
-            const uint32_t bytes = (uint32_t)min(kStageVecs, nvb - v0) * 16u;
-            const ET* Tsrc = reinterpret_cast<const ET*>(P.T) + (size_t)unit * P.V + (size_t)(vb0 + v0) * VEC;
-            unsigned char* dst = ring + (size_t)slot * kStageBytes;
-            const uint64_t pol = kind == 0 ? keep : drop;
-            mbar_expect_tx(&sh.full[slot], bonus ? bytes : 2u * bytes);
-            bulk_load(dst, Tsrc, bytes, &sh.full[slot], pol);
-            if (!bonus) {
-                const ET* Dsrc = reinterpret_cast<const ET*>(P.D) + (size_t)(b * P.k + i) * P.V + (size_t)(vb0 + v0) * VEC;
-                bulk_load(dst + kStageRowBytes, Dsrc, bytes, &sh.full[slot], pol);
-            }
-            st_release_shared(&sh.issued[slot], use + 1u);
-            q_last = q;
-        }
-        if (__any_sync(0xffffffffu, !ok || *abort)) {
-            // giving up: no copy may still be in flight when the block returns
-            for (int slot = lane; slot < R; slot += 32) {
-                long long q = -1;                       // last use this lane issued into the slot
-                for (long long t = slot; t <= q_last; t += R) q = t;
-                if (q >= 0) {
-                    const uint32_t par = (uint32_t)(q / R) & 1u;
-                    for (uint32_t it = 0; it < kWaitLimit && !mbar_try_wait(&sh.full[slot], par); ++it) {}
-                }
-            }
-        }
-    } else if (warp == kStatsWarp) {
+    if (warp == kStatsWarp) {
         // ---- statistics: block partial -> cluster exchange -> row constants
         for (int j = 0; j < nu; ++j) {
             const int unit = u0 + j;
@@ -369,7 +308,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag) {
             if (__any_sync(0xffffffffu, *abort)) break;
         }
     } else if (warp == kResolverWarp) {
-        // ---- resolver: region sums, row reports, tickets; the sequence's last tickets draw the token
+        // ---- resolver: row reports, tickets; the sequence's last tickets draw the token
         int seg = 0;                               // units of the current sequence finished so far
         for (int j = 0; j < nu; ++j) {
             const int unit = u0 + j;
@@ -381,16 +320,6 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag) {
             aop.valid = false;
             if (reports && lane == 0 && !bonus) aop = load_accept_operands<DT>(P, b, i);
             if (!mbar_wait(&sh.s2_done[dslot], (uint32_t)(j / kDoneDepth) & 1u, abort)) break;
-            // mass of this block's 16 regions of the row: lane l adds up half of warp l%16's lanes
-            {
-                const int w = lane & 15, h0 = (lane >> 4) * 16;
-                float ms = 0.f;
-#pragma unroll
-                for (int l = 0; l < 16; ++l) ms += sh.lane_mass[dslot][w][h0 + l];
-                ms += __shfl_xor_sync(0xffffffffu, ms, 16);
-                const int region = rank * kConsumerWarps + w;
-                if (lane < kConsumerWarps && region < P.NR) P.region_sums[(size_t)unit * P.NR + region] = ms;
-            }
             if (reports && lane == 0) finish_row(P, b, i, sh.row[dslot], sh.rc_done[dslot], aop);
             __syncwarp();
             ++seg;
@@ -406,171 +335,179 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag) {
             if (lane == 0) mbar_arrive(&sh.res_free[dslot]);
         }
     } else {
-        // ---- consumers: warp cw owns region 16*rank + cw of every row: groups [g0, g0+ng) of the slice
+        // ---- consumers: warp cw owns stages cw, cw+16, ... of every pass; a stage is a sampling
+        // region.  The warp walks its stages of all passes in order; stage number n of that walk
+        // goes to slot n % 3 of the warp's own ring, and its copies are issued by the warp's first
+        // lane as soon as stage n-3 has been worked on, whatever pass or unit it belongs to.
         const int cw = warp - kFirstConsumerWarp;
-        const int g0 = cw * m;
-        const int ng = max(0, min(m, tg - g0));
-        const int s_first = g0 / kStageGroups, s_last = (g0 + ng - 1) / kStageGroups;   // stages of the region
-        // a stage shared with the neighbouring warp is handed back by both, each counting once
-        const uint32_t w_first = (g0 % kStageGroups != 0) ? 1u : 2u;
-        const uint32_t w_last = ((g0 + ng) % kStageGroups != 0 && g0 + ng < tg) ? 1u : 2u;
-        auto slot_of = [&](int p, int s, uint32_t& use) -> int {
-            const long long q = (long long)p * ns + s;
-            use = (uint32_t)(q / R);
-            return (int)(q % R);
-        };
-        // Wait for use `use` of a slot.  Consumer warps run up to two passes apart, more than the
-        // ring holds, so the parity of the barrier alone could be taken for that of an older use:
-        // first wait until the copies of this very use have been issued (which happens only after
-        // the previous use was handed back), then for them to land.
-        auto wait_stage = [&](int slot, uint32_t use) -> bool {
-            bool seen = false;
-            long long t0 = 0;
-            for (uint32_t it = 0; it < kWaitLimit; ++it) {
-                if (ld_acquire_shared(&sh.issued[slot]) > use) { seen = true; break; }
-                if ((it & 63u) == 63u) {
-                    if (*abort) break;
-                    const long long now = clock64();
-                    if (t0 == 0) t0 = now;
-                    else if (now - t0 > kWaitCycles) break;
-                }
+        const int nst = cw < ns ? (ns - cw + kConsumerWarps - 1) / kConsumerWarps : 0;   // my stages per pass
+        const int n_total = order.count() * nst;
+        unsigned char* myring = ring + (size_t)cw * kWarpSlots * kStageBytes;
+        uint64_t* myfull = &sh.full[cw * kWarpSlots];
+        const uint64_t keep = policy_keep(), normal = policy_normal();
+        // issue cursor (lane 0 only): next stage to fetch, and where it lies
+        int ni = 0, pi = 0, ti = 0;
+        const ET* Tbase = nullptr;
+        const ET* Dbase = nullptr;
+        int kind_i = 0;
+        auto issue_next = [&]() {     // lane 0
+            if (ni >= n_total) return;
+            if (ti == 0) {            // first stage of a pass: where the pass reads from
+                int j;
+                order.decode(pi, j, kind_i);
+                const int unit = u0 + j;
+                const int b = unit / K1, i = unit - b * K1;
+                Tbase = reinterpret_cast<const ET*>(P.T) + (size_t)unit * P.V + (size_t)vb0 * VEC;
+                Dbase = (i == P.k) ? nullptr
+                                   : reinterpret_cast<const ET*>(P.D) + (size_t)(b * P.k + i) * P.V + (size_t)vb0 * VEC;
             }
-            if (!seen) *abort = 1;
-            if (!__all_sync(0xffffffffu, seen ? 1 : 0)) return false;
-            return mbar_wait(&sh.full[slot], use & 1u, abort);
+            const int s = cw + ti * kConsumerWarps;
+            const int v0 = s * kStageVecs;
+            const uint32_t bytes = (uint32_t)min(kStageVecs, nvb - v0) * 16u;
+            const int slot = ni % kWarpSlots;
+            unsigned char* dst = myring + (size_t)slot * kStageBytes;
+            const uint64_t pol = kind_i == 0 ? keep : normal;
+            mbar_expect_tx(&myfull[slot], Dbase ? 2u * bytes : bytes);
+            bulk_load(dst, Tbase + (size_t)v0 * VEC, bytes, &myfull[slot], pol);
+            if (Dbase) bulk_load(dst + kStageRowBytes, Dbase + (size_t)v0 * VEC, bytes, &myfull[slot], pol);
+            ++ni;
+            if (++ti == nst) { ti = 0; ++pi; }
         };
-        auto release = [&](int p, int s) {
-            uint32_t use;
-            const int slot = slot_of(p, s, use);
-            uint32_t n = 2u;
-            if (s == s_first && s == s_last) n = (w_first == 1u || w_last == 1u) ? 1u : 2u;
-            else if (s == s_first) n = w_first;
-            else if (s == s_last) n = w_last;
-            mbar_arrive_n(&sh.empty[slot], n);
+        if (lane == 0)
+            for (int t = 0; t < kWarpSlots; ++t) issue_next();
+        int n = 0;                    // consume cursor: stages worked on so far
+        // hand the slot of stage n back and fetch stage n+3 into it
+        auto recycle = [&]() {
+            __syncwarp();
+            if (lane == 0) {
+                fence_proxy_async();   // the warp's reads of the slot come before the copy that refills it
+                issue_next();
+            }
+            ++n;
         };
         bool ok = true;
         for (int j = 0; j < nu + lag && ok; ++j) {
             if (j < nu) {
-                // pass 1 of unit j.  Sweep A: the region's maxima; sweep B: sums relative to them.
+                // pass 1 of unit j, stage by stage: the stage's maxima first; if they raise the warp's
+                // integer references, the running sums move to the new references (exact: powers of
+                // two); then the stage's sums.
                 const bool bonus = ((u0 + j) % K1 == P.k);
-                const int p = order.index_s1(j);
-                float mT = -3.402823466e+38f, mD = -3.402823466e+38f;
-                int waited = -1;
-                for (int t = 0; t < ng; ++t) {
-                    const int g = g0 + t, st = g / kStageGroups;
-                    uint32_t use;
-                    const int slot = slot_of(p, st, use);
-                    if (st > waited) {
-                        if (!wait_stage(slot, use)) { ok = false; break; }
-                        waited = st;
-                    }
-                    const int vi = (g % kStageGroups) * 32 + lane;
-                    if (g * 32 + lane < nvb) {
-                        const uint4* sT = reinterpret_cast<const uint4*>(ring + (size_t)slot * kStageBytes);
-                        float tv[VEC];
-                        E::unpack(sT[vi], tv);
-                        mT = fmaxf(mT, tree_max<VEC>(tv));
-                        if (!bonus) {
-                            float dv[VEC];
-                            E::unpack(sT[kStageVecs + vi], dv);
-                            mD = fmaxf(mD, tree_max<VEC>(dv));
-                        }
-                    }
-                }
-                if (!ok) break;
-                const float RT = warp_max_ref(ref_of(mT, P.c));
-                const float RD = bonus ? kEmptyRef : warp_max_ref(ref_of(mD, P.c));
+                float RT = kEmptyRef, RD = kEmptyRef;
                 LaneSums ls;
                 ls.init();
-                for (int t = 0; t < ng; ++t) {
-                    const int g = g0 + t;
-                    uint32_t use;
-                    const int slot = slot_of(p, g / kStageGroups, use);
-                    const int vi = (g % kStageGroups) * 32 + lane;
-                    if (g * 32 + lane < nvb) {
-                        const uint4* sT = reinterpret_cast<const uint4*>(ring + (size_t)slot * kStageBytes);
-                        float tv[VEC];
-                        E::unpack(sT[vi], tv);
-                        if (!bonus) {
-                            float dv[VEC];
-                            E::unpack(sT[kStageVecs + vi], dv);
-                            ls.template add_pair<VEC>(tv, dv, P.c, -RT, -RD);
-                        } else {
-                            ls.template add_bonus<VEC>(tv, P.c, -RT);
+                for (int s = cw; s < ns; s += kConsumerWarps) {
+                    const int slot = n % kWarpSlots;
+                    if (!mbar_wait(&myfull[slot], (uint32_t)(n / kWarpSlots) & 1u, abort)) { ok = false; break; }
+                    const uint4* sT = reinterpret_cast<const uint4*>(myring + (size_t)slot * kStageBytes);
+                    const int nv = min(kStageVecs, nvb - s * kStageVecs);     // vectors of this stage
+                    float mT = -3.402823466e+38f, mD = -3.402823466e+38f;
+#pragma unroll
+                    for (int g = 0; g < kStageGroups; ++g) {
+                        const int vi = g * 32 + lane;
+                        if (vi < nv) {
+                            float tv[VEC];
+                            E::unpack(sT[vi], tv);
+                            mT = fmaxf(mT, tree_max<VEC>(tv));
+                            if (!bonus) {
+                                float dv[VEC];
+                                E::unpack(sT[kStageVecs + vi], dv);
+                                mD = fmaxf(mD, tree_max<VEC>(dv));
+                            }
                         }
                     }
+                    const float nT = fmaxf(RT, warp_max_ref(ref_of(mT, P.c)));
+                    const float nD = bonus ? kEmptyRef : fmaxf(RD, warp_max_ref(ref_of(mD, P.c)));
+                    if (nT > RT || nD > RD) {
+                        ls.rescale(nT - RT, nD - RD);
+                        RT = nT;
+                        RD = nD;
+                    }
+#pragma unroll
+                    for (int g = 0; g < kStageGroups; ++g) {
+                        const int vi = g * 32 + lane;
+                        if (vi < nv) {
+                            float tv[VEC];
+                            E::unpack(sT[vi], tv);
+                            if (!bonus) {
+                                float dv[VEC];
+                                E::unpack(sT[kStageVecs + vi], dv);
+                                ls.template add_pair<VEC>(tv, dv, P.c, -RT, -RD);
+                            } else {
+                                ls.template add_bonus<VEC>(tv, P.c, -RT);
+                            }
+                        }
+                    }
+                    recycle();
                 }
+                if (!ok) break;
                 const int parj = j & 1;
                 sh.lane_sums[parj][0][cw][lane] = ls.sT;
                 sh.lane_sums[parj][1][cw][lane] = ls.sD;
                 sh.lane_sums[parj][2][cw][lane] = ls.w;
                 if (lane == 0) { sh.warp_ref[parj][cw][0] = RT; sh.warp_ref[parj][cw][1] = RD; }
                 __syncwarp();
-                if (lane == 0) {
-                    if (ng > 0)
-                        for (int s = s_first; s <= s_last; ++s) release(p, s);
-                    mbar_arrive(&sh.s1_done[parj]);
-                }
+                if (lane == 0) mbar_arrive(&sh.s1_done[parj]);
             }
             if (j >= lag) {
-                // pass 2 of unit j-lag
+                // pass 2 of unit j-lag: gradient out, mass of every stage (= sampling region)
                 const int jj = j - lag;
                 const int unit = u0 + jj;
                 const int b = unit / K1, i = unit - b * K1;
                 const bool bonus = (i == P.k);
                 const int dslot = jj % kDoneDepth;
-                const int p = order.index_s2(jj);
                 if (!mbar_wait(&sh.rc_ready[jj & 1], (uint32_t)(jj >> 1) & 1u, abort)) { ok = false; break; }
                 const RowConst rc = sh.rc[jj & 1];
                 ET* Grow = (P.grad && !bonus)
                                ? reinterpret_cast<ET*>(P.grad) + (size_t)(b * P.k + i) * P.V + (size_t)vb0 * VEC
                                : nullptr;
-                float mass = 0.f;
-                int cur = -1;         // stage being worked on
-                for (int t = 0; t < ng; ++t) {
-                    const int g = g0 + t, st = g / kStageGroups;
-                    uint32_t use;
-                    const int slot = slot_of(p, st, use);
-                    if (st != cur) {
-                        if (cur >= 0) {
-                            __syncwarp();
-                            if (lane == 0) release(p, cur);
-                        }
-                        if (!wait_stage(slot, use)) { ok = false; break; }
-                        cur = st;
-                    }
-                    const int vi = (g % kStageGroups) * 32 + lane;
-                    if (g * 32 + lane < nvb) {
-                        const uint4* sT = reinterpret_cast<const uint4*>(ring + (size_t)slot * kStageBytes);
-                        float tv[VEC], r[VEC];
-                        E::unpack(sT[vi], tv);
-                        if (!bonus) {
-                            float dv[VEC], gv[VEC];
-                            E::unpack(sT[kStageVecs + vi], dv);
+                float* rsum = P.region_sums + (size_t)unit * P.NR + s0;
+                for (int s = cw; s < ns; s += kConsumerWarps) {
+                    const int slot = n % kWarpSlots;
+                    if (!mbar_wait(&myfull[slot], (uint32_t)(n / kWarpSlots) & 1u, abort)) { ok = false; break; }
+                    const uint4* sT = reinterpret_cast<const uint4*>(myring + (size_t)slot * kStageBytes);
+                    const int nv = min(kStageVecs, nvb - s * kStageVecs);
+                    float mass = 0.f;
 #pragma unroll
-                            for (int z = 0; z < VEC; ++z) {
-                                gv[z] = grad_elem(tv[z], dv[z], P.c, rc);
-                                r[z] = fmaxf(-gv[z], 0.f);
+                    for (int g = 0; g < kStageGroups; ++g) {
+                        const int vi = g * 32 + lane;
+                        if (vi < nv) {
+                            float tv[VEC], r[VEC];
+                            E::unpack(sT[vi], tv);
+                            if (!bonus) {
+                                float dv[VEC], gv[VEC];
+                                E::unpack(sT[kStageVecs + vi], dv);
+#pragma unroll
+                                for (int z = 0; z < VEC; ++z) {
+                                    gv[z] = grad_elem(tv[z], dv[z], P.c, rc);
+                                    r[z] = fmaxf(-gv[z], 0.f);
+                                }
+                                if (Grow) store_streaming(Grow + (size_t)(s * kStageVecs + vi) * VEC, E::pack(gv));
+                            } else {
+#pragma unroll
+                                for (int z = 0; z < VEC; ++z) r[z] = prob_elem(tv[z], P.c, rc);
                             }
-                            if (Grow) store_streaming(Grow + (size_t)(g * 32 + lane) * VEC, E::pack(gv));
-                        } else {
-#pragma unroll
-                            for (int z = 0; z < VEC; ++z) r[z] = prob_elem(tv[z], P.c, rc);
+                            mass += tree_sum<VEC>(r);
                         }
-                        mass += tree_sum<VEC>(r);
                     }
+#pragma unroll
+                    for (int off = 16; off > 0; off >>= 1) mass += __shfl_xor_sync(0xffffffffu, mass, off);
+                    if (lane == 0) rsum[s] = mass;
+                    recycle();
                 }
                 if (!ok) break;
-                __syncwarp();
-                if (lane == 0 && cur >= 0) release(p, cur);
-                // the resolver must be done with the slot's last use before the masses are replaced
+                // the resolver's slot of unit jj-4 must be free again before this unit is reported done
                 if (jj >= kDoneDepth &&
                     !mbar_wait(&sh.res_free[dslot], (uint32_t)(jj / kDoneDepth - 1) & 1u, abort)) { ok = false; break; }
-                sh.lane_mass[dslot][cw][lane] = mass;
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.s2_done[dslot]);
             }
         }
+        // leaving early: no copy of this warp may still be in flight when the block returns
+        if (!ok && lane == 0)
+            for (int t = n; t < ni; ++t) {
+                const uint32_t par = (uint32_t)(t / kWarpSlots) & 1u;
+                for (uint32_t it = 0; it < kWaitLimit && !mbar_try_wait(&myfull[t % kWarpSlots], par); ++it) {}
+            }
     }
 
     __syncthreads();
