@@ -70,6 +70,7 @@ struct StageSet {
 };
 
 struct DeviceState {
+    DeviceState() { for (auto& row : max_clusters) for (int& v : row) v = -1; }
     std::mutex mu;
     bool probed = false;
     int cc_major = 0;
@@ -79,7 +80,7 @@ struct DeviceState {
     size_t ws_bytes = 0;
     bool ws_clean = false;   // tickets and status words are zero
     bool attr_set[2] = {false, false};   // shared-memory / cluster attributes of the fast kernel
-    int max_clusters[2][5] = {{-1, -1, -1, -1, -1}, {-1, -1, -1, -1, -1}};   // resident clusters of 1,2,4,8,16 blocks
+    int max_clusters[2][kMaxCluster + 1];   // resident clusters of 1..16 blocks, -1 = not asked yet
     // last launch-shape decision of the fast path
     int dec_dtype = -1, dec_V = 0, dec_forced = 0, dec_C = 0, dec_G = 0, dec_lag = 0, dec_per = 0;
     long long dec_units = 0;
@@ -198,7 +199,8 @@ int choose_stream(DeviceState& d, int V, long long units, int dtype, int* G_out,
     bool best_fits = false;
     Params dummy;
     memset(&dummy, 0, sizeof dummy);
-    for (int ci = 0, C = 1; C <= kMaxCluster; ++ci, C *= 2) {
+    for (int C = 1; C <= kMaxCluster; ++C) {
+        const int ci = C;
         if (forced > 0 && C != forced) continue;
         const int stages_row = (NV + kStageVecs - 1) / kStageVecs;
         const int stages_blk = (stages_row + C - 1) / C;

@@ -89,6 +89,9 @@ template <> struct Elem<SD_DTYPE_F32> {
         return make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]),
                           __float_as_uint(v[3]));
     }
+    static __device__ __forceinline__ uint4 masked() {   // a vector of -inf: adds nothing anywhere
+        return make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u);
+    }
     static __device__ __forceinline__ float load(const void* base, size_t idx) {
         return __ldg(reinterpret_cast<const float*>(base) + idx);
     }
@@ -111,6 +114,9 @@ template <> struct Elem<SD_DTYPE_BF16> {
     }
     static __device__ __forceinline__ uint4 pack(const float (&v)[8]) {
         return make_uint4(pack2(v[0], v[1]), pack2(v[2], v[3]), pack2(v[4], v[5]), pack2(v[6], v[7]));
+    }
+    static __device__ __forceinline__ uint4 masked() {
+        return make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
     }
     static __device__ __forceinline__ float load(const void* base, size_t idx) {
         uint16_t h = __ldg(reinterpret_cast<const uint16_t*>(base) + idx);
@@ -166,11 +172,17 @@ __device__ __forceinline__ float tree_sum(const float (&v)[VEC]) {
     else if constexpr (VEC == 4) return (v[0] + v[1]) + (v[2] + v[3]);
     else return ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
 }
+// Largest of three (one instruction on sm_100).
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
 template <int VEC>
 __device__ __forceinline__ float tree_max(const float (&v)[VEC]) {
     if constexpr (VEC == 1) return v[0];
-    else if constexpr (VEC == 4) return fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3]));
-    else return fmaxf(fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3])), fmaxf(fmaxf(v[4], v[5]), fmaxf(v[6], v[7])));
+    else if constexpr (VEC == 4) return fmaxf(fmax3(v[0], v[1], v[2]), v[3]);
+    else return fmax3(fmax3(v[0], v[1], v[2]), fmax3(v[3], v[4], v[5]), fmaxf(v[6], v[7]));
 }
 
 // Softmax sums of one lane relative to integer references that the lane's whole warp shares:
@@ -201,6 +213,31 @@ struct LaneSums {
         sT += tree_sum<VEC>(eT);
         sD += tree_sum<VEC>(eD);
         w += tree_sum<VEC>(pw);
+    }
+    // The same for one vector, into partial sums of its own (short dependency chains).
+    template <int VEC>
+    static __device__ __forceinline__ void vector_pair(const float (&t)[VEC], const float (&d)[VEC], float c,
+                                                       float negRT, float negRD, float& pT, float& pD, float& pW) {
+        float eT[VEC], eD[VEC];
+        float wv = 0.f;
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) {
+            const float aT = __fmaf_rn(t[e], c, negRT), aD = __fmaf_rn(d[e], c, negRD);
+            eT[e] = ex2f(aT);
+            eD[e] = ex2f(aD);
+            const float diff = (eT[e] > 0.f) ? aT - aD : 0.f;   // masked target entries (p = 0) add nothing
+            wv = __fmaf_rn(eT[e], diff, wv);
+        }
+        pT = tree_sum<VEC>(eT);
+        pD = tree_sum<VEC>(eD);
+        pW = wv;
+    }
+    template <int VEC>
+    static __device__ __forceinline__ float vector_bonus(const float (&t)[VEC], float c, float negRT) {
+        float eT[VEC];
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) eT[e] = exp_term(t[e], c, negRT);
+        return tree_sum<VEC>(eT);
     }
     template <int VEC>
     __device__ __forceinline__ void add_bonus(const float (&t)[VEC], float c, float negRT) {

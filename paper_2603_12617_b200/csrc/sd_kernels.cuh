@@ -102,11 +102,12 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t pa
 // whichever comes first, or as soon as another thread of the block has given up (*abort != 0);
 // the caller then leaves its loop and the kernel returns.  A failed poll is followed by a short
 // sleep, so that waiting warps leave the issue slots and the shared-memory pipe to working ones.
-template <bool CLUSTER>
+template <bool CLUSTER, bool SLEEP = false>
 __device__ __forceinline__ bool mbar_wait_thread(uint64_t* bar, uint32_t parity, volatile int* abort) {
     long long t0 = 0;
     for (uint32_t it = 0; it < kWaitLimit; ++it) {
         if (CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
+        if (SLEEP) __nanosleep(64);   // warps with long waits leave the issue slots to the others
         if ((it & 63u) == 63u) {
             if (*abort) return false;
             const long long now = clock64();
@@ -124,7 +125,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     return __all_sync(0xffffffffu, mbar_wait_thread<false>(bar, parity, abort) ? 1 : 0) != 0;
 }
 __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, volatile int* abort) {
-    return __all_sync(0xffffffffu, mbar_wait_thread<true>(bar, parity, abort) ? 1 : 0) != 0;
+    return __all_sync(0xffffffffu, mbar_wait_thread<true, true>(bar, parity, abort) ? 1 : 0) != 0;
+}
+__device__ __forceinline__ bool mbar_wait_sleepy(uint64_t* bar, uint32_t parity, volatile int* abort) {
+    return __all_sync(0xffffffffu, mbar_wait_thread<false, true>(bar, parity, abort) ? 1 : 0) != 0;
 }
 // 1-D bulk copy global -> shared of this block, completion counted on `bar`, with an L2 eviction
 // policy.  Both addresses 16-byte aligned, bytes a multiple of 16.
@@ -156,6 +160,103 @@ __device__ __forceinline__ void fence_proxy_async() {
 __device__ __forceinline__ void store_streaming(void* p, const uint4& v) {
     asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
                  : "memory");
+}
+
+// ---- the two passes over one stage held in shared memory ------------------------------------
+// A stage is 4 vectors per lane and row.  All of them are loaded before any arithmetic; vectors
+// past the end of the row read as -inf, which adds nothing to any sum and is never stored.
+
+// Pass 1: the stage's maxima; if they raise the warp's integer references (RT, RD), the running
+// sums move to the new references (exact: powers of two); then the stage's sums.
+template <int DT, bool BONUS>
+__device__ __forceinline__ void pass1_stage(const uint4* st, int nv, int lane, float c, float& RT, float& RD,
+                                            LaneSums& ls) {
+    using E = Elem<DT>;
+    constexpr int VEC = E::VEC;
+    uint4 rt[kStageGroups], rd[kStageGroups];
+#pragma unroll
+    for (int g = 0; g < kStageGroups; ++g) {
+        const int vi = g * 32 + lane;
+        rt[g] = vi < nv ? st[vi] : E::masked();
+        if (!BONUS) rd[g] = vi < nv ? st[kStageVecs + vi] : E::masked();
+    }
+    float mT[kStageGroups], mD[kStageGroups];
+#pragma unroll
+    for (int g = 0; g < kStageGroups; ++g) {
+        float v[VEC];
+        E::unpack(rt[g], v);
+        mT[g] = tree_max<VEC>(v);
+        if (!BONUS) {
+            E::unpack(rd[g], v);
+            mD[g] = tree_max<VEC>(v);
+        }
+    }
+    const float nT = fmaxf(RT, warp_max_ref(ref_of(fmaxf(fmax3(mT[0], mT[1], mT[2]), mT[3]), c)));
+    const float nD = BONUS ? kEmptyRef : fmaxf(RD, warp_max_ref(ref_of(fmaxf(fmax3(mD[0], mD[1], mD[2]), mD[3]), c)));
+    if (nT > RT || nD > RD) {
+        ls.rescale(nT - RT, nD - RD);
+        RT = nT;
+        RD = nD;
+    }
+    float pT[kStageGroups], pD[kStageGroups], pW[kStageGroups];
+#pragma unroll
+    for (int g = 0; g < kStageGroups; ++g) {
+        float tv[VEC];
+        E::unpack(rt[g], tv);
+        if (!BONUS) {
+            float dv[VEC];
+            E::unpack(rd[g], dv);
+            LaneSums::vector_pair<VEC>(tv, dv, c, -RT, -RD, pT[g], pD[g], pW[g]);
+        } else {
+            pT[g] = LaneSums::vector_bonus<VEC>(tv, c, -RT);
+        }
+    }
+    ls.sT += (pT[0] + pT[1]) + (pT[2] + pT[3]);
+    if (!BONUS) {
+        ls.sD += (pD[0] + pD[1]) + (pD[2] + pD[3]);
+        ls.w += (pW[0] + pW[1]) + (pW[2] + pW[3]);
+    }
+}
+
+// Pass 2: gradient out (gdst = where the stage's part of the gradient row starts, or null) and
+// the stage's mass (sum of max(0,p-q)/tau, or of p on the bonus row), in every lane.
+template <int DT, bool BONUS>
+__device__ __forceinline__ float pass2_stage(const uint4* st, int nv, int lane, float c, const RowConst& rc,
+                                             typename Elem<DT>::type* gdst) {
+    using E = Elem<DT>;
+    constexpr int VEC = E::VEC;
+    uint4 rt[kStageGroups], rd[kStageGroups];
+#pragma unroll
+    for (int g = 0; g < kStageGroups; ++g) {
+        const int vi = g * 32 + lane;
+        rt[g] = vi < nv ? st[vi] : E::masked();
+        if (!BONUS) rd[g] = vi < nv ? st[kStageVecs + vi] : E::masked();
+    }
+    float ms[kStageGroups];
+#pragma unroll
+    for (int g = 0; g < kStageGroups; ++g) {
+        const int vi = g * 32 + lane;
+        float tv[VEC], r[VEC];
+        E::unpack(rt[g], tv);
+        if (!BONUS) {
+            float dv[VEC], gv[VEC];
+            E::unpack(rd[g], dv);
+#pragma unroll
+            for (int z = 0; z < VEC; ++z) {
+                gv[z] = grad_elem(tv[z], dv[z], c, rc);
+                r[z] = fmaxf(-gv[z], 0.f);
+            }
+            if (gdst && vi < nv) store_streaming(gdst + (size_t)vi * VEC, E::pack(gv));
+        } else {
+#pragma unroll
+            for (int z = 0; z < VEC; ++z) r[z] = prob_elem(tv[z], c, rc);
+        }
+        ms[g] = tree_sum<VEC>(r);
+    }
+    float mass = (ms[0] + ms[1]) + (ms[2] + ms[3]);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) mass += __shfl_xor_sync(0xffffffffu, mass, off);
+    return mass;
 }
 
 // Control block of the fast path; lives in dynamic shared memory after the ring.
@@ -259,7 +360,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag) {
             const int par = j & 1;
             const uint32_t ph = (uint32_t)(j >> 1) & 1u;
             const int dslot = j % kDoneDepth;
-            if (!mbar_wait(&sh.s1_done[par], ph, abort)) break;
+            if (!mbar_wait_sleepy(&sh.s1_done[par], ph, abort)) break;
             // lane l adds up half of the lanes of consumer warp l%16 (they share that warp's
             // references) in fp64; the 16 warp partials then meet in shared memory
             {
@@ -319,7 +420,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag) {
             AcceptOperands aop;
             aop.valid = false;
             if (reports && lane == 0 && !bonus) aop = load_accept_operands<DT>(P, b, i);
-            if (!mbar_wait(&sh.s2_done[dslot], (uint32_t)(j / kDoneDepth) & 1u, abort)) break;
+            if (!mbar_wait_sleepy(&sh.s2_done[dslot], (uint32_t)(j / kDoneDepth) & 1u, abort)) break;
             if (reports && lane == 0) finish_row(P, b, i, sh.row[dslot], sh.rc_done[dslot], aop);
             __syncwarp();
             ++seg;
@@ -400,43 +501,8 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag) {
                     if (!mbar_wait(&myfull[slot], (uint32_t)(n / kWarpSlots) & 1u, abort)) { ok = false; break; }
                     const uint4* sT = reinterpret_cast<const uint4*>(myring + (size_t)slot * kStageBytes);
                     const int nv = min(kStageVecs, nvb - s * kStageVecs);     // vectors of this stage
-                    float mT = -3.402823466e+38f, mD = -3.402823466e+38f;
-#pragma unroll
-                    for (int g = 0; g < kStageGroups; ++g) {
-                        const int vi = g * 32 + lane;
-                        if (vi < nv) {
-                            float tv[VEC];
-                            E::unpack(sT[vi], tv);
-                            mT = fmaxf(mT, tree_max<VEC>(tv));
-                            if (!bonus) {
-                                float dv[VEC];
-                                E::unpack(sT[kStageVecs + vi], dv);
-                                mD = fmaxf(mD, tree_max<VEC>(dv));
-                            }
-                        }
-                    }
-                    const float nT = fmaxf(RT, warp_max_ref(ref_of(mT, P.c)));
-                    const float nD = bonus ? kEmptyRef : fmaxf(RD, warp_max_ref(ref_of(mD, P.c)));
-                    if (nT > RT || nD > RD) {
-                        ls.rescale(nT - RT, nD - RD);
-                        RT = nT;
-                        RD = nD;
-                    }
-#pragma unroll
-                    for (int g = 0; g < kStageGroups; ++g) {
-                        const int vi = g * 32 + lane;
-                        if (vi < nv) {
-                            float tv[VEC];
-                            E::unpack(sT[vi], tv);
-                            if (!bonus) {
-                                float dv[VEC];
-                                E::unpack(sT[kStageVecs + vi], dv);
-                                ls.template add_pair<VEC>(tv, dv, P.c, -RT, -RD);
-                            } else {
-                                ls.template add_bonus<VEC>(tv, P.c, -RT);
-                            }
-                        }
-                    }
+                    if (bonus) pass1_stage<DT, true>(sT, nv, lane, P.c, RT, RD, ls);
+                    else       pass1_stage<DT, false>(sT, nv, lane, P.c, RT, RD, ls);
                     recycle();
                 }
                 if (!ok) break;
@@ -466,31 +532,9 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag) {
                     if (!mbar_wait(&myfull[slot], (uint32_t)(n / kWarpSlots) & 1u, abort)) { ok = false; break; }
                     const uint4* sT = reinterpret_cast<const uint4*>(myring + (size_t)slot * kStageBytes);
                     const int nv = min(kStageVecs, nvb - s * kStageVecs);
-                    float mass = 0.f;
-#pragma unroll
-                    for (int g = 0; g < kStageGroups; ++g) {
-                        const int vi = g * 32 + lane;
-                        if (vi < nv) {
-                            float tv[VEC], r[VEC];
-                            E::unpack(sT[vi], tv);
-                            if (!bonus) {
-                                float dv[VEC], gv[VEC];
-                                E::unpack(sT[kStageVecs + vi], dv);
-#pragma unroll
-                                for (int z = 0; z < VEC; ++z) {
-                                    gv[z] = grad_elem(tv[z], dv[z], P.c, rc);
-                                    r[z] = fmaxf(-gv[z], 0.f);
-                                }
-                                if (Grow) store_streaming(Grow + (size_t)(s * kStageVecs + vi) * VEC, E::pack(gv));
-                            } else {
-#pragma unroll
-                                for (int z = 0; z < VEC; ++z) r[z] = prob_elem(tv[z], P.c, rc);
-                            }
-                            mass += tree_sum<VEC>(r);
-                        }
-                    }
-#pragma unroll
-                    for (int off = 16; off > 0; off >>= 1) mass += __shfl_xor_sync(0xffffffffu, mass, off);
+                    const float mass = bonus ? pass2_stage<DT, true>(sT, nv, lane, P.c, rc, nullptr)
+                                             : pass2_stage<DT, false>(sT, nv, lane, P.c, rc,
+                                                                      Grow ? Grow + (size_t)s * kStageVecs * VEC : nullptr);
                     if (lane == 0) rsum[s] = mass;
                     recycle();
                 }
