@@ -193,7 +193,8 @@ int choose_stream(DeviceState& d, int V, long long units, int dtype, int* G_out,
         return d.dec_C;
     }
     const int NV = V / vec_elems(dtype);
-    const int lag = 1;
+    const char* env_lag = getenv("SD_VERIFY_LAG");
+    const int lag = env_lag ? atoi(env_lag) : 1;   // stages of the next unit before pass 2 of a unit
     int best_C = 0, best_G = 0, best_per = 0;
     long long best_busy = -1;
     bool best_fits = false;
@@ -215,7 +216,7 @@ int choose_stream(DeviceState& d, int V, long long units, int dtype, int* G_out,
         const int G = (int)(units < resident ? units : resident);
         const int used = (stages_row + stages_blk - 1) / stages_blk;   // blocks with work
         const long long busy = (long long)G * (used < C ? used : C);
-        const double in_flight = (double)G * (double)NV * 16.0 * 2.0 * (1 + lag);
+        const double in_flight = (double)G * (double)NV * 16.0 * 2.0 * 1.5;
         const bool fits = in_flight <= l2_budget;
         // a shape that fits L2 beats one that does not; then more busy blocks; then the smaller cluster
         const bool better = best_C == 0 || (fits && !best_fits) || (fits == best_fits && busy > best_busy) ||

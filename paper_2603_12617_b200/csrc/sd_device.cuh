@@ -40,7 +40,7 @@ struct __align__(16) RowConst {
 };
 
 // Softmax statistics of a part of one row pair, relative to integer references RT and RD.
-struct __align__(8) PartialStats {
+struct __align__(16) PartialStats {
     float RT, RD;      // references of the exponentials (integer values)
     double sT, sD;     // sum of eT = 2^aT, aT = t*c - RT; sum of eD likewise
     double w;          // sum of eT*(aT - aD)
@@ -306,6 +306,21 @@ __device__ __forceinline__ PartialStats merge_partials_serial(const PartialStats
     for (int i = 0; i < n; ++i) {
         const PartialStats q = rescaled(p[i], RT, RD);
         r.sT += q.sT; r.sD += q.sD; r.w += q.w;
+    }
+    return r;
+}
+
+// Merge of 32 partials, one per lane (lanes without one pass empty_partial()), by the whole warp:
+// largest references by one redux each, exact rescaling, butterfly sums in a fixed order.  Every
+// lane gets the same bits.
+__device__ __forceinline__ PartialStats warp_merge_lanes(const PartialStats& m) {
+    const float RT = warp_max_ref(m.RT), RD = warp_max_ref(m.RD);
+    PartialStats r = rescaled(m, RT, RD);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        r.sT += shfl_xor_f64(r.sT, off);
+        r.sD += shfl_xor_f64(r.sD, off);
+        r.w += shfl_xor_f64(r.w, off);
     }
     return r;
 }

@@ -76,6 +76,18 @@ __device__ __forceinline__ void mbar_arrive_remote(uint64_t* bar, uint32_t rank)
         "r"(rank)
         : "memory");
 }
+// 16 bytes to the same shared-memory offset in block `rank` of the cluster; their arrival is
+// counted (as 16 bytes) on the barrier at offset `bar` of that block.  One-way: no acknowledgement.
+__device__ __forceinline__ void st_async_remote(void* dst, uint64_t a, uint64_t b, uint64_t* bar, uint32_t rank) {
+    asm volatile(
+        "{\n\t.reg .b32 ra, rb;\n\t"
+        "mapa.shared::cluster.u32 ra, %0, %4;\n\t"
+        "mapa.shared::cluster.u32 rb, %1, %4;\n\t"
+        "st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.b64 [ra], {%2, %3}, [rb];\n\t}" ::"r"(
+            smem_u32(dst)),
+        "r"(smem_u32(bar)), "l"(a), "l"(b), "r"(rank)
+        : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -263,13 +275,11 @@ __device__ __forceinline__ float pass2_stage(const uint4* st, int nv, int lane, 
 struct StreamShared {
     uint64_t full[kRingSlots];          // stage filled by the bulk copies        (1 arrival + bytes)
     uint64_t s1_done[2];                // consumers' sums of a unit posted       (consumer warps)
-    uint64_t xchg_bar[2];               // partials of every block have arrived   (cluster size, remote)
+    uint64_t xchg_bar[2];               // partials of every block have arrived   (1 arrival + bytes, remote)
     uint64_t rc_ready[2];               // row constants published                (1)
     uint64_t s2_done[kDoneDepth];       // unit finished in this block            (consumer warps + 1)
     uint64_t res_free[kDoneDepth];      // resolver is done with the unit         (1)
-    float lane_sums[2][3][kConsumerWarps][33];        // sT, sD, w of every consumer lane (33: no bank conflicts)
-    float warp_ref[2][kConsumerWarps][2];             // RT, RD each consumer warp used
-    PartialStats wpart[kConsumerWarps]; // the consumer warps' partials of the unit being merged
+    PartialStats wpart[2][kConsumerWarps];   // the consumer warps' partials of a unit
     PartialStats xchg[2][kMaxCluster];  // written by every block of the cluster (distributed shared memory)
     PartialStats row[kDoneDepth];       // statistics of the whole row, for the row report
     RowConst rc[2];
@@ -284,28 +294,17 @@ __device__ __host__ __forceinline__ void cluster_units(int units, int G, int cid
     u0 = cid * base + (cid < rem ? cid : rem);
 }
 
-// The passes of a block in the order in which it streams them: with lag 1,
-// S1(0) S1(1) S2(0) S1(2) S2(1) ... S1(n-1) S2(n-2) S2(n-1); with lag 0, S1(0) S2(0) S1(1) ...
-struct PassOrder {
-    int nu, lag;
-    __device__ __forceinline__ int count() const { return 2 * nu; }
-    __device__ __forceinline__ int index_s1(int j) const { return lag ? (j == 0 ? 0 : 2 * j - 1) : 2 * j; }
-    __device__ __forceinline__ int index_s2(int j) const { return lag ? (j == nu - 1 ? 2 * nu - 1 : 2 * j + 2) : 2 * j + 1; }
-    // unit and kind (0 = pass 1, 1 = pass 2) of pass p
-    __device__ __forceinline__ void decode(int p, int& j, int& kind) const {
-        if (!lag) { j = p >> 1; kind = p & 1; return; }
-        if (p == 0) { j = 0; kind = 0; }
-        else if (p == 2 * nu - 1) { j = nu - 1; kind = 1; }
-        else if (p & 1) { j = (p + 1) >> 1; kind = 0; }
-        else { j = (p >> 1) - 1; kind = 1; }
-    }
-};
+// The order in which a consumer warp walks its stages.  The warp has nst stages in every pass.
+// Pass 2 of a unit needs the row constants, which take an exchange between the blocks of the
+// cluster; so it is scheduled after the first L stages of pass 1 of the next unit:
+//   S1(0)[0,nst)  then for j = 1 .. nu-1:  S1(j)[0,L)  S2(j-1)[0,nst)  S1(j)[L,nst)   then  S2(nu-1)[0,nst)
+// The smaller L, the less data lies between the two passes (it has to stay in L2 meanwhile).
 
 // ---- fast path -----------------------------------------------------------------------------
-// lag: 1 if pass 2 of a unit is scheduled after pass 1 of the next unit, else 0.
+// lag_stages: stages (per consumer warp) of pass 1 of the next unit that go before pass 2 of a unit.
 template <int DT>
 __global__ void __launch_bounds__(kStreamThreads, 1)
-sd_stream_kernel(const __grid_constant__ Params P, const int lag) {
+sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
     using E = Elem<DT>;
     using ET = typename E::type;
     constexpr int VEC = E::VEC;
@@ -331,14 +330,13 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag) {
     const int ns = max(0, min(stages_row - s0, stages_blk));     // stages of a pass
     const int vb0 = s0 * kStageVecs;              // first vector of the slice
     const int nvb = max(0, min(NV - vb0, ns * kStageVecs));
-    const PassOrder order{nu, lag};
     volatile int* abort = &sh.abort;
 
     if (tid == 0) {
         for (int s = 0; s < R; ++s) mbar_init(&sh.full[s], 1);
         for (int s = 0; s < 2; ++s) {
             mbar_init(&sh.s1_done[s], kConsumerWarps);
-            mbar_init(&sh.xchg_bar[s], (uint32_t)C);
+            mbar_init(&sh.xchg_bar[s], 1);
             mbar_init(&sh.rc_ready[s], 1);
         }
         for (int s = 0; s < kDoneDepth; ++s) {
@@ -360,38 +358,20 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag) {
             const int par = j & 1;
             const uint32_t ph = (uint32_t)(j >> 1) & 1u;
             const int dslot = j % kDoneDepth;
+            if (lane == 0) mbar_expect_tx(&sh.xchg_bar[par], (uint32_t)C * (uint32_t)sizeof(PartialStats));
             if (!mbar_wait_sleepy(&sh.s1_done[par], ph, abort)) break;
-            // lane l adds up half of the lanes of consumer warp l%16 (they share that warp's
-            // references) in fp64; the 16 warp partials then meet in shared memory
-            {
-                const int w = lane & 15, h0 = (lane >> 4) * 16;
-                double sT = 0.0, sD = 0.0, wv = 0.0;
-#pragma unroll
-                for (int l = 0; l < 16; ++l) {
-                    sT += (double)sh.lane_sums[par][0][w][h0 + l];
-                    sD += (double)sh.lane_sums[par][1][w][h0 + l];
-                    wv += (double)sh.lane_sums[par][2][w][h0 + l];
-                }
-                sT += shfl_xor_f64(sT, 16);
-                sD += shfl_xor_f64(sD, 16);
-                wv += shfl_xor_f64(wv, 16);
-                if (lane < kConsumerWarps) {
-                    PartialStats wp;
-                    wp.RT = sh.warp_ref[par][w][0];
-                    wp.RD = sh.warp_ref[par][w][1];
-                    wp.sT = sT; wp.sD = sD; wp.w = wv;
-                    sh.wpart[lane] = wp;
-                }
-            }
-            __syncwarp();
-            const PartialStats mine = merge_partials_serial(sh.wpart, kConsumerWarps);
-            __syncwarp();
+            // the block's partial from its 16 warp partials, then one copy to every block of the cluster
+            const PartialStats mine = warp_merge_lanes(lane < kConsumerWarps ? sh.wpart[par][lane] : empty_partial());
             if (lane < C) {
-                *cluster.map_shared_rank(&sh.xchg[par][rank], lane) = mine;
-                mbar_arrive_remote(&sh.xchg_bar[par], (uint32_t)lane);
+                uint64_t refs;
+                memcpy(&refs, &mine.RT, 8);
+                PartialStats* dst = &sh.xchg[par][rank];
+                st_async_remote(dst, refs, (uint64_t)__double_as_longlong(mine.sT), &sh.xchg_bar[par], (uint32_t)lane);
+                st_async_remote(&dst->sD, (uint64_t)__double_as_longlong(mine.sD), (uint64_t)__double_as_longlong(mine.w),
+                                &sh.xchg_bar[par], (uint32_t)lane);
             }
             if (!mbar_wait_cluster(&sh.xchg_bar[par], ph, abort)) break;
-            const PartialStats row = merge_partials_serial(sh.xchg[par], C);
+            const PartialStats row = warp_merge_lanes(lane < C ? sh.xchg[par][lane] : empty_partial());
             const RowConst rcw = row_constants(P, bonus, row);
             if (lane == 0) {
                 sh.rc[par] = rcw;
@@ -437,121 +417,149 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag) {
         }
     } else {
         // ---- consumers: warp cw owns stages cw, cw+16, ... of every pass; a stage is a sampling
-        // region.  The warp walks its stages of all passes in order; stage number n of that walk
-        // goes to slot n % 3 of the warp's own ring, and its copies are issued by the warp's first
-        // lane as soon as stage n-3 has been worked on, whatever pass or unit it belongs to.
+        // region.  The warp walks its stages of all passes in a fixed order (Walk); stage number n
+        // of that walk goes to slot n % 3 of the warp's own ring, and its copies are issued by the
+        // warp's first lane as soon as stage n-3 has been worked on, whatever pass or unit it is of.
         const int cw = warp - kFirstConsumerWarp;
         const int nst = cw < ns ? (ns - cw + kConsumerWarps - 1) / kConsumerWarps : 0;   // my stages per pass
-        const int n_total = order.count() * nst;
-        unsigned char* myring = ring + (size_t)cw * kWarpSlots * kStageBytes;
-        uint64_t* myfull = &sh.full[cw * kWarpSlots];
-        const uint64_t keep = policy_keep(), normal = policy_normal();
-        // issue cursor (lane 0 only): next stage to fetch, and where it lies
-        int ni = 0, pi = 0, ti = 0;
-        const ET* Tbase = nullptr;
-        const ET* Dbase = nullptr;
-        int kind_i = 0;
-        auto issue_next = [&]() {     // lane 0
-            if (ni >= n_total) return;
-            if (ti == 0) {            // first stage of a pass: where the pass reads from
-                int j;
-                order.decode(pi, j, kind_i);
-                const int unit = u0 + j;
+        if (nst == 0) {
+            // no data of its own (short rows): the warp only keeps the per-unit protocol going
+            for (int j = 0; j < nu; ++j) {
+                if (lane == 0) { sh.wpart[j & 1][cw] = empty_partial(); mbar_arrive(&sh.s1_done[j & 1]); }
+                const int dslot = j % kDoneDepth;
+                if (!mbar_wait(&sh.rc_ready[j & 1], (uint32_t)(j >> 1) & 1u, abort)) break;
+                if (j >= kDoneDepth && !mbar_wait(&sh.res_free[dslot], (uint32_t)(j / kDoneDepth - 1) & 1u, abort)) break;
+                if (lane == 0) mbar_arrive(&sh.s2_done[dslot]);
+            }
+        } else {
+            const int L = min(max(lag_stages, 0), nst);
+            const int n_total = 2 * nu * nst;
+            unsigned char* myring = ring + (size_t)cw * kWarpSlots * kStageBytes;
+            uint64_t* myfull = &sh.full[cw * kWarpSlots];
+            const uint64_t keep = policy_keep(), normal = policy_normal();
+            // issue cursor (lane 0): the walk S1(0) | S1(j)[0,L) S2(j-1) S1(j)[L,nst) ... | S2(nu-1)
+            // runs of the walk: 0 = S1(0), 1 = head of S1(ji), 2 = S2(ji-1), 3 = rest of S1(ji), 4 = S2(nu-1)
+            int ni = 0, run = 0, ji = 0, ti = 0, endi = nst;   // stage number, run, unit of the run's pass 1, stage, end
+            const ET* Tb = nullptr;       // where the run reads from (this warp's first stage); Db null on a bonus row
+            const ET* Db = nullptr;
+            uint64_t pol = keep;
+            auto begin_run = [&]() {      // lane 0
+                const int unit = u0 + (run == 2 ? ji - 1 : run == 4 ? nu - 1 : ji);
                 const int b = unit / K1, i = unit - b * K1;
-                Tbase = reinterpret_cast<const ET*>(P.T) + (size_t)unit * P.V + (size_t)vb0 * VEC;
-                Dbase = (i == P.k) ? nullptr
-                                   : reinterpret_cast<const ET*>(P.D) + (size_t)(b * P.k + i) * P.V + (size_t)vb0 * VEC;
-            }
-            const int s = cw + ti * kConsumerWarps;
-            const int v0 = s * kStageVecs;
-            const uint32_t bytes = (uint32_t)min(kStageVecs, nvb - v0) * 16u;
-            const int slot = ni % kWarpSlots;
-            unsigned char* dst = myring + (size_t)slot * kStageBytes;
-            const uint64_t pol = kind_i == 0 ? keep : normal;
-            mbar_expect_tx(&myfull[slot], Dbase ? 2u * bytes : bytes);
-            bulk_load(dst, Tbase + (size_t)v0 * VEC, bytes, &myfull[slot], pol);
-            if (Dbase) bulk_load(dst + kStageRowBytes, Dbase + (size_t)v0 * VEC, bytes, &myfull[slot], pol);
-            ++ni;
-            if (++ti == nst) { ti = 0; ++pi; }
-        };
-        if (lane == 0)
-            for (int t = 0; t < kWarpSlots; ++t) issue_next();
-        int n = 0;                    // consume cursor: stages worked on so far
-        // hand the slot of stage n back and fetch stage n+3 into it
-        auto recycle = [&]() {
-            __syncwarp();
-            if (lane == 0) {
-                fence_proxy_async();   // the warp's reads of the slot come before the copy that refills it
-                issue_next();
-            }
-            ++n;
-        };
-        bool ok = true;
-        for (int j = 0; j < nu + lag && ok; ++j) {
-            if (j < nu) {
-                // pass 1 of unit j, stage by stage: the stage's maxima first; if they raise the warp's
-                // integer references, the running sums move to the new references (exact: powers of
-                // two); then the stage's sums.
+                const size_t off = (size_t)(vb0 + cw * kStageVecs) * VEC;
+                Tb = reinterpret_cast<const ET*>(P.T) + (size_t)unit * P.V + off;
+                Db = (i == P.k) ? nullptr : reinterpret_cast<const ET*>(P.D) + (size_t)(b * P.k + i) * P.V + off;
+                pol = (run == 2 || run == 4) ? normal : keep;
+            };
+            auto issue_next = [&]() {     // lane 0
+                if (ni >= n_total) return;
+                const int v0 = (cw + ti * kConsumerWarps) * kStageVecs;
+                const uint32_t bytes = (uint32_t)min(kStageVecs, nvb - v0) * 16u;
+                const int slot = ni % kWarpSlots;
+                unsigned char* dst = myring + (size_t)slot * kStageBytes;
+                const size_t off = (size_t)ti * (kConsumerWarps * kStageVecs * VEC);
+                mbar_expect_tx(&myfull[slot], Db ? 2u * bytes : bytes);
+                bulk_load(dst, Tb + off, bytes, &myfull[slot], pol);
+                if (Db) bulk_load(dst + kStageRowBytes, Db + off, bytes, &myfull[slot], pol);
+                ++ni;
+                ++ti;
+                if (ti >= endi) {
+                    while (ti >= endi && run != 5) {
+                        // the next run that is not empty
+                        if (run == 0) { if (nu > 1) { run = 1; ji = 1; } else run = 4; }
+                        else if (run == 1) run = 2;
+                        else if (run == 2) run = 3;
+                        else if (run == 3) { if (ji + 1 < nu) { run = 1; ++ji; } else run = 4; }
+                        else run = 5;
+                        if (run == 1) { ti = 0; endi = L; }
+                        else if (run == 3) { ti = L; endi = nst; }
+                        else { ti = 0; endi = nst; }
+                    }
+                    if (run != 5) begin_run();
+                }
+            };
+            if (lane == 0) begin_run();
+            if (lane == 0)
+                for (int t = 0; t < kWarpSlots; ++t) issue_next();
+            int n = 0;                    // consume cursor: stages worked on so far
+            bool ok = true;
+            // hand the slot of stage n back and fetch stage n+3 of the walk into it
+            auto recycle = [&]() {
+                __syncwarp();
+                if (lane == 0) {
+                    fence_proxy_async();   // the warp's reads of the slot come before the copy that refills it
+                    issue_next();
+                }
+                ++n;
+            };
+            float RT = kEmptyRef, RD = kEmptyRef;
+            LaneSums ls;
+            ls.init();
+            auto run_pass1 = [&](int j, int t0, int t1) {
                 const bool bonus = ((u0 + j) % K1 == P.k);
-                float RT = kEmptyRef, RD = kEmptyRef;
-                LaneSums ls;
-                ls.init();
-                for (int s = cw; s < ns; s += kConsumerWarps) {
+                for (int t = t0; t < t1 && ok; ++t) {
                     const int slot = n % kWarpSlots;
                     if (!mbar_wait(&myfull[slot], (uint32_t)(n / kWarpSlots) & 1u, abort)) { ok = false; break; }
-                    const uint4* sT = reinterpret_cast<const uint4*>(myring + (size_t)slot * kStageBytes);
+                    const uint4* st = reinterpret_cast<const uint4*>(myring + (size_t)slot * kStageBytes);
+                    const int s = cw + t * kConsumerWarps;
                     const int nv = min(kStageVecs, nvb - s * kStageVecs);     // vectors of this stage
-                    if (bonus) pass1_stage<DT, true>(sT, nv, lane, P.c, RT, RD, ls);
-                    else       pass1_stage<DT, false>(sT, nv, lane, P.c, RT, RD, ls);
+                    if (bonus) pass1_stage<DT, true>(st, nv, lane, P.c, RT, RD, ls);
+                    else       pass1_stage<DT, false>(st, nv, lane, P.c, RT, RD, ls);
                     recycle();
                 }
-                if (!ok) break;
-                const int parj = j & 1;
-                sh.lane_sums[parj][0][cw][lane] = ls.sT;
-                sh.lane_sums[parj][1][cw][lane] = ls.sD;
-                sh.lane_sums[parj][2][cw][lane] = ls.w;
-                if (lane == 0) { sh.warp_ref[parj][cw][0] = RT; sh.warp_ref[parj][cw][1] = RD; }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sh.s1_done[parj]);
-            }
-            if (j >= lag) {
-                // pass 2 of unit j-lag: gradient out, mass of every stage (= sampling region)
-                const int jj = j - lag;
-                const int unit = u0 + jj;
+            };
+            auto run_pass2 = [&](int j) {
+                const int unit = u0 + j;
                 const int b = unit / K1, i = unit - b * K1;
                 const bool bonus = (i == P.k);
-                const int dslot = jj % kDoneDepth;
-                if (!mbar_wait(&sh.rc_ready[jj & 1], (uint32_t)(jj >> 1) & 1u, abort)) { ok = false; break; }
-                const RowConst rc = sh.rc[jj & 1];
+                const int dslot = j % kDoneDepth;
+                if (!mbar_wait(&sh.rc_ready[j & 1], (uint32_t)(j >> 1) & 1u, abort)) { ok = false; return; }
+                const RowConst rc = sh.rc[j & 1];
                 ET* Grow = (P.grad && !bonus)
                                ? reinterpret_cast<ET*>(P.grad) + (size_t)(b * P.k + i) * P.V + (size_t)vb0 * VEC
                                : nullptr;
                 float* rsum = P.region_sums + (size_t)unit * P.NR + s0;
-                for (int s = cw; s < ns; s += kConsumerWarps) {
+                for (int t = 0; t < nst; ++t) {
                     const int slot = n % kWarpSlots;
-                    if (!mbar_wait(&myfull[slot], (uint32_t)(n / kWarpSlots) & 1u, abort)) { ok = false; break; }
-                    const uint4* sT = reinterpret_cast<const uint4*>(myring + (size_t)slot * kStageBytes);
+                    if (!mbar_wait(&myfull[slot], (uint32_t)(n / kWarpSlots) & 1u, abort)) { ok = false; return; }
+                    const uint4* st = reinterpret_cast<const uint4*>(myring + (size_t)slot * kStageBytes);
+                    const int s = cw + t * kConsumerWarps;
                     const int nv = min(kStageVecs, nvb - s * kStageVecs);
-                    const float mass = bonus ? pass2_stage<DT, true>(sT, nv, lane, P.c, rc, nullptr)
-                                             : pass2_stage<DT, false>(sT, nv, lane, P.c, rc,
+                    const float mass = bonus ? pass2_stage<DT, true>(st, nv, lane, P.c, rc, nullptr)
+                                             : pass2_stage<DT, false>(st, nv, lane, P.c, rc,
                                                                       Grow ? Grow + (size_t)s * kStageVecs * VEC : nullptr);
                     if (lane == 0) rsum[s] = mass;
                     recycle();
                 }
-                if (!ok) break;
-                // the resolver's slot of unit jj-4 must be free again before this unit is reported done
-                if (jj >= kDoneDepth &&
-                    !mbar_wait(&sh.res_free[dslot], (uint32_t)(jj / kDoneDepth - 1) & 1u, abort)) { ok = false; break; }
+                // the resolver's slot of unit j-4 must be free again before this unit is reported done
+                if (j >= kDoneDepth &&
+                    !mbar_wait(&sh.res_free[dslot], (uint32_t)(j / kDoneDepth - 1) & 1u, abort)) { ok = false; return; }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.s2_done[dslot]);
+            };
+            for (int j = 0; j < nu && ok; ++j) {
+                const int head = (j == 0) ? nst : L;
+                run_pass1(j, 0, head);
+                if (ok && j > 0) run_pass2(j - 1);
+                if (ok) run_pass1(j, head, nst);
+                if (!ok) break;
+                // pass 1 of the unit is over: the warp's partial for the statistics warp
+                const PartialStats part = warp_sum_lanes(ls, RT, RD);
+                if (lane == 0) {
+                    sh.wpart[j & 1][cw] = part;
+                    mbar_arrive(&sh.s1_done[j & 1]);
+                }
+                RT = RD = kEmptyRef;
+                ls.init();
             }
+            if (ok) run_pass2(nu - 1);
+            // leaving early: no copy of this warp may still be in flight when the block returns
+            if (!ok && lane == 0)
+                for (int t = n; t < ni; ++t) {
+                    const uint32_t par = (uint32_t)(t / kWarpSlots) & 1u;
+                    for (uint32_t it = 0; it < kWaitLimit && !mbar_try_wait(&myfull[t % kWarpSlots], par); ++it) {}
+                }
         }
-        // leaving early: no copy of this warp may still be in flight when the block returns
-        if (!ok && lane == 0)
-            for (int t = n; t < ni; ++t) {
-                const uint32_t par = (uint32_t)(t / kWarpSlots) & 1u;
-                for (uint32_t it = 0; it < kWaitLimit && !mbar_try_wait(&myfull[t % kWarpSlots], par); ++it) {}
-            }
     }
 
     __syncthreads();
