@@ -127,6 +127,42 @@ int sd_verify_feedback_ex(const void* target_logits, const void* draft_logits,
                           float* out_acc_prob, uint32_t* out_status, void* workspace,
                           size_t workspace_bytes, void* stream);
 
+/*
+ * sd_verify_feedback_static -- the same computation as sd_verify_feedback_ex for callers that
+ * cannot allocate device memory.  (The paper has no counterpart of this entry point; it exists
+ * for the way the library is embedded.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a serving loop whose
+ * memory is handed out once at start-up by a pool that owns the whole device, in a process that
+ * has been told to stay within a fixed footprint, or in a callback that may not call anything
+ * that can synchronise the device or fail for lack of memory.  sd_verify_feedback allocates its
+ * scratch on first use and sd_verify_feedback_ex wants a buffer from the caller; this entry point
+ * needs neither, because its scratch is a fixed array of SD_STATIC_SCRATCH_BYTES bytes inside the
+ * library itself.  The price: every GPU on which the library is loaded gives up that much memory
+ * for as long as the process lives, whether this entry point is used or not.
+ *
+ * Arguments and results are those of sd_verify_feedback_ex without workspace/workspace_bytes.
+ * It never calls cudaMalloc, cudaFree or any other allocating routine.
+ *
+ *   - Shapes whose sd_workspace_bytes(B,k,V,dtype) exceeds SD_STATIC_SCRATCH_BYTES are refused
+ *     with SD_ERR_WORKSPACE (sd_last_cuda_error() says how many bytes were needed); nothing is
+ *     enqueued.  4 MiB covers, for instance, B*(k+1) up to about 3900 rows at V <= 131072.
+ *   - The first call on each device looks up the device address of the array
+ *     (cudaGetSymbolAddress, with that device current).  Make that first call outside any stream
+ *     capture; later calls only enqueue a small memset and the kernel.
+ *   - All calls on a device share the one array, and it keeps what the last call left in it.  The
+ *     words that must start at zero are cleared on `stream` at the start of every call.  Two calls
+ *     that overlap on the GPU (different streams without an ordering between them, or different
+ *     host threads) race on the array and give wrong results: serialise them, or use
+ *     sd_verify_feedback_ex with a scratch buffer per stream.
+ */
+#define SD_STATIC_SCRATCH_BYTES (4 * 1024 * 1024)
+int sd_verify_feedback_static(const void* target_logits, const void* draft_logits,
+                              const int32_t* draft_tokens, const float* uniforms, float temperature,
+                              int B, int k, int V, int dtype, int32_t* out_accept_len,
+                              int32_t* out_tokens, float* out_loss, void* out_grad_draft,
+                              float* out_acc_prob, uint32_t* out_status, void* stream);
+
 /* Bytes of scratch sd_verify_feedback_ex needs for this shape; 0 if the shape is invalid. */
 size_t sd_workspace_bytes(int B, int k, int V, int dtype);
 

@@ -47,6 +47,8 @@ def _load() -> ctypes.CDLL:
     lib.sd_verify_feedback_bf16.argtypes = [P, P, P, P, F, I, I, I, P, P, P, P, P]
     lib.sd_verify_feedback_ex.restype = I
     lib.sd_verify_feedback_ex.argtypes = [P, P, P, P, F, I, I, I, I, P, P, P, P, P, P, P, Z, P]
+    lib.sd_verify_feedback_static.restype = I
+    lib.sd_verify_feedback_static.argtypes = [P, P, P, P, F, I, I, I, I, P, P, P, P, P, P, P]
     lib.sd_verify_feedback_host.restype = I
     lib.sd_verify_feedback_host.argtypes = [P, P, P, P, F, I, I, I, I, P, P, P, P, P, P]
     lib.sd_workspace_bytes.restype = Z
@@ -187,6 +189,35 @@ def sd_verify_feedback_ex(target_logits: torch.Tensor, draft_logits: torch.Tenso
             _stream_ptr(stream))
     if rc != 0:
         raise SdVerifyError(rc, "sd_verify_feedback_ex")
+    return out
+
+
+SD_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
+
+
+def sd_verify_feedback_static(target_logits: torch.Tensor, draft_logits: torch.Tensor,
+                              draft_tokens: torch.Tensor, uniforms: torch.Tensor, temperature: float, *,
+                              out: StepOutputs, stream: Optional[torch.cuda.Stream] = None) -> StepOutputs:
+    """``sd_verify_feedback_static``: the step with the scratch that is built into the library.
+
+    For callers that may not allocate device memory: the C entry point allocates nothing, and
+    neither does this wrapper, which is why ``out`` (every output tensor the caller wants, made
+    beforehand) is required here instead of being created on the fly.  Shapes that need more than
+    ``SD_STATIC_SCRATCH_BYTES`` of scratch raise ``SdVerifyError`` (SD_ERR_WORKSPACE).  Calls that
+    overlap on the GPU share the one scratch array and must be serialised by the caller.
+    """
+    B, k, V = _shapes(target_logits, draft_logits, draft_tokens, uniforms)
+    dev = target_logits.device
+    if dev.type != "cuda":
+        raise ValueError("device tensors required")
+    code = _dtype_code(target_logits)
+    with torch.cuda.device(dev):
+        rc = _lib.sd_verify_feedback_static(
+            _ptr(target_logits), _ptr(draft_logits), _ptr(draft_tokens), _ptr(uniforms), float(temperature),
+            B, k, V, code, _ptr(out.accept_len), _ptr(out.tokens), _ptr(out.loss), _ptr(out.grad_draft),
+            _ptr(out.acc_prob), _ptr(out.status), _stream_ptr(stream))
+    if rc != 0:
+        raise SdVerifyError(rc, "sd_verify_feedback_static")
     return out
 
 

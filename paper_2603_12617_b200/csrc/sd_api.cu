@@ -325,6 +325,34 @@ int run_cached(const void* T, const void* D, const int32_t* x, const float* u, f
     return rc;
 }
 
+// ---- scratch that nobody allocates --------------------------------------------------------
+// For callers that must not allocate device memory (see sd_verify_feedback_static in the header):
+// the scratch of the step lives in the library's own image.  Every GPU that loads the library
+// holds these bytes until the process exits.
+static __device__ __align__(256) unsigned char g_static_scratch[SD_STATIC_SCRATCH_BYTES];
+
+// In host code the name g_static_scratch is only a handle of the symbol, not a device address:
+// the address on a given GPU comes from cudaGetSymbolAddress, asked once per device while that
+// device is current.
+std::mutex g_static_mu;
+unsigned char* g_static_ptr[kMaxDevices] = {};
+
+int static_scratch(int dev, unsigned char** out) {
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        void* ptr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress(g_static_scratch)");
+        if (!ptr || !aligned(ptr, kAlign)) {
+            snprintf(tl_cuda_error, sizeof tl_cuda_error, "static scratch has no usable device address");
+            return SD_ERR_CUDA;
+        }
+        g_static_ptr[dev] = static_cast<unsigned char*>(ptr);
+    }
+    *out = g_static_ptr[dev];
+    return SD_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -367,6 +395,35 @@ int sd_verify_feedback_ex(const void* target_logits, const void* draft_logits, c
     return run_device(*d, target_logits, draft_logits, draft_tokens, uniforms, temperature, B, k, V, dtype,
                       out_accept_len, out_tokens, out_loss, out_grad_draft, out_acc_prob, out_status,
                       static_cast<unsigned char*>(workspace), L, false, static_cast<cudaStream_t>(stream));
+}
+
+int sd_verify_feedback_static(const void* target_logits, const void* draft_logits, const int32_t* draft_tokens,
+                              const float* uniforms, float temperature, int B, int k, int V, int dtype,
+                              int32_t* out_accept_len, int32_t* out_tokens, float* out_loss, void* out_grad_draft,
+                              float* out_acc_prob, uint32_t* out_status, void* stream) {
+    int rc = check_args(target_logits, draft_logits, draft_tokens, uniforms, temperature, B, k, V, dtype,
+                        out_accept_len, out_tokens, out_loss, out_grad_draft, out_acc_prob, out_status);
+    if (rc != SD_OK) return rc;
+    const WorkspaceLayout L = workspace_layout(B, k, V, dtype);
+    if (L.total > (size_t)SD_STATIC_SCRATCH_BYTES) {
+        snprintf(tl_cuda_error, sizeof tl_cuda_error,
+                 "this shape needs %zu bytes of scratch, the built-in scratch has %d: use sd_verify_feedback_ex",
+                 L.total, SD_STATIC_SCRATCH_BYTES);
+        return SD_ERR_WORKSPACE;
+    }
+    int dev;
+    DeviceState* d = nullptr;
+    rc = current_device(&dev, &d);
+    if (rc != SD_OK) return rc;
+    unsigned char* scratch = nullptr;
+    rc = static_scratch(dev, &scratch);   // first call on this device: looks the address up
+    if (rc != SD_OK) return rc;
+    std::lock_guard<std::mutex> lock(d->mu);
+    // clean = false: the tickets, status words and error flag at the head of the scratch are zeroed
+    // on the stream before the kernel, whatever the previous call left there
+    return run_device(*d, target_logits, draft_logits, draft_tokens, uniforms, temperature, B, k, V, dtype,
+                      out_accept_len, out_tokens, out_loss, out_grad_draft, out_acc_prob, out_status, scratch, L, false,
+                      static_cast<cudaStream_t>(stream));
 }
 
 int sd_verify_feedback_host(const void* target_logits, const void* draft_logits, const int32_t* draft_tokens,

@@ -113,13 +113,13 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t pa
 // Bounded wait of one thread.  It gives up after kWaitLimit polls or kWaitCycles clock cycles,
 // whichever comes first, or as soon as another thread of the block has given up (*abort != 0);
 // the caller then leaves its loop and the kernel returns.  A failed poll is followed by a short
-// sleep, so that waiting warps leave the issue slots and the shared-memory pipe to working ones.
+// sleep (longer for the warps whose waits are long by design).
 template <bool CLUSTER, bool SLEEP = false>
 __device__ __forceinline__ bool mbar_wait_thread(uint64_t* bar, uint32_t parity, volatile int* abort) {
     long long t0 = 0;
     for (uint32_t it = 0; it < kWaitLimit; ++it) {
         if (CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
-        if (SLEEP) __nanosleep(64);   // warps with long waits leave the issue slots to the others
+        __nanosleep(SLEEP ? 64 : 20);   // waiting warps leave the issue slots to the working ones
         if ((it & 63u) == 63u) {
             if (*abort) return false;
             const long long now = clock64();
