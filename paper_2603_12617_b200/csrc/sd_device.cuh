@@ -149,6 +149,16 @@ __device__ __forceinline__ float grad_elem(float t, float d, float c, const RowC
     float eD = exp_term(d, c, rc.negRD);
     return __fmaf_rn(eD, rc.kD, -__fmul_rn(eT, rc.kT));
 }
+// The same for two elements at once (packed fp32 instructions, same rounding).
+__device__ __forceinline__ float2 grad_elem2(float2 t, float2 d, float c, const RowConst& rc) {
+    const float2 c2 = make_float2(c, c);
+    const float2 aT = __ffma2_rn(t, c2, make_float2(rc.negRT, rc.negRT));
+    const float2 aD = __ffma2_rn(d, c2, make_float2(rc.negRD, rc.negRD));
+    const float2 eT = make_float2(ex2f(aT.x), ex2f(aT.y));
+    const float2 eD = make_float2(ex2f(aD.x), ex2f(aD.y));
+    const float2 pT = __fmul2_rn(eT, make_float2(-rc.kT, -rc.kT));        // -(eT*kT), exact negation
+    return __ffma2_rn(eD, make_float2(rc.kD, rc.kD), pT);
+}
 // p of one element of a bonus row
 __device__ __forceinline__ float prob_elem(float t, float c, const RowConst& rc) {
     return __fmul_rn(exp_term(t, c, rc.negRT), rc.kT);
@@ -214,23 +224,32 @@ struct LaneSums {
         sD += tree_sum<VEC>(eD);
         w += tree_sum<VEC>(pw);
     }
-    // The same for one vector, into partial sums of its own (short dependency chains).
+    // The same for one vector, into partial sums of its own (short dependency chains).  Entries are
+    // taken two at a time with the packed fp32 instructions of sm_100 (same rounding as the scalar
+    // ones); even and odd entries are summed separately and meet at the end.
     template <int VEC>
     static __device__ __forceinline__ void vector_pair(const float (&t)[VEC], const float (&d)[VEC], float c,
                                                        float negRT, float negRD, float& pT, float& pD, float& pW) {
-        float eT[VEC], eD[VEC];
-        float wv = 0.f;
+        static_assert(VEC % 2 == 0, "packed arithmetic takes entries in pairs");
+        const float2 c2 = make_float2(c, c), nT2 = make_float2(negRT, negRT), nD2 = make_float2(negRD, negRD);
+        const float2 m1 = make_float2(-1.f, -1.f);
+        float2 accT = make_float2(0.f, 0.f), accD = make_float2(0.f, 0.f);
+        float w0 = 0.f, w1 = 0.f;
 #pragma unroll
-        for (int e = 0; e < VEC; ++e) {
-            const float aT = __fmaf_rn(t[e], c, negRT), aD = __fmaf_rn(d[e], c, negRD);
-            eT[e] = ex2f(aT);
-            eD[e] = ex2f(aD);
-            const float diff = (eT[e] > 0.f) ? aT - aD : 0.f;   // masked target entries (p = 0) add nothing
-            wv = __fmaf_rn(eT[e], diff, wv);
+        for (int e = 0; e < VEC; e += 2) {
+            const float2 aT = __ffma2_rn(make_float2(t[e], t[e + 1]), c2, nT2);
+            const float2 aD = __ffma2_rn(make_float2(d[e], d[e + 1]), c2, nD2);
+            const float2 eT = make_float2(ex2f(aT.x), ex2f(aT.y));
+            const float2 eD = make_float2(ex2f(aD.x), ex2f(aD.y));
+            const float2 diff = __ffma2_rn(aD, m1, aT);          // aT - aD
+            if (eT.x > 0.f) w0 = __fmaf_rn(eT.x, diff.x, w0);    // masked target entries (p = 0) add nothing
+            if (eT.y > 0.f) w1 = __fmaf_rn(eT.y, diff.y, w1);
+            accT = __fadd2_rn(accT, eT);
+            accD = __fadd2_rn(accD, eD);
         }
-        pT = tree_sum<VEC>(eT);
-        pD = tree_sum<VEC>(eD);
-        pW = wv;
+        pT = accT.x + accT.y;
+        pD = accD.x + accD.y;
+        pW = w0 + w1;
     }
     template <int VEC>
     static __device__ __forceinline__ float vector_bonus(const float (&t)[VEC], float c, float negRT) {

@@ -254,9 +254,12 @@ __device__ __forceinline__ float pass2_stage(const uint4* st, int nv, int lane, 
             float dv[VEC], gv[VEC];
             E::unpack(rd[g], dv);
 #pragma unroll
-            for (int z = 0; z < VEC; ++z) {
-                gv[z] = grad_elem(tv[z], dv[z], c, rc);
-                r[z] = fmaxf(-gv[z], 0.f);
+            for (int z = 0; z < VEC; z += 2) {
+                const float2 g2 = grad_elem2(make_float2(tv[z], tv[z + 1]), make_float2(dv[z], dv[z + 1]), c, rc);
+                gv[z] = g2.x;
+                gv[z + 1] = g2.y;
+                r[z] = fmaxf(-g2.x, 0.f);
+                r[z + 1] = fmaxf(-g2.y, 0.f);
             }
             if (gdst && vi < nv) store_streaming(gdst + (size_t)vi * VEC, E::pack(gv));
         } else {
