@@ -17,7 +17,7 @@ constexpr int kMaxDevices = 64;
 constexpr size_t kAlign = 256;
 constexpr int kStreamSmem = kRingSlots * kStageBytes + (int)sizeof(StreamShared);
 static_assert(kStreamSmem <= 227 * 1024, "ring does not fit the shared memory of a block");
-constexpr double kL2BudgetMiB = 48.0;             // slices in flight between their two passes should fit this
+constexpr double kL2BudgetMiB = 80.0;              // row pairs in flight between their two passes should fit this
 
 thread_local char tl_cuda_error[256] = "";
 thread_local int tl_info[6] = {0, 0, 0, 0, 0, 0};
@@ -171,15 +171,18 @@ int launch_generic(const Params& P, cudaStream_t stream) {
 }
 
 // Launch shape of the fast path: cluster size C (0 if the fast path cannot run), number of
-// clusters G, vectors per sampling region, and whether pass 2 of a unit is scheduled after pass 1
-// of the next one.
+// clusters G, vectors per sampling region, and how many stages of pass 1 of the next unit a
+// consumer warp takes before pass 2 of a unit.
 //
-// A row is cut into stages of 128 vectors and block r of a cluster of C takes every C-th share of
-// them.  A block's slice lives in L2 between its two passes, so the row pairs all resident
-// clusters have in flight (two each, with the lag) should fit a part of L2.  Among the cluster
-// sizes that qualify, take the one that keeps most blocks busy (resident clusters, but no more
-// clusters than units), then the smaller cluster: larger slices spread the per-unit costs
-// (exchange, row report) over more bytes.  If none qualifies, the largest cluster.
+// A row is cut into stages and block r of a cluster of C takes every C-th share of them.  A
+// block's slice lives in L2 between its two passes, so the row pairs the resident clusters work on
+// at the same time should fit the part of L2 that holds on to them (about 80 MiB of the 126 MiB,
+// measured: beyond it the second pass goes back to HBM).  Among the cluster sizes that fit, take
+// the one that keeps most blocks busy (resident clusters, but no more clusters than units; 128
+// busy blocks or more count alike), then the smaller cluster: larger slices spread the per-unit
+// costs (exchange, row report) over more bytes and small clusters pack the GPU best (resident
+// blocks: 148 for C = 1 and 2, 135 for 3, 132 for 4, 120 for 8, 112 for 16).  If none fits, the
+// largest cluster.
 int choose_stream(DeviceState& d, int V, long long units, int dtype, int* G_out, int* per_out, int* lag_out) {
     const char* env = getenv("SD_VERIFY_CLUSTER");
     const int forced = env ? atoi(env) : 0;
@@ -215,8 +218,9 @@ int choose_stream(DeviceState& d, int V, long long units, int dtype, int* G_out,
         if (resident < 1) continue;
         const int G = (int)(units < resident ? units : resident);
         const int used = (stages_row + stages_blk - 1) / stages_blk;   // blocks with work
-        const long long busy = (long long)G * (used < C ? used : C);
-        const double in_flight = (double)G * (double)NV * 16.0 * 2.0 * 1.5;
+        long long busy = (long long)G * (used < C ? used : C);
+        if (busy > 128) busy = 128;
+        const double in_flight = (double)G * (double)NV * 16.0 * 2.0;
         const bool fits = in_flight <= l2_budget;
         // a shape that fits L2 beats one that does not; then more busy blocks; then the smaller cluster
         const bool better = best_C == 0 || (fits && !best_fits) || (fits == best_fits && busy > best_busy) ||

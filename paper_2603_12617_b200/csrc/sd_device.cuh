@@ -179,6 +179,7 @@ __device__ __forceinline__ float pow2_neg_f32(float d) {
 template <int VEC>
 __device__ __forceinline__ float tree_sum(const float (&v)[VEC]) {
     if constexpr (VEC == 1) return v[0];
+    else if constexpr (VEC == 2) return v[0] + v[1];
     else if constexpr (VEC == 4) return (v[0] + v[1]) + (v[2] + v[3]);
     else return ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
 }
@@ -191,6 +192,7 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
 template <int VEC>
 __device__ __forceinline__ float tree_max(const float (&v)[VEC]) {
     if constexpr (VEC == 1) return v[0];
+    else if constexpr (VEC == 2) return fmaxf(v[0], v[1]);
     else if constexpr (VEC == 4) return fmaxf(fmax3(v[0], v[1], v[2]), v[3]);
     else return fmax3(fmax3(v[0], v[1], v[2]), fmax3(v[3], v[4], v[5]), fmaxf(v[6], v[7]));
 }

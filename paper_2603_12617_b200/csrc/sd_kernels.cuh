@@ -35,17 +35,17 @@
 namespace sdv {
 
 // ---- geometry of the fast path -------------------------------------------------------------
-// A row is cut into stages of 128 16-byte vectors (2 KiB); a stage is also a sampling region.
+// A row is cut into stages of 256 16-byte vectors (4 KiB); a stage is also a sampling region.
 // Block r of a cluster of C owns the stages [r*S, (r+1)*S) of every row it works on, S =
-// ceil(stages per row / C); stage s of the slice belongs to consumer warp s % 16, so sixteen
+// ceil(stages per row / C); stage s of the slice belongs to consumer warp s % 8, so eight
 // consecutive stages are worked on at the same time.  Every consumer warp has a ring of its own.
-constexpr int kConsumerWarps = 16;
+constexpr int kConsumerWarps = 14;
 constexpr int kStageGroups = 4;                               // groups of 32 vectors in a stage
 constexpr int kStageVecs = 32 * kStageGroups;                 // vectors of one row in a stage
-constexpr int kStageRowBytes = kStageVecs * 16;               // 2 KiB of one row
+constexpr int kStageRowBytes = kStageVecs * 16;               // 4 KiB of one row
 constexpr int kStageBytes = 2 * kStageRowBytes;               // target part + draft part
 constexpr int kWarpSlots = 3;                                 // stages a consumer warp has in flight or in use
-constexpr int kRingSlots = kConsumerWarps * kWarpSlots;       // 48 slots, 192 KiB
+constexpr int kRingSlots = kConsumerWarps * kWarpSlots;       // 24 slots, 192 KiB
 constexpr int kDoneDepth = 4;                                 // units the resolver may lag behind
 constexpr int kStatsWarp = 0, kResolverWarp = 1, kFirstConsumerWarp = 2;
 constexpr int kStreamThreads = (kFirstConsumerWarp + kConsumerWarps) * 32;
@@ -114,12 +114,12 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t pa
 // whichever comes first, or as soon as another thread of the block has given up (*abort != 0);
 // the caller then leaves its loop and the kernel returns.  A failed poll is followed by a short
 // sleep (longer for the warps whose waits are long by design).
-template <bool CLUSTER, bool SLEEP = false>
+template <bool CLUSTER, int SLEEP_NS = 20>
 __device__ __forceinline__ bool mbar_wait_thread(uint64_t* bar, uint32_t parity, volatile int* abort) {
     long long t0 = 0;
     for (uint32_t it = 0; it < kWaitLimit; ++it) {
         if (CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
-        __nanosleep(SLEEP ? 64 : 20);   // waiting warps leave the issue slots to the working ones
+        __nanosleep(SLEEP_NS);   // waiting warps leave the issue slots to the working ones
         if ((it & 63u) == 63u) {
             if (*abort) return false;
             const long long now = clock64();
@@ -137,10 +137,11 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     return __all_sync(0xffffffffu, mbar_wait_thread<false>(bar, parity, abort) ? 1 : 0) != 0;
 }
 __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, volatile int* abort) {
-    return __all_sync(0xffffffffu, mbar_wait_thread<true, true>(bar, parity, abort) ? 1 : 0) != 0;
+    return __all_sync(0xffffffffu, mbar_wait_thread<true, 100>(bar, parity, abort) ? 1 : 0) != 0;
 }
+template <int SLEEP_NS>
 __device__ __forceinline__ bool mbar_wait_sleepy(uint64_t* bar, uint32_t parity, volatile int* abort) {
-    return __all_sync(0xffffffffu, mbar_wait_thread<false, true>(bar, parity, abort) ? 1 : 0) != 0;
+    return __all_sync(0xffffffffu, mbar_wait_thread<false, SLEEP_NS>(bar, parity, abort) ? 1 : 0) != 0;
 }
 // 1-D bulk copy global -> shared of this block, completion counted on `bar`, with an L2 eviction
 // policy.  Both addresses 16-byte aligned, bytes a multiple of 16.
@@ -175,7 +176,7 @@ __device__ __forceinline__ void store_streaming(void* p, const uint4& v) {
 }
 
 // ---- the two passes over one stage held in shared memory ------------------------------------
-// A stage is 4 vectors per lane and row.  All of them are loaded before any arithmetic; vectors
+// A stage is kStageGroups vectors per lane and row.  All of them are loaded before any arithmetic; vectors
 // past the end of the row read as -inf, which adds nothing to any sum and is never stored.
 
 // Pass 1: the stage's maxima; if they raise the warp's integer references (RT, RD), the running
@@ -186,11 +187,19 @@ __device__ __forceinline__ void pass1_stage(const uint4* st, int nv, int lane, f
     using E = Elem<DT>;
     constexpr int VEC = E::VEC;
     uint4 rt[kStageGroups], rd[kStageGroups];
+    if (nv == kStageVecs) {
 #pragma unroll
-    for (int g = 0; g < kStageGroups; ++g) {
-        const int vi = g * 32 + lane;
-        rt[g] = vi < nv ? st[vi] : E::masked();
-        if (!BONUS) rd[g] = vi < nv ? st[kStageVecs + vi] : E::masked();
+        for (int g = 0; g < kStageGroups; ++g) {
+            rt[g] = st[g * 32 + lane];
+            if (!BONUS) rd[g] = st[kStageVecs + g * 32 + lane];
+        }
+    } else {
+#pragma unroll
+        for (int g = 0; g < kStageGroups; ++g) {
+            const int vi = g * 32 + lane;
+            rt[g] = vi < nv ? st[vi] : E::masked();
+            if (!BONUS) rd[g] = vi < nv ? st[kStageVecs + vi] : E::masked();
+        }
     }
     float mT[kStageGroups], mD[kStageGroups];
 #pragma unroll
@@ -203,9 +212,11 @@ __device__ __forceinline__ void pass1_stage(const uint4* st, int nv, int lane, f
             mD[g] = tree_max<VEC>(v);
         }
     }
-    const float nT = fmaxf(RT, warp_max_ref(ref_of(fmaxf(fmax3(mT[0], mT[1], mT[2]), mT[3]), c)));
-    const float nD = BONUS ? kEmptyRef : fmaxf(RD, warp_max_ref(ref_of(fmaxf(fmax3(mD[0], mD[1], mD[2]), mD[3]), c)));
-    if (nT > RT || nD > RD) {
+    const float lT = tree_max<kStageGroups>(mT), lD = BONUS ? 0.f : tree_max<kStageGroups>(mD);
+    // the references only move when some lane has an entry above them (rare after the first stages)
+    if (__any_sync(0xffffffffu, __fmul_rn(lT, c) > RT || (!BONUS && __fmul_rn(lD, c) > RD))) {
+        const float nT = fmaxf(RT, warp_max_ref(ref_of(lT, c)));
+        const float nD = BONUS ? kEmptyRef : fmaxf(RD, warp_max_ref(ref_of(lD, c)));
         ls.rescale(nT - RT, nD - RD);
         RT = nT;
         RD = nD;
@@ -223,10 +234,10 @@ __device__ __forceinline__ void pass1_stage(const uint4* st, int nv, int lane, f
             pT[g] = LaneSums::vector_bonus<VEC>(tv, c, -RT);
         }
     }
-    ls.sT += (pT[0] + pT[1]) + (pT[2] + pT[3]);
+    ls.sT += tree_sum<kStageGroups>(pT);
     if (!BONUS) {
-        ls.sD += (pD[0] + pD[1]) + (pD[2] + pD[3]);
-        ls.w += (pW[0] + pW[1]) + (pW[2] + pW[3]);
+        ls.sD += tree_sum<kStageGroups>(pD);
+        ls.w += tree_sum<kStageGroups>(pW);
     }
 }
 
@@ -238,11 +249,19 @@ __device__ __forceinline__ float pass2_stage(const uint4* st, int nv, int lane, 
     using E = Elem<DT>;
     constexpr int VEC = E::VEC;
     uint4 rt[kStageGroups], rd[kStageGroups];
+    if (nv == kStageVecs) {
 #pragma unroll
-    for (int g = 0; g < kStageGroups; ++g) {
-        const int vi = g * 32 + lane;
-        rt[g] = vi < nv ? st[vi] : E::masked();
-        if (!BONUS) rd[g] = vi < nv ? st[kStageVecs + vi] : E::masked();
+        for (int g = 0; g < kStageGroups; ++g) {
+            rt[g] = st[g * 32 + lane];
+            if (!BONUS) rd[g] = st[kStageVecs + g * 32 + lane];
+        }
+    } else {
+#pragma unroll
+        for (int g = 0; g < kStageGroups; ++g) {
+            const int vi = g * 32 + lane;
+            rt[g] = vi < nv ? st[vi] : E::masked();
+            if (!BONUS) rd[g] = vi < nv ? st[kStageVecs + vi] : E::masked();
+        }
     }
     float ms[kStageGroups];
 #pragma unroll
@@ -268,7 +287,7 @@ __device__ __forceinline__ float pass2_stage(const uint4* st, int nv, int lane, 
         }
         ms[g] = tree_sum<VEC>(r);
     }
-    float mass = (ms[0] + ms[1]) + (ms[2] + ms[3]);
+    float mass = tree_sum<kStageGroups>(ms);
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) mass += __shfl_xor_sync(0xffffffffu, mass, off);
     return mass;
@@ -362,7 +381,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
             const uint32_t ph = (uint32_t)(j >> 1) & 1u;
             const int dslot = j % kDoneDepth;
             if (lane == 0) mbar_expect_tx(&sh.xchg_bar[par], (uint32_t)C * (uint32_t)sizeof(PartialStats));
-            if (!mbar_wait_sleepy(&sh.s1_done[par], ph, abort)) break;
+            if (!mbar_wait_sleepy<100>(&sh.s1_done[par], ph, abort)) break;
             // the block's partial from its 16 warp partials, then one copy to every block of the cluster
             const PartialStats mine = warp_merge_lanes(lane < kConsumerWarps ? sh.wpart[par][lane] : empty_partial());
             if (lane < C) {
@@ -403,7 +422,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
             AcceptOperands aop;
             aop.valid = false;
             if (reports && lane == 0 && !bonus) aop = load_accept_operands<DT>(P, b, i);
-            if (!mbar_wait_sleepy(&sh.s2_done[dslot], (uint32_t)(j / kDoneDepth) & 1u, abort)) break;
+            if (!mbar_wait_sleepy<500>(&sh.s2_done[dslot], (uint32_t)(j / kDoneDepth) & 1u, abort)) break;
             if (reports && lane == 0) finish_row(P, b, i, sh.row[dslot], sh.rc_done[dslot], aop);
             __syncwarp();
             ++seg;
@@ -443,27 +462,28 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
             // issue cursor (lane 0): the walk S1(0) | S1(j)[0,L) S2(j-1) S1(j)[L,nst) ... | S2(nu-1)
             // runs of the walk: 0 = S1(0), 1 = head of S1(ji), 2 = S2(ji-1), 3 = rest of S1(ji), 4 = S2(nu-1)
             int ni = 0, run = 0, ji = 0, ti = 0, endi = nst;   // stage number, run, unit of the run's pass 1, stage, end
-            const ET* Tb = nullptr;       // where the run reads from (this warp's first stage); Db null on a bonus row
+            const ET* Tb = nullptr;       // where the next copy of the run reads from; Db null on a bonus row
             const ET* Db = nullptr;
             uint64_t pol = keep;
+            int slot_i = 0;               // ring slot of the next copy
+            constexpr size_t kStride = (size_t)kConsumerWarps * kStageVecs * VEC;   // from one of my stages to the next
             auto begin_run = [&]() {      // lane 0
                 const int unit = u0 + (run == 2 ? ji - 1 : run == 4 ? nu - 1 : ji);
                 const int b = unit / K1, i = unit - b * K1;
-                const size_t off = (size_t)(vb0 + cw * kStageVecs) * VEC;
+                const size_t off = (size_t)(vb0 + cw * kStageVecs) * VEC + (size_t)ti * kStride;
                 Tb = reinterpret_cast<const ET*>(P.T) + (size_t)unit * P.V + off;
                 Db = (i == P.k) ? nullptr : reinterpret_cast<const ET*>(P.D) + (size_t)(b * P.k + i) * P.V + off;
                 pol = (run == 2 || run == 4) ? normal : keep;
             };
             auto issue_next = [&]() {     // lane 0
                 if (ni >= n_total) return;
-                const int v0 = (cw + ti * kConsumerWarps) * kStageVecs;
-                const uint32_t bytes = (uint32_t)min(kStageVecs, nvb - v0) * 16u;
-                const int slot = ni % kWarpSlots;
-                unsigned char* dst = myring + (size_t)slot * kStageBytes;
-                const size_t off = (size_t)ti * (kConsumerWarps * kStageVecs * VEC);
-                mbar_expect_tx(&myfull[slot], Db ? 2u * bytes : bytes);
-                bulk_load(dst, Tb + off, bytes, &myfull[slot], pol);
-                if (Db) bulk_load(dst + kStageRowBytes, Db + off, bytes, &myfull[slot], pol);
+                const uint32_t bytes = (uint32_t)min(kStageVecs, nvb - (cw + ti * kConsumerWarps) * kStageVecs) * 16u;
+                unsigned char* dst = myring + (size_t)slot_i * kStageBytes;
+                mbar_expect_tx(&myfull[slot_i], Db ? 2u * bytes : bytes);
+                bulk_load(dst, Tb, bytes, &myfull[slot_i], pol);
+                if (Db) { bulk_load(dst + kStageRowBytes, Db, bytes, &myfull[slot_i], pol); Db += kStride; }
+                Tb += kStride;
+                if (++slot_i == kWarpSlots) slot_i = 0;
                 ++ni;
                 ++ti;
                 if (ti >= endi) {
@@ -484,7 +504,9 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
             if (lane == 0) begin_run();
             if (lane == 0)
                 for (int t = 0; t < kWarpSlots; ++t) issue_next();
-            int n = 0;                    // consume cursor: stages worked on so far
+            int n = 0;                    // consume cursor: stages worked on so far, its slot and parity
+            int slot_c = 0;
+            uint32_t par_c = 0;
             bool ok = true;
             // hand the slot of stage n back and fetch stage n+3 of the walk into it
             auto recycle = [&]() {
@@ -494,6 +516,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
                     issue_next();
                 }
                 ++n;
+                if (++slot_c == kWarpSlots) { slot_c = 0; par_c ^= 1u; }
             };
             float RT = kEmptyRef, RD = kEmptyRef;
             LaneSums ls;
@@ -501,8 +524,8 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
             auto run_pass1 = [&](int j, int t0, int t1) {
                 const bool bonus = ((u0 + j) % K1 == P.k);
                 for (int t = t0; t < t1 && ok; ++t) {
-                    const int slot = n % kWarpSlots;
-                    if (!mbar_wait(&myfull[slot], (uint32_t)(n / kWarpSlots) & 1u, abort)) { ok = false; break; }
+                    const int slot = slot_c;
+                    if (!mbar_wait(&myfull[slot], par_c, abort)) { ok = false; break; }
                     const uint4* st = reinterpret_cast<const uint4*>(myring + (size_t)slot * kStageBytes);
                     const int s = cw + t * kConsumerWarps;
                     const int nv = min(kStageVecs, nvb - s * kStageVecs);     // vectors of this stage
@@ -523,8 +546,8 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
                                : nullptr;
                 float* rsum = P.region_sums + (size_t)unit * P.NR + s0;
                 for (int t = 0; t < nst; ++t) {
-                    const int slot = n % kWarpSlots;
-                    if (!mbar_wait(&myfull[slot], (uint32_t)(n / kWarpSlots) & 1u, abort)) { ok = false; return; }
+                    const int slot = slot_c;
+                    if (!mbar_wait(&myfull[slot], par_c, abort)) { ok = false; return; }
                     const uint4* st = reinterpret_cast<const uint4*>(myring + (size_t)slot * kStageBytes);
                     const int s = cw + t * kConsumerWarps;
                     const int nv = min(kStageVecs, nvb - s * kStageVecs);
