@@ -179,28 +179,24 @@ __device__ __forceinline__ void store_streaming(void* p, const uint4& v) {
 // A stage is kStageGroups vectors per lane and row.  All of them are loaded before any arithmetic; vectors
 // past the end of the row read as -inf, which adds nothing to any sum and is never stored.
 
-// Pass 1: the stage's maxima; if they raise the warp's integer references (RT, RD), the running
-// sums move to the new references (exact: powers of two); then the stage's sums.
+// Pass 1: the stage's softmax sums relative to the warp's integer references (RT, RD), added to
+// the running sums.  References need not be the exact maxima: any integers work as long as nothing
+// overflows, and sums under different references are merged exactly later.  So only the first
+// stage of a unit looks for its maxima first; later stages reuse the references, and a stage whose
+// sums come out too large for comfort (an entry far above everything the warp has seen: rare) is
+// done again by pass1_stage_again after its maxima have raised the references and the running
+// sums have moved with them (exact: powers of two).
+struct Pass1State {
+    float RT, RD;
+    LaneSums ls;
+};
+
+// The stage's maxima raise the references; the running sums follow.
 template <int DT, bool BONUS>
-__device__ __forceinline__ void pass1_stage(const uint4* st, int nv, int lane, float c, float& RT, float& RD,
-                                            LaneSums& ls) {
+__device__ __forceinline__ void raise_references(const uint4 (&rt)[kStageGroups], const uint4 (&rd)[kStageGroups],
+                                                 float c, Pass1State& s) {
     using E = Elem<DT>;
     constexpr int VEC = E::VEC;
-    uint4 rt[kStageGroups], rd[kStageGroups];
-    if (nv == kStageVecs) {
-#pragma unroll
-        for (int g = 0; g < kStageGroups; ++g) {
-            rt[g] = st[g * 32 + lane];
-            if (!BONUS) rd[g] = st[kStageVecs + g * 32 + lane];
-        }
-    } else {
-#pragma unroll
-        for (int g = 0; g < kStageGroups; ++g) {
-            const int vi = g * 32 + lane;
-            rt[g] = vi < nv ? st[vi] : E::masked();
-            if (!BONUS) rd[g] = vi < nv ? st[kStageVecs + vi] : E::masked();
-        }
-    }
     float mT[kStageGroups], mD[kStageGroups];
 #pragma unroll
     for (int g = 0; g < kStageGroups; ++g) {
@@ -212,43 +208,17 @@ __device__ __forceinline__ void pass1_stage(const uint4* st, int nv, int lane, f
             mD[g] = tree_max<VEC>(v);
         }
     }
-    const float lT = tree_max<kStageGroups>(mT), lD = BONUS ? 0.f : tree_max<kStageGroups>(mD);
-    // the references only move when some lane has an entry above them (rare after the first stages)
-    if (__any_sync(0xffffffffu, __fmul_rn(lT, c) > RT || (!BONUS && __fmul_rn(lD, c) > RD))) {
-        const float nT = fmaxf(RT, warp_max_ref(ref_of(lT, c)));
-        const float nD = BONUS ? kEmptyRef : fmaxf(RD, warp_max_ref(ref_of(lD, c)));
-        ls.rescale(nT - RT, nD - RD);
-        RT = nT;
-        RD = nD;
-    }
-    float pT[kStageGroups], pD[kStageGroups], pW[kStageGroups];
-#pragma unroll
-    for (int g = 0; g < kStageGroups; ++g) {
-        float tv[VEC];
-        E::unpack(rt[g], tv);
-        if (!BONUS) {
-            float dv[VEC];
-            E::unpack(rd[g], dv);
-            LaneSums::vector_pair<VEC>(tv, dv, c, -RT, -RD, pT[g], pD[g], pW[g]);
-        } else {
-            pT[g] = LaneSums::vector_bonus<VEC>(tv, c, -RT);
-        }
-    }
-    ls.sT += tree_sum<kStageGroups>(pT);
-    if (!BONUS) {
-        ls.sD += tree_sum<kStageGroups>(pD);
-        ls.w += tree_sum<kStageGroups>(pW);
-    }
+    const float nT = fmaxf(s.RT, warp_max_ref(ref_of(tree_max<kStageGroups>(mT), c)));
+    const float nD = BONUS ? kEmptyRef : fmaxf(s.RD, warp_max_ref(ref_of(tree_max<kStageGroups>(mD), c)));
+    s.ls.rescale(nT - s.RT, nD - s.RD);
+    s.RT = nT;
+    s.RD = nD;
 }
 
-// Pass 2: gradient out (gdst = where the stage's part of the gradient row starts, or null) and
-// the stage's mass (sum of max(0,p-q)/tau, or of p on the bonus row), in every lane.
 template <int DT, bool BONUS>
-__device__ __forceinline__ float pass2_stage(const uint4* st, int nv, int lane, float c, const RowConst& rc,
-                                             typename Elem<DT>::type* gdst) {
+__device__ __forceinline__ void load_stage(const uint4* st, int nv, int lane, uint4 (&rt)[kStageGroups],
+                                           uint4 (&rd)[kStageGroups]) {
     using E = Elem<DT>;
-    constexpr int VEC = E::VEC;
-    uint4 rt[kStageGroups], rd[kStageGroups];
     if (nv == kStageVecs) {
 #pragma unroll
         for (int g = 0; g < kStageGroups; ++g) {
@@ -263,6 +233,72 @@ __device__ __forceinline__ float pass2_stage(const uint4* st, int nv, int lane, 
             if (!BONUS) rd[g] = vi < nv ? st[kStageVecs + vi] : E::masked();
         }
     }
+}
+
+template <int DT, bool BONUS>
+__device__ __forceinline__ void stage_sums(const uint4 (&rt)[kStageGroups], const uint4 (&rd)[kStageGroups], float c,
+                                           float RT, float RD, float& sT, float& sD, float& sW) {
+    using E = Elem<DT>;
+    constexpr int VEC = E::VEC;
+    sT = sD = sW = 0.f;
+#pragma unroll
+    for (int g = 0; g < kStageGroups; ++g) {
+        float tv[VEC];
+        E::unpack(rt[g], tv);
+        if (!BONUS) {
+            float dv[VEC], pT, pD, pW;
+            E::unpack(rd[g], dv);
+            LaneSums::vector_pair<VEC>(tv, dv, c, -RT, -RD, pT, pD, pW);
+            sT += pT;
+            sD += pD;
+            sW += pW;
+        } else {
+            sT += LaneSums::vector_bonus<VEC>(tv, c, -RT);
+        }
+    }
+}
+
+// The slow way, out of line: maxima first, then the sums.
+template <int DT, bool BONUS>
+__device__ __noinline__ Pass1State pass1_stage_again(const uint4* st, int nv, int lane, float c, Pass1State s) {
+    uint4 rt[kStageGroups], rd[kStageGroups];
+    load_stage<DT, BONUS>(st, nv, lane, rt, rd);
+    raise_references<DT, BONUS>(rt, rd, c, s);
+    float sT, sD, sW;
+    stage_sums<DT, BONUS>(rt, rd, c, s.RT, s.RD, sT, sD, sW);
+    s.ls.sT += sT;
+    s.ls.sD += sD;
+    s.ls.w += sW;
+    return s;
+}
+
+template <int DT, bool BONUS>
+__device__ __forceinline__ void pass1_stage(const uint4* st, int nv, int lane, float c, bool first, Pass1State& s) {
+    constexpr float kTooLarge = 1.152921504606846976e18f;   // 2^60
+    uint4 rt[kStageGroups], rd[kStageGroups];
+    load_stage<DT, BONUS>(st, nv, lane, rt, rd);
+    if (first) raise_references<DT, BONUS>(rt, rd, c, s);
+    float sT, sD, sW;
+    stage_sums<DT, BONUS>(rt, rd, c, s.RT, s.RD, sT, sD, sW);
+    // (written so that a NaN counts as too large)
+    if (!first && __any_sync(0xffffffffu, !(sT < kTooLarge) || !(sD < kTooLarge))) {
+        s = pass1_stage_again<DT, BONUS>(st, nv, lane, c, s);
+        return;
+    }
+    s.ls.sT += sT;
+    s.ls.sD += sD;
+    s.ls.w += sW;
+}
+
+// Pass 2: gradient out (gdst = where the stage's part of the gradient row starts, or null) and
+// the stage's mass (sum of max(0,p-q)/tau, or of p on the bonus row), in every lane.
+template <int DT, bool BONUS>
+__device__ __forceinline__ float pass2_stage(const uint4* st, int nv, int lane, float c, const RowConst& rc,
+                                             typename Elem<DT>::type* gdst) {
+    using E = Elem<DT>;
+    constexpr int VEC = E::VEC;
+    uint4 rt[kStageGroups], rd[kStageGroups];
+    load_stage<DT, BONUS>(st, nv, lane, rt, rd);
     float ms[kStageGroups];
 #pragma unroll
     for (int g = 0; g < kStageGroups; ++g) {
@@ -518,9 +554,9 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
                 ++n;
                 if (++slot_c == kWarpSlots) { slot_c = 0; par_c ^= 1u; }
             };
-            float RT = kEmptyRef, RD = kEmptyRef;
-            LaneSums ls;
-            ls.init();
+            Pass1State ps;
+            ps.RT = ps.RD = kEmptyRef;
+            ps.ls.init();
             auto run_pass1 = [&](int j, int t0, int t1) {
                 const bool bonus = ((u0 + j) % K1 == P.k);
                 for (int t = t0; t < t1 && ok; ++t) {
@@ -529,8 +565,8 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
                     const uint4* st = reinterpret_cast<const uint4*>(myring + (size_t)slot * kStageBytes);
                     const int s = cw + t * kConsumerWarps;
                     const int nv = min(kStageVecs, nvb - s * kStageVecs);     // vectors of this stage
-                    if (bonus) pass1_stage<DT, true>(st, nv, lane, P.c, RT, RD, ls);
-                    else       pass1_stage<DT, false>(st, nv, lane, P.c, RT, RD, ls);
+                    if (bonus) pass1_stage<DT, true>(st, nv, lane, P.c, t == 0, ps);
+                    else       pass1_stage<DT, false>(st, nv, lane, P.c, t == 0, ps);
                     recycle();
                 }
             };
@@ -570,13 +606,13 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
                 if (ok) run_pass1(j, head, nst);
                 if (!ok) break;
                 // pass 1 of the unit is over: the warp's partial for the statistics warp
-                const PartialStats part = warp_sum_lanes(ls, RT, RD);
+                const PartialStats part = warp_sum_lanes(ps.ls, ps.RT, ps.RD);
                 if (lane == 0) {
                     sh.wpart[j & 1][cw] = part;
                     mbar_arrive(&sh.s1_done[j & 1]);
                 }
-                RT = RD = kEmptyRef;
-                ls.init();
+                ps.RT = ps.RD = kEmptyRef;
+                ps.ls.init();
             }
             if (ok) run_pass2(nu - 1);
             // leaving early: no copy of this warp may still be in flight when the block returns

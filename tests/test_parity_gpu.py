@@ -273,6 +273,26 @@ def test_shifted_and_huge_logits(binding):
     check(inp, out, oracle_of(inp), max_band_frac=1.0)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_late_spike_far_above_everything_seen(binding, dtype, monkeypatch):
+    """A logit that towers over all earlier ones late in a row: the fast path works with the
+    references it has and must notice that this stage needs new ones."""
+    monkeypatch.setenv("SD_VERIFY_CLUSTER", "1")          # one block per row: many stages per warp
+    cfg = synth.custom_config(B=3, k=2, V=131072, dtype=dtype, t_sigma=1.0, d_sigma=0.5, index=64)
+    inp = synth.make_inputs(cfg)
+    big = np.float32(300.0) if dtype == "f32" else synth.f32_to_bf16_bits(np.array([300.0], np.float32))[0]
+    inp.target_logits[0, 0, 120000] = big                  # target only
+    inp.draft_logits[1, 1, 99999] = big                    # draft only
+    inp.target_logits[2, 1, 70001] = big                   # both, different places
+    inp.draft_logits[2, 1, 130000] = big
+    inp.target_logits[2, 2, 131071] = big                  # bonus row, last entry
+    T, D, x, u = to_device(inp)
+    out = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
+    torch.cuda.synchronize()
+    assert binding.sd_launch_info()["path"] == 1
+    check(inp, out, oracle_of(inp), max_band_frac=1.0)
+
+
 def test_all_equal_logits(binding):
     cfg = synth.custom_config(B=2, k=2, V=777, dtype="f32", index=57)
     inp = synth.make_inputs(cfg)
