@@ -235,6 +235,19 @@ __device__ __forceinline__ void load_stage(const uint4* st, int nv, int lane, ui
     }
 }
 
+// Returns only when every vector of the stage has arrived in this lane's registers (the value
+// depends on all of them), so that the stage's slot may be overwritten afterwards.
+template <bool BONUS>
+__device__ __forceinline__ void await_stage_registers(const uint4 (&rt)[kStageGroups], const uint4 (&rd)[kStageGroups]) {
+    uint32_t dep = 0;
+#pragma unroll
+    for (int g = 0; g < kStageGroups; ++g) {
+        dep ^= rt[g].w;
+        if (!BONUS) dep ^= rd[g].w;
+    }
+    asm volatile("" ::"r"(dep) : "memory");
+}
+
 template <int DT, bool BONUS>
 __device__ __forceinline__ void stage_sums(const uint4 (&rt)[kStageGroups], const uint4 (&rd)[kStageGroups], float c,
                                            float RT, float RD, float& sT, float& sD, float& sW) {
@@ -258,11 +271,20 @@ __device__ __forceinline__ void stage_sums(const uint4 (&rt)[kStageGroups], cons
     }
 }
 
-// The slow way, out of line: maxima first, then the sums.
+// The slow way, out of line: maxima first, then the sums.  By now the stage's slot in the ring
+// has been handed back, so the stage is read once more from global memory (gT, gD: where it
+// starts in the two rows).
 template <int DT, bool BONUS>
-__device__ __noinline__ Pass1State pass1_stage_again(const uint4* st, int nv, int lane, float c, Pass1State s) {
+__device__ __noinline__ Pass1State pass1_stage_again(const uint4* gT, const uint4* gD, int nv, int lane, float c,
+                                                     Pass1State s) {
+    using E = Elem<DT>;
     uint4 rt[kStageGroups], rd[kStageGroups];
-    load_stage<DT, BONUS>(st, nv, lane, rt, rd);
+#pragma unroll
+    for (int g = 0; g < kStageGroups; ++g) {
+        const int vi = g * 32 + lane;
+        rt[g] = vi < nv ? __ldg(gT + vi) : E::masked();
+        if (!BONUS) rd[g] = vi < nv ? __ldg(gD + vi) : E::masked();
+    }
     raise_references<DT, BONUS>(rt, rd, c, s);
     float sT, sD, sW;
     stage_sums<DT, BONUS>(rt, rd, c, s.RT, s.RD, sT, sD, sW);
@@ -272,17 +294,21 @@ __device__ __noinline__ Pass1State pass1_stage_again(const uint4* st, int nv, in
     return s;
 }
 
-template <int DT, bool BONUS>
-__device__ __forceinline__ void pass1_stage(const uint4* st, int nv, int lane, float c, bool first, Pass1State& s) {
+// `handed_back` is called once the stage is in registers: the caller refills the slot then.
+template <int DT, bool BONUS, class F>
+__device__ __forceinline__ void pass1_stage(const uint4* st, const uint4* gT, const uint4* gD, int nv, int lane, float c,
+                                            bool first, Pass1State& s, F&& handed_back) {
     constexpr float kTooLarge = 1.152921504606846976e18f;   // 2^60
     uint4 rt[kStageGroups], rd[kStageGroups];
     load_stage<DT, BONUS>(st, nv, lane, rt, rd);
+    await_stage_registers<BONUS>(rt, rd);
+    handed_back();
     if (first) raise_references<DT, BONUS>(rt, rd, c, s);
     float sT, sD, sW;
     stage_sums<DT, BONUS>(rt, rd, c, s.RT, s.RD, sT, sD, sW);
     // (written so that a NaN counts as too large)
     if (!first && __any_sync(0xffffffffu, !(sT < kTooLarge) || !(sD < kTooLarge))) {
-        s = pass1_stage_again<DT, BONUS>(st, nv, lane, c, s);
+        s = pass1_stage_again<DT, BONUS>(gT, gD, nv, lane, c, s);
         return;
     }
     s.ls.sT += sT;
@@ -292,13 +318,15 @@ __device__ __forceinline__ void pass1_stage(const uint4* st, int nv, int lane, f
 
 // Pass 2: gradient out (gdst = where the stage's part of the gradient row starts, or null) and
 // the stage's mass (sum of max(0,p-q)/tau, or of p on the bonus row), in every lane.
-template <int DT, bool BONUS>
+template <int DT, bool BONUS, class F>
 __device__ __forceinline__ float pass2_stage(const uint4* st, int nv, int lane, float c, const RowConst& rc,
-                                             typename Elem<DT>::type* gdst) {
+                                             typename Elem<DT>::type* gdst, F&& handed_back) {
     using E = Elem<DT>;
     constexpr int VEC = E::VEC;
     uint4 rt[kStageGroups], rd[kStageGroups];
     load_stage<DT, BONUS>(st, nv, lane, rt, rd);
+    await_stage_registers<BONUS>(rt, rd);
+    handed_back();
     float ms[kStageGroups];
 #pragma unroll
     for (int g = 0; g < kStageGroups; ++g) {
@@ -544,13 +572,11 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
             int slot_c = 0;
             uint32_t par_c = 0;
             bool ok = true;
-            // hand the slot of stage n back and fetch stage n+3 of the walk into it
+            // The stage is in registers: hand its slot back and fetch stage n+3 of the walk into it.
+            // (Every lane's loads from the slot have returned their values before the copy is issued.)
             auto recycle = [&]() {
                 __syncwarp();
-                if (lane == 0) {
-                    fence_proxy_async();   // the warp's reads of the slot come before the copy that refills it
-                    issue_next();
-                }
+                if (lane == 0) issue_next();
                 ++n;
                 if (++slot_c == kWarpSlots) { slot_c = 0; par_c ^= 1u; }
             };
@@ -558,16 +584,22 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
             ps.RT = ps.RD = kEmptyRef;
             ps.ls.init();
             auto run_pass1 = [&](int j, int t0, int t1) {
-                const bool bonus = ((u0 + j) % K1 == P.k);
+                const int unit = u0 + j;
+                const int b = unit / K1, i = unit - b * K1;
+                const bool bonus = (i == P.k);
+                // the block's slice of the two rows in global memory (for the rare second try of a stage)
+                const ET* Trow = reinterpret_cast<const ET*>(P.T) + (size_t)unit * P.V + (size_t)vb0 * VEC;
+                const ET* Drow = reinterpret_cast<const ET*>(P.D) + (size_t)(b * P.k + (bonus ? 0 : i)) * P.V + (size_t)vb0 * VEC;
                 for (int t = t0; t < t1 && ok; ++t) {
                     const int slot = slot_c;
                     if (!mbar_wait(&myfull[slot], par_c, abort)) { ok = false; break; }
                     const uint4* st = reinterpret_cast<const uint4*>(myring + (size_t)slot * kStageBytes);
                     const int s = cw + t * kConsumerWarps;
                     const int nv = min(kStageVecs, nvb - s * kStageVecs);     // vectors of this stage
-                    if (bonus) pass1_stage<DT, true>(st, nv, lane, P.c, t == 0, ps);
-                    else       pass1_stage<DT, false>(st, nv, lane, P.c, t == 0, ps);
-                    recycle();
+                    const uint4* gT = reinterpret_cast<const uint4*>(Trow) + (size_t)s * kStageVecs;
+                    const uint4* gD = reinterpret_cast<const uint4*>(Drow) + (size_t)s * kStageVecs;
+                    if (bonus) pass1_stage<DT, true>(st, gT, gD, nv, lane, P.c, t == 0, ps, recycle);
+                    else       pass1_stage<DT, false>(st, gT, gD, nv, lane, P.c, t == 0, ps, recycle);
                 }
             };
             auto run_pass2 = [&](int j) {
@@ -587,11 +619,11 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
                     const uint4* st = reinterpret_cast<const uint4*>(myring + (size_t)slot * kStageBytes);
                     const int s = cw + t * kConsumerWarps;
                     const int nv = min(kStageVecs, nvb - s * kStageVecs);
-                    const float mass = bonus ? pass2_stage<DT, true>(st, nv, lane, P.c, rc, nullptr)
+                    const float mass = bonus ? pass2_stage<DT, true>(st, nv, lane, P.c, rc, nullptr, recycle)
                                              : pass2_stage<DT, false>(st, nv, lane, P.c, rc,
-                                                                      Grow ? Grow + (size_t)s * kStageVecs * VEC : nullptr);
+                                                                      Grow ? Grow + (size_t)s * kStageVecs * VEC : nullptr,
+                                                                      recycle);
                     if (lane == 0) rsum[s] = mass;
-                    recycle();
                 }
                 // the resolver's slot of unit j-4 must be free again before this unit is reported done
                 if (j >= kDoneDepth &&
