@@ -188,16 +188,16 @@ int choose_stream(DeviceState& d, int V, long long units, int dtype, int* G_out,
     const int forced = env ? atoi(env) : 0;
     const char* env_l2 = getenv("SD_VERIFY_L2_MIB");
     const double l2_budget = (env_l2 ? atof(env_l2) : kL2BudgetMiB) * 1048576.0;
+    const char* env_lag = getenv("SD_VERIFY_LAG");
+    const int lag = env_lag ? atoi(env_lag) : 1;   // stages of the next unit before pass 2 of a unit
     if (d.dec_dtype == dtype && d.dec_V == V && d.dec_units == units && d.dec_forced == forced &&
-        d.dec_l2 == l2_budget) {
+        d.dec_l2 == l2_budget && d.dec_lag == lag) {
         *G_out = d.dec_G;
         *per_out = d.dec_per;
         *lag_out = d.dec_lag;
         return d.dec_C;
     }
     const int NV = V / vec_elems(dtype);
-    const char* env_lag = getenv("SD_VERIFY_LAG");
-    const int lag = env_lag ? atoi(env_lag) : 1;   // stages of the next unit before pass 2 of a unit
     int best_C = 0, best_G = 0, best_per = 0;
     long long best_busy = -1;
     bool best_fits = false;

@@ -192,13 +192,42 @@ def test_largest_k(binding):
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-@pytest.mark.parametrize("cluster", [1, 2, 4, 8, 16])
+@pytest.mark.parametrize("cluster", [1, 2, 3, 4, 5, 8, 9, 16])
 def test_every_cluster_size_gives_the_same_answer(binding, dtype, cluster, monkeypatch):
     cfg = synth.custom_config(B=3, k=3, V=24000 if dtype == "f32" else 48000, dtype=dtype, tau=1.2, index=52)
     monkeypatch.setenv("SD_VERIFY_CLUSTER", str(cluster))
     inp, out, ref = run_and_check(binding, cfg, ex=True, max_band_frac=1.0)
     info = binding.sd_launch_info()
     assert info["path"] == 1 and info["cluster_size"] == cluster
+
+
+@pytest.mark.parametrize("lag", [0, 1, 2, 100])
+@pytest.mark.parametrize("cluster", [1, 3])
+def test_every_order_of_the_two_passes_gives_the_same_answer(binding, lag, cluster, monkeypatch):
+    """Pass 2 of a unit may come 0, 1, 2 ... stages (per warp) into pass 1 of the next unit, or after
+    all of it; several units per cluster, rows long enough for several stages per warp."""
+    cfg = synth.custom_config(B=40, k=3, V=100000, dtype="bf16", tau=1.1, index=65)
+    monkeypatch.setenv("SD_VERIFY_CLUSTER", str(cluster))
+    monkeypatch.setenv("SD_VERIFY_LAG", str(lag))
+    inp = synth.make_inputs(cfg)
+    T, D, x, u = to_device(inp)
+    out = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
+    torch.cuda.synchronize()
+    info = binding.sd_launch_info()
+    assert info["path"] == 1 and info["cluster_size"] == cluster
+    seqs = [0, 1, 13, 26, 39]
+    check(inp, out, oracle_of(inp, seqs), seqs=seqs, max_band_frac=1.0)
+    base = getattr(test_every_order_of_the_two_passes_gives_the_same_answer, "_base", None)
+    key = (cluster,)
+    if base is None or key not in base:
+        base = base or {}
+        base[key] = out
+        test_every_order_of_the_two_passes_gives_the_same_answer._base = base
+    else:   # the order of the passes changes no bit of any output
+        ref = base[key]
+        assert torch.equal(ref.accept_len, out.accept_len) and torch.equal(ref.tokens, out.tokens)
+        assert torch.equal(ref.loss, out.loss)
+        assert torch.equal(ref.grad_draft.view(torch.int16), out.grad_draft.view(torch.int16))
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
