@@ -39,9 +39,9 @@ from paper_2603_12617_b200 import synth  # noqa: E402
 METRIC = "verified draft positions/sec"
 UNIT = "positions/s"
 L2_BYTES = 126 * 1024 * 1024
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
-# profiles/ (bytes; None = not captured for that workload)
-NCU_TRAFFIC_BYTES = {}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch at full size, from the ncu captures
+# summarised under profiles/ (bytes; a workload that is not listed has not been captured)
+NCU_TRAFFIC_BYTES = {"cfg5": 2692059136 + 756199936, "cfg3": 174112768 + 33039360, "cfg4": 190112000 + 46578176}
 
 
 def measured_peak_gbs():
@@ -294,9 +294,9 @@ def run_ours(args, cfg):
     peak, peak_src = measured_peak_gbs()
     achieved = cfg.algorithmic_bytes / (mean_kernel_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": NCU_TRAFFIC_BYTES.get(cfg.name), "peak_source": peak_src,
+                "traffic": NCU_TRAFFIC_BYTES.get(cfg.name) if not args.batch else None, "peak_source": peak_src,
                 "algorithmic_bytes_per_launch": cfg.algorithmic_bytes, "kernel_ms_mean": mean_kernel_ms,
-                "kernel_ms_min": float(np.min(kernel_ms)), "kernel": "sd_cluster_kernel" if info["path"] == 1 else "sd_generic_kernel",
+                "kernel_ms_min": float(np.min(kernel_ms)), "kernel": "sd_stream_kernel" if info["path"] == 1 else "sd_generic_kernel",
                 "frac_of_nominal_8000_GBps": achieved / 8000.0}
     base = cpu_baseline(cfg, inp) if not args.no_cpu_baseline else None
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
