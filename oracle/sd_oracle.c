@@ -248,6 +248,51 @@ int sd_oracle(const void* T, const void* D, int dtype, const int32_t* x, const f
     return failed ? -1 : 0;
 }
 
+/*
+ * sd_oracle_greedy -- verification under greedy decoding (the setting of the paper's experiments,
+ * "greedy decoding is adopted unless otherwise specified", Sec. 4.1): Algorithm 1 in the limit
+ * tau -> 0, where the target distribution of every position is the point mass on its largest
+ * logit.  The rejection test then accepts a draft token iff it is the target's argmax of its
+ * position (p/q is 1 for it when the draft was decoded greedily too, 0 for anything else), and
+ * the residual max(0, p - q) as well as the bonus distribution are the point mass on the target's
+ * argmax, so no random numbers are involved.
+ *   argmax[b,i]   = smallest v with T[b,i,v] = max_w T[b,i,w], i = 0..k   (ties: first index)
+ *   n_b           = first i < k with x[b,i] != argmax[b,i], else k
+ *   tokens[b]     = x[b,0..n_b-1], argmax[b,n_b], -1 ...
+ * T [B,k+1,V] in `dtype`, x [B,k]; out_accept_len [B], out_tokens [B,k+1], out_argmax [B,k+1] or
+ * NULL.  A row without any entry above -inf (or with only NaN) has argmax 0.  Returns 0, or -1 on
+ * a bad argument.
+ */
+int sd_oracle_greedy(const void* T, int dtype, const int32_t* x, int B, int k, int V,
+                     int32_t* out_accept_len, int32_t* out_tokens, int32_t* out_argmax) {
+    if (!T || !x || !out_accept_len || !out_tokens) return -1;
+    if (B < 1 || k < 1 || V < 1) return -1;
+    if (dtype != SD_ORACLE_F32 && dtype != SD_ORACLE_BF16) return -1;
+    for (int b = 0; b < B; ++b) {
+        int n = k;
+        int32_t* tok = out_tokens + (size_t)b * (k + 1);
+        for (int i = 0; i <= k; ++i) {
+            size_t off = ((size_t)b * (k + 1) + i) * (size_t)V;
+            int best = 0;
+            double bestv = -INFINITY;
+            for (int v = 0; v < V; ++v) {
+                double z = logit_at(T, dtype, off + (size_t)v);
+                if (z > bestv) {
+                    bestv = z;
+                    best = v;
+                }
+            }
+            if (out_argmax) out_argmax[(size_t)b * (k + 1) + i] = best;
+            tok[i] = best; /* for now: the argmax of every row */
+            if (i < k && n == k && x[(size_t)b * k + i] != best) n = i;
+        }
+        out_accept_len[b] = n;
+        int32_t y = tok[n];
+        for (int i = 0; i <= k; ++i) tok[i] = (i < n) ? x[(size_t)b * k + i] : (i == n ? y : -1);
+    }
+    return 0;
+}
+
 /* Threads the build can use: 1 without OpenMP. */
 int sd_oracle_max_threads(void) {
 #ifdef _OPENMP

