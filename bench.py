@@ -18,6 +18,10 @@ draw, KL loss and its gradient) over one batch.  Prints ONE JSON line (rank 0).
 
 With N > 1 (launched by torch.distributed.run) every rank runs the full batch of its own
 (weak scaling: sequences are independent, no collective on the path).
+
+  --path greedy   times greedy verification instead (Algorithm 1 in the limit tau -> 0, the decoding
+             mode of the paper's experiments): only the target logits are read, (k+1)*V*B entries per
+             launch; the line has the same keys, with "path": "greedy" in config.  Not the headline.
 """
 from __future__ import annotations
 
@@ -313,6 +317,119 @@ def run_ours(args, cfg):
         dist.destroy_process_group()
 
 
+def run_greedy(args, cfg):
+    """--path greedy: sd_verify_greedy on the target logits of the workload, one GPU per rank."""
+    import torch
+    import torch.distributed as dist
+
+    import __graft_entry__ as entry
+    entry.build()
+    from paper_2603_12617_b200 import binding, shard
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    inp = synth.make_inputs(cfg, seed=synth.BASE_SEED + 1000 * rank)
+    hT = torch.from_numpy(inp.target_logits)
+    if inp.target_logits.dtype == np.uint16:
+        hT = hT.view(torch.bfloat16)
+    hT = hT.pin_memory()
+    # greedy drafting proposes the draft's argmax; the inputs carry sampled tokens, which serves as well:
+    # the work does not depend on the tokens
+    hx = torch.from_numpy(inp.draft_tokens).pin_memory()
+    in_bytes = hT.numel() * hT.element_size()
+    nsets = 1 if in_bytes > 2 * L2_BYTES else int(min(64, -(-3 * L2_BYTES // in_bytes)))
+    sets = [(hT.to(dev), hx.to(dev)) for _ in range(nsets)]
+    out = binding.sd_verify_greedy(*sets[0])
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(3, args.warmup)):
+        binding.sd_verify_greedy(*sets[i % nsets], out=out)
+    info = binding.sd_launch_info()
+    barrier()
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        t_begin.record()
+        for i in range(args.steps):
+            starts[i].record()
+            binding.sd_verify_greedy(*sets[i % nsets], out=out)
+            ends[i].record()
+        t_end.record()
+        barrier()
+    total_ms = shard.max_over_ranks(t_begin.elapsed_time(t_end), device=str(dev) if world > 1 else "cpu")
+    kernel_ms = [s.elapsed_time(e) for s, e in zip(starts, ends)]
+    mean_kernel_ms = float(np.mean(kernel_ms))
+    positions = cfg.B * cfg.k * world
+    value = positions * args.steps / (total_ms * 1e-3)
+
+    # end to end: pinned host logits in, results back to the host, every copy inside the region
+    e2e_steps = max(1, min(args.steps, 10))
+    dT, dx = torch.empty_like(sets[0][0]), torch.empty_like(sets[0][1])
+    h_n = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
+    h_tok = torch.empty((cfg.B, cfg.k + 1), dtype=torch.int32).pin_memory()
+
+    def e2e_step():
+        dT.copy_(hT, non_blocking=True)
+        dx.copy_(hx, non_blocking=True)
+        binding.sd_verify_greedy(dT, dx, out=out)
+        h_n.copy_(out.accept_len, non_blocking=True)
+        h_tok.copy_(out.tokens, non_blocking=True)
+        torch.cuda.synchronize()
+
+    e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    barrier()
+    e2e_s = shard.max_over_ranks(time.perf_counter() - t0, device=str(dev) if world > 1 else "cpu")
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    from oracle import sd_oracle
+    t0 = time.perf_counter()
+    ref = sd_oracle.verify_greedy(inp.target_logits, inp.draft_tokens)
+    t_cpu = time.perf_counter() - t0
+    verified = bool((h_n.numpy() == ref.accept_len).all() and (h_tok.numpy() == ref.tokens).all()
+                    and (out.argmax.cpu().numpy() == ref.argmax).all())
+    algo = (cfg.k + 1) * cfg.V * cfg.B * cfg.elem_bytes
+    peak, peak_src = measured_peak_gbs()
+    achieved = algo / (mean_kernel_ms * 1e-3) / 1e9
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32 comparisons" if cfg.dtype == "f32" else "bf16 comparisons",
+            "data": "synthetic",
+            "config": workload_config(cfg, path="greedy", l2="inputs larger than L2" if nsets == 1 else f"{nsets} rotating input sets larger than L2 together",
+                                      parallelism=f"replicas x{world}, sequences independent, no collective", launch=info),
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": None, "peak_source": peak_src, "algorithmic_bytes_per_launch": algo,
+                         "kernel_ms_mean": mean_kernel_ms, "kernel_ms_min": float(np.min(kernel_ms)),
+                         "kernel": "sd_greedy_kernel"},
+            "cpu_baseline": {"value": cfg.B * cfg.k / t_cpu, "unit": UNIT, "cores": 1, "kind": "oracle",
+                             "sample": f"all {cfg.B} sequences of {cfg.name}, one call, {t_cpu:.2f} s"},
+            "e2e": {"value": positions * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": int(in_bytes + hx.numel() * 4),
+                    "d2h_bytes_per_step": int(h_n.numel() * 4 + h_tok.numel() * 4), "steps": e2e_steps,
+                    "ms_per_step": e2e_s / e2e_steps * 1e3, "entry_point": "sd_verify_greedy between pinned-memory copies"},
+            "gpu_launches": args.steps * info["kernels"], "clocks": clocks.summary(),
+            "outputs_verified_against_oracle": verified}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -322,12 +439,16 @@ def main():
     ap.add_argument("--config", default="cfg5", choices=sorted(synth.CONFIGS))
     ap.add_argument("--batch", type=int, default=0, help="override B (profiling on a smaller case)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--path", choices=["sample", "greedy"], default="sample",
+                    help="sample: the verify-and-feedback step (the headline); greedy: greedy verification")
     args = ap.parse_args()
     cfg = synth.CONFIGS[args.config]
     if args.batch:
         cfg = cfg.with_batch(args.batch)
     if args.impl == "reference":
         run_reference(args, cfg)
+    elif args.path == "greedy":
+        run_greedy(args, cfg)
     else:
         run_ours(args, cfg)
 

@@ -167,6 +167,36 @@ int sd_verify_feedback_static(const void* target_logits, const void* draft_logit
 size_t sd_workspace_bytes(int B, int k, int V, int dtype);
 
 /*
+ * sd_verify_greedy -- verification under greedy decoding: Algorithm 1 in the limit tau -> 0, the
+ * decoding mode of the paper's experiments ("greedy decoding is adopted unless otherwise
+ * specified", Sec. 4.1 Implementation Details).  The target distribution of a position is then
+ * the point mass on its largest logit: a draft token is accepted iff it is the target's argmax of
+ * its position, and the extra token is the target's argmax at the first mismatch, or at the bonus
+ * position when everything was accepted.  No random numbers, no draft logits; only the target
+ * logits are read, once.  (For the feedback loss of the same round call sd_verify_feedback_ex
+ * with the temperature of the loss.)
+ *
+ *   target_logits  [B, k+1, V]  in   `dtype`; ties go to the smallest index; NaN entries are
+ *                                    ignored; a row without an entry above -inf has argmax 0
+ *   draft_tokens   [B, k]       in   int32; a token outside [0,V) simply matches nothing
+ *   out_accept_len [B]          out  int32 n_b in [0,k]
+ *   out_tokens     [B, k+1]     out  int32: x[b,0..n_b-1], argmax T[b,n_b,:] at index n_b, then -1
+ *   out_argmax     [B, k+1]     out  int32 argmax of every target row, or NULL
+ *   workspace                   in   device scratch of at least sd_greedy_workspace_bytes(B,k) bytes,
+ *                                    aligned to 256 bytes, or NULL to use the library's own scratch
+ *                                    (allocated and grown on demand, shared with sd_verify_feedback)
+ *   stream                      in   cudaStream_t
+ * Rows whose byte length and base address are multiples of 16 are read with 16-byte loads, all
+ * others element by element.  Returns SD_OK or a negative SD_ERR_* code (nothing enqueued).
+ */
+int sd_verify_greedy(const void* target_logits, const int32_t* draft_tokens, int B, int k, int V,
+                     int dtype, int32_t* out_accept_len, int32_t* out_tokens, int32_t* out_argmax,
+                     void* workspace, size_t workspace_bytes, void* stream);
+
+/* Bytes of scratch sd_verify_greedy needs for this shape; 0 if the shape is invalid. */
+size_t sd_greedy_workspace_bytes(int B, int k);
+
+/*
  * sd_verify_feedback_host -- the same step for callers whose tensors live in HOST memory.
  * Every pointer is a HOST pointer (pinned memory gives asynchronous copies, pageable memory
  * works too).  The call copies the inputs to device buffers the library keeps per device
@@ -182,7 +212,7 @@ int sd_verify_feedback_host(const void* target_logits, const void* draft_logits,
 
 /*
  * sd_launch_info -- HOST out-parameters describing how the last successful device call on this
- * thread was launched: path (0 = generic, 1 = cluster fast path), cluster size, threads per
+ * thread was launched: path (0 = generic, 1 = stream fast path, 2 = greedy verification), cluster size, threads per
  * block, dynamic shared memory per block, blocks launched, kernels launched.  Any pointer may
  * be NULL.  Diagnostic only.
  */

@@ -49,6 +49,10 @@ def _load() -> ctypes.CDLL:
     lib.sd_verify_feedback_ex.argtypes = [P, P, P, P, F, I, I, I, I, P, P, P, P, P, P, P, Z, P]
     lib.sd_verify_feedback_static.restype = I
     lib.sd_verify_feedback_static.argtypes = [P, P, P, P, F, I, I, I, I, P, P, P, P, P, P, P]
+    lib.sd_verify_greedy.restype = I
+    lib.sd_verify_greedy.argtypes = [P, P, I, I, I, I, P, P, P, P, Z, P]
+    lib.sd_greedy_workspace_bytes.restype = Z
+    lib.sd_greedy_workspace_bytes.argtypes = [I, I]
     lib.sd_verify_feedback_host.restype = I
     lib.sd_verify_feedback_host.argtypes = [P, P, P, P, F, I, I, I, I, P, P, P, P, P, P]
     lib.sd_workspace_bytes.restype = Z
@@ -189,6 +193,45 @@ def sd_verify_feedback_ex(target_logits: torch.Tensor, draft_logits: torch.Tenso
             _stream_ptr(stream))
     if rc != 0:
         raise SdVerifyError(rc, "sd_verify_feedback_ex")
+    return out
+
+
+@dataclass
+class GreedyOutputs:
+    accept_len: torch.Tensor            # [B] int32
+    tokens: torch.Tensor                # [B,k+1] int32, -1 padded
+    argmax: Optional[torch.Tensor]      # [B,k+1] int32
+
+
+def sd_greedy_workspace_bytes(B: int, k: int) -> int:
+    return int(_lib.sd_greedy_workspace_bytes(B, k))
+
+
+def sd_verify_greedy(target_logits: torch.Tensor, draft_tokens: torch.Tensor, *, want_argmax: bool = True,
+                     workspace: Optional[torch.Tensor] = None, out: Optional[GreedyOutputs] = None,
+                     stream: Optional[torch.cuda.Stream] = None) -> GreedyOutputs:
+    """``sd_verify_greedy`` on device tensors: accept iff the draft token is the target's argmax."""
+    if target_logits.dim() != 3 or not target_logits.is_contiguous():
+        raise ValueError("target logits must be contiguous [B,k+1,V]")
+    B, k1, V = target_logits.shape
+    k = k1 - 1
+    if tuple(draft_tokens.shape) != (B, k) or draft_tokens.dtype != torch.int32 or not draft_tokens.is_contiguous():
+        raise ValueError("draft_tokens must be contiguous int32 [B,k]")
+    dev = target_logits.device
+    if dev.type != "cuda":
+        raise ValueError("device tensors required")
+    code = _dtype_code(target_logits)
+    if out is None:
+        out = GreedyOutputs(accept_len=torch.empty(B, dtype=torch.int32, device=dev),
+                            tokens=torch.empty((B, k + 1), dtype=torch.int32, device=dev),
+                            argmax=torch.empty((B, k + 1), dtype=torch.int32, device=dev) if want_argmax else None)
+    with torch.cuda.device(dev):
+        rc = _lib.sd_verify_greedy(_ptr(target_logits), _ptr(draft_tokens), B, k, V, code, _ptr(out.accept_len),
+                                   _ptr(out.tokens), _ptr(out.argmax), _ptr(workspace),
+                                   0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                   _stream_ptr(stream))
+    if rc != 0:
+        raise SdVerifyError(rc, "sd_verify_greedy")
     return out
 
 

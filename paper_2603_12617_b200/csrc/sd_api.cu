@@ -8,6 +8,7 @@
 #include <mutex>
 
 #include "sd_kernels.cuh"
+#include "sd_greedy.cuh"
 
 namespace {
 
@@ -79,6 +80,7 @@ struct DeviceState {
     void* ws = nullptr;
     size_t ws_bytes = 0;
     bool ws_clean = false;   // tickets and status words are zero
+    size_t ws_zero_bytes = 0;   // leading bytes of ws known to be zero (what greedy verification needs)
     bool attr_set[2] = {false, false};   // shared-memory / cluster attributes of the fast kernel
     int max_clusters[2][kMaxCluster + 1];   // resident clusters of 1..16 blocks, -1 = not asked yet
     // last launch-shape decision of the fast path
@@ -323,6 +325,7 @@ int run_cached(const void* T, const void* D, const int32_t* x, const float* u, f
         SD_CUDA(cudaDeviceSynchronize());
         d->ws_clean = true;
     }
+    d->ws_zero_bytes = 0;   // row constants and sums of this call stay behind
     rc = run_device(*d, T, D, x, u, tau, B, k, V, dtype, accept_len, tokens, loss, grad, nullptr, nullptr,
                     static_cast<unsigned char*>(d->ws), L, d->ws_clean, static_cast<cudaStream_t>(stream));
     d->ws_clean = (rc == SD_OK);   // a failed launch may leave tickets behind: zero them next time
@@ -428,6 +431,85 @@ int sd_verify_feedback_static(const void* target_logits, const void* draft_logit
     return run_device(*d, target_logits, draft_logits, draft_tokens, uniforms, temperature, B, k, V, dtype,
                       out_accept_len, out_tokens, out_loss, out_grad_draft, out_acc_prob, out_status, scratch, L, false,
                       static_cast<cudaStream_t>(stream));
+}
+
+size_t sd_greedy_workspace_bytes(int B, int k) {
+    if (B < 1 || k < 1 || k > SD_MAX_K || (long double)B * (k + 1) >= 2.0e9L) return 0;
+    return kAlign + align_up((size_t)B * (k + 1) * 8, kAlign);   // ticket word, keys
+}
+
+int sd_verify_greedy(const void* target_logits, const int32_t* draft_tokens, int B, int k, int V, int dtype,
+                     int32_t* out_accept_len, int32_t* out_tokens, int32_t* out_argmax, void* workspace,
+                     size_t workspace_bytes, void* stream) {
+    if (dtype != SD_DTYPE_F32 && dtype != SD_DTYPE_BF16) return SD_ERR_DTYPE;
+    if (!target_logits || !draft_tokens || !out_accept_len || !out_tokens) return SD_ERR_NULL;
+    if (!shape_ok(B, k, V)) return SD_ERR_SHAPE;
+    const size_t es = (size_t)elem_bytes(dtype);
+    if (!aligned(target_logits, es) || !aligned(draft_tokens, 4) || !aligned(out_accept_len, 4) ||
+        !aligned(out_tokens, 4) || (out_argmax && !aligned(out_argmax, 4)))
+        return SD_ERR_ALIGN;
+    const size_t need = sd_greedy_workspace_bytes(B, k);
+    if (workspace && (!aligned(workspace, kAlign) || workspace_bytes < need)) return SD_ERR_WORKSPACE;
+    int dev;
+    DeviceState* d = nullptr;
+    int rc = current_device(&dev, &d);
+    if (rc != SD_OK) return rc;
+    std::lock_guard<std::mutex> lock(d->mu);
+    unsigned char* ws = static_cast<unsigned char*>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // The kernel wants its ticket word and keys zero and leaves them zero.  A caller's workspace is
+    // cleared every call; the library's own scratch (shared with sd_verify_feedback, grown on
+    // demand) only when something else has written there since.
+    bool clean = false;
+    if (!ws) {
+        if (d->ws_bytes < need) {
+            if (d->ws) {
+                SD_CUDA(cudaDeviceSynchronize());
+                SD_CUDA(cudaFree(d->ws));
+                d->ws = nullptr;
+                d->ws_bytes = 0;
+            }
+            const size_t want = align_up(need + need / 4, 1 << 20);
+            SD_CUDA(cudaMalloc(&d->ws, want));
+            d->ws_bytes = want;
+            SD_CUDA(cudaMemset(d->ws, 0, want));
+            SD_CUDA(cudaDeviceSynchronize());
+            d->ws_clean = true;
+            d->ws_zero_bytes = want;
+        }
+        ws = static_cast<unsigned char*>(d->ws);
+        clean = d->ws_zero_bytes >= need;
+    }
+    if (!clean) SD_CUDA(cudaMemsetAsync(ws, 0, need, st));
+    GreedyParams P;
+    memset(&P, 0, sizeof P);
+    P.T = target_logits; P.x = draft_tokens;
+    P.B = B; P.k = k; P.V = V;
+    P.accept_len = out_accept_len; P.tokens = out_tokens; P.argmax = out_argmax;
+    P.ticket = reinterpret_cast<uint32_t*>(ws);
+    P.keys = reinterpret_cast<unsigned long long*>(ws + kAlign);
+    const int item_elems = kGreedyItemVecs * vec_elems(dtype);
+    P.items_per_row = (V + item_elems - 1) / item_elems;
+    P.vectorised = (((size_t)V * es) % 16 == 0 && aligned(target_logits, 16)) ? 1 : 0;
+    const long long items = (long long)B * (k + 1) * P.items_per_row;
+    // blocks per SM: 4 of 256 threads, 8 loads of 16 bytes in flight per thread, measured best among 2..8
+    // on the largest workload (more blocks disturb the DRAM page locality of the streams);
+    // SD_GREEDY_BLOCKS_PER_SM (1..8) overrides it
+    int per_sm = 4;
+    if (const char* env = getenv("SD_GREEDY_BLOCKS_PER_SM")) {
+        const int v = atoi(env);
+        if (v >= 1 && v <= 8) per_sm = v;
+    }
+    const long long cap = (long long)d->sm_count * per_sm;
+    const unsigned grid = (unsigned)(items < cap ? items : cap);
+    if (dtype == SD_DTYPE_F32) sd_greedy_kernel<SD_DTYPE_F32><<<grid, kGreedyThreads, 0, st>>>(P);
+    else                       sd_greedy_kernel<SD_DTYPE_BF16><<<grid, kGreedyThreads, 0, st>>>(P);
+    const cudaError_t launched = cudaGetLastError();
+    if (!workspace) d->ws_zero_bytes = launched == cudaSuccess ? (d->ws_zero_bytes > need ? d->ws_zero_bytes : need) : 0;
+    SD_CUDA(launched);
+    tl_info[0] = 2; tl_info[1] = 1; tl_info[2] = kGreedyThreads; tl_info[3] = 0;
+    tl_info[4] = (int)grid; tl_info[5] = 1;
+    return SD_OK;
 }
 
 int sd_verify_feedback_host(const void* target_logits, const void* draft_logits, const int32_t* draft_tokens,
@@ -562,7 +644,7 @@ void sd_release_cached_buffers(void) {
         if (cudaGetDevice(&prev) != cudaSuccess) continue;
         if (cudaSetDevice(i) != cudaSuccess) continue;
         cudaDeviceSynchronize();
-        if (d.ws) { cudaFree(d.ws); d.ws = nullptr; d.ws_bytes = 0; d.ws_clean = false; }
+        if (d.ws) { cudaFree(d.ws); d.ws = nullptr; d.ws_bytes = 0; d.ws_clean = false; d.ws_zero_bytes = 0; }
         for (StageSet& st : d.stage)
             if (st.base) { cudaFree(st.base); st.base = nullptr; st.bytes = 0; }
         cudaSetDevice(prev);
