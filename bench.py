@@ -45,6 +45,7 @@ UNIT = "positions/s"
 L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum per launch at full size, from the ncu captures
 # summarised under profiles/ (bytes; a workload that is not listed has not been captured)
+NCU_TRAFFIC_GREEDY = {"cfg5": 919481088 + 244224}
 NCU_TRAFFIC_BYTES = {"cfg5": 2692059136 + 756199936, "cfg3": 174112768 + 33039360, "cfg4": 190112000 + 46578176}
 
 
@@ -415,7 +416,8 @@ def run_greedy(args, cfg):
             "config": workload_config(cfg, path="greedy", l2="inputs larger than L2" if nsets == 1 else f"{nsets} rotating input sets larger than L2 together",
                                       parallelism=f"replicas x{world}, sequences independent, no collective", launch=info),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None, "peak_source": peak_src, "algorithmic_bytes_per_launch": algo,
+                         "traffic": NCU_TRAFFIC_GREEDY.get(cfg.name) if not args.batch else None,
+                         "peak_source": peak_src, "algorithmic_bytes_per_launch": algo,
                          "kernel_ms_mean": mean_kernel_ms, "kernel_ms_min": float(np.min(kernel_ms)),
                          "kernel": "sd_greedy_kernel"},
             "cpu_baseline": {"value": cfg.B * cfg.k / t_cpu, "unit": UNIT, "cores": 1, "kind": "oracle",
