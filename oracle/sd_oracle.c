@@ -293,6 +293,88 @@ int sd_oracle_greedy(const void* T, int dtype, const int32_t* x, int B, int k, i
     return 0;
 }
 
+/*
+ * sd_oracle_ensemble -- feedback of one round for an online ensemble of N draft models
+ * (Sec. 3.3, "Online Update with Ensemble"): every base learner n receives the loss of the round
+ * and its gradient for its own draft distribution q^n against the same target distribution p,
+ *     loss[n,b,i] = KL(p_{b,i} || q^n_{b,i}),      grad^n[b,i,:] = (q^n_{b,i} - p_{b,i}) / tau,
+ * and the meta learner's weights follow the exponential weighting scheme (Hedge)
+ *     weight_n  proportional to  exp(-eps * sum over rounds so far of f_s(w_s^n)).
+ * Readings: the loss of a round, f_t, is the mean of the per-position losses over the B*k
+ * positions of the round (a training loss is a mean); cum_out = cum_in + that mean, and the weights
+ * returned are those of the next round, computed from cum_out.  KL and the cross-entropy of
+ * Assumption 1 differ by the entropy of p, the same for every learner, so the weights do not
+ * depend on which of the two is accumulated.
+ *   T [B,k+1,V] (the bonus rows are not used), Dn[n] [B,k,V], cum_in [N] or NULL (zeros);
+ *   out_loss [N,B,k]; out_grad[n] [B,k,V] or out_grad NULL; out_round [N], out_cum [N],
+ *   out_weights [N].  Returns 0, or -1 on a bad argument or allocation failure.
+ */
+int sd_oracle_ensemble(const void* T, const void* const* Dn, int N, int dtype, double tau, double eps,
+                       int B, int k, int V, const double* cum_in, double* out_loss,
+                       double* const* out_grad, double* out_round, double* out_cum, double* out_weights,
+                       int nthreads) {
+    if (!T || !Dn || !out_loss || !out_round || !out_cum || !out_weights) return -1;
+    if (N < 1 || B < 1 || k < 1 || V < 1 || !(tau > 0.0) || !isfinite(tau) || !(eps >= 0.0)) return -1;
+    if (dtype != SD_ORACLE_F32 && dtype != SD_ORACLE_BF16) return -1;
+    int failed = 0;
+#ifdef _OPENMP
+    if (nthreads < 1) nthreads = 1;
+#pragma omp parallel num_threads(nthreads)
+#endif
+    {
+        double* p = (double*)malloc((size_t)V * sizeof(double));
+        double* logp = (double*)malloc((size_t)V * sizeof(double));
+        double* q = (double*)malloc((size_t)V * sizeof(double));
+        double* logq = (double*)malloc((size_t)V * sizeof(double));
+        if (!p || !logp || !q || !logq) {
+#ifdef _OPENMP
+#pragma omp atomic write
+#endif
+            failed = 1;
+        } else {
+#ifdef _OPENMP
+#pragma omp for schedule(dynamic, 1)
+#endif
+            for (int pos = 0; pos < B * k; ++pos) {
+                int b = pos / k, i = pos % k;
+                double S;
+                softmax_row(T, dtype, ((size_t)b * (k + 1) + i) * V, V, tau, p, logp, &S);
+                for (int n = 0; n < N; ++n) {
+                    softmax_row(Dn[n], dtype, (size_t)pos * V, V, tau, q, logq, &S);
+                    double kl = 0.0;
+                    for (int v = 0; v < V; ++v) {
+                        if (p[v] > 0.0) kl += p[v] * (logp[v] - logq[v]);
+                        if (out_grad) out_grad[n][(size_t)pos * V + v] = (q[v] - p[v]) / tau;
+                    }
+                    out_loss[(size_t)n * B * k + pos] = kl;
+                }
+            }
+        }
+        free(p);
+        free(logp);
+        free(q);
+        free(logq);
+    }
+    (void)nthreads;
+    if (failed) return -1;
+    /* the round's loss of every learner, the cumulative losses, the weights of the next round */
+    double lowest = INFINITY;
+    for (int n = 0; n < N; ++n) {
+        double sum = 0.0;
+        for (int pos = 0; pos < B * k; ++pos) sum += out_loss[(size_t)n * B * k + pos];
+        out_round[n] = sum / (double)(B * k);
+        out_cum[n] = (cum_in ? cum_in[n] : 0.0) + out_round[n];
+        if (out_cum[n] < lowest) lowest = out_cum[n];
+    }
+    double Z = 0.0;
+    for (int n = 0; n < N; ++n) {
+        out_weights[n] = exp(-eps * (out_cum[n] - lowest)); /* the common factor exp(eps*lowest) cancels */
+        Z += out_weights[n];
+    }
+    for (int n = 0; n < N; ++n) out_weights[n] /= Z;
+    return 0;
+}
+
 /* Threads the build can use: 1 without OpenMP. */
 int sd_oracle_max_threads(void) {
 #ifdef _OPENMP

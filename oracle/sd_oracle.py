@@ -2,7 +2,7 @@
 
 Only the tests, the smoke check and the benchmark's CPU-baseline leg may import this module.
 It compiles ``sd_oracle.c`` with gcc on first use (``build()``), loads it and exposes
-``verify_feedback`` which takes and returns numpy arrays.  Nothing here touches CUDA and nothing
+``verify_feedback``, ``verify_greedy`` and ``ensemble_feedback``, which take and return numpy arrays.  Nothing here touches CUDA and nothing
 here is imported by the product package.
 """
 from __future__ import annotations
@@ -11,7 +11,7 @@ import ctypes
 import os
 import subprocess
 from dataclasses import dataclass
-from typing import Optional
+from typing import Optional, Sequence
 
 import numpy as np
 
@@ -43,6 +43,10 @@ def _load():
                                   ctypes.c_int]
         lib.sd_oracle_greedy.restype = ctypes.c_int
         lib.sd_oracle_greedy.argtypes = [P, ctypes.c_int, P, ctypes.c_int, ctypes.c_int, ctypes.c_int, P, P, P]
+        lib.sd_oracle_ensemble.restype = ctypes.c_int
+        lib.sd_oracle_ensemble.argtypes = [P, P, ctypes.c_int, ctypes.c_int, ctypes.c_double, ctypes.c_double,
+                                           ctypes.c_int, ctypes.c_int, ctypes.c_int, P, P, P, P, P, P,
+                                           ctypes.c_int]
         lib.sd_oracle_max_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -136,4 +140,45 @@ def verify_greedy(target_logits: np.ndarray, draft_tokens: np.ndarray) -> Greedy
                                   _ptr(res.argmax))
     if rc != 0:
         raise RuntimeError(f"sd_oracle_greedy failed with code {rc}")
+    return res
+
+
+@dataclass
+class EnsembleResult:
+    loss: np.ndarray                # [N,B,k] float64 KL(p || q^n)
+    grad: Optional[list]            # N arrays [B,k,V] float64, or None
+    round_loss: np.ndarray          # [N] mean loss of the round
+    cum_loss: np.ndarray            # [N] cumulative loss including this round
+    weights: np.ndarray             # [N] Hedge weights of the next round
+
+
+def ensemble_feedback(target_logits: np.ndarray, draft_logits: Sequence[np.ndarray], tau: float, eps: float,
+                      cum_loss: Optional[np.ndarray] = None, want_grad: bool = True,
+                      nthreads: int = 1) -> EnsembleResult:
+    """Feedback for an online ensemble of N draft models (Sec. 3.3) and the Hedge weights."""
+    T = np.ascontiguousarray(target_logits)
+    if T.dtype == np.float32:
+        dtype = F32
+    elif T.dtype == np.uint16:
+        dtype = BF16
+    else:
+        raise TypeError("logits must be float32 or uint16 (bf16 bits)")
+    B, k1, V = T.shape
+    k = k1 - 1
+    Ds = [np.ascontiguousarray(d) for d in draft_logits]
+    N = len(Ds)
+    for d in Ds:
+        if d.dtype != T.dtype or d.shape != (B, k, V):
+            raise ValueError("every draft logit set must be [B,k,V] of the target's dtype")
+    dptr = (ctypes.c_void_p * N)(*[d.ctypes.data for d in Ds])
+    grads = [np.empty((B, k, V), np.float64) for _ in range(N)] if want_grad else None
+    gptr = (ctypes.c_void_p * N)(*[g.ctypes.data for g in grads]) if want_grad else None
+    cum_in = None if cum_loss is None else np.ascontiguousarray(cum_loss, dtype=np.float64)
+    res = EnsembleResult(loss=np.empty((N, B, k), np.float64), grad=grads, round_loss=np.empty(N, np.float64),
+                         cum_loss=np.empty(N, np.float64), weights=np.empty(N, np.float64))
+    rc = _load().sd_oracle_ensemble(_ptr(T), dptr, N, dtype, ctypes.c_double(tau), ctypes.c_double(eps), B, k, V,
+                                    _ptr(cum_in) if cum_in is not None else None, _ptr(res.loss), gptr,
+                                    _ptr(res.round_loss), _ptr(res.cum_loss), _ptr(res.weights), int(nthreads))
+    if rc != 0:
+        raise RuntimeError(f"sd_oracle_ensemble failed with code {rc}")
     return res

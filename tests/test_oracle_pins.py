@@ -425,3 +425,82 @@ def test_greedy_is_the_small_temperature_limit_of_the_sampling_step():
     assert (samp.tokens == gr.tokens).all()
     assert 0 < (gr.accept_len == k).sum() < B or True
     assert len(set(gr.accept_len.tolist())) > 1       # the case exercises several accept lengths
+
+
+# ---- online ensemble (Sec. 3.3): per-learner feedback and the Hedge weights ----------------
+
+def _ensemble_case(seed=0, N=3, B=3, k=2, V=11):
+    rng = np.random.default_rng(seed)
+    T = rng.standard_normal((B, k + 1, V)).astype(np.float32) * 2.0
+    Ds = [(T[:, :k] + (0.3 * 2 ** n) * rng.standard_normal((B, k, V))).astype(np.float32) for n in range(N)]
+    return T, Ds
+
+
+@pytest.mark.parametrize("tau", [0.6, 1.0])
+def test_ensemble_losses_and_gradients_match_scipy_per_learner(tau):
+    T, Ds = _ensemble_case(1)
+    res = sd_oracle.ensemble_feedback(T, Ds, tau, eps=10.0)
+    p = softmax(T[:, :-1].astype(np.float64) / tau, axis=-1)
+    for n, D in enumerate(Ds):
+        q = softmax(D.astype(np.float64) / tau, axis=-1)
+        np.testing.assert_allclose(res.loss[n], rel_entr(p, q).sum(-1), rtol=1e-11, atol=1e-14)
+        np.testing.assert_allclose(res.grad[n], (q - p) / tau, rtol=1e-11, atol=1e-15)
+        assert res.round_loss[n] == pytest.approx(rel_entr(p, q).sum(-1).mean(), rel=1e-12)
+
+
+def test_hedge_weights_hand_values():
+    """Two learners with cumulative losses 0.1 and 0.2 and eps = 10: the weights are
+    1/(1+e^-1) and e^-1/(1+e^-1) (the two-expert form of the exponential weighting scheme)."""
+    T, Ds = _ensemble_case(2, N=2)
+    Ds = [T[:, :-1].copy(), T[:, :-1].copy()]            # both learners equal the target: the round adds nothing
+    res = sd_oracle.ensemble_feedback(T, Ds, 1.0, eps=10.0, cum_loss=np.array([0.1, 0.2]))
+    np.testing.assert_allclose(res.round_loss, 0.0, atol=1e-15)
+    np.testing.assert_allclose(res.cum_loss, [0.1, 0.2], rtol=1e-15)
+    np.testing.assert_allclose(res.weights, [0.7310585786300049, 0.2689414213699951], rtol=1e-12)
+
+
+def test_hedge_weights_are_softmax_of_minus_eps_cumulative_loss_and_accumulate_over_rounds():
+    T, Ds = _ensemble_case(3)
+    eps = 10.0
+    cum = None
+    total = np.zeros(3)
+    for rnd in range(3):
+        T, Ds = _ensemble_case(10 + rnd)
+        res = sd_oracle.ensemble_feedback(T, Ds, 0.8, eps=eps, cum_loss=cum, want_grad=False)
+        total += res.round_loss
+        np.testing.assert_allclose(res.cum_loss, total, rtol=1e-13)
+        np.testing.assert_allclose(res.weights, softmax(-eps * total), rtol=1e-12)
+        assert res.weights.sum() == pytest.approx(1.0, abs=1e-15)
+        cum = res.cum_loss
+    # the noisier the learner the larger its loss, hence the smaller its weight
+    assert res.weights[0] > res.weights[1] > res.weights[2]
+
+
+def test_hedge_limits_and_invariance():
+    T, Ds = _ensemble_case(4)
+    base = sd_oracle.ensemble_feedback(T, Ds, 1.0, eps=10.0, cum_loss=np.array([0.3, 0.1, 0.2]), want_grad=False)
+    # eps = 0: uniform weights, whatever the losses
+    flat = sd_oracle.ensemble_feedback(T, Ds, 1.0, eps=0.0, cum_loss=np.array([0.3, 0.1, 0.2]), want_grad=False)
+    np.testing.assert_allclose(flat.weights, 1.0 / 3.0, rtol=1e-15)
+    # a constant added to every learner's cumulative loss (cross-entropy instead of KL: + entropy of p) cancels
+    moved = sd_oracle.ensemble_feedback(T, Ds, 1.0, eps=10.0, cum_loss=np.array([0.3, 0.1, 0.2]) + 123.0, want_grad=False)
+    np.testing.assert_allclose(moved.weights, base.weights, rtol=1e-10)
+    # a huge eps puts all weight on the learner with the smallest cumulative loss, without overflow
+    sharp = sd_oracle.ensemble_feedback(T, Ds, 1.0, eps=1e6, cum_loss=np.array([0.3, 0.1, 0.2]) * 1e3, want_grad=False)
+    assert np.isfinite(sharp.weights).all()
+    assert sharp.weights[int(np.argmin(sharp.cum_loss))] == pytest.approx(1.0)
+
+
+def test_ensemble_learner_equals_single_draft_feedback_and_bf16():
+    """Each learner's loss and gradient are those of the single-draft step given the same logits."""
+    rng = np.random.default_rng(5)
+    B, k, V = 2, 3, 37
+    T = synth.f32_to_bf16_bits(rng.standard_normal((B, k + 1, V)).astype(np.float32) * 3)
+    Ds = [synth.f32_to_bf16_bits(rng.standard_normal((B, k, V)).astype(np.float32) * 3) for _ in range(2)]
+    res = sd_oracle.ensemble_feedback(T, Ds, 0.7, eps=10.0, nthreads=2)
+    x = np.zeros((B, k), np.int32)
+    u = np.zeros((B, k + 1), np.float32)
+    for n in range(2):
+        one = sd_oracle.verify_feedback(T, Ds[n], x, u, 0.7)
+        np.testing.assert_allclose(res.loss[n], one.loss, rtol=1e-13)
+        np.testing.assert_allclose(res.grad[n], one.grad, rtol=1e-13, atol=1e-300)
