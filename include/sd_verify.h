@@ -71,6 +71,8 @@ extern "C" {
 #define SD_ERR_ALIGN (-8)       /* a pointer is not aligned to its element type */
 
 #define SD_MAX_K 64 /* largest number of draft tokens per sequence */
+#define SD_MAX_LEARNERS 8 /* largest number of draft models of an online ensemble */
+#define SD_ENSEMBLE_SCRATCH_BYTES 256 /* device scratch of sd_ensemble_feedback */
 
 /* bits of out_status[b] */
 #define SD_STATUS_BAD_TOKEN 1u      /* some draft token of the sequence is outside [0,V): treated as rejected */
@@ -197,6 +199,44 @@ int sd_verify_greedy(const void* target_logits, const int32_t* draft_tokens, int
 size_t sd_greedy_workspace_bytes(int B, int k);
 
 /*
+ * sd_ensemble_feedback -- the feedback of one round for an online ensemble of N draft models
+ * (Sec. 3.3, "Online Update with Ensemble"; N = 3 and epsilon = 10 in the paper's experiments).
+ * Every base learner n gets the loss and the gradient of its own draft distribution
+ * q^n = softmax(D^n/tau) against the same target distribution p = softmax(T/tau),
+ *     loss[n,b,i] = KL(p_{b,i} || q^n_{b,i}),     grad^n[b,i,:] = (q^n_{b,i} - p_{b,i}) / tau,
+ * each target row being fetched from HBM once for all N learners, and the meta learner's weights
+ * follow the exponential weighting scheme  weight_n ~ exp(-epsilon * cumulative loss of learner n).
+ * The loss of a round is the mean of the B*k per-position losses; out_cum_loss = cum_loss_in + that
+ * mean, and out_weights are the weights of the NEXT round, computed from out_cum_loss.  Nothing is
+ * verified or drawn here (use sd_verify_feedback / sd_verify_greedy with the logits of the combined
+ * draft for that); the bonus rows of target_logits are not read.
+ *
+ *   target_logits   [B, k+1, V]   in   device, `dtype`
+ *   draft_logits    [N]           in   HOST array of N device pointers, each [B, k, V] in `dtype`
+ *   n_learners                    in   N, 1 .. SD_MAX_LEARNERS
+ *   temperature, epsilon          in   tau > 0; epsilon >= 0 (SD_ERR_TEMPERATURE otherwise)
+ *   cum_loss_in     [N] double    in   device, cumulative losses before this round, or NULL for zeros
+ *   out_loss        [N, B, k]     out  device fp32
+ *   out_grad        [N]           in   HOST array of N device pointers, each [B, k, V] in `dtype`
+ *                                      (an entry may be NULL: no gradient for that learner), or NULL
+ *   out_round_loss  [N] double    out  device, mean loss of the round per learner
+ *   out_cum_loss    [N] double    out  device; may be the same buffer as cum_loss_in
+ *   out_weights     [N] float     out  device, sums to 1
+ *   out_status      [B] uint32    out  device SD_STATUS_BAD_ROW / SD_STATUS_TIMEOUT bits, or NULL
+ *   workspace                     in   device scratch of SD_ENSEMBLE_SCRATCH_BYTES, aligned to 256
+ *                                      bytes, or NULL for the library's own
+ *   stream                        in   cudaStream_t
+ * Rows must be whole 16-byte vectors and every tensor 16-byte aligned (SD_ERR_ALIGN otherwise:
+ * there is no element-wise path for this entry point).  Two kernels are enqueued: the streaming
+ * kernel of sd_verify_feedback over (sequence, row, learner) units, then a one-block reduction.
+ */
+int sd_ensemble_feedback(const void* target_logits, const void* const* draft_logits, int n_learners,
+                         float temperature, float epsilon, int B, int k, int V, int dtype,
+                         const double* cum_loss_in, float* out_loss, void* const* out_grad,
+                         double* out_round_loss, double* out_cum_loss, float* out_weights,
+                         uint32_t* out_status, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * sd_verify_feedback_host -- the same step for callers whose tensors live in HOST memory.
  * Every pointer is a HOST pointer (pinned memory gives asynchronous copies, pageable memory
  * works too).  The call copies the inputs to device buffers the library keeps per device
@@ -212,7 +252,7 @@ int sd_verify_feedback_host(const void* target_logits, const void* draft_logits,
 
 /*
  * sd_launch_info -- HOST out-parameters describing how the last successful device call on this
- * thread was launched: path (0 = generic, 1 = stream fast path, 2 = greedy verification), cluster size, threads per
+ * thread was launched: path (0 = generic, 1 = stream fast path, 2 = greedy verification, 3 = ensemble feedback), cluster size, threads per
  * block, dynamic shared memory per block, blocks launched, kernels launched.  Any pointer may
  * be NULL.  Diagnostic only.
  */

@@ -53,6 +53,9 @@ def _load() -> ctypes.CDLL:
     lib.sd_verify_greedy.argtypes = [P, P, I, I, I, I, P, P, P, P, Z, P]
     lib.sd_greedy_workspace_bytes.restype = Z
     lib.sd_greedy_workspace_bytes.argtypes = [I, I]
+    lib.sd_ensemble_feedback.restype = I
+    lib.sd_ensemble_feedback.argtypes = [P, P, I, ctypes.c_float, ctypes.c_float, I, I, I, I, P, P, P, P, P, P, P,
+                                         P, Z, P]
     lib.sd_verify_feedback_host.restype = I
     lib.sd_verify_feedback_host.argtypes = [P, P, P, P, F, I, I, I, I, P, P, P, P, P, P]
     lib.sd_workspace_bytes.restype = Z
@@ -232,6 +235,55 @@ def sd_verify_greedy(target_logits: torch.Tensor, draft_tokens: torch.Tensor, *,
                                    _stream_ptr(stream))
     if rc != 0:
         raise SdVerifyError(rc, "sd_verify_greedy")
+    return out
+
+
+@dataclass
+class EnsembleOutputs:
+    loss: torch.Tensor                  # [N,B,k] float32 KL(p || q^n)
+    grad: Optional[list]                # N tensors [B,k,V] in the dtype of the logits, or None
+    round_loss: torch.Tensor            # [N] float64 mean loss of the round
+    cum_loss: torch.Tensor              # [N] float64 cumulative loss including this round
+    weights: torch.Tensor               # [N] float32 Hedge weights of the next round
+    status: Optional[torch.Tensor]      # [B] int32 view of the status words
+
+
+def sd_ensemble_feedback(target_logits: torch.Tensor, draft_logits, temperature: float, epsilon: float, *,
+                         cum_loss: Optional[torch.Tensor] = None, want_grad: bool = True,
+                         want_status: bool = False, out: Optional[EnsembleOutputs] = None,
+                         stream: Optional[torch.cuda.Stream] = None) -> EnsembleOutputs:
+    """``sd_ensemble_feedback`` on device tensors: N draft logit sets against one target."""
+    if target_logits.dim() != 3 or not target_logits.is_contiguous():
+        raise ValueError("target logits must be contiguous [B,k+1,V]")
+    B, k1, V = target_logits.shape
+    k = k1 - 1
+    N = len(draft_logits)
+    dev = target_logits.device
+    if dev.type != "cuda":
+        raise ValueError("device tensors required")
+    for d in draft_logits:
+        if tuple(d.shape) != (B, k, V) or d.dtype != target_logits.dtype or not d.is_contiguous() or d.device != dev:
+            raise ValueError("every draft logit set must be contiguous [B,k,V] of the target's dtype and device")
+    if cum_loss is not None and (cum_loss.dtype != torch.float64 or tuple(cum_loss.shape) != (N,) or cum_loss.device != dev):
+        raise ValueError("cum_loss must be float64 [N] on the device")
+    code = _dtype_code(target_logits)
+    if out is None:
+        out = EnsembleOutputs(
+            loss=torch.empty((N, B, k), dtype=torch.float32, device=dev),
+            grad=[torch.empty((B, k, V), dtype=target_logits.dtype, device=dev) for _ in range(N)] if want_grad else None,
+            round_loss=torch.empty(N, dtype=torch.float64, device=dev),
+            cum_loss=torch.empty(N, dtype=torch.float64, device=dev),
+            weights=torch.empty(N, dtype=torch.float32, device=dev),
+            status=torch.empty(B, dtype=torch.int32, device=dev) if want_status else None)
+    dptr = (ctypes.c_void_p * N)(*[d.data_ptr() for d in draft_logits])
+    gptr = (ctypes.c_void_p * N)(*[g.data_ptr() for g in out.grad]) if out.grad is not None else None
+    with torch.cuda.device(dev):
+        rc = _lib.sd_ensemble_feedback(_ptr(target_logits), dptr, N, float(temperature), float(epsilon), B, k, V, code,
+                                       _ptr(cum_loss), _ptr(out.loss), gptr, _ptr(out.round_loss),
+                                       _ptr(out.cum_loss), _ptr(out.weights), _ptr(out.status), None, 0,
+                                       _stream_ptr(stream))
+    if rc != 0:
+        raise SdVerifyError(rc, "sd_ensemble_feedback")
     return out
 
 

@@ -81,7 +81,7 @@ struct DeviceState {
     size_t ws_bytes = 0;
     bool ws_clean = false;   // tickets and status words are zero
     size_t ws_zero_bytes = 0;   // leading bytes of ws known to be zero (what greedy verification needs)
-    bool attr_set[2] = {false, false};   // shared-memory / cluster attributes of the fast kernel
+    bool attr_set[2][2] = {{false, false}, {false, false}};   // shared-memory / cluster attributes of the fast kernels
     int max_clusters[2][kMaxCluster + 1];   // resident clusters of 1..16 blocks, -1 = not asked yet
     // last launch-shape decision of the fast path
     int dec_dtype = -1, dec_V = 0, dec_forced = 0, dec_C = 0, dec_G = 0, dec_lag = 0, dec_per = 0;
@@ -124,14 +124,14 @@ int current_device(int* dev, DeviceState** st) {
 
 // Launches the fast path with G clusters of C blocks, or (query_only) asks how many such
 // clusters the device can hold at once.
-template <int DT>
+template <int DT, bool ENS = false>
 int launch_stream(DeviceState& d, const Params& P, int C, int G, int lag, cudaStream_t stream, bool query_only,
                   int* max_clusters) {
-    auto kern = sd_stream_kernel<DT>;
-    if (!d.attr_set[DT]) {
+    auto kern = sd_stream_kernel<DT, ENS>;
+    if (!d.attr_set[DT][ENS]) {
         SD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmem));
         SD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
-        d.attr_set[DT] = true;
+        d.attr_set[DT][ENS] = true;
     }
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
@@ -431,6 +431,80 @@ int sd_verify_feedback_static(const void* target_logits, const void* draft_logit
     return run_device(*d, target_logits, draft_logits, draft_tokens, uniforms, temperature, B, k, V, dtype,
                       out_accept_len, out_tokens, out_loss, out_grad_draft, out_acc_prob, out_status, scratch, L, false,
                       static_cast<cudaStream_t>(stream));
+}
+
+// ---- online ensemble -------------------------------------------------------------------------
+int sd_ensemble_feedback(const void* target_logits, const void* const* draft_logits, int n_learners,
+                         float temperature, float epsilon, int B, int k, int V, int dtype,
+                         const double* cum_loss_in, float* out_loss, void* const* out_grad,
+                         double* out_round_loss, double* out_cum_loss, float* out_weights, uint32_t* out_status,
+                         void* workspace, size_t workspace_bytes, void* stream) {
+    if (dtype != SD_DTYPE_F32 && dtype != SD_DTYPE_BF16) return SD_ERR_DTYPE;
+    if (!target_logits || !draft_logits || !out_loss || !out_round_loss || !out_cum_loss || !out_weights)
+        return SD_ERR_NULL;
+    if (n_learners < 1 || n_learners > SD_MAX_LEARNERS || !shape_ok(B, k, V)) return SD_ERR_SHAPE;
+    if ((long double)B * k * n_learners >= 2.0e9L) return SD_ERR_SHAPE;
+    if (!(temperature > 0.f) || !isfinite(temperature)) return SD_ERR_TEMPERATURE;
+    if (!(epsilon >= 0.f) || !isfinite(epsilon)) return SD_ERR_TEMPERATURE;
+    const size_t row_bytes = (size_t)V * elem_bytes(dtype);
+    if (row_bytes % 16 != 0 || !aligned(target_logits, 16)) return SD_ERR_ALIGN;
+    for (int n = 0; n < n_learners; ++n) {
+        if (!draft_logits[n]) return SD_ERR_NULL;
+        if (!aligned(draft_logits[n], 16) || (out_grad && out_grad[n] && !aligned(out_grad[n], 16))) return SD_ERR_ALIGN;
+    }
+    if (!aligned(out_loss, 4) || !aligned(out_round_loss, 8) || !aligned(out_cum_loss, 8) || !aligned(out_weights, 4) ||
+        (cum_loss_in && !aligned(cum_loss_in, 8)) || (out_status && !aligned(out_status, 4)))
+        return SD_ERR_ALIGN;
+    if (workspace && (!aligned(workspace, kAlign) || workspace_bytes < SD_ENSEMBLE_SCRATCH_BYTES)) return SD_ERR_WORKSPACE;
+    int dev;
+    DeviceState* d = nullptr;
+    int rc = current_device(&dev, &d);
+    if (rc != SD_OK) return rc;
+    std::lock_guard<std::mutex> lock(d->mu);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char* ws = static_cast<unsigned char*>(workspace);
+    if (!ws) {
+        if (!d->ws) {
+            const size_t want = 1 << 20;
+            SD_CUDA(cudaMalloc(&d->ws, want));
+            d->ws_bytes = want;
+        }
+        ws = static_cast<unsigned char*>(d->ws);
+        d->ws_clean = false;       // the flag word of this call sits where other entry points expect zeros
+        d->ws_zero_bytes = 0;
+    }
+    SD_CUDA(cudaMemsetAsync(ws, 0, SD_ENSEMBLE_SCRATCH_BYTES, st));
+    if (out_status) SD_CUDA(cudaMemsetAsync(out_status, 0, (size_t)B * 4, st));
+
+    Params P;
+    memset(&P, 0, sizeof P);
+    P.T = target_logits;
+    P.B = B; P.k = k; P.V = V;
+    P.c = (float)(1.4426950408889634 / (double)temperature);
+    P.tau = temperature;
+    P.inv_tau = 1.0 / (double)temperature;
+    P.loss = out_loss;
+    P.status = out_status;
+    P.sticky = reinterpret_cast<uint32_t*>(ws);
+    P.learners = n_learners;
+    for (int n = 0; n < n_learners; ++n) {
+        P.Dn[n] = draft_logits[n];
+        P.Gn[n] = out_grad ? out_grad[n] : nullptr;
+    }
+    int G = 0, lag = 0, per = 0;
+    const int C = choose_stream(*d, V, (long long)B * k * n_learners, dtype, &G, &per, &lag);
+    if (C <= 0) return SD_ERR_CUDA;
+    P.blocks_per_unit = C;
+    P.RE = per * vec_elems(dtype);
+    P.NR = (V + P.RE - 1) / P.RE;
+    rc = dtype == SD_DTYPE_F32 ? launch_stream<SD_DTYPE_F32, true>(*d, P, C, G, lag, st, false, nullptr)
+                               : launch_stream<SD_DTYPE_BF16, true>(*d, P, C, G, lag, st, false, nullptr);
+    if (rc != SD_OK) return rc;
+    sd_hedge_kernel<<<1, 256, 0, st>>>(out_loss, n_learners, (long long)B * k, (double)epsilon, cum_loss_in,
+                                       out_round_loss, out_cum_loss, out_weights, P.sticky, out_status, B);
+    SD_CUDA(cudaGetLastError());
+    tl_info[0] = 3; tl_info[5] = 2;
+    return SD_OK;
 }
 
 size_t sd_greedy_workspace_bytes(int B, int k) {

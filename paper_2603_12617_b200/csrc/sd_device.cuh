@@ -26,6 +26,7 @@ namespace sdv {
 namespace cg = cooperative_groups;
 
 constexpr int kMaxCluster = 16;
+constexpr int kMaxLearners = 8;                  // draft models of an online ensemble
 constexpr int kGenericRegionElems = 512;         // sampling region of the generic path
 constexpr uint32_t kStatusTimeout = 0x80000000u; // a bounded wait gave up
 constexpr uint32_t kWaitLimit = 1u << 21;        // polls of an mbarrier before giving up
@@ -73,7 +74,48 @@ struct Params {
     RowConst* rowc;          // [B*(k+1)]
     float* region_sums;      // [B*(k+1)*NR] mass of each sampling region of each row
     int blocks_per_unit;     // blocks that take a ticket per (sequence, row)
+    // online ensemble: feedback of `learners` draft models against one target (0: the plain step).
+    // Then loss is [learners,B,k], D and grad above are unused, and nothing is verified or drawn.
+    int learners;
+    const void* Dn[kMaxLearners];   // [B,k,V] each
+    void* Gn[kMaxLearners];         // [B,k,V] each, or null
 };
+
+// What a unit of the fast path works on.  Plain step: unit = (sequence, row) with the bonus row
+// last.  Ensemble: unit = (sequence, row, learner) with the learner running fastest, so that the
+// units that read the same target row follow one another and find it in L2.
+struct UnitRef {
+    int b, i, n;
+    bool bonus;
+    size_t t_row;            // row of T
+    size_t d_row;            // row of the draft logits and of the gradient (a valid row on a bonus unit too)
+};
+template <bool ENS>
+__device__ __forceinline__ UnitRef unit_ref(const Params& P, int unit) {
+    UnitRef r;
+    if constexpr (ENS) {
+        const int pos = unit / P.learners;
+        r.n = unit - pos * P.learners;
+        r.b = pos / P.k;
+        r.i = pos - r.b * P.k;
+        r.bonus = false;
+        r.t_row = (size_t)r.b * (P.k + 1) + r.i;
+        r.d_row = (size_t)pos;
+    } else {
+        const int K1 = P.k + 1;
+        r.n = 0;
+        r.b = unit / K1;
+        r.i = unit - r.b * K1;
+        r.bonus = (r.i == P.k);
+        r.t_row = (size_t)unit;
+        r.d_row = (size_t)r.b * P.k + (r.bonus ? 0 : r.i);
+    }
+    return r;
+}
+template <bool ENS>
+__device__ __forceinline__ int total_units(const Params& P) {
+    return ENS ? P.B * P.k * P.learners : P.B * (P.k + 1);
+}
 
 // ------------------------------------------------------------------------------------------
 // element types
@@ -432,6 +474,14 @@ __device__ inline void finish_row(const Params& P, int b, int i, const PartialSt
         P.accept[b * P.k + i] = acc ? 1 : 0;
     }
     if (flags) atomicOr(&P.wstatus[b], flags);
+}
+
+// End of a (sequence, row, learner) unit of the ensemble feedback, by one thread: the learner's loss.
+__device__ inline void finish_row_ensemble(const Params& P, const UnitRef& ur, const PartialStats& st) {
+    const bool ok = (st.sT > 0.0) && isfinite(st.sT) && (st.sD > 0.0) && isfinite(st.sD);
+    if (!ok && P.status) atomicOr(&P.status[ur.b], SD_STATUS_BAD_ROW);
+    const double kl = 0.6931471805599453 * (st.w / st.sT - log2(st.sT) + log2(st.sD));
+    P.loss[(size_t)ur.n * P.B * P.k + ur.d_row] = (float)kl;
 }
 
 // ------------------------------------------------------------------------------------------

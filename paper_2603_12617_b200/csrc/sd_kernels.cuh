@@ -388,7 +388,8 @@ __device__ __host__ __forceinline__ void cluster_units(int units, int G, int cid
 
 // ---- fast path -----------------------------------------------------------------------------
 // lag_stages: stages (per consumer warp) of pass 1 of the next unit that go before pass 2 of a unit.
-template <int DT>
+// ENS: the units are those of the ensemble feedback (see UnitRef); nothing is verified or drawn.
+template <int DT, bool ENS>
 __global__ void __launch_bounds__(kStreamThreads, 1)
 sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
     using E = Elem<DT>;
@@ -407,7 +408,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int K1 = P.k + 1;
     int u0, nu;
-    cluster_units(P.B * K1, G, cid, u0, nu);      // this cluster works on units u0 .. u0+nu-1
+    cluster_units(total_units<ENS>(P), G, cid, u0, nu);   // this cluster works on units u0 .. u0+nu-1
 
     const int NV = P.V / VEC;                     // vectors per row
     const int stages_row = (NV + kStageVecs - 1) / kStageVecs;   // = sampling regions per row
@@ -440,7 +441,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
         // ---- statistics: block partial -> cluster exchange -> row constants
         for (int j = 0; j < nu; ++j) {
             const int unit = u0 + j;
-            const bool bonus = (unit % K1 == P.k);
+            const bool bonus = !ENS && (unit % K1 == P.k);
             const int par = j & 1;
             const uint32_t ph = (uint32_t)(j >> 1) & 1u;
             const int dslot = j % kDoneDepth;
@@ -479,10 +480,17 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
         int seg = 0;                               // units of the current sequence finished so far
         for (int j = 0; j < nu; ++j) {
             const int unit = u0 + j;
-            const int b = unit / K1, i = unit - b * K1;
-            const bool bonus = (i == P.k);
             const int dslot = j % kDoneDepth;
             const bool reports = (j % C == rank);   // the blocks of the cluster take turns
+            if constexpr (ENS) {
+                if (!mbar_wait_sleepy<500>(&sh.s2_done[dslot], (uint32_t)(j / kDoneDepth) & 1u, abort)) break;
+                if (reports && lane == 0) finish_row_ensemble(P, unit_ref<true>(P, unit), sh.row[dslot]);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.res_free[dslot]);
+                continue;
+            }
+            const int b = unit / K1, i = unit - b * K1;
+            const bool bonus = (i == P.k);
             AcceptOperands aop;
             aop.valid = false;
             if (reports && lane == 0 && !bonus) aop = load_accept_operands<DT>(P, b, i);
@@ -532,11 +540,10 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
             int slot_i = 0;               // ring slot of the next copy
             constexpr size_t kStride = (size_t)kConsumerWarps * kStageVecs * VEC;   // from one of my stages to the next
             auto begin_run = [&]() {      // lane 0
-                const int unit = u0 + (run == 2 ? ji - 1 : run == 4 ? nu - 1 : ji);
-                const int b = unit / K1, i = unit - b * K1;
+                const UnitRef ur = unit_ref<ENS>(P, u0 + (run == 2 ? ji - 1 : run == 4 ? nu - 1 : ji));
                 const size_t off = (size_t)(vb0 + cw * kStageVecs) * VEC + (size_t)ti * kStride;
-                Tb = reinterpret_cast<const ET*>(P.T) + (size_t)unit * P.V + off;
-                Db = (i == P.k) ? nullptr : reinterpret_cast<const ET*>(P.D) + (size_t)(b * P.k + i) * P.V + off;
+                Tb = reinterpret_cast<const ET*>(P.T) + ur.t_row * P.V + off;
+                Db = ur.bonus ? nullptr : reinterpret_cast<const ET*>(ENS ? P.Dn[ur.n] : P.D) + ur.d_row * P.V + off;
                 pol = (run == 2 || run == 4) ? normal : keep;
             };
             auto issue_next = [&]() {     // lane 0
@@ -584,12 +591,11 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
             ps.RT = ps.RD = kEmptyRef;
             ps.ls.init();
             auto run_pass1 = [&](int j, int t0, int t1) {
-                const int unit = u0 + j;
-                const int b = unit / K1, i = unit - b * K1;
-                const bool bonus = (i == P.k);
+                const UnitRef ur = unit_ref<ENS>(P, u0 + j);
+                const bool bonus = ur.bonus;
                 // the block's slice of the two rows in global memory (for the rare second try of a stage)
-                const ET* Trow = reinterpret_cast<const ET*>(P.T) + (size_t)unit * P.V + (size_t)vb0 * VEC;
-                const ET* Drow = reinterpret_cast<const ET*>(P.D) + (size_t)(b * P.k + (bonus ? 0 : i)) * P.V + (size_t)vb0 * VEC;
+                const ET* Trow = reinterpret_cast<const ET*>(P.T) + ur.t_row * P.V + (size_t)vb0 * VEC;
+                const ET* Drow = reinterpret_cast<const ET*>(ENS ? P.Dn[ur.n] : P.D) + ur.d_row * P.V + (size_t)vb0 * VEC;
                 for (int t = t0; t < t1 && ok; ++t) {
                     const int slot = slot_c;
                     if (!mbar_wait(&myfull[slot], par_c, abort)) { ok = false; break; }
@@ -604,15 +610,14 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
             };
             auto run_pass2 = [&](int j) {
                 const int unit = u0 + j;
-                const int b = unit / K1, i = unit - b * K1;
-                const bool bonus = (i == P.k);
+                const UnitRef ur = unit_ref<ENS>(P, unit);
+                const bool bonus = ur.bonus;
                 const int dslot = j % kDoneDepth;
                 if (!mbar_wait(&sh.rc_ready[j & 1], (uint32_t)(j >> 1) & 1u, abort)) { ok = false; return; }
                 const RowConst rc = sh.rc[j & 1];
-                ET* Grow = (P.grad && !bonus)
-                               ? reinterpret_cast<ET*>(P.grad) + (size_t)(b * P.k + i) * P.V + (size_t)vb0 * VEC
-                               : nullptr;
-                float* rsum = P.region_sums + (size_t)unit * P.NR + s0;
+                void* const gbase = ENS ? P.Gn[ur.n] : P.grad;
+                ET* Grow = (gbase && !bonus) ? reinterpret_cast<ET*>(gbase) + ur.d_row * P.V + (size_t)vb0 * VEC : nullptr;
+                float* rsum = ENS ? nullptr : P.region_sums + (size_t)unit * P.NR + s0;
                 for (int t = 0; t < nst; ++t) {
                     const int slot = slot_c;
                     if (!mbar_wait(&myfull[slot], par_c, abort)) { ok = false; return; }
@@ -623,7 +628,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
                                              : pass2_stage<DT, false>(st, nv, lane, P.c, rc,
                                                                       Grow ? Grow + (size_t)s * kStageVecs * VEC : nullptr,
                                                                       recycle);
-                    if (lane == 0) rsum[s] = mass;
+                    if (!ENS && lane == 0) rsum[s] = mass;
                 }
                 // the resolver's slot of unit j-4 must be free again before this unit is reported done
                 if (j >= kDoneDepth &&
@@ -662,7 +667,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
         // sequence resolved from now on
         if (tid == 0) atomicExch(P.sticky, 1u);
         if (P.status)
-            for (int j = tid; j < nu; j += kStreamThreads) atomicOr(P.status + (u0 + j) / K1, kStatusTimeout);
+            for (int j = tid; j < nu; j += kStreamThreads) atomicOr(P.status + unit_ref<ENS>(P, u0 + j).b, kStatusTimeout);
     }
     // no block leaves while another may still write to its shared memory
     cluster.sync();
@@ -760,6 +765,45 @@ __global__ void __launch_bounds__(kGenericThreads) sd_generic_kernel(const __gri
     if (tid == 0) sh.last = take_tickets(P, b, 1u) ? 1 : 0;
     __syncthreads();
     if (sh.last && warp == 0) resolve_sequence<DT>(P, b);
+}
+
+// ---- online ensemble ---------------------------------------------------------------------
+// Mean loss of the round per learner (fixed summation order), cumulative losses, Hedge weights.
+__global__ void __launch_bounds__(256) sd_hedge_kernel(const float* loss, int N, long long per, double eps,
+                                                       const double* cum_in, double* round_loss, double* cum_out,
+                                                       float* weights, const uint32_t* sticky, uint32_t* status,
+                                                       int B) {
+    __shared__ double part[256];
+    __shared__ double mean[kMaxLearners];
+    const int tid = threadIdx.x;
+    for (int n = 0; n < N; ++n) {
+        double s = 0.0;
+        for (long long j = tid; j < per; j += 256) s += (double)loss[(size_t)n * per + j];
+        part[tid] = s;
+        __syncthreads();
+        for (int w = 128; w > 0; w >>= 1) {
+            if (tid < w) part[tid] += part[tid + w];
+            __syncthreads();
+        }
+        if (tid == 0) mean[n] = part[0] / (double)per;
+        __syncthreads();
+    }
+    if (tid == 0) {
+        double cum[kMaxLearners], lowest = INFINITY, Z = 0.0;
+        for (int n = 0; n < N; ++n) {
+            cum[n] = (cum_in ? cum_in[n] : 0.0) + mean[n];
+            if (cum[n] < lowest) lowest = cum[n];
+        }
+        for (int n = 0; n < N; ++n) Z += exp(-eps * (cum[n] - lowest));
+        for (int n = 0; n < N; ++n) {
+            round_loss[n] = mean[n];
+            cum_out[n] = cum[n];
+            weights[n] = (float)(exp(-eps * (cum[n] - lowest)) / Z);
+        }
+    }
+    // a bounded wait gave up somewhere in the feedback kernel: nothing of this round is valid
+    if (status && *sticky != 0)
+        for (int b = tid; b < B; b += 256) atomicOr(status + b, kStatusTimeout);
 }
 
 }  // namespace sdv

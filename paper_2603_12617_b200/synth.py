@@ -175,3 +175,22 @@ def custom_config(B: int, k: int, V: int, dtype: str = "f32", tau: float = 1.0,
     return Config(f"custom_B{B}_k{k}_V{V}_{dtype}", B=B, k=k, V=V, dtype=dtype, tau=tau,
                   recipe=recipe, t_sigma=t_sigma, d_sigma=d_sigma, d_scale=d_scale, zipf_s=zipf_s,
                   index=index)
+
+
+def ensemble_drafts(inp: Inputs, n_learners: int, seed: int = BASE_SEED) -> list:
+    """Draft logits of ``n_learners`` base learners for the inputs of one round: learner 0 is the
+    workload's own draft, learner n > 0 is the target's rows plus Gaussian noise whose standard
+    deviation doubles from learner to learner (base learners that track the target ever more
+    loosely, like draft heads trained with ever larger step sizes).  Same dtype as the inputs."""
+    cfg = inp.cfg
+    k = cfg.k
+    T = inp.target_logits[:, :k]
+    Tf = bf16_bits_to_f32(T) if cfg.dtype == "bf16" else T
+    out = [inp.draft_logits]
+    sigma0 = cfg.d_sigma if cfg.d_sigma > 0 else 0.5
+    for n in range(1, n_learners):
+        rng = _rng(seed, cfg.index, 1000 + n)
+        noise = rng.standard_normal(Tf.shape, dtype=np.float32) * np.float32(sigma0 * 2.0 ** n)
+        D = Tf + noise
+        out.append(f32_to_bf16_bits(D) if cfg.dtype == "bf16" else D.astype(np.float32))
+    return out
