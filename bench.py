@@ -22,6 +22,9 @@ With N > 1 (launched by torch.distributed.run) every rank runs the full batch of
   --path greedy   times greedy verification instead (Algorithm 1 in the limit tau -> 0, the decoding
              mode of the paper's experiments): only the target logits are read, (k+1)*V*B entries per
              launch; the line has the same keys, with "path": "greedy" in config.  Not the headline.
+  --path ensemble  times the feedback of an online ensemble of --learners N draft models (Sec. 3.3):
+             (k + N*k)*V*B logits in, N*k*V*B gradient entries out per launch; value counts the B*k
+             positions of the round (each served for all N learners).  Not the headline.
 """
 from __future__ import annotations
 
@@ -45,6 +48,7 @@ UNIT = "positions/s"
 L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum per launch at full size, from the ncu captures
 # summarised under profiles/ (bytes; a workload that is not listed has not been captured)
+NCU_TRAFFIC_ENSEMBLE = {}
 NCU_TRAFFIC_GREEDY = {"cfg5": 919481088 + 244224}
 NCU_TRAFFIC_BYTES = {"cfg5": 2692059136 + 756199936, "cfg3": 174112768 + 33039360, "cfg4": 190112000 + 46578176}
 
@@ -432,6 +436,142 @@ def run_greedy(args, cfg):
         dist.destroy_process_group()
 
 
+def run_ensemble(args, cfg):
+    """--path ensemble: sd_ensemble_feedback with N learners on the workload, one GPU per rank."""
+    import torch
+    import torch.distributed as dist
+
+    import __graft_entry__ as entry
+    entry.build()
+    from paper_2603_12617_b200 import binding, shard
+
+    N = args.learners
+    eps = 10.0
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    inp = synth.make_inputs(cfg, seed=synth.BASE_SEED + 1000 * rank)
+    drafts = synth.ensemble_drafts(inp, N, seed=synth.BASE_SEED + 1000 * rank)
+
+    def as_torch(a):
+        t = torch.from_numpy(a)
+        return t.view(torch.bfloat16) if a.dtype == np.uint16 else t
+
+    hT = as_torch(inp.target_logits).pin_memory()
+    hD = [as_torch(d).pin_memory() for d in drafts]
+    in_bytes = hT.numel() * hT.element_size() + sum(d.numel() * d.element_size() for d in hD)
+    nsets = 1 if in_bytes > 2 * L2_BYTES else int(min(64, -(-3 * L2_BYTES // in_bytes)))
+    sets = [(hT.to(dev), [d.to(dev) for d in hD]) for _ in range(nsets)]
+    out = binding.sd_ensemble_feedback(sets[0][0], sets[0][1], inp.tau, eps)
+    cum = torch.zeros(N, dtype=torch.float64, device=dev)
+
+    def step(i):
+        T, Ds = sets[i % nsets]
+        binding.sd_ensemble_feedback(T, Ds, inp.tau, eps, cum_loss=cum, out=out)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(3, args.warmup)):
+        step(i)
+    info = binding.sd_launch_info()
+    barrier()
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        t_begin.record()
+        for i in range(args.steps):
+            starts[i].record()
+            step(i)
+            ends[i].record()
+        t_end.record()
+        barrier()
+    total_ms = shard.max_over_ranks(t_begin.elapsed_time(t_end), device=str(dev) if world > 1 else "cpu")
+    kernel_ms = [s.elapsed_time(e) for s, e in zip(starts, ends)]
+    mean_kernel_ms = float(np.mean(kernel_ms))
+    positions = cfg.B * cfg.k * world
+    value = positions * args.steps / (total_ms * 1e-3)
+
+    # end to end: pinned host logits in, losses, weights and gradients back to the host
+    e2e_steps = max(1, min(args.steps, 5))
+    dT, dD = torch.empty_like(sets[0][0]), [torch.empty_like(d) for d in sets[0][1]]
+    h_loss = torch.empty((N, cfg.B, cfg.k), dtype=torch.float32).pin_memory()
+    h_w = torch.empty(N, dtype=torch.float32).pin_memory()
+    h_grad = [torch.empty_like(d).pin_memory() for d in hD]
+
+    def e2e_step():
+        dT.copy_(hT, non_blocking=True)
+        for a, b in zip(dD, hD):
+            a.copy_(b, non_blocking=True)
+        binding.sd_ensemble_feedback(dT, dD, inp.tau, eps, cum_loss=cum, out=out)
+        h_loss.copy_(out.loss, non_blocking=True)
+        h_w.copy_(out.weights, non_blocking=True)
+        for a, b in zip(h_grad, out.grad):
+            a.copy_(b, non_blocking=True)
+        torch.cuda.synchronize()
+
+    e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    barrier()
+    e2e_s = shard.max_over_ranks(time.perf_counter() - t0, device=str(dev) if world > 1 else "cpu")
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # the timed outputs against the oracle on a few sequences, and the oracle's own speed
+    from oracle import sd_oracle
+    cores = min(sd_oracle.max_threads(), os.cpu_count() or 1)
+    nseq = min(cfg.B, max(1, cores // cfg.k))
+    sl = np.arange(nseq)
+    t0 = time.perf_counter()
+    ref = sd_oracle.ensemble_feedback(inp.target_logits[sl], [d[sl] for d in drafts], inp.tau, eps, want_grad=False,
+                                      nthreads=cores)
+    t_cpu = time.perf_counter() - t0
+    loss = h_loss.numpy()[:, :nseq].astype(np.float64)
+    verified = bool(np.allclose(loss, ref.loss, rtol=2e-2 if cfg.dtype == "bf16" else 1e-5, atol=4e-7)
+                    and abs(float(h_w.sum()) - 1.0) < 1e-5)
+    s = cfg.elem_bytes
+    algo = ((cfg.k + N * cfg.k) + N * cfg.k) * cfg.V * cfg.B * s
+    d2h = h_loss.numel() * 4 + h_w.numel() * 4 + sum(g.numel() * g.element_size() for g in h_grad)
+    peak, peak_src = measured_peak_gbs()
+    achieved = algo / (mean_kernel_ms * 1e-3) / 1e9
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32" if cfg.dtype == "f32" else "f32 (bf16 storage)",
+            "data": "synthetic",
+            "config": workload_config(cfg, path="ensemble", learners=N, epsilon=eps,
+                                      l2="inputs larger than L2" if nsets == 1 else f"{nsets} rotating input sets larger than L2 together",
+                                      parallelism=f"replicas x{world}, sequences independent, no collective", launch=info),
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": NCU_TRAFFIC_ENSEMBLE.get((cfg.name, N)) if not args.batch else None,
+                         "peak_source": peak_src, "algorithmic_bytes_per_launch": algo,
+                         "kernel_ms_mean": mean_kernel_ms, "kernel_ms_min": float(np.min(kernel_ms)),
+                         "kernel": "sd_stream_kernel<ensemble> + sd_hedge_kernel"},
+            "cpu_baseline": {"value": nseq * cfg.k / t_cpu, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": f"{nseq} of {cfg.B} sequences of {cfg.name}, {N} learners, no gradients, "
+                                       f"one call, {t_cpu:.2f} s"},
+            "e2e": {"value": positions * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": int(in_bytes),
+                    "d2h_bytes_per_step": int(d2h), "steps": e2e_steps, "ms_per_step": e2e_s / e2e_steps * 1e3,
+                    "entry_point": "sd_ensemble_feedback between pinned-memory copies"},
+            "gpu_launches": args.steps * info["kernels"], "clocks": clocks.summary(),
+            "outputs_verified_against_oracle": verified}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -441,8 +581,10 @@ def main():
     ap.add_argument("--config", default="cfg5", choices=sorted(synth.CONFIGS))
     ap.add_argument("--batch", type=int, default=0, help="override B (profiling on a smaller case)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--path", choices=["sample", "greedy"], default="sample",
-                    help="sample: the verify-and-feedback step (the headline); greedy: greedy verification")
+    ap.add_argument("--path", choices=["sample", "greedy", "ensemble"], default="sample",
+                    help="sample: the verify-and-feedback step (the headline); greedy: greedy verification; "
+                         "ensemble: feedback of an online ensemble of draft models")
+    ap.add_argument("--learners", type=int, default=3, help="draft models of --path ensemble")
     args = ap.parse_args()
     cfg = synth.CONFIGS[args.config]
     if args.batch:
@@ -451,6 +593,8 @@ def main():
         run_reference(args, cfg)
     elif args.path == "greedy":
         run_greedy(args, cfg)
+    elif args.path == "ensemble":
+        run_ensemble(args, cfg)
     else:
         run_ours(args, cfg)
 

@@ -42,6 +42,14 @@
  *     logit tensors and for out_grad_draft.  Arithmetic is fp32 per element with fp64 row
  *     scalars in both cases.
  *   - Calls that share a workspace must not overlap on the GPU.
+ *   - Side effect on the CUDA context: the first call on a device sets the context's limit
+ *     cudaLimitPersistingL2CacheSize to 52 MiB (capped by the device's maximum), because the fast
+ *     path fetches with the L2 evict_last policy what its second pass reads again, and that
+ *     policy only holds lines inside such a set-aside.  The limit belongs to this process's
+ *     context and ends with it.  Environment: SD_VERIFY_L2_PERSIST_MIB=<MiB> chooses another
+ *     size, 0 leaves the limit untouched.  Other tuning knobs read from the environment (never
+ *     needed for correctness): SD_VERIFY_CLUSTER (cluster size of the fast path),
+ *     SD_VERIFY_LAG, SD_VERIFY_L2_MIB, SD_VERIFY_FORCE_GENERIC, SD_GREEDY_BLOCKS_PER_SM.
  */
 #ifndef SD_VERIFY_H
 #define SD_VERIFY_H

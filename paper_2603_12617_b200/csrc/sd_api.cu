@@ -18,6 +18,7 @@ constexpr int kMaxDevices = 64;
 constexpr size_t kAlign = 256;
 constexpr int kStreamSmem = kRingSlots * kStageBytes + (int)sizeof(StreamShared);
 static_assert(kStreamSmem <= 227 * 1024, "ring does not fit the shared memory of a block");
+constexpr int kL2PersistMiB = 52;
 constexpr double kL2BudgetMiB = 80.0;              // row pairs in flight between their two passes should fit this
 
 thread_local char tl_cuda_error[256] = "";
@@ -111,6 +112,18 @@ int current_device(int* dev, DeviceState** st) {
         }
         d.cc_major = prop.major;
         d.sm_count = prop.multiProcessorCount;
+        // Part of L2 set aside for lines fetched with the evict_last policy (pass 1 of the fast
+        // path fetches with it what pass 2 reads again): without a set-aside the policy has no
+        // effect and pass 2 of the largest workloads goes back to HBM for most of its lines.  52 MiB
+        // (granted as 58 MB) measured best on the 126 MB L2: larger ones starve everything else.
+        // A limit of this process's context only; SD_VERIFY_L2_PERSIST_MIB=0 leaves it alone.
+        {
+            const char* env = getenv("SD_VERIFY_L2_PERSIST_MIB");
+            size_t want = (size_t)(env ? atoi(env) : kL2PersistMiB) << 20;
+            if (want > (size_t)prop.persistingL2CacheMaxSize) want = (size_t)prop.persistingL2CacheMaxSize;
+            if (want > 0 && cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, want) != cudaSuccess)
+                (void)cudaGetLastError();   // not fatal: the path is only slower without it
+        }
         d.probed = true;
     }
     if (d.cc_major != 10) {

@@ -35,17 +35,17 @@
 namespace sdv {
 
 // ---- geometry of the fast path -------------------------------------------------------------
-// A row is cut into stages of 256 16-byte vectors (4 KiB); a stage is also a sampling region.
+// A row is cut into stages of 128 16-byte vectors (2 KiB); a stage is also a sampling region.
 // Block r of a cluster of C owns the stages [r*S, (r+1)*S) of every row it works on, S =
-// ceil(stages per row / C); stage s of the slice belongs to consumer warp s % 8, so eight
+// ceil(stages per row / C); stage s of the slice belongs to consumer warp s % 14, so fourteen
 // consecutive stages are worked on at the same time.  Every consumer warp has a ring of its own.
 constexpr int kConsumerWarps = 14;
 constexpr int kStageGroups = 4;                               // groups of 32 vectors in a stage
 constexpr int kStageVecs = 32 * kStageGroups;                 // vectors of one row in a stage
-constexpr int kStageRowBytes = kStageVecs * 16;               // 4 KiB of one row
+constexpr int kStageRowBytes = kStageVecs * 16;               // 2 KiB of one row
 constexpr int kStageBytes = 2 * kStageRowBytes;               // target part + draft part
 constexpr int kWarpSlots = 3;                                 // stages a consumer warp has in flight or in use
-constexpr int kRingSlots = kConsumerWarps * kWarpSlots;       // 24 slots, 192 KiB
+constexpr int kRingSlots = kConsumerWarps * kWarpSlots;       // 42 slots, 168 KiB
 constexpr int kDoneDepth = 4;                                 // units the resolver may lag behind
 constexpr int kStatsWarp = 0, kResolverWarp = 1, kFirstConsumerWarp = 2;
 constexpr int kStreamThreads = (kFirstConsumerWarp + kConsumerWarps) * 32;
