@@ -48,9 +48,9 @@ UNIT = "positions/s"
 L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum per launch at full size, from the ncu captures
 # summarised under profiles/ (bytes; a workload that is not listed has not been captured)
-NCU_TRAFFIC_ENSEMBLE = {}
+NCU_TRAFFIC_ENSEMBLE = {("cfg5", 3): 4938604544 + 2329972736}
 NCU_TRAFFIC_GREEDY = {"cfg5": 919481088 + 244224}
-NCU_TRAFFIC_BYTES = {"cfg5": 2692059136 + 756199936, "cfg3": 174112768 + 33039360, "cfg4": 190112000 + 46578176}
+NCU_TRAFFIC_BYTES = {"cfg5": 2089991936 + 759110400, "cfg3": 155516160 + 35080448, "cfg4": 179646464 + 49013248}
 
 
 def measured_peak_gbs():
@@ -255,6 +255,9 @@ def run_ours(args, cfg):
     total_ms = shard.max_over_ranks(t_begin.elapsed_time(t_end), device=str(dev) if world > 1 else "cpu")
     kernel_ms = [s.elapsed_time(e) for s, e in zip(starts, ends)]
     mean_kernel_ms = float(np.mean(kernel_ms))
+    if args.times_out and rank == 0:
+        with open(args.times_out, "w") as fh:
+            json.dump(kernel_ms, fh)
     positions = cfg.B * cfg.k * world
     value = positions * args.steps / (total_ms * 1e-3)
 
@@ -585,6 +588,7 @@ def main():
                     help="sample: the verify-and-feedback step (the headline); greedy: greedy verification; "
                          "ensemble: feedback of an online ensemble of draft models")
     ap.add_argument("--learners", type=int, default=3, help="draft models of --path ensemble")
+    ap.add_argument("--times-out", default="", help="write the per-step device times (ms) of the headline path here")
     args = ap.parse_args()
     cfg = synth.CONFIGS[args.config]
     if args.batch:
