@@ -636,22 +636,31 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.s2_done[dslot]);
             };
-            for (int j = 0; j < nu && ok; ++j) {
+            // The walk, segment by segment (each pass has one call site, which keeps the hot code small):
+            // unit j contributes  [pass 1 head]  [pass 2 of unit j-1]  [pass 1 rest];  then pass 2 of the last unit.
+            for (int seg = 0; seg <= 3 * nu && ok; ++seg) {
+                const int j = seg / 3, kind = seg - 3 * j;
+                int p1 = -1, p2 = -1, t0 = 0, t1 = 0;
                 const int head = (j == 0) ? nst : L;
-                run_pass1(j, 0, head);
-                if (ok && j > 0) run_pass2(j - 1);
-                if (ok) run_pass1(j, head, nst);
-                if (!ok) break;
-                // pass 1 of the unit is over: the warp's partial for the statistics warp
-                const PartialStats part = warp_sum_lanes(ps.ls, ps.RT, ps.RD);
-                if (lane == 0) {
-                    sh.wpart[j & 1][cw] = part;
-                    mbar_arrive(&sh.s1_done[j & 1]);
+                if (j == nu) p2 = nu - 1;
+                else if (kind == 0) { p1 = j; t0 = 0; t1 = head; }
+                else if (kind == 1) { if (j > 0) p2 = j - 1; }
+                else { p1 = j; t0 = head; t1 = nst; }
+                if (p2 >= 0) run_pass2(p2);
+                if (p1 >= 0) {
+                    run_pass1(p1, t0, t1);
+                    if (ok && kind == 2) {
+                        // pass 1 of the unit is over: the warp's partial for the statistics warp
+                        const PartialStats part = warp_sum_lanes(ps.ls, ps.RT, ps.RD);
+                        if (lane == 0) {
+                            sh.wpart[j & 1][cw] = part;
+                            mbar_arrive(&sh.s1_done[j & 1]);
+                        }
+                        ps.RT = ps.RD = kEmptyRef;
+                        ps.ls.init();
+                    }
                 }
-                ps.RT = ps.RD = kEmptyRef;
-                ps.ls.init();
             }
-            if (ok) run_pass2(nu - 1);
             // leaving early: no copy of this warp may still be in flight when the block returns
             if (!ok && lane == 0)
                 for (int t = n; t < ni; ++t) {
