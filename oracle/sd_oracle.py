@@ -182,3 +182,25 @@ def ensemble_feedback(target_logits: np.ndarray, draft_logits: Sequence[np.ndarr
     if rc != 0:
         raise RuntimeError(f"sd_oracle_ensemble failed with code {rc}")
     return res
+
+
+@dataclass
+class ErrorFeedbackResult:
+    full: OracleResult              # the whole step (accept lengths, tokens, losses of every position, bands)
+    error_grad: np.ndarray          # [B,V] float64: gradient row of the first rejected position, zeros if none
+
+
+def error_position_feedback(target_logits: np.ndarray, draft_logits: np.ndarray, draft_tokens: np.ndarray,
+                            uniforms: np.ndarray, tau: float, nthreads: int = 1) -> ErrorFeedbackResult:
+    """The step with the feedback restricted to the error position (what OSD collects, Sec. 3.1):
+    verification as in ``verify_feedback``; of the gradient only the row of the first rejected
+    position n_b of every sequence, a zero row where every draft token was accepted."""
+    full = verify_feedback(target_logits, draft_logits, draft_tokens, uniforms, tau, want_grad=True,
+                           nthreads=nthreads)
+    B, k, V = full.grad.shape
+    eg = np.zeros((B, V), np.float64)
+    for b in range(B):
+        n = int(full.accept_len[b])
+        if n < k:
+            eg[b] = full.grad[b, n]
+    return ErrorFeedbackResult(full=full, error_grad=eg)

@@ -504,3 +504,43 @@ def test_ensemble_learner_equals_single_draft_feedback_and_bf16():
         one = sd_oracle.verify_feedback(T, Ds[n], x, u, 0.7)
         np.testing.assert_allclose(res.loss[n], one.loss, rtol=1e-13)
         np.testing.assert_allclose(res.grad[n], one.grad, rtol=1e-13, atol=1e-300)
+
+
+# ---- error-position feedback (what OSD collects, Sec. 3.1) ---------------------------------
+
+def test_error_position_feedback_hand_cases():
+    """Two-token vocabulary, tau = 1, logits = log-probabilities.  Sequence 0: p = (1/2,1/2),
+    q = (3/4,1/4), x = 0, u = 0.7 > 2/3 rejects at position 0: the gradient row is q - p =
+    (1/4,-1/4).  Sequence 1: the same pair accepted (u = 0.1), then q = (1/4,3/4) with x = 1 and
+    ratio 2/3 rejected (u = 0.9): the row of position 1, (-1/4, 1/4).  Sequence 2: everything
+    accepted: a zero row."""
+    lp = lambda *a: np.log(np.array(a, np.float64))
+    T = np.empty((3, 3, 2), np.float32)
+    D = np.empty((3, 2, 2), np.float32)
+    T[:] = lp(0.5, 0.5)
+    D[0] = [lp(0.75, 0.25), lp(0.75, 0.25)]
+    D[1] = [lp(0.75, 0.25), lp(0.25, 0.75)]
+    D[2] = [lp(0.75, 0.25), lp(0.25, 0.75)]
+    x = np.array([[0, 0], [0, 1], [0, 1]], np.int32)
+    u = np.array([[0.7, 0.0, 0.3], [0.1, 0.9, 0.3], [0.1, 0.2, 0.3]], np.float32)
+    res = sd_oracle.error_position_feedback(T, D, x, u, 1.0)
+    assert list(res.full.accept_len) == [0, 1, 2]
+    np.testing.assert_allclose(res.error_grad, [[0.25, -0.25], [-0.25, 0.25], [0.0, 0.0]], atol=1e-7)
+    # a later rejection does not move the error position: sequence 0 would also reject at position 1 (u = 0.0 accepts; make it reject)
+    u2 = u.copy(); u2[0, 1] = 0.99
+    res2 = sd_oracle.error_position_feedback(T, D, x, u2, 1.0)
+    np.testing.assert_allclose(res2.error_grad[0], [0.25, -0.25], atol=1e-7)
+
+
+def test_error_position_feedback_is_a_selection_of_the_full_step():
+    cfg = synth.custom_config(6, 4, 257, dtype="bf16", tau=0.7, recipe="peaks")
+    inp = synth.make_inputs(cfg)
+    res = sd_oracle.error_position_feedback(inp.target_logits, inp.draft_logits, inp.draft_tokens, inp.uniforms, inp.tau)
+    full = sd_oracle.verify_feedback(inp.target_logits, inp.draft_logits, inp.draft_tokens, inp.uniforms, inp.tau)
+    assert (res.full.tokens == full.tokens).all()
+    for b in range(cfg.B):
+        n = int(full.accept_len[b])
+        expect = full.grad[b, n] if n < cfg.k else np.zeros(cfg.V)
+        assert (res.error_grad[b] == expect).all()
+        if n < cfg.k:
+            assert abs(res.error_grad[b].sum()) < 1e-12          # a difference of two distributions
