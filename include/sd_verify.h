@@ -245,6 +245,33 @@ int sd_ensemble_feedback(const void* target_logits, const void* const* draft_log
                          uint32_t* out_status, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * sd_verify_error_feedback -- the step with the feedback restricted to the error position, the
+ * signal OSD collects (Sec. 3.1, "Online Update with Gradient Descent": the token positions where
+ * the draft model was wrong, with the target's logits there, for a distillation loss on these
+ * errors).  Verification is that of sd_verify_feedback, bit for bit: accept lengths and emitted
+ * tokens are the same.  Of the gradient only the row of the first rejected position n_b of every
+ * sequence is produced,
+ *     out_error_grad[b, :] = (q_{b,n_b} - p_{b,n_b}) / tau      if n_b < k,      0 otherwise,
+ * so the position it belongs to is out_accept_len[b].  The losses of all k positions are still
+ * returned (the rejection tests need every row's softmax sums anyway).  Compared with the full step
+ * the second pass runs over one row per sequence instead of k+1 and B*V instead of B*k*V gradient
+ * entries are written.
+ *
+ *   target_logits, draft_logits, draft_tokens, uniforms, temperature, B, k, V, dtype,
+ *   out_accept_len, out_tokens, out_loss (or NULL), out_status (or NULL): as in sd_verify_feedback_ex
+ *   out_error_grad  [B, V]   out  `dtype`, or NULL
+ *   workspace                in   device scratch of at least sd_workspace_bytes(B,k,V,dtype) bytes,
+ *                                 aligned to 256 bytes, or NULL for the library's own
+ * Rows must be whole 16-byte vectors and every tensor 16-byte aligned (SD_ERR_ALIGN otherwise: there
+ * is no element-wise path for this entry point).  Two kernels are enqueued.
+ */
+int sd_verify_error_feedback(const void* target_logits, const void* draft_logits, const int32_t* draft_tokens,
+                             const float* uniforms, float temperature, int B, int k, int V, int dtype,
+                             int32_t* out_accept_len, int32_t* out_tokens, float* out_loss,
+                             void* out_error_grad, uint32_t* out_status, void* workspace,
+                             size_t workspace_bytes, void* stream);
+
+/*
  * sd_verify_feedback_host -- the same step for callers whose tensors live in HOST memory.
  * Every pointer is a HOST pointer (pinned memory gives asynchronous copies, pageable memory
  * works too).  The call copies the inputs to device buffers the library keeps per device
@@ -260,7 +287,7 @@ int sd_verify_feedback_host(const void* target_logits, const void* draft_logits,
 
 /*
  * sd_launch_info -- HOST out-parameters describing how the last successful device call on this
- * thread was launched: path (0 = generic, 1 = stream fast path, 2 = greedy verification, 3 = ensemble feedback), cluster size, threads per
+ * thread was launched: path (0 = generic, 1 = stream fast path, 2 = greedy verification, 3 = ensemble feedback, 4 = error-position feedback), cluster size, threads per
  * block, dynamic shared memory per block, blocks launched, kernels launched.  Any pointer may
  * be NULL.  Diagnostic only.
  */

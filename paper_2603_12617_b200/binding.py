@@ -53,6 +53,8 @@ def _load() -> ctypes.CDLL:
     lib.sd_verify_greedy.argtypes = [P, P, I, I, I, I, P, P, P, P, Z, P]
     lib.sd_greedy_workspace_bytes.restype = Z
     lib.sd_greedy_workspace_bytes.argtypes = [I, I]
+    lib.sd_verify_error_feedback.restype = I
+    lib.sd_verify_error_feedback.argtypes = [P, P, P, P, ctypes.c_float, I, I, I, I, P, P, P, P, P, P, Z, P]
     lib.sd_ensemble_feedback.restype = I
     lib.sd_ensemble_feedback.argtypes = [P, P, I, ctypes.c_float, ctypes.c_float, I, I, I, I, P, P, P, P, P, P, P,
                                          P, Z, P]
@@ -235,6 +237,43 @@ def sd_verify_greedy(target_logits: torch.Tensor, draft_tokens: torch.Tensor, *,
                                    _stream_ptr(stream))
     if rc != 0:
         raise SdVerifyError(rc, "sd_verify_greedy")
+    return out
+
+
+@dataclass
+class ErrorFeedbackOutputs:
+    accept_len: torch.Tensor            # [B] int32: also the position the gradient row belongs to
+    tokens: torch.Tensor                # [B,k+1] int32, -1 padded
+    loss: Optional[torch.Tensor]        # [B,k] float32 KL(p||q), every position
+    error_grad: Optional[torch.Tensor]  # [B,V] gradient row of the first rejected position (zeros if none)
+    status: Optional[torch.Tensor]      # [B] int32 view of the status words
+
+
+def sd_verify_error_feedback(target_logits: torch.Tensor, draft_logits: torch.Tensor, draft_tokens: torch.Tensor,
+                             uniforms: torch.Tensor, temperature: float, *, want_loss: bool = True,
+                             want_grad: bool = True, want_status: bool = True,
+                             out: Optional[ErrorFeedbackOutputs] = None,
+                             stream: Optional[torch.cuda.Stream] = None) -> ErrorFeedbackOutputs:
+    """``sd_verify_error_feedback`` on device tensors (library scratch)."""
+    B, k, V = _shapes(target_logits, draft_logits, draft_tokens, uniforms)
+    dev = target_logits.device
+    if dev.type != "cuda":
+        raise ValueError("device tensors required")
+    code = _dtype_code(target_logits)
+    if out is None:
+        out = ErrorFeedbackOutputs(
+            accept_len=torch.empty(B, dtype=torch.int32, device=dev),
+            tokens=torch.empty((B, k + 1), dtype=torch.int32, device=dev),
+            loss=torch.empty((B, k), dtype=torch.float32, device=dev) if want_loss else None,
+            error_grad=torch.empty((B, V), dtype=target_logits.dtype, device=dev) if want_grad else None,
+            status=torch.empty(B, dtype=torch.int32, device=dev) if want_status else None)
+    with torch.cuda.device(dev):
+        rc = _lib.sd_verify_error_feedback(_ptr(target_logits), _ptr(draft_logits), _ptr(draft_tokens), _ptr(uniforms),
+                                           float(temperature), B, k, V, code, _ptr(out.accept_len), _ptr(out.tokens),
+                                           _ptr(out.loss), _ptr(out.error_grad), _ptr(out.status), None, 0,
+                                           _stream_ptr(stream))
+    if rc != 0:
+        raise SdVerifyError(rc, "sd_verify_error_feedback")
     return out
 
 

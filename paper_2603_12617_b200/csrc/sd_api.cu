@@ -9,6 +9,7 @@
 
 #include "sd_kernels.cuh"
 #include "sd_greedy.cuh"
+#include "sd_errpos.cuh"
 
 namespace {
 
@@ -82,7 +83,7 @@ struct DeviceState {
     size_t ws_bytes = 0;
     bool ws_clean = false;   // tickets and status words are zero
     size_t ws_zero_bytes = 0;   // leading bytes of ws known to be zero (what greedy verification needs)
-    bool attr_set[2][2] = {{false, false}, {false, false}};   // shared-memory / cluster attributes of the fast kernels
+    bool attr_set[2][3] = {{false, false, false}, {false, false, false}};   // shared-memory / cluster attributes of the fast kernels
     int max_clusters[2][kMaxCluster + 1];   // resident clusters of 1..16 blocks, -1 = not asked yet
     // last launch-shape decision of the fast path
     int dec_dtype = -1, dec_V = 0, dec_forced = 0, dec_C = 0, dec_G = 0, dec_lag = 0, dec_per = 0;
@@ -137,14 +138,15 @@ int current_device(int* dev, DeviceState** st) {
 
 // Launches the fast path with G clusters of C blocks, or (query_only) asks how many such
 // clusters the device can hold at once.
-template <int DT, bool ENS = false>
+template <int DT, bool ENS = false, bool STATS = false>
 int launch_stream(DeviceState& d, const Params& P, int C, int G, int lag, cudaStream_t stream, bool query_only,
                   int* max_clusters) {
-    auto kern = sd_stream_kernel<DT, ENS>;
-    if (!d.attr_set[DT][ENS]) {
+    auto kern = sd_stream_kernel<DT, ENS, STATS>;
+    constexpr int kVariant = ENS ? 1 : STATS ? 2 : 0;
+    if (!d.attr_set[DT][kVariant]) {
         SD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmem));
         SD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
-        d.attr_set[DT][ENS] = true;
+        d.attr_set[DT][kVariant] = true;
     }
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
@@ -517,6 +519,78 @@ int sd_ensemble_feedback(const void* target_logits, const void* const* draft_log
                                        out_round_loss, out_cum_loss, out_weights, P.sticky, out_status, B);
     SD_CUDA(cudaGetLastError());
     tl_info[0] = 3; tl_info[5] = 2;
+    return SD_OK;
+}
+
+// ---- error-position feedback -------------------------------------------------------------------
+int sd_verify_error_feedback(const void* target_logits, const void* draft_logits, const int32_t* draft_tokens,
+                             const float* uniforms, float temperature, int B, int k, int V, int dtype,
+                             int32_t* out_accept_len, int32_t* out_tokens, float* out_loss, void* out_error_grad,
+                             uint32_t* out_status, void* workspace, size_t workspace_bytes, void* stream) {
+    int rc = check_args(target_logits, draft_logits, draft_tokens, uniforms, temperature, B, k, V, dtype,
+                        out_accept_len, out_tokens, out_loss, out_error_grad, nullptr, out_status);
+    if (rc != SD_OK) return rc;
+    const size_t row_bytes = (size_t)V * elem_bytes(dtype);
+    if (row_bytes % 16 != 0 || !aligned(target_logits, 16) || !aligned(draft_logits, 16) ||
+        (out_error_grad && !aligned(out_error_grad, 16)))
+        return SD_ERR_ALIGN;
+    const WorkspaceLayout L = workspace_layout(B, k, V, dtype);
+    if (workspace && (!aligned(workspace, kAlign) || workspace_bytes < L.total)) return SD_ERR_WORKSPACE;
+    int dev;
+    DeviceState* d = nullptr;
+    rc = current_device(&dev, &d);
+    if (rc != SD_OK) return rc;
+    std::lock_guard<std::mutex> lock(d->mu);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char* ws = static_cast<unsigned char*>(workspace);
+    if (!ws) {
+        // the library's own scratch, shared with the other entry points and grown on demand
+        if (d->ws_bytes < L.total) {
+            if (d->ws) {
+                SD_CUDA(cudaDeviceSynchronize());
+                SD_CUDA(cudaFree(d->ws));
+                d->ws = nullptr;
+                d->ws_bytes = 0;
+            }
+            const size_t want = align_up(L.total + L.total / 4, 1 << 20);
+            SD_CUDA(cudaMalloc(&d->ws, want));
+            d->ws_bytes = want;
+        }
+        ws = static_cast<unsigned char*>(d->ws);
+        d->ws_clean = false;      // cleared below for this call; say so to the others
+        d->ws_zero_bytes = 0;
+    }
+    Params P;
+    memset(&P, 0, sizeof P);
+    P.T = target_logits; P.D = draft_logits; P.x = draft_tokens; P.u = uniforms;
+    P.B = B; P.k = k; P.V = V;
+    P.c = (float)(1.4426950408889634 / (double)temperature);
+    P.tau = temperature;
+    P.inv_tau = 1.0 / (double)temperature;
+    P.accept_len = out_accept_len; P.tokens = out_tokens; P.loss = out_loss; P.grad = out_error_grad;
+    P.status = out_status;
+    P.ticket = reinterpret_cast<uint32_t*>(ws + L.ticket);
+    P.wstatus = reinterpret_cast<uint32_t*>(ws + L.wstatus);
+    P.sticky = reinterpret_cast<uint32_t*>(ws + L.sticky);
+    P.accept = ws + L.accept;
+    P.rowc = reinterpret_cast<RowConst*>(ws + L.rowc);
+    P.region_sums = reinterpret_cast<float*>(ws + L.region_sums);
+    SD_CUDA(cudaMemsetAsync(ws, 0, L.accept, st));   // tickets, status words, sticky flag
+    int G = 0, lag = 0, per = 0;
+    const int C = choose_stream(*d, V, (long long)B * (k + 1), dtype, &G, &per, &lag);
+    if (C <= 0) return SD_ERR_CUDA;
+    P.blocks_per_unit = C;
+    P.RE = per * vec_elems(dtype);
+    P.NR = (V + P.RE - 1) / P.RE;
+    rc = dtype == SD_DTYPE_F32 ? launch_stream<SD_DTYPE_F32, false, true>(*d, P, C, G, lag, st, false, nullptr)
+                               : launch_stream<SD_DTYPE_BF16, false, true>(*d, P, C, G, lag, st, false, nullptr);
+    if (rc != SD_OK) return rc;
+    const int slices = (P.NR + kErrSliceRegions - 1) / kErrSliceRegions;
+    const unsigned grid = (unsigned)B * (unsigned)slices;
+    if (dtype == SD_DTYPE_F32) sd_errpos_kernel<SD_DTYPE_F32><<<grid, kErrThreads, 0, st>>>(P, slices);
+    else                       sd_errpos_kernel<SD_DTYPE_BF16><<<grid, kErrThreads, 0, st>>>(P, slices);
+    SD_CUDA(cudaGetLastError());
+    tl_info[0] = 4; tl_info[5] = 2;
     return SD_OK;
 }
 

@@ -389,7 +389,9 @@ __device__ __host__ __forceinline__ void cluster_units(int units, int G, int cid
 // ---- fast path -----------------------------------------------------------------------------
 // lag_stages: stages (per consumer warp) of pass 1 of the next unit that go before pass 2 of a unit.
 // ENS: the units are those of the ensemble feedback (see UnitRef); nothing is verified or drawn.
-template <int DT, bool ENS>
+// STATS: pass 1 only -- row constants, losses and rejection tests of every row; no gradient, no
+// masses, no draw (the error-position feedback finishes the one row it needs in a kernel of its own).
+template <int DT, bool ENS, bool STATS = false>
 __global__ void __launch_bounds__(kStreamThreads, 1)
 sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
     using E = Elem<DT>;
@@ -497,6 +499,10 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
             if (!mbar_wait_sleepy<500>(&sh.s2_done[dslot], (uint32_t)(j / kDoneDepth) & 1u, abort)) break;
             if (reports && lane == 0) finish_row(P, b, i, sh.row[dslot], sh.rc_done[dslot], aop);
             __syncwarp();
+            if constexpr (STATS) {
+                if (lane == 0) mbar_arrive(&sh.res_free[dslot]);
+                continue;
+            }
             ++seg;
             const bool leaves = (i == P.k) || (j == nu - 1);   // last unit of the sequence in this cluster
             if (leaves) {
@@ -527,7 +533,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
             }
         } else {
             const int L = min(max(lag_stages, 0), nst);
-            const int n_total = 2 * nu * nst;
+            const int n_total = (STATS ? 1 : 2) * nu * nst;
             unsigned char* myring = ring + (size_t)cw * kWarpSlots * kStageBytes;
             uint64_t* myfull = &sh.full[cw * kWarpSlots];
             const uint64_t keep = policy_keep(), normal = policy_normal();
@@ -560,10 +566,11 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
                 if (ti >= endi) {
                     while (ti >= endi && run != 5) {
                         // the next run that is not empty
-                        if (run == 0) { if (nu > 1) { run = 1; ji = 1; } else run = 4; }
-                        else if (run == 1) run = 2;
+                        constexpr int kLast = STATS ? 5 : 4;          // no pass 2 to fetch for in a pass-1-only walk
+                        if (run == 0) { if (nu > 1) { run = 1; ji = 1; } else run = kLast; }
+                        else if (run == 1) run = STATS ? 3 : 2;
                         else if (run == 2) run = 3;
-                        else if (run == 3) { if (ji + 1 < nu) { run = 1; ++ji; } else run = 4; }
+                        else if (run == 3) { if (ji + 1 < nu) { run = 1; ++ji; } else run = kLast; }
                         else run = 5;
                         if (run == 1) { ti = 0; endi = L; }
                         else if (run == 3) { ti = L; endi = nst; }
@@ -646,7 +653,18 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
                 else if (kind == 0) { p1 = j; t0 = 0; t1 = head; }
                 else if (kind == 1) { if (j > 0) p2 = j - 1; }
                 else { p1 = j; t0 = head; t1 = nst; }
-                if (p2 >= 0) run_pass2(p2);
+                if (p2 >= 0) {
+                    if constexpr (STATS) {
+                        // nothing to do for the unit but to report it finished
+                        const int dslot = p2 % kDoneDepth;
+                        if (p2 >= kDoneDepth &&
+                            !mbar_wait(&sh.res_free[dslot], (uint32_t)(p2 / kDoneDepth - 1) & 1u, abort)) { ok = false; break; }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&sh.s2_done[dslot]);
+                    } else {
+                        run_pass2(p2);
+                    }
+                }
                 if (p1 >= 0) {
                     run_pass1(p1, t0, t1);
                     if (ok && kind == 2) {
