@@ -25,6 +25,8 @@ With N > 1 (launched by torch.distributed.run) every rank runs the full batch of
   --path ensemble  times the feedback of an online ensemble of --learners N draft models (Sec. 3.3):
              (k + N*k)*V*B logits in, N*k*V*B gradient entries out per launch; value counts the B*k
              positions of the round (each served for all N learners).  Not the headline.
+  --path errors   times the step with the feedback restricted to the error position (what OSD
+             collects, Sec. 3.1): (2k+1)*V*B logits in, B*V gradient entries out.  Not the headline.
 """
 from __future__ import annotations
 
@@ -49,6 +51,7 @@ L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum per launch at full size, from the ncu captures
 # summarised under profiles/ (bytes; a workload that is not listed has not been captured)
 NCU_TRAFFIC_ENSEMBLE = {("cfg5", 3): 4938604544 + 2329972736}
+NCU_TRAFFIC_ERRORS = {}
 NCU_TRAFFIC_GREEDY = {"cfg5": 919481088 + 244224}
 NCU_TRAFFIC_BYTES = {"cfg5": 2089991936 + 759110400, "cfg3": 155516160 + 35080448, "cfg4": 179646464 + 49013248}
 
@@ -439,6 +442,138 @@ def run_greedy(args, cfg):
         dist.destroy_process_group()
 
 
+def run_errors(args, cfg):
+    """--path errors: sd_verify_error_feedback on the workload, one GPU per rank."""
+    import torch
+    import torch.distributed as dist
+
+    import __graft_entry__ as entry
+    entry.build()
+    from paper_2603_12617_b200 import binding, shard
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    inp = synth.make_inputs(cfg, seed=synth.BASE_SEED + 1000 * rank)
+
+    def as_torch(a):
+        t = torch.from_numpy(a)
+        return t.view(torch.bfloat16) if a.dtype == np.uint16 else t
+
+    hT, hD = as_torch(inp.target_logits).pin_memory(), as_torch(inp.draft_logits).pin_memory()
+    hx, hu = torch.from_numpy(inp.draft_tokens).pin_memory(), torch.from_numpy(inp.uniforms).pin_memory()
+    in_bytes = hT.numel() * hT.element_size() + hD.numel() * hD.element_size()
+    nsets = 1 if in_bytes > 2 * L2_BYTES else int(min(64, -(-3 * L2_BYTES // in_bytes)))
+    sets = [(hT.to(dev), hD.to(dev), hx.to(dev), hu.to(dev)) for _ in range(nsets)]
+    out = binding.sd_verify_error_feedback(*sets[0], inp.tau)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(3, args.warmup)):
+        binding.sd_verify_error_feedback(*sets[i % nsets], inp.tau, out=out)
+    info = binding.sd_launch_info()
+    barrier()
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        t_begin.record()
+        for i in range(args.steps):
+            starts[i].record()
+            binding.sd_verify_error_feedback(*sets[i % nsets], inp.tau, out=out)
+            ends[i].record()
+        t_end.record()
+        barrier()
+    total_ms = shard.max_over_ranks(t_begin.elapsed_time(t_end), device=str(dev) if world > 1 else "cpu")
+    kernel_ms = [s.elapsed_time(e) for s, e in zip(starts, ends)]
+    mean_kernel_ms = float(np.mean(kernel_ms))
+    positions = cfg.B * cfg.k * world
+    value = positions * args.steps / (total_ms * 1e-3)
+
+    # end to end: pinned host logits in, results and the gradient rows back to the host
+    e2e_steps = max(1, min(args.steps, 10))
+    dbuf = [torch.empty_like(t) for t in sets[0]]
+    h_n = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
+    h_tok = torch.empty((cfg.B, cfg.k + 1), dtype=torch.int32).pin_memory()
+    h_loss = torch.empty((cfg.B, cfg.k), dtype=torch.float32).pin_memory()
+    h_g = torch.empty((cfg.B, cfg.V), dtype=hT.dtype).pin_memory()
+
+    def e2e_step():
+        for a, b in zip(dbuf, (hT, hD, hx, hu)):
+            a.copy_(b, non_blocking=True)
+        binding.sd_verify_error_feedback(*dbuf, inp.tau, out=out)
+        h_n.copy_(out.accept_len, non_blocking=True)
+        h_tok.copy_(out.tokens, non_blocking=True)
+        h_loss.copy_(out.loss, non_blocking=True)
+        h_g.copy_(out.error_grad, non_blocking=True)
+        torch.cuda.synchronize()
+
+    e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    barrier()
+    e2e_s = shard.max_over_ranks(time.perf_counter() - t0, device=str(dev) if world > 1 else "cpu")
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    from oracle import sd_oracle
+    cores = min(sd_oracle.max_threads(), os.cpu_count() or 1)
+    nseq = min(cfg.B, cores)
+    sl = np.arange(nseq)
+    t0 = time.perf_counter()
+    ref = sd_oracle.error_position_feedback(inp.target_logits[sl], inp.draft_logits[sl], inp.draft_tokens[sl],
+                                            inp.uniforms[sl], inp.tau, nthreads=cores)
+    t_cpu = time.perf_counter() - t0
+    safe = (ref.full.accept_band.sum(1) == 0) & (ref.full.cdf_margin > 1e-6)
+    g = h_g[:nseq].float().numpy().astype(np.float64)
+    tol = 2e-2 if cfg.dtype == "bf16" else 1e-5
+    verified = bool((h_n.numpy()[sl][safe] == ref.full.accept_len[safe]).all()
+                    and (h_tok.numpy()[sl][safe] == ref.full.tokens[safe]).all()
+                    and np.allclose(h_loss.numpy()[sl], ref.full.loss, rtol=tol, atol=4e-7)
+                    and all(np.abs(g[b] - ref.error_grad[b]).max() <= tol * np.abs(ref.error_grad[b]).max() + 1e-6
+                            for b in range(nseq) if safe[b]))
+    s = cfg.elem_bytes
+    algo = ((2 * cfg.k + 1) + 1) * cfg.V * cfg.B * s
+    peak, peak_src = measured_peak_gbs()
+    achieved = algo / (mean_kernel_ms * 1e-3) / 1e9
+    d2h = h_n.numel() * 4 + h_tok.numel() * 4 + h_loss.numel() * 4 + h_g.numel() * h_g.element_size()
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32" if cfg.dtype == "f32" else "f32 (bf16 storage)",
+            "data": "synthetic",
+            "config": workload_config(cfg, path="errors", mean_accept_len=float(h_n.float().mean()),
+                                      l2="inputs larger than L2" if nsets == 1 else f"{nsets} rotating input sets larger than L2 together",
+                                      parallelism=f"replicas x{world}, sequences independent, no collective", launch=info),
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": NCU_TRAFFIC_ERRORS.get(cfg.name) if not args.batch else None,
+                         "peak_source": peak_src, "algorithmic_bytes_per_launch": algo,
+                         "kernel_ms_mean": mean_kernel_ms, "kernel_ms_min": float(np.min(kernel_ms)),
+                         "kernel": "sd_stream_kernel<pass 1 only> + sd_errpos_kernel"},
+            "cpu_baseline": {"value": nseq * cfg.k / t_cpu, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": f"{nseq} of {cfg.B} sequences of {cfg.name}, one call, {t_cpu:.2f} s"},
+            "e2e": {"value": positions * e2e_steps / e2e_s, "unit": UNIT,
+                    "h2d_bytes_per_step": int(in_bytes + hx.numel() * 4 + hu.numel() * 4), "d2h_bytes_per_step": int(d2h),
+                    "steps": e2e_steps, "ms_per_step": e2e_s / e2e_steps * 1e3,
+                    "entry_point": "sd_verify_error_feedback between pinned-memory copies"},
+            "gpu_launches": args.steps * info["kernels"], "clocks": clocks.summary(),
+            "outputs_verified_against_oracle": verified}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def run_ensemble(args, cfg):
     """--path ensemble: sd_ensemble_feedback with N learners on the workload, one GPU per rank."""
     import torch
@@ -584,9 +719,9 @@ def main():
     ap.add_argument("--config", default="cfg5", choices=sorted(synth.CONFIGS))
     ap.add_argument("--batch", type=int, default=0, help="override B (profiling on a smaller case)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--path", choices=["sample", "greedy", "ensemble"], default="sample",
+    ap.add_argument("--path", choices=["sample", "greedy", "ensemble", "errors"], default="sample",
                     help="sample: the verify-and-feedback step (the headline); greedy: greedy verification; "
-                         "ensemble: feedback of an online ensemble of draft models")
+                         "ensemble: feedback of an online ensemble of draft models; errors: feedback at the error position only")
     ap.add_argument("--learners", type=int, default=3, help="draft models of --path ensemble")
     ap.add_argument("--times-out", default="", help="write the per-step device times (ms) of the headline path here")
     args = ap.parse_args()
@@ -599,6 +734,8 @@ def main():
         run_greedy(args, cfg)
     elif args.path == "ensemble":
         run_ensemble(args, cfg)
+    elif args.path == "errors":
+        run_errors(args, cfg)
     else:
         run_ours(args, cfg)
 

@@ -655,8 +655,11 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
                 else { p1 = j; t0 = head; t1 = nst; }
                 if (p2 >= 0) {
                     if constexpr (STATS) {
-                        // nothing to do for the unit but to report it finished
+                        // nothing to do for the unit but to report it finished -- after its row
+                        // constants are out, as in the full walk: the statistics warp is then done
+                        // with the partials of the unit, whose slots the unit after next reuses
                         const int dslot = p2 % kDoneDepth;
+                        if (!mbar_wait(&sh.rc_ready[p2 & 1], (uint32_t)(p2 >> 1) & 1u, abort)) { ok = false; break; }
                         if (p2 >= kDoneDepth &&
                             !mbar_wait(&sh.res_free[dslot], (uint32_t)(p2 / kDoneDepth - 1) & 1u, abort)) { ok = false; break; }
                         __syncwarp();

@@ -169,3 +169,30 @@ def test_refusals(binding):
     out = binding.sd_ensemble_feedback(T, [D, T[:, :2].contiguous()], 1.0, EPS)
     torch.cuda.synchronize()
     assert float(out.round_loss[1]) < 1e-9 and float(out.weights[1]) > float(out.weights[0])
+
+
+def test_full_size_bench_shape_equals_the_single_draft_step(binding, monkeypatch):
+    """The bench shape with 3 learners (B=256, k=6, V=128256, fp32; 62 units per cluster): every
+    learner's loss and gradient bit-equal to the single-draft step on the same logits, and the
+    weights from the device's own losses."""
+    monkeypatch.setenv("SD_VERIFY_CLUSTER", "2")
+    cfg = synth.CONFIGS["cfg5"]
+    inp = synth.make_inputs(cfg)
+    Ds = synth.ensemble_drafts(inp, 3)
+    T = dev(inp.target_logits)
+    x = torch.from_numpy(inp.draft_tokens).cuda()
+    u = torch.from_numpy(inp.uniforms).cuda()
+    dDs = [dev(d) for d in Ds]
+    out = binding.sd_ensemble_feedback(T, dDs, inp.tau, EPS, want_status=True)
+    torch.cuda.synchronize()
+    assert (out.status.cpu().numpy() == 0).all()
+    for n in range(3):
+        one = binding.sd_verify_feedback(T, dDs[n], x, u, inp.tau)
+        torch.cuda.synchronize()
+        assert torch.equal(one.loss, out.loss[n])
+        assert torch.equal(one.grad_draft, out.grad[n])
+        del one
+    mean = out.loss.double().mean(dim=(1, 2)).cpu().numpy()
+    np.testing.assert_allclose(out.round_loss.cpu().numpy(), mean, rtol=1e-12)
+    w = np.exp(-EPS * (mean - mean.min()))
+    np.testing.assert_allclose(out.weights.cpu().numpy(), w / w.sum(), rtol=3e-7, atol=1e-12)

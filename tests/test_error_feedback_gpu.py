@@ -145,3 +145,35 @@ def test_refusals(binding):
         binding.sd_verify_error_feedback(dev(inp.target_logits), dev(inp.draft_logits),
                                          torch.from_numpy(inp.draft_tokens).cuda(),
                                          torch.from_numpy(inp.uniforms).cuda(), 1.0)
+
+
+def test_full_size_bench_shape_equals_the_full_step(binding):
+    """The bench shape (B=256, k=6, V=128256, fp32; 24-25 units per cluster, so every ring and every
+    double-buffered slot of the kernel wraps many times): everything bit-equal to the full step, and
+    a sample of sequences against the oracle."""
+    cfg = synth.CONFIGS["cfg5"]
+    inp = synth.make_inputs(cfg)
+    T, D = dev(inp.target_logits), dev(inp.draft_logits)
+    x, u = torch.from_numpy(inp.draft_tokens).cuda(), torch.from_numpy(inp.uniforms).cuda()
+    out = binding.sd_verify_error_feedback(T, D, x, u, inp.tau)
+    full = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
+    torch.cuda.synchronize()
+    assert torch.equal(out.accept_len, full.accept_len)
+    assert torch.equal(out.tokens, full.tokens)
+    assert torch.equal(out.loss, full.loss)
+    assert torch.equal(out.status, full.status)
+    n = out.accept_len.long()
+    rows = full.grad_draft[torch.arange(cfg.B, device="cuda"), n.clamp(max=cfg.k - 1)]
+    rows[n == cfg.k] = 0
+    assert torch.equal(out.error_grad, rows)
+    seqs = np.array([0, 9, 77, 128, 201, 255])
+    ref = sd_oracle.error_position_feedback(inp.target_logits[seqs], inp.draft_logits[seqs], inp.draft_tokens[seqs],
+                                            inp.uniforms[seqs], inp.tau, nthreads=min(6, sd_oracle.max_threads()))
+    safe = (ref.full.accept_band.sum(1) == 0) & (ref.full.cdf_margin > 1e-6)
+    assert (out.accept_len.cpu().numpy()[seqs][safe] == ref.full.accept_len[safe]).all()
+    assert (out.tokens.cpu().numpy()[seqs][safe] == ref.full.tokens[safe]).all()
+    assert np.allclose(out.loss.cpu().numpy()[seqs], ref.full.loss, rtol=1e-5, atol=4e-7)
+    g = out.error_grad.cpu().numpy()[seqs].astype(np.float64)
+    for j in range(len(seqs)):
+        if safe[j]:
+            assert np.abs(g[j] - ref.error_grad[j]).max() <= 1e-5 * np.abs(ref.error_grad[j]).max() + 1e-7
