@@ -196,3 +196,22 @@ def test_full_size_bench_shape_equals_the_single_draft_step(binding, monkeypatch
     np.testing.assert_allclose(out.round_loss.cpu().numpy(), mean, rtol=1e-12)
     w = np.exp(-EPS * (mean - mean.min()))
     np.testing.assert_allclose(out.weights.cpu().numpy(), w / w.sum(), rtol=3e-7, atol=1e-12)
+
+
+@pytest.mark.parametrize("lag,cluster", [(0, 2), (2, 1), (100, 3)])
+def test_orders_of_the_walk_with_many_units_per_cluster(binding, lag, cluster, monkeypatch):
+    monkeypatch.setenv("SD_VERIFY_LAG", str(lag))
+    monkeypatch.setenv("SD_VERIFY_CLUSTER", str(cluster))
+    cfg = synth.custom_config(300, 4, 8192, dtype="bf16", tau=0.9, recipe="peaks")
+    inp = synth.make_inputs(cfg)
+    Ds = synth.ensemble_drafts(inp, 3)
+    T = dev(inp.target_logits)
+    x = torch.from_numpy(inp.draft_tokens).cuda()
+    u = torch.from_numpy(inp.uniforms).cuda()
+    dDs = [dev(d) for d in Ds]
+    out = binding.sd_ensemble_feedback(T, dDs, inp.tau, EPS)
+    for n in range(3):
+        one = binding.sd_verify_feedback(T, dDs[n], x, u, inp.tau)
+        torch.cuda.synchronize()
+        assert torch.equal(one.loss, out.loss[n])
+        assert torch.equal(one.grad_draft.view(torch.int16), out.grad[n].view(torch.int16))

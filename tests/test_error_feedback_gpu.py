@@ -177,3 +177,26 @@ def test_full_size_bench_shape_equals_the_full_step(binding):
     for j in range(len(seqs)):
         if safe[j]:
             assert np.abs(g[j] - ref.error_grad[j]).max() <= 1e-5 * np.abs(ref.error_grad[j]).max() + 1e-7
+
+
+@pytest.mark.parametrize("lag,cluster", [(0, 2), (2, 1), (100, 3), (1, 4)])
+def test_orders_of_the_walk_and_cluster_sizes_with_many_units_per_cluster(binding, lag, cluster, monkeypatch):
+    """Many units per cluster (about 60 here) in every order of the walk: bit-equal to the full step
+    run with the same settings."""
+    monkeypatch.setenv("SD_VERIFY_LAG", str(lag))
+    monkeypatch.setenv("SD_VERIFY_CLUSTER", str(cluster))
+    cfg = synth.custom_config(600, 5, 8192, dtype="bf16", tau=0.9, recipe="peaks")
+    inp = synth.make_inputs(cfg)
+    T, D = dev(inp.target_logits), dev(inp.draft_logits)
+    x, u = torch.from_numpy(inp.draft_tokens).cuda(), torch.from_numpy(inp.uniforms).cuda()
+    out = binding.sd_verify_error_feedback(T, D, x, u, inp.tau)
+    full = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
+    torch.cuda.synchronize()
+    assert torch.equal(out.accept_len, full.accept_len)
+    assert torch.equal(out.tokens, full.tokens)
+    assert torch.equal(out.loss, full.loss)
+    assert torch.equal(out.status, full.status)
+    n = out.accept_len.long()
+    rows = full.grad_draft[torch.arange(cfg.B, device="cuda"), n.clamp(max=cfg.k - 1)]
+    rows[n == cfg.k] = 0
+    assert torch.equal(out.error_grad.view(torch.int16), rows.view(torch.int16))
