@@ -313,6 +313,13 @@ def run_ours(args, cfg):
                 "algorithmic_bytes_per_launch": cfg.algorithmic_bytes, "kernel_ms_mean": mean_kernel_ms,
                 "kernel_ms_min": float(np.min(kernel_ms)), "kernel": "sd_stream_kernel" if info["path"] == 1 else "sd_generic_kernel",
                 "frac_of_nominal_8000_GBps": achieved / 8000.0}
+    # second ceiling: the special-function units (4 ex2 per entry pair and 2 per bonus entry; 16 results per
+    # clock and SM, 148 SMs at the maximum SM clock): what binds when entries are 2 bytes
+    ex2 = (4 * cfg.k + 2) * cfg.V * cfg.B
+    sfu_peak = 148 * 16 * 1.965e9
+    roofline["sfu"] = {"ex2_per_launch": ex2, "achieved_per_s": ex2 / (mean_kernel_ms * 1e-3), "peak_per_s": sfu_peak,
+                       "frac": ex2 / (mean_kernel_ms * 1e-3) / sfu_peak,
+                       "peak_source": "148 SMs x 16 ex2/clk x 1965 MHz (nominal unit count and maximum clock)"}
     base = cpu_baseline(cfg, inp) if not args.no_cpu_baseline else None
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": total_ms / args.steps, "higher_is_better": True,

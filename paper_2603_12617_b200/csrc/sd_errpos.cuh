@@ -22,7 +22,7 @@ constexpr int kErrThreads = 256;
 constexpr int kErrSliceRegions = 32;
 
 template <int DT>
-__global__ void __launch_bounds__(kErrThreads) sd_errpos_kernel(const __grid_constant__ Params P, const int slices) {
+__global__ void __launch_bounds__(kErrThreads, 4) sd_errpos_kernel(const __grid_constant__ Params P, const int slices) {
     using E = Elem<DT>;
     using ET = typename E::type;
     constexpr int VEC = E::VEC;
