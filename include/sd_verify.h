@@ -46,7 +46,9 @@
  *     cudaLimitPersistingL2CacheSize to 52 MiB (capped by the device's maximum), because the fast
  *     path fetches with the L2 evict_last policy what its second pass reads again, and that
  *     policy only holds lines inside such a set-aside.  The limit belongs to this process's
- *     context and ends with it.  Environment: SD_VERIFY_L2_PERSIST_MIB=<MiB> chooses another
+ *     context and ends with it; lines kept that way stay until later ones displace them, so a
+ *     process whose other kernels want all of L2 may call cudaCtxResetPersistingL2Cache()
+ *     between its own phases.  Environment: SD_VERIFY_L2_PERSIST_MIB=<MiB> chooses another
  *     size, 0 leaves the limit untouched.  Other tuning knobs read from the environment (never
  *     needed for correctness): SD_VERIFY_CLUSTER (cluster size of the fast path),
  *     SD_VERIFY_LAG, SD_VERIFY_L2_MIB, SD_VERIFY_FORCE_GENERIC, SD_GREEDY_BLOCKS_PER_SM.
