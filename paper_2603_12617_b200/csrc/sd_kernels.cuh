@@ -409,8 +409,19 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
     const int cid = (int)blockIdx.x / C;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int K1 = P.k + 1;
-    int u0, nu;
-    cluster_units(total_units<ENS>(P), G, cid, u0, nu);   // this cluster works on units u0 .. u0+nu-1
+    // The plain step gives a cluster a contiguous range of units (the rows of a sequence stay
+    // together: fewer tickets).  The ensemble deals its units round the clusters instead: the units
+    // that read the same target row then run on neighbouring clusters at about the same time, and all
+    // but the first find the row in L2.
+    int u0, nu, ustep = 1;
+    if constexpr (ENS) {
+        const int units = total_units<true>(P);
+        u0 = cid;
+        ustep = G;
+        nu = cid < units ? (units - cid + G - 1) / G : 0;
+    } else {
+        cluster_units(total_units<false>(P), G, cid, u0, nu);   // this cluster works on units u0 .. u0+nu-1
+    }
 
     const int NV = P.V / VEC;                     // vectors per row
     const int stages_row = (NV + kStageVecs - 1) / kStageVecs;   // = sampling regions per row
@@ -442,7 +453,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
     if (warp == kStatsWarp) {
         // ---- statistics: block partial -> cluster exchange -> row constants
         for (int j = 0; j < nu; ++j) {
-            const int unit = u0 + j;
+            const int unit = u0 + j * ustep;
             const bool bonus = !ENS && (unit % K1 == P.k);
             const int par = j & 1;
             const uint32_t ph = (uint32_t)(j >> 1) & 1u;
@@ -481,7 +492,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
         // ---- resolver: row reports, tickets; the sequence's last tickets draw the token
         int seg = 0;                               // units of the current sequence finished so far
         for (int j = 0; j < nu; ++j) {
-            const int unit = u0 + j;
+            const int unit = u0 + j * ustep;
             const int dslot = j % kDoneDepth;
             const bool reports = (j % C == rank);   // the blocks of the cluster take turns
             if constexpr (ENS) {
@@ -546,7 +557,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
             int slot_i = 0;               // ring slot of the next copy
             constexpr size_t kStride = (size_t)kConsumerWarps * kStageVecs * VEC;   // from one of my stages to the next
             auto begin_run = [&]() {      // lane 0
-                const UnitRef ur = unit_ref<ENS>(P, u0 + (run == 2 ? ji - 1 : run == 4 ? nu - 1 : ji));
+                const UnitRef ur = unit_ref<ENS>(P, u0 + (run == 2 ? ji - 1 : run == 4 ? nu - 1 : ji) * ustep);
                 const size_t off = (size_t)(vb0 + cw * kStageVecs) * VEC + (size_t)ti * kStride;
                 Tb = reinterpret_cast<const ET*>(P.T) + ur.t_row * P.V + off;
                 Db = ur.bonus ? nullptr : reinterpret_cast<const ET*>(ENS ? P.Dn[ur.n] : P.D) + ur.d_row * P.V + off;
@@ -598,7 +609,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
             ps.RT = ps.RD = kEmptyRef;
             ps.ls.init();
             auto run_pass1 = [&](int j, int t0, int t1) {
-                const UnitRef ur = unit_ref<ENS>(P, u0 + j);
+                const UnitRef ur = unit_ref<ENS>(P, u0 + j * ustep);
                 const bool bonus = ur.bonus;
                 // the block's slice of the two rows in global memory (for the rare second try of a stage)
                 const ET* Trow = reinterpret_cast<const ET*>(P.T) + ur.t_row * P.V + (size_t)vb0 * VEC;
@@ -616,7 +627,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
                 }
             };
             auto run_pass2 = [&](int j) {
-                const int unit = u0 + j;
+                const int unit = u0 + j * ustep;
                 const UnitRef ur = unit_ref<ENS>(P, unit);
                 const bool bonus = ur.bonus;
                 const int dslot = j % kDoneDepth;
@@ -697,7 +708,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
         // sequence resolved from now on
         if (tid == 0) atomicExch(P.sticky, 1u);
         if (P.status)
-            for (int j = tid; j < nu; j += kStreamThreads) atomicOr(P.status + unit_ref<ENS>(P, u0 + j).b, kStatusTimeout);
+            for (int j = tid; j < nu; j += kStreamThreads) atomicOr(P.status + unit_ref<ENS>(P, u0 + j * ustep).b, kStatusTimeout);
     }
     // no block leaves while another may still write to its shared memory
     cluster.sync();
