@@ -482,3 +482,19 @@ def test_host_entry_point_slices_large_batches(binding):
     seqs = [0, 7, 8, 23, 39]
     ref = oracle_of(inp, seqs)
     check(inp, host, ref, seqs=seqs, max_band_frac=1.0)
+
+
+@pytest.mark.parametrize("name", ["cfg3", "cfg4"])
+def test_pinsker_ties_acceptance_probability_to_the_loss_on_every_row(binding, name):
+    """TV(p,q) <= sqrt(KL(p||q)/2) (used in the proof of Lemma 1), with TV = 1 - acc_prob (Eq. 1):
+    holds for every row of a full-size workload whatever the oracle says; also 0 <= acc_prob <= 1."""
+    cfg = synth.CONFIGS[name]
+    inp = synth.make_inputs(cfg)
+    T, D, x, u = to_device(inp)
+    out = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau, want_grad=False)
+    torch.cuda.synchronize()
+    acc = out.acc_prob.cpu().numpy().astype(np.float64)
+    loss = out.loss.cpu().numpy().astype(np.float64)
+    assert ((acc >= -1e-6) & (acc <= 1 + 1e-6)).all()
+    assert ((1.0 - acc) <= np.sqrt(loss / 2.0) + 1e-5).all()
+    assert (out.status.cpu().numpy() == 0).all()
