@@ -28,8 +28,8 @@
  *     caller.  The library never frees or reallocates caller memory.
  *   - Tensors are dense, row-major, contiguous.  Logit rows may start at any element-aligned
  *     address; rows whose byte length and base address are multiples of 16 take the fast
- *     (bulk-copy, cluster) path, everything else takes a slower generic path with the same
- *     results.
+ *     (bulk-copy, cluster) path, everything else takes a generic path with the same results
+ *     that is about three times slower: pad the vocabulary to a multiple of 8 entries if you can.
  *   - Work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = the legacy default
  *     stream).  The call does not synchronise; outputs are valid once the stream reaches the
  *     end of the enqueued work.
