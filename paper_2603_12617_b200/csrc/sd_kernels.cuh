@@ -716,7 +716,6 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
 
 // ---- generic path --------------------------------------------------------------------------
 struct GenericShared {
-    float wmax[2][kGenericWarps];
     PartialStats warp_part[kGenericWarps];
     RowConst rc;
     int last;
@@ -734,30 +733,36 @@ __global__ void __launch_bounds__(kGenericThreads) sd_generic_kernel(const __gri
     const size_t offT = (size_t)unit * P.V;
     const size_t offD = (size_t)(b * P.k + (bonus ? 0 : i)) * P.V;
 
-    // sweep 0: the row maxima give the references of every exponential
-    float mT = -3.402823466e+38f, mD = -3.402823466e+38f;
-    for (int v = tid; v < P.V; v += kGenericThreads) {
-        mT = fmaxf(mT, E::load(P.T, offT + v));
-        if (!bonus) mD = fmaxf(mD, E::load(P.D, offD + v));
-    }
-    mT = warp_max_f32(mT);
-    mD = warp_max_f32(mD);
-    if (lane == 0) { sh.wmax[0][warp] = mT; sh.wmax[1][warp] = mD; }
-    __syncthreads();
-#pragma unroll
-    for (int w = 0; w < kGenericWarps; ++w) { mT = fmaxf(mT, sh.wmax[0][w]); mD = fmaxf(mD, sh.wmax[1][w]); }
-    const float RT = ref_of(mT, P.c), RD = bonus ? kEmptyRef : ref_of(mD, P.c);
-
-    // sweep 1: softmax sums
+    // sweep 1: softmax sums relative to integer references that every warp raises as it goes (the
+    // sums follow by exact powers of two), eight entries per thread at a time; the warps' partial
+    // sums, each under its own references, are merged exactly afterwards
+    constexpr int kPer = (DT == SD_DTYPE_BF16) ? 16 : 8;
+    float RT = kEmptyRef, RD = kEmptyRef;
     LaneSums ls;
     ls.init();
-    for (int v = tid; v < P.V; v += kGenericThreads) {
-        float t[1] = {E::load(P.T, offT + v)};
-        if (!bonus) {
-            float d[1] = {E::load(P.D, offD + v)};
-            ls.template add_pair<1>(t, d, P.c, -RT, -RD);
-        } else {
-            ls.template add_bonus<1>(t, P.c, -RT);
+    for (int base = 0; base < P.V; base += kPer * kGenericThreads) {
+        float t[kPer], d[kPer];
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) {
+            const int v = base + j * kGenericThreads + tid;
+            t[j] = v < P.V ? E::load(P.T, offT + v) : -INFINITY;
+            d[j] = (!bonus && v < P.V) ? E::load(P.D, offD + v) : -INFINITY;
+        }
+        float mt = t[0], md = d[0];
+#pragma unroll
+        for (int j = 1; j < kPer; ++j) { mt = fmaxf(mt, t[j]); md = fmaxf(md, d[j]); }
+        const float nT = fmaxf(RT, warp_max_ref(ref_of(mt, P.c)));
+        const float nD = bonus ? kEmptyRef : fmaxf(RD, warp_max_ref(ref_of(md, P.c)));
+        ls.rescale(nT - RT, nD - RD);
+        RT = nT;
+        RD = nD;
+#pragma unroll
+        for (int j0 = 0; j0 < kPer; j0 += 8) {
+            float t8[8], d8[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { t8[j] = t[j0 + j]; d8[j] = d[j0 + j]; }
+            if (!bonus) ls.template add_pair<8>(t8, d8, P.c, -RT, -RD);
+            else        ls.template add_bonus<8>(t8, P.c, -RT);
         }
     }
     {
@@ -782,6 +787,7 @@ __global__ void __launch_bounds__(kGenericThreads) sd_generic_kernel(const __gri
     for (int q = warp; q < P.NR; q += kGenericWarps) {
         const int ebase = q * P.RE;
         float mass = 0.f;
+#pragma unroll 8
         for (int j = lane; j < P.RE; j += 32) {
             const int v = ebase + j;
             if (v < P.V) {
