@@ -50,10 +50,10 @@ UNIT = "positions/s"
 L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum per launch at full size, from the ncu captures
 # summarised under profiles/ (bytes; a workload that is not listed has not been captured)
-NCU_TRAFFIC_ENSEMBLE = {("cfg5", 3): 3432264448 + 2326029056}
+NCU_TRAFFIC_ENSEMBLE = {("cfg5", 3): 3388811776 + 2325275904}
 NCU_TRAFFIC_ERRORS = {"cfg5": 1707537664 + 3327232 + 251808256 + 99995904}   # both kernels of the step
 NCU_TRAFFIC_GREEDY = {"cfg5": 919481088 + 244224}
-NCU_TRAFFIC_BYTES = {"cfg5": 2081561856 + 758121728, "cfg3": 155340544 + 37302016, "cfg4": 179461376 + 50529024}
+NCU_TRAFFIC_BYTES = {"cfg5": 2078492160 + 758877952, "cfg3": 155482368 + 36729856, "cfg4": 179505152 + 50643456}
 
 
 def measured_peak_gbs():
