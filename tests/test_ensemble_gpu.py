@@ -215,3 +215,28 @@ def test_orders_of_the_walk_with_many_units_per_cluster(binding, lag, cluster, m
         torch.cuda.synchronize()
         assert torch.equal(one.loss, out.loss[n])
         assert torch.equal(one.grad_draft.view(torch.int16), out.grad[n].view(torch.int16))
+
+
+def test_gradients_of_some_learners_can_be_left_out(binding):
+    """A NULL entry in the array of gradient pointers: no gradient for that learner, the rest unchanged."""
+    import ctypes
+    cfg = synth.custom_config(4, 3, 8192, dtype="f32")
+    inp = synth.make_inputs(cfg)
+    Ds = synth.ensemble_drafts(inp, 3)
+    T, dDs = dev(inp.target_logits), [dev(d) for d in Ds]
+    full = binding.sd_ensemble_feedback(T, dDs, inp.tau, EPS)
+    torch.cuda.synchronize()
+    out = binding.EnsembleOutputs(loss=torch.empty_like(full.loss), grad=None,
+                                  round_loss=torch.empty_like(full.round_loss), cum_loss=torch.empty_like(full.cum_loss),
+                                  weights=torch.empty_like(full.weights), status=None)
+    g0 = torch.full_like(full.grad[0], 7.0)
+    g2 = torch.empty_like(full.grad[2])
+    dptr = (ctypes.c_void_p * 3)(*[d.data_ptr() for d in dDs])
+    gptr = (ctypes.c_void_p * 3)(None, None, g2.data_ptr())
+    rc = binding._lib.sd_ensemble_feedback(T.data_ptr(), dptr, 3, float(inp.tau), EPS, cfg.B, cfg.k, cfg.V, 0, None,
+                                           out.loss.data_ptr(), gptr, out.round_loss.data_ptr(),
+                                           out.cum_loss.data_ptr(), out.weights.data_ptr(), None, None, 0, None)
+    torch.cuda.synchronize()
+    assert rc == 0
+    assert torch.equal(out.loss, full.loss) and torch.equal(out.weights, full.weights)
+    assert torch.equal(g2, full.grad[2]) and (g0 == 7.0).all()

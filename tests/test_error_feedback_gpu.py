@@ -200,3 +200,20 @@ def test_orders_of_the_walk_and_cluster_sizes_with_many_units_per_cluster(bindin
     rows = full.grad_draft[torch.arange(cfg.B, device="cuda"), n.clamp(max=cfg.k - 1)]
     rows[n == cfg.k] = 0
     assert torch.equal(out.error_grad.view(torch.int16), rows.view(torch.int16))
+
+
+def test_optional_outputs_can_be_left_out(binding):
+    cfg = synth.CONFIGS["cfg2"]
+    inp = synth.make_inputs(cfg)
+    T, D = dev(inp.target_logits), dev(inp.draft_logits)
+    x, u = torch.from_numpy(inp.draft_tokens).cuda(), torch.from_numpy(inp.uniforms).cuda()
+    full = binding.sd_verify_error_feedback(T, D, x, u, inp.tau)
+    for kw in (dict(want_loss=False), dict(want_grad=False), dict(want_status=False),
+               dict(want_loss=False, want_grad=False, want_status=False)):
+        out = binding.sd_verify_error_feedback(T, D, x, u, inp.tau, **kw)
+        torch.cuda.synchronize()
+        assert torch.equal(out.accept_len, full.accept_len) and torch.equal(out.tokens, full.tokens)
+        if out.loss is not None:
+            assert torch.equal(out.loss, full.loss)
+        if out.error_grad is not None:
+            assert torch.equal(out.error_grad.view(torch.int16), full.error_grad.view(torch.int16))
