@@ -48,10 +48,10 @@
  *     policy only holds lines inside such a set-aside.  The limit belongs to this process's
  *     context and ends with it; lines kept that way stay until later ones displace them, so a
  *     process whose other kernels want all of L2 may call cudaCtxResetPersistingL2Cache()
- *     between its own phases.  Environment: SD_VERIFY_L2_PERSIST_MIB=<MiB> chooses another
- *     size, 0 leaves the limit untouched.  Other tuning knobs read from the environment (never
- *     needed for correctness): SD_VERIFY_CLUSTER (cluster size of the fast path),
- *     SD_VERIFY_LAG, SD_VERIFY_L2_MIB, SD_VERIFY_FORCE_GENERIC, SD_GREEDY_BLOCKS_PER_SM.
+ *     between its own phases.  A caller that wants its context left alone calls
+ *     sd_set_option(SD_OPT_L2_PERSIST_MIB, 0) before the first call on the device (any other
+ *     value chooses another size).  See sd_set_option for the other tuning options; none is ever
+ *     needed for correctness.
  */
 #ifndef SD_VERIFY_H
 #define SD_VERIFY_H
@@ -154,7 +154,9 @@ int sd_verify_feedback_ex(const void* target_logits, const void* draft_logits,
  * for as long as the process lives, whether this entry point is used or not.
  *
  * Arguments and results are those of sd_verify_feedback_ex without workspace/workspace_bytes.
- * It never calls cudaMalloc, cudaFree or any other allocating routine.
+ * It never calls cudaMalloc, cudaFree or any other allocating routine.  (The array itself becomes
+ * resident when the CUDA runtime loads the library's device code on a GPU -- at the latest during
+ * the first call of any entry point on that GPU -- not through a call of this function.)
  *
  *   - Shapes whose sd_workspace_bytes(B,k,V,dtype) exceeds SD_STATIC_SCRATCH_BYTES are refused
  *     with SD_ERR_WORKSPACE (sd_last_cuda_error() says how many bytes were needed); nothing is
@@ -286,6 +288,39 @@ int sd_verify_feedback_host(const void* target_logits, const void* draft_logits,
                             int B, int k, int V, int dtype, int32_t* out_accept_len,
                             int32_t* out_tokens, float* out_loss, void* out_grad_draft,
                             float* out_acc_prob, uint32_t* out_status);
+
+/*
+ * Tuning options.  Each has a default, which an environment variable of the process (read once,
+ * at the first use of the library) replaces, and which sd_set_option replaces at any time; a
+ * change applies to the calls made after it.  Results never depend on them beyond rounding
+ * (sums are taken in another order when the launch shape changes).
+ *   SD_OPT_L2_PERSIST_MIB        env SD_VERIFY_L2_PERSIST_MIB   default 52   L2 set-aside requested on the
+ *                                first call on a device; 0 = leave the context's limit untouched
+ *   SD_OPT_CLUSTER               env SD_VERIFY_CLUSTER          default 0    cluster size of the fast path
+ *                                (1..16), 0 = chosen per shape
+ *   SD_OPT_LAG                   env SD_VERIFY_LAG              default 1    stages of the next row pair
+ *                                that go before the second pass over a row pair
+ *   SD_OPT_L2_BUDGET_MIB         env SD_VERIFY_L2_MIB           default 80   bytes of row pairs in flight
+ *                                between their two passes that the launch shape may assume L2 holds
+ *   SD_OPT_FORCE_GENERIC         env SD_VERIFY_FORCE_GENERIC    default 0    non-zero: element-wise path
+ *                                even for aligned rows
+ *   SD_OPT_GREEDY_BLOCKS_PER_SM  env SD_GREEDY_BLOCKS_PER_SM    default 4    resident blocks of sd_verify_greedy
+ *   SD_OPT_WAIT_POLLS            env SD_VERIFY_WAIT_POLLS       default 2^21 polls after which a wait
+ *                                inside the fast path gives up (the sequences concerned then carry
+ *                                SD_STATUS_TIMEOUT); the wait also ends after about a second
+ * sd_set_option returns SD_OK, or SD_ERR_SHAPE for an unknown option; sd_get_option returns the
+ * value in force, or -1 for an unknown option.
+ */
+#define SD_OPT_L2_PERSIST_MIB 0
+#define SD_OPT_CLUSTER 1
+#define SD_OPT_LAG 2
+#define SD_OPT_L2_BUDGET_MIB 3
+#define SD_OPT_FORCE_GENERIC 4
+#define SD_OPT_GREEDY_BLOCKS_PER_SM 5
+#define SD_OPT_WAIT_POLLS 6
+#define SD_OPT_COUNT 7
+int sd_set_option(int option_id, long long value);
+long long sd_get_option(int option_id);
 
 /*
  * sd_launch_info -- HOST out-parameters describing how the last successful device call on this

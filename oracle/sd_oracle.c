@@ -375,6 +375,57 @@ int sd_oracle_ensemble(const void* T, const void* const* Dn, int N, int dtype, d
     return 0;
 }
 
+/*
+ * sd_oracle_draw_interval -- where token y sits on the inverse CDF that Algorithm 1 draws the extra
+ * token from ("Verify and update the draft sequence") when the accept length of the sequence is n:
+ * the residual max(0, p_n - q_n) for n < k (p_n itself when the residual has no mass, as in
+ * sd_oracle), the bonus distribution p_k for n = k.  Sums are sequential in vocabulary order:
+ *     out[0] = c_{y-1} = sum_{w<y} r_w,   out[1] = c_y = c_{y-1} + r_y,   out[2] = R = sum_w r_w.
+ * The draw with uniform u returns y exactly when c_{y-1} <= u*R < c_y.  T [k+1,V] and D [k,V] are
+ * the logits of ONE sequence.  Used by the tests to decide whether an answer that differs from
+ * sd_oracle's on a sequence flagged as sitting on a decision threshold is still a valid one.
+ * Returns 0, or -1 on a bad argument or allocation failure.
+ */
+int sd_oracle_draw_interval(const void* T, const void* D, int dtype, double tau, int k, int V, int n,
+                            int y, double* out) {
+    if (!T || !D || !out || k < 1 || V < 1 || n < 0 || n > k || y < 0 || y >= V) return -1;
+    if (!(tau > 0.0) || !isfinite(tau)) return -1;
+    if (dtype != SD_ORACLE_F32 && dtype != SD_ORACLE_BF16) return -1;
+    double* p = (double*)malloc((size_t)V * sizeof(double));
+    double* q = (double*)malloc((size_t)V * sizeof(double));
+    double* lg = (double*)malloc((size_t)V * sizeof(double));
+    if (!p || !q || !lg) {
+        free(p); free(q); free(lg);
+        return -1;
+    }
+    double S;
+    softmax_row(T, dtype, (size_t)n * V, V, tau, p, lg, &S);
+    double R = 0.0;
+    if (n < k) {
+        softmax_row(D, dtype, (size_t)n * V, V, tau, q, lg, &S);
+        for (int v = 0; v < V; ++v) {
+            double d = p[v] - q[v];
+            q[v] = d > 0.0 ? d : 0.0;          /* q now holds the residual */
+            R += q[v];
+        }
+        if (!(R > 0.0))
+            for (int v = 0; v < V; ++v) q[v] = p[v];
+    } else {
+        for (int v = 0; v < V; ++v) q[v] = p[v];
+    }
+    double c = 0.0, before = 0.0, after = 0.0;
+    for (int v = 0; v < V; ++v) {
+        if (v == y) before = c;
+        c += q[v];
+        if (v == y) after = c;
+    }
+    out[0] = before;
+    out[1] = after;
+    out[2] = c;
+    free(p); free(q); free(lg);
+    return 0;
+}
+
 /* Threads the build can use: 1 without OpenMP. */
 int sd_oracle_max_threads(void) {
 #ifdef _OPENMP

@@ -2,7 +2,7 @@
 
 Only the tests, the smoke check and the benchmark's CPU-baseline leg may import this module.
 It compiles ``sd_oracle.c`` with gcc on first use (``build()``), loads it and exposes
-``verify_feedback``, ``verify_greedy`` and ``ensemble_feedback``, which take and return numpy arrays.  Nothing here touches CUDA and nothing
+``verify_feedback``, ``draw_interval``, ``verify_greedy`` and ``ensemble_feedback``, which take and return numpy arrays.  Nothing here touches CUDA and nothing
 here is imported by the product package.
 """
 from __future__ import annotations
@@ -41,6 +41,9 @@ def _load():
         lib.sd_oracle.argtypes = [P, P, ctypes.c_int, P, P, ctypes.c_double, ctypes.c_int,
                                   ctypes.c_int, ctypes.c_int, P, P, P, P, P, P, P, P, P,
                                   ctypes.c_int]
+        lib.sd_oracle_draw_interval.restype = ctypes.c_int
+        lib.sd_oracle_draw_interval.argtypes = [P, P, ctypes.c_int, ctypes.c_double, ctypes.c_int, ctypes.c_int,
+                                                ctypes.c_int, ctypes.c_int, P]
         lib.sd_oracle_greedy.restype = ctypes.c_int
         lib.sd_oracle_greedy.argtypes = [P, ctypes.c_int, P, ctypes.c_int, ctypes.c_int, ctypes.c_int, P, P, P]
         lib.sd_oracle_ensemble.restype = ctypes.c_int
@@ -109,6 +112,28 @@ def verify_feedback(target_logits: np.ndarray, draft_logits: np.ndarray, draft_t
     if rc != 0:
         raise RuntimeError(f"sd_oracle failed with code {rc}")
     return res
+
+
+def draw_interval(target_logits: np.ndarray, draft_logits: np.ndarray, temperature: float, n: int, y: int):
+    """Where token ``y`` sits on the inverse CDF the extra token of ONE sequence ([k+1,V] and [k,V]
+    logits) is drawn from when its accept length is ``n``: returns (c_before, c_after, R); the draw
+    with uniform u gives ``y`` exactly when c_before <= u*R < c_after."""
+    T = np.ascontiguousarray(target_logits)
+    D = np.ascontiguousarray(draft_logits)
+    if T.dtype == np.float32 and D.dtype == np.float32:
+        dtype = F32
+    elif T.dtype == np.uint16 and D.dtype == np.uint16:
+        dtype = BF16
+    else:
+        raise TypeError("logits must both be float32 or both be uint16 (bf16 bits)")
+    if T.ndim != 2 or D.ndim != 2 or T.shape[0] != D.shape[0] + 1 or T.shape[1] != D.shape[1]:
+        raise ValueError("logits of one sequence: [k+1,V] and [k,V]")
+    out = np.empty(3, np.float64)
+    rc = _load().sd_oracle_draw_interval(_ptr(T), _ptr(D), dtype, float(temperature), D.shape[0], T.shape[1],
+                                         int(n), int(y), _ptr(out))
+    if rc != 0:
+        raise RuntimeError(f"sd_oracle_draw_interval failed with code {rc}")
+    return float(out[0]), float(out[1]), float(out[2])
 
 
 @dataclass

@@ -17,6 +17,14 @@ import torch
 SD_DTYPE_F32 = 0
 SD_DTYPE_BF16 = 1
 
+SD_OPT_L2_PERSIST_MIB = 0
+SD_OPT_CLUSTER = 1
+SD_OPT_LAG = 2
+SD_OPT_L2_BUDGET_MIB = 3
+SD_OPT_FORCE_GENERIC = 4
+SD_OPT_GREEDY_BLOCKS_PER_SM = 5
+SD_OPT_WAIT_POLLS = 6
+
 SD_STATUS_BAD_TOKEN = 1
 SD_STATUS_BAD_ROW = 2
 SD_STATUS_ZERO_RESIDUAL = 4
@@ -62,6 +70,10 @@ def _load() -> ctypes.CDLL:
     lib.sd_verify_feedback_host.argtypes = [P, P, P, P, F, I, I, I, I, P, P, P, P, P, P]
     lib.sd_workspace_bytes.restype = Z
     lib.sd_workspace_bytes.argtypes = [I, I, I, I]
+    lib.sd_set_option.restype = I
+    lib.sd_set_option.argtypes = [I, ctypes.c_longlong]
+    lib.sd_get_option.restype = ctypes.c_longlong
+    lib.sd_get_option.argtypes = [I]
     lib.sd_launch_info.restype = None
     lib.sd_launch_info.argtypes = [P] * 6
     lib.sd_release_cached_buffers.restype = None
@@ -137,6 +149,16 @@ def sd_launch_info() -> dict:
     _lib.sd_launch_info(*[ctypes.byref(v) for v in vals])
     keys = ["path", "cluster_size", "threads", "smem_bytes", "blocks", "kernels"]
     return {k: v.value for k, v in zip(keys, vals)}
+
+
+def sd_set_option(option_id: int, value: int) -> None:
+    rc = _lib.sd_set_option(int(option_id), int(value))
+    if rc != 0:
+        raise SdVerifyError(rc, "sd_set_option")
+
+
+def sd_get_option(option_id: int) -> int:
+    return int(_lib.sd_get_option(int(option_id)))
 
 
 def sd_release_cached_buffers() -> None:

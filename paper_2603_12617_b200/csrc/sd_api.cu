@@ -20,7 +20,38 @@ constexpr size_t kAlign = 256;
 constexpr int kStreamSmem = kRingSlots * kStageBytes + (int)sizeof(StreamShared);
 static_assert(kStreamSmem <= 227 * 1024, "ring does not fit the shared memory of a block");
 constexpr int kL2PersistMiB = 52;
-constexpr double kL2BudgetMiB = 80.0;              // row pairs in flight between their two passes should fit this
+constexpr long long kL2BudgetMiB = 80;             // row pairs in flight between their two passes should fit this
+
+// Tuning options: defaults, overridden once per process by the environment, then by sd_set_option.
+struct Options {
+    long long v[SD_OPT_COUNT];
+};
+std::once_flag g_opt_once;
+std::mutex g_opt_mu;
+Options g_opt;
+
+void init_options() {
+    std::call_once(g_opt_once, [] {
+        static const struct { int id; const char* env; long long dflt; } table[] = {
+            {SD_OPT_L2_PERSIST_MIB, "SD_VERIFY_L2_PERSIST_MIB", kL2PersistMiB},
+            {SD_OPT_CLUSTER, "SD_VERIFY_CLUSTER", 0},
+            {SD_OPT_LAG, "SD_VERIFY_LAG", 1},
+            {SD_OPT_L2_BUDGET_MIB, "SD_VERIFY_L2_MIB", kL2BudgetMiB},
+            {SD_OPT_FORCE_GENERIC, "SD_VERIFY_FORCE_GENERIC", 0},
+            {SD_OPT_GREEDY_BLOCKS_PER_SM, "SD_GREEDY_BLOCKS_PER_SM", 4},
+            {SD_OPT_WAIT_POLLS, "SD_VERIFY_WAIT_POLLS", (long long)kWaitLimit},
+        };
+        for (const auto& t : table) {
+            const char* e = getenv(t.env);
+            g_opt.v[t.id] = (e && *e) ? atoll(e) : t.dflt;
+        }
+    });
+}
+long long option(int id) {
+    init_options();
+    std::lock_guard<std::mutex> lock(g_opt_mu);
+    return g_opt.v[id];
+}
 
 thread_local char tl_cuda_error[256] = "";
 thread_local int tl_info[6] = {0, 0, 0, 0, 0, 0};
@@ -81,8 +112,11 @@ struct DeviceState {
     // grow-only scratch of the 13-argument entry points
     void* ws = nullptr;
     size_t ws_bytes = 0;
-    bool ws_clean = false;   // tickets and status words are zero
-    size_t ws_zero_bytes = 0;   // leading bytes of ws known to be zero (what greedy verification needs)
+    // Leading bytes of ws known to be zero.  Every entry point wants the head of its own layout
+    // zero (tickets, status words, error flag; keys of the greedy path), leaves that head zero and
+    // writes whatever it likes behind it -- and where the head ends depends on the shape.  So a call
+    // whose head is longer than this clears it first, and afterwards its own head is what is known.
+    size_t ws_zero_bytes = 0;
     bool attr_set[2][3] = {{false, false, false}, {false, false, false}};   // shared-memory / cluster attributes of the fast kernels
     int max_clusters[2][kMaxCluster + 1];   // resident clusters of 1..16 blocks, -1 = not asked yet
     // last launch-shape decision of the fast path
@@ -117,10 +151,10 @@ int current_device(int* dev, DeviceState** st) {
         // path fetches with it what pass 2 reads again): without a set-aside the policy has no
         // effect and pass 2 of the largest workloads goes back to HBM for most of its lines.  52 MiB
         // (granted as 58 MB) measured best on the 126 MB L2: larger ones starve everything else.
-        // A limit of this process's context only; SD_VERIFY_L2_PERSIST_MIB=0 leaves it alone.
+        // A limit of this process's context only; option SD_OPT_L2_PERSIST_MIB = 0 leaves it alone.
         {
-            const char* env = getenv("SD_VERIFY_L2_PERSIST_MIB");
-            size_t want = (size_t)(env ? atoi(env) : kL2PersistMiB) << 20;
+            const long long mib = option(SD_OPT_L2_PERSIST_MIB);
+            size_t want = (size_t)(mib > 0 ? mib : 0) << 20;
             if (want > (size_t)prop.persistingL2CacheMaxSize) want = (size_t)prop.persistingL2CacheMaxSize;
             if (want > 0 && cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, want) != cudaSuccess)
                 (void)cudaGetLastError();   // not fatal: the path is only slower without it
@@ -201,12 +235,9 @@ int launch_generic(const Params& P, cudaStream_t stream) {
 // blocks: 148 for C = 1 and 2, 135 for 3, 132 for 4, 120 for 8, 112 for 16).  If none fits, the
 // largest cluster.
 int choose_stream(DeviceState& d, int V, long long units, int dtype, int* G_out, int* per_out, int* lag_out) {
-    const char* env = getenv("SD_VERIFY_CLUSTER");
-    const int forced = env ? atoi(env) : 0;
-    const char* env_l2 = getenv("SD_VERIFY_L2_MIB");
-    const double l2_budget = (env_l2 ? atof(env_l2) : kL2BudgetMiB) * 1048576.0;
-    const char* env_lag = getenv("SD_VERIFY_LAG");
-    const int lag = env_lag ? atoi(env_lag) : 1;   // stages of the next unit before pass 2 of a unit
+    const int forced = (int)option(SD_OPT_CLUSTER);
+    const double l2_budget = (double)option(SD_OPT_L2_BUDGET_MIB) * 1048576.0;
+    const int lag = (int)option(SD_OPT_LAG);       // stages of the next unit before pass 2 of a unit
     if (d.dec_dtype == dtype && d.dec_V == V && d.dec_units == units && d.dec_forced == forced &&
         d.dec_l2 == l2_budget && d.dec_lag == lag) {
         *G_out = d.dec_G;
@@ -291,10 +322,11 @@ int run_device(DeviceState& d, const void* T, const void* D, const int32_t* x, c
     P.region_sums = reinterpret_cast<float*>(ws + L.region_sums);
 
     if (!clean) SD_CUDA(cudaMemsetAsync(ws, 0, L.accept, stream));   // tickets, status words, sticky flag
+    if (status) SD_CUDA(cudaMemsetAsync(status, 0, (size_t)B * 4, stream));   // bits are ORed in on the device
 
     const size_t row_bytes = (size_t)V * elem_bytes(dtype);
     const bool fast = (row_bytes % 16 == 0) && aligned(T, 16) && aligned(D, 16) && (!grad || aligned(grad, 16)) &&
-                      !getenv("SD_VERIFY_FORCE_GENERIC");
+                      option(SD_OPT_FORCE_GENERIC) == 0;
     int C = 0, G = 0, lag = 0, per = 0;
     if (fast) C = choose_stream(d, V, (long long)B * (k + 1), dtype, &G, &per, &lag);
     int rc;
@@ -334,16 +366,15 @@ int run_cached(const void* T, const void* D, const int32_t* x, const float* u, f
         const size_t want = align_up(L.total + L.total / 4, 1 << 20);
         SD_CUDA(cudaMalloc(&d->ws, want));
         d->ws_bytes = want;
-        // Zero all of it once: every call leaves its ticket and status words at zero again, so
-        // later calls of any shape find zeros wherever their layout puts those words.
-        SD_CUDA(cudaMemset(d->ws, 0, want));
-        SD_CUDA(cudaDeviceSynchronize());
-        d->ws_clean = true;
+        d->ws_zero_bytes = 0;
     }
-    d->ws_zero_bytes = 0;   // row constants and sums of this call stay behind
+    // the head of this layout (tickets, status words, error flag) must be zero on entry; the kernel
+    // leaves it zero again and dirties everything behind it
+    const bool clean = d->ws_zero_bytes >= L.accept;
+    d->ws_zero_bytes = 0;
     rc = run_device(*d, T, D, x, u, tau, B, k, V, dtype, accept_len, tokens, loss, grad, nullptr, nullptr,
-                    static_cast<unsigned char*>(d->ws), L, d->ws_clean, static_cast<cudaStream_t>(stream));
-    d->ws_clean = (rc == SD_OK);   // a failed launch may leave tickets behind: zero them next time
+                    static_cast<unsigned char*>(d->ws), L, clean, static_cast<cudaStream_t>(stream));
+    if (rc == SD_OK) d->ws_zero_bytes = L.accept;   // a failed launch may leave anything behind
     return rc;
 }
 
@@ -483,10 +514,10 @@ int sd_ensemble_feedback(const void* target_logits, const void* const* draft_log
             const size_t want = 1 << 20;
             SD_CUDA(cudaMalloc(&d->ws, want));
             d->ws_bytes = want;
+            d->ws_zero_bytes = 0;
         }
         ws = static_cast<unsigned char*>(d->ws);
-        d->ws_clean = false;       // the flag word of this call sits where other entry points expect zeros
-        d->ws_zero_bytes = 0;
+        d->ws_zero_bytes = 0;      // the flag word of this call sits where other entry points expect zeros
     }
     SD_CUDA(cudaMemsetAsync(ws, 0, SD_ENSEMBLE_SCRATCH_BYTES, st));
     if (out_status) SD_CUDA(cudaMemsetAsync(out_status, 0, (size_t)B * 4, st));
@@ -557,8 +588,7 @@ int sd_verify_error_feedback(const void* target_logits, const void* draft_logits
             d->ws_bytes = want;
         }
         ws = static_cast<unsigned char*>(d->ws);
-        d->ws_clean = false;      // cleared below for this call; say so to the others
-        d->ws_zero_bytes = 0;
+        d->ws_zero_bytes = 0;     // cleared below for this call; what it leaves behind is not tracked
     }
     Params P;
     memset(&P, 0, sizeof P);
@@ -576,6 +606,7 @@ int sd_verify_error_feedback(const void* target_logits, const void* draft_logits
     P.rowc = reinterpret_cast<RowConst*>(ws + L.rowc);
     P.region_sums = reinterpret_cast<float*>(ws + L.region_sums);
     SD_CUDA(cudaMemsetAsync(ws, 0, L.accept, st));   // tickets, status words, sticky flag
+    if (out_status) SD_CUDA(cudaMemsetAsync(out_status, 0, (size_t)B * 4, st));   // bits are ORed in on the device
     int G = 0, lag = 0, per = 0;
     const int C = choose_stream(*d, V, (long long)B * (k + 1), dtype, &G, &per, &lag);
     if (C <= 0) return SD_ERR_CUDA;
@@ -635,7 +666,6 @@ int sd_verify_greedy(const void* target_logits, const int32_t* draft_tokens, int
             d->ws_bytes = want;
             SD_CUDA(cudaMemset(d->ws, 0, want));
             SD_CUDA(cudaDeviceSynchronize());
-            d->ws_clean = true;
             d->ws_zero_bytes = want;
         }
         ws = static_cast<unsigned char*>(d->ws);
@@ -655,18 +685,15 @@ int sd_verify_greedy(const void* target_logits, const int32_t* draft_tokens, int
     const long long items = (long long)B * (k + 1) * P.items_per_row;
     // blocks per SM: 4 of 256 threads, 8 loads of 16 bytes in flight per thread, measured best among 2..8
     // on the largest workload (more blocks disturb the DRAM page locality of the streams);
-    // SD_GREEDY_BLOCKS_PER_SM (1..8) overrides it
-    int per_sm = 4;
-    if (const char* env = getenv("SD_GREEDY_BLOCKS_PER_SM")) {
-        const int v = atoi(env);
-        if (v >= 1 && v <= 8) per_sm = v;
-    }
+    // option SD_OPT_GREEDY_BLOCKS_PER_SM (1..8) overrides it
+    int per_sm = (int)option(SD_OPT_GREEDY_BLOCKS_PER_SM);
+    if (per_sm < 1 || per_sm > 8) per_sm = 4;
     const long long cap = (long long)d->sm_count * per_sm;
     const unsigned grid = (unsigned)(items < cap ? items : cap);
     if (dtype == SD_DTYPE_F32) sd_greedy_kernel<SD_DTYPE_F32><<<grid, kGreedyThreads, 0, st>>>(P);
     else                       sd_greedy_kernel<SD_DTYPE_BF16><<<grid, kGreedyThreads, 0, st>>>(P);
     const cudaError_t launched = cudaGetLastError();
-    if (!workspace) d->ws_zero_bytes = launched == cudaSuccess ? (d->ws_zero_bytes > need ? d->ws_zero_bytes : need) : 0;
+    if (!workspace) d->ws_zero_bytes = launched == cudaSuccess ? (clean ? d->ws_zero_bytes : need) : 0;
     SD_CUDA(launched);
     tl_info[0] = 2; tl_info[1] = 1; tl_info[2] = kGreedyThreads; tl_info[3] = 0;
     tl_info[4] = (int)grid; tl_info[5] = 1;
@@ -787,6 +814,19 @@ int sd_verify_feedback_host(const void* target_logits, const void* draft_logits,
     return SD_OK;
 }
 
+int sd_set_option(int option_id, long long value) {
+    if (option_id < 0 || option_id >= SD_OPT_COUNT) return SD_ERR_SHAPE;
+    init_options();
+    std::lock_guard<std::mutex> lock(g_opt_mu);
+    g_opt.v[option_id] = value;
+    return SD_OK;
+}
+
+long long sd_get_option(int option_id) {
+    if (option_id < 0 || option_id >= SD_OPT_COUNT) return -1;
+    return option(option_id);
+}
+
 void sd_launch_info(int* path, int* cluster_size, int* threads, int* smem_bytes, int* blocks, int* kernels) {
     if (path) *path = tl_info[0];
     if (cluster_size) *cluster_size = tl_info[1];
@@ -805,7 +845,7 @@ void sd_release_cached_buffers(void) {
         if (cudaGetDevice(&prev) != cudaSuccess) continue;
         if (cudaSetDevice(i) != cudaSuccess) continue;
         cudaDeviceSynchronize();
-        if (d.ws) { cudaFree(d.ws); d.ws = nullptr; d.ws_bytes = 0; d.ws_clean = false; d.ws_zero_bytes = 0; }
+        if (d.ws) { cudaFree(d.ws); d.ws = nullptr; d.ws_bytes = 0; d.ws_zero_bytes = 0; }
         for (StageSet& st : d.stage)
             if (st.base) { cudaFree(st.base); st.base = nullptr; st.bytes = 0; }
         cudaSetDevice(prev);

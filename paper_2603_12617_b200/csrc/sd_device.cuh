@@ -28,6 +28,8 @@ namespace cg = cooperative_groups;
 constexpr int kMaxCluster = 16;
 constexpr int kMaxLearners = 8;                  // draft models of an online ensemble
 constexpr int kGenericRegionElems = 512;         // sampling region of the generic path
+constexpr int kRegionRows = 2;                   // fast path: 16-byte vectors per lane and row in a sampling region
+constexpr int kRegionVecs = 32 * kRegionRows;    // ... so a region is 64 vectors (1 KiB) of a row
 constexpr uint32_t kStatusTimeout = 0x80000000u; // a bounded wait gave up
 constexpr uint32_t kWaitLimit = 1u << 21;        // polls of an mbarrier before giving up
 constexpr long long kWaitCycles = 2000000000ll;  // ... or about a second of waiting
@@ -74,6 +76,7 @@ struct Params {
     RowConst* rowc;          // [B*(k+1)]
     float* region_sums;      // [B*(k+1)*NR] mass of each sampling region of each row
     int blocks_per_unit;     // blocks that take a ticket per (sequence, row)
+    uint32_t wait_polls;     // polls after which a bounded wait gives up (kWaitLimit unless a caller asks otherwise)
     // online ensemble: feedback of `learners` draft models against one target (0: the plain step).
     // Then loss is [learners,B,k], D and grad above are unused, and nothing is verified or drawn.
     int learners;
@@ -659,7 +662,7 @@ __device__ void resolve_sequence(const Params& P, int b) {
         P.accept_len[b] = n;
         uint32_t st = __ldcg(P.wstatus + b) | flags;
         if (__ldcg(P.sticky) != 0) st |= kStatusTimeout;
-        if (P.status) P.status[b] = st;
+        if (P.status && st) atomicOr(P.status + b, st);   // zero on entry; a block that gave up may have set its bit already
         // leave the workspace ready for the next call
         P.wstatus[b] = 0;
         P.ticket[b] = 0;

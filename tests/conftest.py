@@ -24,3 +24,19 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture
+def options():
+    """Sets tuning options of the library for one test (``options(option_id, value)``) and puts the
+    previous values back afterwards."""
+    from paper_2603_12617_b200 import binding
+    saved = {}
+
+    def set_option(option_id, value):
+        saved.setdefault(option_id, binding.sd_get_option(option_id))
+        binding.sd_set_option(option_id, value)
+
+    yield set_option
+    for option_id, value in saved.items():
+        binding.sd_set_option(option_id, value)

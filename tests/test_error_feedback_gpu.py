@@ -44,7 +44,7 @@ def pmax_of(z, tau):
     return 1.0 / e.sum(axis=-1)
 
 
-def run(binding, cfg, seqs=None, seed=synth.BASE_SEED):
+def run(binding, cfg, seqs=None, seed=synth.BASE_SEED, loss_floor=LOSS_FLOOR, grad_floor=GRAD_FLOOR):
     inp = synth.make_inputs(cfg, seed, sequences=seqs)
     T, D = dev(inp.target_logits), dev(inp.draft_logits)
     x, u = torch.from_numpy(inp.draft_tokens).cuda(), torch.from_numpy(inp.uniforms).cuda()
@@ -66,7 +66,7 @@ def run(binding, cfg, seqs=None, seed=synth.BASE_SEED):
     assert (n_gpu[~band] == ref.full.accept_len[~band]).all()
     assert (out.tokens.cpu().numpy()[~band] == ref.full.tokens[~band]).all()
     loss = out.loss.cpu().numpy().astype(np.float64)
-    assert (np.abs(loss - ref.full.loss) <= tol * np.abs(ref.full.loss) + LOSS_FLOOR).all()
+    assert (np.abs(loss - ref.full.loss) <= tol * np.maximum(np.abs(ref.full.loss), 1e-6) + loss_floor).all()
     g = out.error_grad.cpu().float().numpy().astype(np.float64)
     Tf, Df = f64(inp.target_logits), f64(inp.draft_logits)
     for b in range(B):
@@ -75,7 +75,7 @@ def run(binding, cfg, seqs=None, seed=synth.BASE_SEED):
             assert (g[b] == 0).all()
             continue
         want = ref.full.grad[b, n]
-        bound = tol * np.abs(want).max() + GRAD_FLOOR * max(pmax_of(Tf[b, n], inp.tau), pmax_of(Df[b, n], inp.tau)) / inp.tau
+        bound = tol * np.abs(want).max() + grad_floor * max(pmax_of(Tf[b, n], inp.tau), pmax_of(Df[b, n], inp.tau)) / inp.tau
         assert np.abs(g[b] - want).max() <= bound, (b, n, np.abs(g[b] - want).max() / bound)
         # and the row is the full step's row of that position, bit for bit
         assert torch.equal(out.error_grad[b].view(torch.int16), full.grad_draft[b, n].view(torch.int16))
@@ -85,7 +85,8 @@ def run(binding, cfg, seqs=None, seed=synth.BASE_SEED):
 @pytest.mark.parametrize("name,seqs", [("cfg1", None), ("cfg2", None), ("cfg3", range(0, 32, 5)),
                                        ("cfg4", range(1, 64, 9)), ("cfg5", range(0, 256, 41))])
 def test_workloads(binding, name, seqs):
-    run(binding, synth.CONFIGS[name], seqs=seqs)
+    # the workloads at the contract's tolerance: no absolute term on the loss, no floor on the gradient
+    run(binding, synth.CONFIGS[name], seqs=seqs, loss_floor=0.0, grad_floor=0.0)
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
@@ -126,8 +127,8 @@ def test_every_accept_length_occurs_and_fully_accepted_rows_are_zero(binding):
 
 
 @pytest.mark.parametrize("cluster", [1, 2, 3, 5, 16])
-def test_every_cluster_size(binding, cluster, monkeypatch):
-    monkeypatch.setenv("SD_VERIFY_CLUSTER", str(cluster))
+def test_every_cluster_size(binding, cluster, options):
+    options(binding.SD_OPT_CLUSTER, cluster)
     run(binding, synth.custom_config(9, 3, 50000, dtype="bf16", tau=0.9))
 
 
@@ -180,11 +181,11 @@ def test_full_size_bench_shape_equals_the_full_step(binding):
 
 
 @pytest.mark.parametrize("lag,cluster", [(0, 2), (2, 1), (100, 3), (1, 4)])
-def test_orders_of_the_walk_and_cluster_sizes_with_many_units_per_cluster(binding, lag, cluster, monkeypatch):
+def test_orders_of_the_walk_and_cluster_sizes_with_many_units_per_cluster(binding, lag, cluster, options):
     """Many units per cluster (about 60 here) in every order of the walk: bit-equal to the full step
     run with the same settings."""
-    monkeypatch.setenv("SD_VERIFY_LAG", str(lag))
-    monkeypatch.setenv("SD_VERIFY_CLUSTER", str(cluster))
+    options(binding.SD_OPT_LAG, lag)
+    options(binding.SD_OPT_CLUSTER, cluster)
     cfg = synth.custom_config(600, 5, 8192, dtype="bf16", tau=0.9, recipe="peaks")
     inp = synth.make_inputs(cfg)
     T, D = dev(inp.target_logits), dev(inp.draft_logits)

@@ -6,14 +6,20 @@ Bars (stated here, derived in the design notes):
     sitting on a decision threshold: a reached accept test with |u - p/q| < 1e-6, or an
     inverse-CDF draw whose target lies within 1e-6 (relative to the total mass) of an interval
     edge.  Those sequences are counted, must be rare, and must still produce a valid answer.
-  * loss: |gpu - ref| <= tol * |ref| + 4e-7, tol = 1e-5 (fp32 logits) / 2e-2 (bf16 logits).  The
-    absolute term is the rounding floor of the method in fp32: KL is log S_D - log S_T plus a mean,
-    and each softmax denominator S carries a relative error of a few 2^-24 (2^-22 per term from the
-    hardware exp2, averaged over the row), whatever the size of KL.
+  * loss: on the five workloads |gpu - ref| <= tol * max(|ref|, 1e-6), tol = 1e-5 (fp32 logits) /
+    2e-2 (bf16 logits), nothing added.  The edge-case tests (rows with KL near zero: identical or
+    nearly identical models, tiny vocabularies) add an absolute 4e-7, the rounding floor of the
+    method in fp32: KL is log S_D - log S_T plus a mean, and each softmax denominator S carries a
+    relative error of a few 2^-24 (2^-22 per term from the hardware exp2, averaged over the row),
+    whatever the size of KL.
   * gradient, per row: max|gpu - ref| <= tol * max|ref| + floor and the same in the L2 norm, the
     reference being the fp64 value before any rounding to bf16.  floor = 8 * 2^-24 * max(p,q)/tau
     is the rounding of p and q themselves: it only matters when q - p is a difference of two
-    nearly equal large probabilities (near one-hot rows), never on the five workloads.
+    nearly equal large probabilities (near one-hot rows); the five workloads are checked without it.
+  * inside the band a sequence may differ from the oracle's answer only in the way the band
+    allows: the accept lengths part at a flagged test, and the extra token is one whose interval
+    of the oracle's inverse CDF (for the accept length the device took) lies within 1e-6 of the
+    total mass from u_k times the total mass.
 """
 import os
 
@@ -69,20 +75,44 @@ def oracle_of(inp, seqs=None, want_grad=True):
                                      nthreads=min(8, sd_oracle.max_threads()))
 
 
-def check(inp, out, ref, seqs=None, max_band_frac=0.02, check_grad=True, check_loss=True):
+BAND = 1e-6
+COUNTS = {}     # per workload: what the five-workload tests print at the end
+
+
+def check_band_answer(inp, b_global, n_gpu, tok_gpu, ref, j):
+    """A sequence whose answer differs from the oracle's: it must be one the threshold band allows."""
+    k = inp.cfg.k
+    n_ref = int(ref.accept_len[j])
+    if n_gpu != n_ref:
+        first = min(n_gpu, n_ref)
+        assert first < k and ref.accept_band[j, first], \
+            f"sequence {b_global}: accept length {n_gpu} vs {n_ref} without a flagged test at position {first}"
+    y = int(tok_gpu[n_gpu])
+    lo, hi, R = sd_oracle.draw_interval(inp.target_logits[b_global], inp.draft_logits[b_global], inp.tau, n_gpu, y)
+    t = float(inp.uniforms[b_global, k]) * R
+    assert hi > lo, f"sequence {b_global}: token {y} has no mass in the distribution it was drawn from"
+    assert lo - BAND * R <= t <= hi + BAND * R, \
+        f"sequence {b_global}: token {y} owns [{lo / R:.9f}, {hi / R:.9f}) of the CDF, u_k = {t / R:.9f}"
+
+
+def check(inp, out, ref, seqs=None, max_band_frac=0.02, check_grad=True, check_loss=True,
+          loss_floor=LOSS_FLOOR, grad_floor=GRAD_FLOOR):
     """Compare device outputs (for sequences `seqs`, default all) with the oracle's."""
     dtype = inp.cfg.dtype
     tol = TOL[dtype]
-    sl = slice(None) if seqs is None else torch.as_tensor(np.asarray(seqs))
+    idx = np.arange(ref.tokens.shape[0]) if seqs is None else np.asarray(seqs)
+    sl = torch.as_tensor(idx)
     n_gpu = out.accept_len.cpu()[sl].numpy()
     tok_gpu = out.tokens.cpu()[sl].numpy()
     B, k, V = ref.tokens.shape[0], inp.cfg.k, inp.cfg.V
-    x = inp.draft_tokens if seqs is None else inp.draft_tokens[np.asarray(seqs)]
+    x = inp.draft_tokens[idx]
 
     # A draw that lands in a token of mass < 2e-6 is inside the sample band by construction, so with
     # V > 10^5 the band itself is not rare; what must be rare is a disagreement, and every
-    # disagreement must sit inside the band.
-    band = (ref.accept_band.sum(1) > 0) | (ref.cdf_margin <= 1e-6)
+    # disagreement must sit inside the band and be an answer the band allows.
+    accept_band = ref.accept_band.sum(1) > 0
+    sample_band = ref.cdf_margin <= BAND
+    band = accept_band | sample_band
     safe = ~band
     assert (n_gpu[safe] == ref.accept_len[safe]).all(), "accept lengths differ off the threshold band"
     assert (tok_gpu[safe] == ref.tokens[safe]).all(), "emitted tokens differ off the threshold band"
@@ -92,37 +122,54 @@ def check(inp, out, ref, seqs=None, max_band_frac=0.02, check_grad=True, check_l
     assert ref.accept_band.sum() <= max(1, int(max_band_frac * B * k)), "accept band is not rare"
     # every sequence, band or not, has a well-formed answer
     assert ((n_gpu >= 0) & (n_gpu <= k)).all()
-    for b in range(B):
-        n = int(n_gpu[b])
-        assert (tok_gpu[b, :n] == x[b, :n]).all()
-        assert 0 <= tok_gpu[b, n] < V
-        assert (tok_gpu[b, n + 1:] == -1).all()
+    for j in range(B):
+        n = int(n_gpu[j])
+        assert (tok_gpu[j, :n] == x[j, :n]).all()
+        assert 0 <= tok_gpu[j, n] < V
+        assert (tok_gpu[j, n + 1:] == -1).all()
+    for j in np.nonzero(mismatch)[0]:
+        check_band_answer(inp, int(idx[j]), int(n_gpu[j]), tok_gpu[j], ref, int(j))
 
     if check_loss and out.loss is not None:
         loss = out.loss.cpu()[sl].numpy().astype(np.float64)
         err = np.abs(loss - ref.loss)
-        bound = tol * np.abs(ref.loss) + LOSS_FLOOR
+        bound = tol * np.maximum(np.abs(ref.loss), 1e-6) + loss_floor
         ok = (err <= bound) | (loss == ref.loss)          # the second term covers +inf == +inf
         assert ok.all(), f"loss: worst ratio {np.nanmax(err / bound):.3g}"
     if check_grad and out.grad_draft is not None and ref.grad is not None:
         g = out.grad_draft.cpu()[sl].float().numpy().astype(np.float64)
         d = g - ref.grad
-        T64, D64 = logits_f64(inp, seqs)
+        T64, D64 = logits_f64(inp, idx)
         pmax, p2 = prob_max_and_l2(T64[:, :k], inp.tau)
         qmax, q2 = prob_max_and_l2(D64, inp.tau)
         gmax = np.abs(ref.grad).max(axis=2)
-        bound = tol * gmax + GRAD_FLOOR * np.maximum(pmax, qmax) / inp.tau
+        bound = tol * gmax + grad_floor * np.maximum(pmax, qmax) / inp.tau
         worst = np.abs(d).max(axis=2)
         assert (worst <= bound).all(), f"grad max-norm: worst ratio {np.max(worst / bound):.3g}"
         l2 = np.sqrt((d * d).sum(axis=2))
         ref_l2 = np.sqrt((ref.grad * ref.grad).sum(axis=2))
-        assert (l2 <= tol * ref_l2 + GRAD_FLOOR * (p2 + q2) / inp.tau).all(), "grad L2 norm"
+        assert (l2 <= tol * ref_l2 + grad_floor * (p2 + q2) / inp.tau).all(), "grad L2 norm"
     if out.acc_prob is not None:
         acc = out.acc_prob.cpu()[sl].numpy().astype(np.float64)
         assert np.abs(acc - ref.acc_prob).max() < 2e-5
     if out.status is not None:
         assert (out.status.cpu()[sl].numpy() == ref.status.astype(np.int32)).all()
-    return int(band.sum()), int(mismatch.sum())
+    return {"sequences": int(B), "accept_band_rows": int(ref.accept_band.sum()),
+            "sample_band_rows": int(sample_band.sum()), "mismatches": int(mismatch.sum()),
+            "mean_accept_len": float(n_gpu.mean()), "mean_acc_prob": float(ref.acc_prob.mean())}
+
+
+def add_counts(name, c):
+    t = COUNTS.setdefault(name, {"sequences": 0, "accept_band_rows": 0, "sample_band_rows": 0, "mismatches": 0,
+                                 "accept_len_sum": 0.0, "acc_prob_sum": 0.0})
+    for key in ("sequences", "accept_band_rows", "sample_band_rows", "mismatches"):
+        t[key] += c[key]
+    t["accept_len_sum"] += c["mean_accept_len"] * c["sequences"]
+    t["acc_prob_sum"] += c["mean_acc_prob"] * c["sequences"]
+    print(f"[parity] {name}: {t['sequences']} sequences compared, accept-band rows {t['accept_band_rows']}, "
+          f"sample-band rows {t['sample_band_rows']}, mismatches (all inside the band, all valid) {t['mismatches']}, "
+          f"mean accept length {t['accept_len_sum'] / t['sequences']:.3f}, "
+          f"mean sum min(p,q) {t['acc_prob_sum'] / t['sequences']:.4f}")
 
 
 def run_and_check(binding, cfg, seed=synth.BASE_SEED, ex=False, **kw):
@@ -131,48 +178,48 @@ def run_and_check(binding, cfg, seed=synth.BASE_SEED, ex=False, **kw):
     out = (binding.sd_verify_feedback_ex if ex else binding.sd_verify_feedback)(T, D, x, u, inp.tau)
     torch.cuda.synchronize()
     ref = oracle_of(inp)
-    check(inp, out, ref, **kw)
-    return inp, out, ref
+    counts = check(inp, out, ref, **kw)
+    return inp, out, ref, counts
 
 
 # ------------------------------------------------------------------ the five workloads
 @pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg3", "cfg4"])
 @pytest.mark.parametrize("seed_off", [0, 1])
 def test_config_full_parity(binding, name, seed_off):
+    """Every sequence of the workload, both seeds, at the tolerance the contract states: no
+    absolute term on the loss, no floor on the gradient."""
     cfg = synth.CONFIGS[name]
-    if seed_off and name in ("cfg3", "cfg4"):
-        cfg = cfg.with_batch(8)   # second seed on a slice of the batch keeps the CPU time down
-    inp, out, ref = run_and_check(binding, cfg, synth.BASE_SEED + seed_off, ex=True)
+    inp, out, ref, counts = run_and_check(binding, cfg, synth.BASE_SEED + seed_off, ex=True,
+                                          loss_floor=0.0, grad_floor=0.0)
+    add_counts(f"{name} seed+{seed_off}", counts)
     info = binding.sd_launch_info()
     assert info["path"] == 1, "the five workloads must take the cluster fast path"
 
 
-def test_config5_full_size_sampled_parity(binding):
-    """B=256, k=6, V=128256 fp32 in the launch configuration the benchmark times; the oracle
-    checks a sample of sequences element by element, properties cover the rest."""
+def test_config5_full_size_every_sequence(binding):
+    """B=256, k=6, V=128256 fp32 in the launch configuration the benchmark times, every sequence
+    against the oracle element by element (in slices of 32 sequences: the fp64 gradient of a slice
+    is 0.2 GB), at the contract's tolerance without floors."""
     cfg = synth.CONFIGS["cfg5"]
     inp = synth.make_inputs(cfg)
     T, D, x, u = to_device(inp)
     out = binding.sd_verify_feedback(T, D, x, u, inp.tau)
     torch.cuda.synchronize()
     assert binding.sd_launch_info()["path"] == 1
-    seqs = [0, 1, 17, 63, 64, 100, 128, 191, 200, 254, 255]
-    ref = oracle_of(inp, seqs)
-    check(inp, out, ref, seqs=seqs, max_band_frac=0.1)
-    # properties that hold for every sequence at any size
+    acc_sum = 0.0
+    for b0 in range(0, cfg.B, 32):
+        seqs = list(range(b0, min(cfg.B, b0 + 32)))
+        ref = oracle_of(inp, seqs)
+        counts = check(inp, out, ref, seqs=seqs, max_band_frac=0.1, loss_floor=0.0, grad_floor=0.0)
+        add_counts("cfg5", counts)
+        acc_sum += ref.acc_prob.sum()
+        del ref
     n = out.accept_len.cpu().numpy()
-    tok = out.tokens.cpu().numpy()
-    assert ((n >= 0) & (n <= cfg.k)).all()
-    for b in range(cfg.B):
-        assert (tok[b, :n[b]] == inp.draft_tokens[b, :n[b]]).all()
-        assert 0 <= tok[b, n[b]] < cfg.V and (tok[b, n[b] + 1:] == -1).all()
-    loss = out.loss.cpu().numpy()
-    assert np.isfinite(loss).all() and (loss > 0).all()
     gsum = out.grad_draft.sum(dim=2).abs().max().item()
     assert gsum < 1e-4                     # rows of (q-p)/tau sum to zero
     # expected mean accepted length from the closed form of the proof of Lemma 1, with the
-    # per-position acceptance probabilities of the sampled sequences
-    acc = ref.acc_prob.mean()
+    # per-position acceptance probabilities of the workload
+    acc = acc_sum / (cfg.B * cfg.k)
     expect = (1 - acc ** (cfg.k + 1)) / (1 - acc)
     assert abs((n + 1).mean() - expect) < 0.35
 
@@ -193,22 +240,22 @@ def test_largest_k(binding):
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("cluster", [1, 2, 3, 4, 5, 8, 9, 16])
-def test_every_cluster_size_gives_the_same_answer(binding, dtype, cluster, monkeypatch):
+def test_every_cluster_size_gives_the_same_answer(binding, dtype, cluster, options):
     cfg = synth.custom_config(B=3, k=3, V=24000 if dtype == "f32" else 48000, dtype=dtype, tau=1.2, index=52)
-    monkeypatch.setenv("SD_VERIFY_CLUSTER", str(cluster))
-    inp, out, ref = run_and_check(binding, cfg, ex=True, max_band_frac=1.0)
+    options(binding.SD_OPT_CLUSTER, cluster)
+    inp, out, ref, _ = run_and_check(binding, cfg, ex=True, max_band_frac=1.0)
     info = binding.sd_launch_info()
     assert info["path"] == 1 and info["cluster_size"] == cluster
 
 
 @pytest.mark.parametrize("lag", [0, 1, 2, 100])
 @pytest.mark.parametrize("cluster", [1, 3])
-def test_every_order_of_the_two_passes_gives_the_same_answer(binding, lag, cluster, monkeypatch):
+def test_every_order_of_the_two_passes_gives_the_same_answer(binding, lag, cluster, options):
     """Pass 2 of a unit may come 0, 1, 2 ... stages (per warp) into pass 1 of the next unit, or after
     all of it; several units per cluster, rows long enough for several stages per warp."""
     cfg = synth.custom_config(B=40, k=3, V=100000, dtype="bf16", tau=1.1, index=65)
-    monkeypatch.setenv("SD_VERIFY_CLUSTER", str(cluster))
-    monkeypatch.setenv("SD_VERIFY_LAG", str(lag))
+    options(binding.SD_OPT_CLUSTER, cluster)
+    options(binding.SD_OPT_LAG, lag)
     inp = synth.make_inputs(cfg)
     T, D, x, u = to_device(inp)
     out = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
@@ -231,14 +278,14 @@ def test_every_order_of_the_two_passes_gives_the_same_answer(binding, lag, clust
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_generic_path_matches_fast_path(binding, dtype, monkeypatch):
+def test_generic_path_matches_fast_path(binding, dtype, options):
     cfg = synth.custom_config(B=3, k=3, V=20000, dtype=dtype, tau=0.9, index=53)
     inp = synth.make_inputs(cfg)
     T, D, x, u = to_device(inp)
     fast = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
     torch.cuda.synchronize()
     assert binding.sd_launch_info()["path"] == 1
-    monkeypatch.setenv("SD_VERIFY_FORCE_GENERIC", "1")
+    options(binding.SD_OPT_FORCE_GENERIC, 1)
     slow = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
     torch.cuda.synchronize()
     assert binding.sd_launch_info()["path"] == 0
@@ -303,10 +350,10 @@ def test_shifted_and_huge_logits(binding):
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_late_spike_far_above_everything_seen(binding, dtype, monkeypatch):
+def test_late_spike_far_above_everything_seen(binding, dtype, options):
     """A logit that towers over all earlier ones late in a row: the fast path works with the
     references it has and must notice that this stage needs new ones."""
-    monkeypatch.setenv("SD_VERIFY_CLUSTER", "1")          # one block per row: many stages per warp
+    options(binding.SD_OPT_CLUSTER, 1)          # one block per row: many stages per warp
     cfg = synth.custom_config(B=3, k=2, V=131072, dtype=dtype, t_sigma=1.0, d_sigma=0.5, index=64)
     inp = synth.make_inputs(cfg)
     big = np.float32(300.0) if dtype == "f32" else synth.f32_to_bf16_bits(np.array([300.0], np.float32))[0]
@@ -383,7 +430,107 @@ def test_bad_token_sets_status(binding):
     check(inp, out, ref, max_band_frac=1.0)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("V", [4096, 777])
+def test_zero_residual_at_a_forced_rejection(binding, dtype, V):
+    """q = p exactly and a draft token outside the vocabulary: the rejection leaves a residual
+    without mass, and the extra token is drawn from p_n instead (status BAD_TOKEN | ZERO_RESIDUAL).
+    With all logits zero every product in the gradient is exact, so the device sees a residual of
+    exactly zero as well and takes its own fallback (a draw over the whole row by one warp);
+    V = 4096 goes through the cluster path, V = 777 through the element-wise one."""
+    cfg = synth.custom_config(B=6, k=3, V=V, dtype=dtype, tau=0.9, index=66)
+    inp = synth.make_inputs(cfg)
+    inp.target_logits[:] = 0
+    inp.draft_logits[:] = 0
+    inp.draft_tokens[1, 1] = V            # rejected at position 1
+    inp.draft_tokens[2, 0] = -1           # rejected at position 0
+    inp.draft_tokens[4, 2] = V + 5        # rejected at the last position
+    T, D, x, u = to_device(inp)
+    out = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
+    torch.cuda.synchronize()
+    ref = oracle_of(inp)
+    assert ref.status.tolist() == [0, 5, 5, 0, 5, 0]
+    assert ref.accept_len.tolist() == [3, 1, 0, 3, 2, 3]
+    check(inp, out, ref, max_band_frac=1.0)
+    st = out.status.cpu().numpy()
+    assert st.tolist() == [0, 5, 5, 0, 5, 0]
+    # uniform p_n: the token is floor(u_k * V) wherever u_k * V is not within rounding of an integer
+    tok = out.tokens.cpu().numpy()
+    for b, n in [(1, 1), (2, 0), (4, 2)]:
+        t = float(inp.uniforms[b, cfg.k]) * V
+        if abs(t - round(t)) > 1e-3:
+            assert tok[b, n] == int(t)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_row_without_finite_entries_sets_bad_row(binding, dtype):
+    """A target or draft row of -inf only: the sequence carries SD_STATUS_BAD_ROW, its other outputs
+    are unspecified but well-formed, and its neighbours are exact."""
+    cfg = synth.custom_config(B=4, k=2, V=2048, dtype=dtype, index=67)
+    inp = synth.make_inputs(cfg)
+    ninf = np.float32(-np.inf) if dtype == "f32" else np.uint16(0xFF80)
+    inp.target_logits[1, 0, :] = ninf
+    inp.draft_logits[2, 1, :] = ninf
+    T, D, x, u = to_device(inp)
+    out = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
+    torch.cuda.synchronize()
+    ref = oracle_of(inp)
+    assert ref.status.tolist() == [0, 2, 2, 0]
+    st = out.status.cpu().numpy()
+    assert st[0] == 0 and st[3] == 0 and (st[1] & binding.SD_STATUS_BAD_ROW) and (st[2] & binding.SD_STATUS_BAD_ROW)
+    n = out.accept_len.cpu().numpy()
+    tok = out.tokens.cpu().numpy()
+    assert ((n >= 0) & (n <= cfg.k)).all()
+    for b in range(cfg.B):
+        assert 0 <= tok[b, n[b]] < cfg.V and (tok[b, n[b] + 1:] == -1).all()
+    good = [0, 3]
+    check(inp, out, oracle_of(inp, good), seqs=good, max_band_frac=1.0)
+
+
 # ------------------------------------------------------------------ modes and plumbing
+def test_library_scratch_survives_changing_batch_sizes_and_other_entry_points(binding):
+    """The 13-argument entry point keeps one scratch buffer per device, and where the words that must
+    start at zero end depends on the batch size: a small batch, then a larger one in the same
+    buffer, then a smaller one, then after each of the other entry points that borrow the buffer.
+    Every call must equal the call with a fresh caller workspace, bit for bit."""
+    binding.sd_release_cached_buffers()
+    k, V = 3, 8192
+
+    def one(B, index):
+        cfg = synth.custom_config(B=B, k=k, V=V, dtype="f32", index=index)
+        inp = synth.make_inputs(cfg)
+        T, D, x, u = to_device(inp)
+        ref = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau, want_acc_prob=False, want_status=False)
+        out = binding.sd_verify_feedback(T, D, x, u, inp.tau,
+                                         out=binding.StepOutputs(accept_len=torch.full_like(ref.accept_len, -9),
+                                                                 tokens=torch.full_like(ref.tokens, -9),
+                                                                 loss=torch.full_like(ref.loss, -9.0),
+                                                                 grad_draft=torch.full_like(ref.grad_draft, -9.0)))
+        torch.cuda.synchronize()
+        assert torch.equal(out.accept_len, ref.accept_len), f"B={B}: accept lengths"
+        assert torch.equal(out.tokens, ref.tokens), f"B={B}: tokens"
+        assert torch.equal(out.loss, ref.loss), f"B={B}: loss"
+        assert torch.equal(out.grad_draft, ref.grad_draft), f"B={B}: gradient"
+        return T, D, x, u, inp
+
+    one(4, 80)
+    one(200, 81)          # same buffer (under 1 MiB): the head of the layout is longer now
+    one(70, 82)
+    T, D, x, u, inp = one(130, 83)
+    binding.sd_verify_error_feedback(T, D, x, u, inp.tau)          # borrows the library's buffer
+    one(200, 84)
+    one(5, 85)
+    binding.sd_verify_greedy(T, x)
+    one(190, 86)
+    binding.sd_ensemble_feedback(T, [D, D], inp.tau, 10.0)
+    one(66, 87)
+    one(3, 88)
+    binding.sd_verify_greedy(T, x)
+    binding.sd_verify_greedy(T, x)
+    torch.cuda.synchronize()
+
+
+
 def test_verify_only_mode(binding):
     cfg = synth.custom_config(B=4, k=3, V=16000, dtype="bf16", index=61)
     inp = synth.make_inputs(cfg)

@@ -83,3 +83,34 @@ def test_static_scratch_matches_caller_scratch_twice_in_a_row(binding, dtype, B,
         bound = tol * np.abs(rg).max(axis=2, keepdims=True) + 1e-12
         assert (np.abs(g - rg) <= bound).all(), f"call {call}: gradient differs"
         assert torch.allclose(out.acc_prob, ref.acc_prob, rtol=0, atol=2e-5), f"call {call}: acc_prob differs"
+
+
+@pytest.mark.gpu
+def test_static_entry_point_allocates_nothing_and_survives_a_change_of_shape(binding):
+    """What the entry point is for: once it has been called on a device, further calls leave the
+    device's free memory exactly where it was -- also when the shape changes so that the words at
+    the head of the built-in scratch move (batch sizes either side of 64) -- and still give the
+    answers of sd_verify_feedback_ex."""
+    dev = torch.device("cuda", 0)
+    cases = []
+    for i, (B, k, V) in enumerate([(5, 2, 4096), (130, 2, 4096), (5, 2, 4096), (64, 3, 2048), (65, 3, 2048)]):
+        cfg = synth.custom_config(B=B, k=k, V=V, dtype="f32", tau=0.8, index=95 + i)
+        inp = synth.make_inputs(cfg)
+        T = torch.from_numpy(inp.target_logits).to(dev)
+        D = torch.from_numpy(inp.draft_logits).to(dev)
+        x = torch.from_numpy(inp.draft_tokens).to(dev)
+        u = torch.from_numpy(inp.uniforms).to(dev)
+        ref = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
+        cases.append((cfg, inp, T, D, x, u, ref, _outputs(binding, cfg, dev)))
+    cfg, inp, T, D, x, u, ref, out = cases[0]
+    binding.sd_verify_feedback_static(T, D, x, u, inp.tau, out=out)      # the set-up call of this device
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info(dev)[0]
+    for cfg, inp, T, D, x, u, ref, out in cases:
+        binding.sd_verify_feedback_static(T, D, x, u, inp.tau, out=out)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info(dev)[0] == free_before, "a call of the static entry point changed the free device memory"
+    for cfg, inp, T, D, x, u, ref, out in cases:
+        assert torch.equal(out.accept_len, ref.accept_len) and torch.equal(out.tokens, ref.tokens)
+        assert torch.equal(out.status, ref.status)
+        assert torch.equal(out.loss, ref.loss) and torch.equal(out.grad_draft, ref.grad_draft)
