@@ -17,7 +17,7 @@ using namespace sdv;
 
 constexpr int kMaxDevices = 64;
 constexpr size_t kAlign = 256;
-constexpr int kStreamSmem = kRingSlots * kStageBytes + (int)sizeof(StreamShared);
+constexpr int kStreamSmem = kRingStages * kStageBytes + (int)sizeof(StreamShared);
 static_assert(kStreamSmem <= 227 * 1024, "ring does not fit the shared memory of a block");
 constexpr int kL2PersistMiB = 52;
 constexpr long long kL2BudgetMiB = 80;             // row pairs in flight between their two passes should fit this
@@ -83,9 +83,11 @@ bool shape_ok(int B, int k, int V) {
 
 WorkspaceLayout workspace_layout(int B, int k, int V, int dtype) {
     WorkspaceLayout L;
-    (void)dtype;
-    const int generic_regions = (V + kGenericRegionElems - 1) / kGenericRegionElems;
-    L.NRmax = generic_regions > kMaxCluster * kConsumerWarps ? generic_regions : kMaxCluster * kConsumerWarps;
+    // room for region sums per row: enough for either path (the fast path's regions are 64 vectors,
+    // 256 fp32 or 512 bf16 entries; the generic path's 512 entries)
+    const int fast_elems = kRegionVecs * vec_elems(dtype);
+    const int per = fast_elems < kGenericRegionElems ? fast_elems : kGenericRegionElems;
+    L.NRmax = (V + per - 1) / per;
     size_t off = 0;
     L.ticket = off;      off = align_up(off + (size_t)B * 4, kAlign);
     L.wstatus = off;     off = align_up(off + (size_t)B * 4, kAlign);
@@ -254,8 +256,8 @@ int choose_stream(DeviceState& d, int V, long long units, int dtype, int* G_out,
     for (int C = 1; C <= kMaxCluster; ++C) {
         const int ci = C;
         if (forced > 0 && C != forced) continue;
-        const int stages_row = (NV + kStageVecs - 1) / kStageVecs;
-        const int stages_blk = (stages_row + C - 1) / C;
+        const int regions_row = (NV + kRegionVecs - 1) / kRegionVecs;
+        const int regions_blk = (regions_row + C - 1) / C;
         if (d.max_clusters[dtype][ci] < 0) {
             int n = 0;
             int rc = dtype == SD_DTYPE_F32 ? launch_stream<SD_DTYPE_F32>(d, dummy, C, 1, 0, nullptr, true, &n)
@@ -265,7 +267,7 @@ int choose_stream(DeviceState& d, int V, long long units, int dtype, int* G_out,
         const int resident = d.max_clusters[dtype][ci];
         if (resident < 1) continue;
         const int G = (int)(units < resident ? units : resident);
-        const int used = (stages_row + stages_blk - 1) / stages_blk;   // blocks with work
+        const int used = (regions_row + regions_blk - 1) / regions_blk;   // blocks with work
         long long busy = (long long)G * (used < C ? used : C);
         if (busy > 128) busy = 128;
         const double in_flight = (double)G * (double)NV * 16.0 * 2.0;
@@ -273,7 +275,7 @@ int choose_stream(DeviceState& d, int V, long long units, int dtype, int* G_out,
         // a shape that fits L2 beats one that does not; then more busy blocks; then the smaller cluster
         const bool better = best_C == 0 || (fits && !best_fits) || (fits == best_fits && busy > best_busy) ||
                             (!fits && !best_fits);
-        if (better) { best_C = C; best_G = G; best_per = kStageVecs; best_busy = busy; best_fits = fits; }
+        if (better) { best_C = C; best_G = G; best_per = kRegionVecs; best_busy = busy; best_fits = fits; }
     }
     d.dec_dtype = dtype; d.dec_V = V; d.dec_units = units; d.dec_forced = forced; d.dec_l2 = l2_budget;
     d.dec_C = best_C; d.dec_G = best_G; d.dec_lag = lag; d.dec_per = best_per;
@@ -281,6 +283,11 @@ int choose_stream(DeviceState& d, int V, long long units, int dtype, int* G_out,
     *per_out = best_per;
     *lag_out = lag;
     return best_C;
+}
+
+uint32_t wait_polls() {
+    const long long v = option(SD_OPT_WAIT_POLLS);
+    return (uint32_t)(v < 1 ? 1 : v > (long long)kWaitLimit ? (long long)kWaitLimit : v);
 }
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
@@ -320,6 +327,7 @@ int run_device(DeviceState& d, const void* T, const void* D, const int32_t* x, c
     P.accept = ws + L.accept;
     P.rowc = reinterpret_cast<RowConst*>(ws + L.rowc);
     P.region_sums = reinterpret_cast<float*>(ws + L.region_sums);
+    P.wait_polls = wait_polls();
 
     if (!clean) SD_CUDA(cudaMemsetAsync(ws, 0, L.accept, stream));   // tickets, status words, sticky flag
     if (status) SD_CUDA(cudaMemsetAsync(status, 0, (size_t)B * 4, stream));   // bits are ORed in on the device
@@ -533,6 +541,7 @@ int sd_ensemble_feedback(const void* target_logits, const void* const* draft_log
     P.status = out_status;
     P.sticky = reinterpret_cast<uint32_t*>(ws);
     P.learners = n_learners;
+    P.wait_polls = wait_polls();
     for (int n = 0; n < n_learners; ++n) {
         P.Dn[n] = draft_logits[n];
         P.Gn[n] = out_grad ? out_grad[n] : nullptr;
@@ -605,6 +614,7 @@ int sd_verify_error_feedback(const void* target_logits, const void* draft_logits
     P.accept = ws + L.accept;
     P.rowc = reinterpret_cast<RowConst*>(ws + L.rowc);
     P.region_sums = reinterpret_cast<float*>(ws + L.region_sums);
+    P.wait_polls = wait_polls();
     SD_CUDA(cudaMemsetAsync(ws, 0, L.accept, st));   // tickets, status words, sticky flag
     if (out_status) SD_CUDA(cudaMemsetAsync(out_status, 0, (size_t)B * 4, st));   // bits are ORed in on the device
     int G = 0, lag = 0, per = 0;

@@ -492,50 +492,92 @@ __device__ inline void finish_row_ensemble(const Params& P, const UnitRef& ur, c
 // processed: accept length, emitted tokens, the residual / bonus draw.  It reads what other
 // blocks wrote (after their fence + ticket), so those loads bypass L1.
 
-// Unnormalised mass of vocabulary entry v in the distribution the extra token is drawn from.
+// Unnormalised mass of a vocabulary entry with target logit t and draft logit d in the distribution
+// the extra token is drawn from.
 //   mode 0: pair row, max(0,p-q)/tau     mode 1: bonus row, p     mode 2: pair row, p/tau
-template <int DT>
-__device__ __forceinline__ float mass_elem(const Params& P, const RowConst& rc, int mode,
-                                           size_t offT, size_t offD, int v) {
-    if (v >= P.V) return 0.f;
-    const float t = Elem<DT>::load(P.T, offT + v);
-    if (mode != 0) return prob_elem(t, P.c, rc);
-    const float d = Elem<DT>::load(P.D, offD + v);
-    return fmaxf(-grad_elem(t, d, P.c, rc), 0.f);
+__device__ __forceinline__ float mass_of(float t, float d, float c, const RowConst& rc, int mode) {
+    if (mode != 0) return prob_elem(t, c, rc);
+    return fmaxf(-grad_elem(t, d, c, rc), 0.f);
+}
+
+// Masses of the PER consecutive entries from v0 on (this lane's share of a sampling region), with
+// every load in flight before the first is used: the warp that draws is on the critical path of
+// its sequence, and one round trip to L2 is all it should pay per region.  VECTOR: rows are whole
+// 16-byte vectors and PER is a multiple of the entries of a vector (fast path); otherwise element
+// loads.  Entries past the end of the row have mass 0.
+template <int DT, int PER, bool VECTOR>
+__device__ __forceinline__ void lane_masses(const Params& P, const RowConst& rc, int mode, size_t offT, size_t offD,
+                                            int v0, float (&m)[PER]) {
+    using E = Elem<DT>;
+    using ET = typename E::type;
+    float t[PER], d[PER];
+    if constexpr (VECTOR) {
+        constexpr int VEC = E::VEC;
+        static_assert(PER % VEC == 0, "a lane's share is whole vectors");
+        const uint4* pT = reinterpret_cast<const uint4*>(reinterpret_cast<const ET*>(P.T) + offT + v0);
+        const uint4* pD = reinterpret_cast<const uint4*>(reinterpret_cast<const ET*>(P.D) + offD + v0);
+        uint4 qt[PER / VEC], qd[PER / VEC];
+#pragma unroll
+        for (int g = 0; g < PER / VEC; ++g) {
+            const bool in = v0 + g * VEC < P.V;
+            qt[g] = in ? __ldg(pT + g) : E::masked();
+            qd[g] = (in && mode == 0) ? __ldg(pD + g) : E::masked();
+        }
+#pragma unroll
+        for (int g = 0; g < PER / VEC; ++g) {
+            float a[VEC], b[VEC];
+            E::unpack(qt[g], a);
+            E::unpack(qd[g], b);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) { t[g * VEC + e] = a[e]; d[g * VEC + e] = b[e]; }
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < PER; ++e) {
+            const bool in = v0 + e < P.V;
+            t[e] = in ? E::load(P.T, offT + v0 + e) : -INFINITY;
+            d[e] = (in && mode == 0) ? E::load(P.D, offD + v0 + e) : -INFINITY;
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < PER; ++e) m[e] = (v0 + e < P.V) ? mass_of(t[e], d[e], P.c, rc, mode) : 0.f;
 }
 
 // Inverse-CDF search inside one sampling region.  prefix = mass before the region, t = target.
 // last_with_mass: ignore t and return the last entry of the region that has mass.
-// Every lane takes a contiguous run of RE/32 entries and visits it twice (sum, then search), so
-// nothing is kept per entry.  Returns (in every lane) the vocabulary index, or -1 if the region
-// has no qualifying entry.
-template <int DT>
+// Every lane takes a contiguous run of PER = RE/32 entries.  Returns (in every lane) the
+// vocabulary index, or -1 if the region has no qualifying entry.
+template <int DT, int PER, bool VECTOR>
 __device__ int search_region(const Params& P, const RowConst& rc, int mode, size_t offT, size_t offD,
                              int region, double prefix, double t, bool last_with_mass, double* region_total) {
     const int lane = threadIdx.x & 31;
-    const int per = P.RE / 32;                    // contiguous entries per lane
-    const int v0 = region * P.RE + lane * per;
+    const int v0 = region * (32 * PER) + lane * PER;
+    float m[PER];
+    lane_masses<DT, PER, VECTOR>(P, rc, mode, offT, offD, v0, m);
     double loc = 0.0;
-    for (int e = 0; e < per; ++e) loc += (double)mass_elem<DT>(P, rc, mode, offT, offD, v0 + e);
+#pragma unroll
+    for (int e = 0; e < PER; ++e) loc += (double)m[e];
     const double incl = warp_inclusive_scan(loc);
     *region_total = __shfl_sync(0xffffffffu, incl, 31);
     int cand = last_with_mass ? -1 : 0x7fffffff;
     if (!last_with_mass) {
         double run = prefix + (incl - loc);
         if (run + loc > t) {                      // the crossing can only be in a lane whose run reaches t
-            for (int e = 0; e < per; ++e) {
-                const float r = mass_elem<DT>(P, rc, mode, offT, offD, v0 + e);
-                run += (double)r;
-                if (run > t && r > 0.f) { cand = v0 + e; break; }
+#pragma unroll
+            for (int e = 0; e < PER; ++e) {
+                run += (double)m[e];
+                if (cand == 0x7fffffff && run > t && m[e] > 0.f) cand = v0 + e;
             }
         }
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) cand = min(cand, __shfl_xor_sync(0xffffffffu, cand, off));
         return cand == 0x7fffffff ? -1 : cand;
     }
-    if (loc > 0.0)
-        for (int e = 0; e < per; ++e)
-            if (mass_elem<DT>(P, rc, mode, offT, offD, v0 + e) > 0.f) cand = v0 + e;
+    if (loc > 0.0) {
+#pragma unroll
+        for (int e = 0; e < PER; ++e)
+            if (m[e] > 0.f) cand = v0 + e;
+    }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) cand = max(cand, __shfl_xor_sync(0xffffffffu, cand, off));
     return cand;
@@ -543,12 +585,12 @@ __device__ int search_region(const Params& P, const RowConst& rc, int mode, size
 
 // Draw from a row without region sums (two sweeps over the row by one warp).  Only used when a
 // rejection leaves no residual mass in fp32, which exact arithmetic rules out.
-template <int DT>
+template <int DT, int PER, bool VECTOR>
 __device__ int draw_row_slow(const Params& P, const RowConst& rc, int mode, size_t offT,
                              size_t offD, double u) {
     double total = 0.0, rtot;
     for (int j = 0; j < P.NR; ++j) {
-        search_region<DT>(P, rc, mode, offT, offD, j, 0.0, 0.0, true, &rtot);
+        search_region<DT, PER, VECTOR>(P, rc, mode, offT, offD, j, 0.0, 0.0, true, &rtot);
         total += rtot;
     }
     if (!(total > 0.0) || !isfinite(total)) return 0;
@@ -556,18 +598,21 @@ __device__ int draw_row_slow(const Params& P, const RowConst& rc, int mode, size
     double prefix = 0.0;
     int last_mass = -1;
     for (int j = 0; j < P.NR; ++j) {
-        const int y = search_region<DT>(P, rc, mode, offT, offD, j, prefix, t, false, &rtot);
+        const int y = search_region<DT, PER, VECTOR>(P, rc, mode, offT, offD, j, prefix, t, false, &rtot);
         if (y >= 0) return y;
         if (rtot > 0.0) last_mass = j;
         prefix += rtot;
     }
     if (last_mass < 0) return 0;
-    const int y = search_region<DT>(P, rc, mode, offT, offD, last_mass, 0.0, 0.0, true, &rtot);
+    const int y = search_region<DT, PER, VECTOR>(P, rc, mode, offT, offD, last_mass, 0.0, 0.0, true, &rtot);
     return y < 0 ? 0 : y;
 }
 
-template <int DT>
-__device__ void resolve_sequence(const Params& P, int b) {
+// FAST: the regions are those of the fast path (kRegionVecs vectors, rows of whole vectors);
+// otherwise those of the generic path (kGenericRegionElems entries, any alignment).
+template <int DT, bool FAST>
+__device__ __noinline__ void resolve_sequence(const Params& P, int b) {
+    constexpr int PER = FAST ? kRegionVecs * Elem<DT>::VEC / 32 : kGenericRegionElems / 32;
     const int lane = threadIdx.x & 31;
     const int k = P.k, NR = P.NR;
 
@@ -586,7 +631,13 @@ __device__ void resolve_sequence(const Params& P, int b) {
         for (int i = 0; i < k; ++i) {
             const float* rsi = P.region_sums + (size_t)(b * (k + 1) + i) * NR;
             double part = 0.0;
-            for (int j = lane; j < NR; j += 32) part += (double)__ldcg(rsi + j);
+            for (int j = lane; j < NR; j += 32 * 4) {
+                float v[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) v[q] = (j + 32 * q < NR) ? __ldcg(rsi + j + 32 * q) : 0.f;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) part += (double)v[q];
+            }
             const double R = warp_sum(part) * (double)P.tau;
             if (lane == 0) P.acc_prob[b * k + i] = (float)(1.0 - R);
         }
@@ -601,11 +652,18 @@ __device__ void resolve_sequence(const Params& P, int b) {
     const size_t offD = (size_t)(b * k + (bonus ? 0 : n)) * P.V;
     const double uk = (double)P.u[b * (k + 1) + k];
 
-    // prefix over the region sums: each lane owns a contiguous run of regions
+    // prefix over the region sums: each lane owns a contiguous run of regions, which it reads eight
+    // at a time (all eight loads in flight together) and adds up in index order
     const int per = (NR + 31) / 32;
     const int j0 = min(NR, lane * per), j1 = min(NR, j0 + per);
     double mine = 0.0;
-    for (int j = j0; j < j1; ++j) mine += (double)__ldcg(rs + j);
+    for (int c = j0; c < j1; c += 8) {
+        float v[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) v[q] = (c + q < j1) ? __ldcg(rs + c + q) : 0.f;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) mine += (double)v[q];
+    }
     const double incl = warp_inclusive_scan(mine);
     const double before = incl - mine;
     const double total = __shfl_sync(0xffffffffu, incl, 31);
@@ -617,18 +675,26 @@ __device__ void resolve_sequence(const Params& P, int b) {
             flags |= SD_STATUS_BAD_ROW;
         } else {
             flags |= SD_STATUS_ZERO_RESIDUAL;   // draw from p_n instead
-            y = draw_row_slow<DT>(P, rc, 2, offT, offD, uk);
+            y = draw_row_slow<DT, PER, FAST>(P, rc, 2, offT, offD, uk);
         }
     } else {
         // first region whose running sum exceeds t, and the mass before it
         int cand = 0x7fffffff;
         double cand_prefix = 0.0;
-        {
+        if (before + mine > t) {                  // the crossing can only be in a lane whose run reaches t
             double run = before;
-            for (int j = j0; j < j1; ++j) {
-                const double next = run + (double)__ldcg(rs + j);
-                if (next > t) { cand = j; cand_prefix = run; break; }
-                run = next;
+            for (int c = j0; c < j1 && cand == 0x7fffffff; c += 8) {
+                float v[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) v[q] = (c + q < j1) ? __ldcg(rs + c + q) : 0.f;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    if (cand == 0x7fffffff && c + q < j1) {
+                        const double next = run + (double)v[q];
+                        if (next > t) { cand = c + q; cand_prefix = run; }
+                        else run = next;
+                    }
+                }
             }
         }
         const unsigned has = __ballot_sync(0xffffffffu, cand != 0x7fffffff);
@@ -651,9 +717,9 @@ __device__ void resolve_sequence(const Params& P, int b) {
         }
         if (region >= 0) {
             double rtot;
-            y = search_region<DT>(P, rc, bonus ? 1 : 0, offT, offD, region, prefix, t, past_end, &rtot);
+            y = search_region<DT, PER, FAST>(P, rc, bonus ? 1 : 0, offT, offD, region, prefix, t, past_end, &rtot);
             // region sum and re-summed entries may disagree in the last bits: last entry with mass
-            if (y < 0) y = search_region<DT>(P, rc, bonus ? 1 : 0, offT, offD, region, 0.0, 0.0, true, &rtot);
+            if (y < 0) y = search_region<DT, PER, FAST>(P, rc, bonus ? 1 : 0, offT, offD, region, 0.0, 0.0, true, &rtot);
             if (y < 0) y = 0;
         }
     }

@@ -10,7 +10,7 @@
 //                                        full step), the masses of its sampling regions, and the
 //                                        draw by the block that takes the sequence's last ticket.
 //
-// The row is read straight from global memory (eight 16-byte loads in flight per lane); a block
+// The row is read straight from global memory (2 x kRegionRows 16-byte loads in flight per lane); a block
 // takes a slice of kErrSliceRegions sampling regions, a warp one region at a time.
 #pragma once
 
@@ -26,7 +26,7 @@ __global__ void __launch_bounds__(kErrThreads, 4) sd_errpos_kernel(const __grid_
     using E = Elem<DT>;
     using ET = typename E::type;
     constexpr int VEC = E::VEC;
-    constexpr int kGroups = 4;                      // a region is 4 x 32 vectors, as in the streaming kernel
+    constexpr int kGroups = kRegionRows;            // a region is kRegionRows x 32 vectors, as in the streaming kernel
     __shared__ int is_last;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = (int)blockIdx.x / slices, sl = (int)blockIdx.x - b * slices;
@@ -97,7 +97,7 @@ __global__ void __launch_bounds__(kErrThreads, 4) sd_errpos_kernel(const __grid_
         if (is_last) __threadfence();
     }
     __syncthreads();
-    if (is_last && warp == 0) resolve_sequence<DT>(P, b);   // also sets ticket and status words back to zero
+    if (is_last && warp == 0) resolve_sequence<DT, true>(P, b);   // also sets ticket and status words back to zero
 }
 
 }  // namespace sdv

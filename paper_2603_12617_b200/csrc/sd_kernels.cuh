@@ -2,17 +2,23 @@
 //
 //   sd_stream_kernel   fast path.  A persistent kernel of thread-block clusters.  A cluster takes a
 //                      contiguous range of (sequence, row) units, one after the other; each block
-//                      of the cluster owns a contiguous slice of the vocabulary, cut into stages
-//                      of 2 KiB per row that its 16 consumer warps take in turn.
-//                      A slice is streamed through a ring of small shared-memory stages twice:
-//                      pass 1 (maxima, then softmax sums relative to integer references) reads it
-//                      from HBM, pass 2 (gradient out, residual mass) reads it again a few
-//                      microseconds later, when it is still in L2, so HBM sees each logit once.
+//                      of the cluster owns a contiguous slice of the vocabulary, cut into sampling
+//                      regions of 64 16-byte vectors (1 KiB of a row) and into stages of 28 regions.
+//                      A slice is read twice: pass 1 (softmax sums relative to integer references)
+//                      streams it from HBM through a ring of three shared-memory stages, pass 2
+//                      (gradient out, residual mass) reads it again a few microseconds later with
+//                      plain 16-byte loads, last stage first, when it is still in L2, so HBM sees
+//                      each logit once.  (One SM takes in about 48 bytes per clock through bulk
+//                      copies of this size and about as much again through plain loads; the two
+//                      passes together need 30 at the HBM roofline, so they use one path each.)
 //                      Inside a block the warps are specialised:
-//                        consumers  each works through its own stages, which it fetches itself into
-//                                   a private ring of three slots with bulk asynchronous copies
-//                                   (cp.async.bulk + mbarrier), always three stages ahead, across
-//                                   passes and units; warps meet only once per unit and pass;
+//                        producer   one thread fetches the pass-1 stages of unit after unit, each
+//                                   with two bulk asynchronous copies (cp.async.bulk + mbarrier),
+//                                   as soon as the consumers have handed the slot back;
+//                        consumers  28 warps; warp w takes region w of every stage into registers
+//                                   (pass 1: from the ring, handing the slot back at once; pass 2:
+//                                   from global memory, one region ahead) and works from registers;
+//                                   warps meet only through the ring's barriers and once per unit and pass;
 //                        statistics adds up the consumers' sums, exchanges the block's partial
 //                                   with the other blocks of the cluster through distributed
 //                                   shared memory (remote stores + remote mbarrier arrivals, no
@@ -20,8 +26,8 @@
 //                        resolver   reports rows (loss, rejection test), takes the sequence's tickets when
 //                                   the block leaves a sequence and, if they were the last ones,
 //                                   draws the extra token.
-//                      Pass 2 of a unit is scheduled after pass 1 of the next unit (lag 1), which
-//                      hides the exchange.
+//                      Pass 2 of a unit is scheduled after the first stages of pass 1 of the next
+//                      unit (the lag), which hides the exchange.
 //   sd_generic_kernel  any V and any alignment.  One block per unit, sweeps over global memory
 //                      with element loads.  Same arithmetic, same workspace, same resolver.
 //
@@ -35,20 +41,19 @@
 namespace sdv {
 
 // ---- geometry of the fast path -------------------------------------------------------------
-// A row is cut into stages of 128 16-byte vectors (2 KiB); a stage is also a sampling region.
-// Block r of a cluster of C owns the stages [r*S, (r+1)*S) of every row it works on, S =
-// ceil(stages per row / C); stage s of the slice belongs to consumer warp s % 14, so fourteen
-// consecutive stages are worked on at the same time.  Every consumer warp has a ring of its own.
-constexpr int kConsumerWarps = 14;
-constexpr int kStageGroups = 4;                               // groups of 32 vectors in a stage
-constexpr int kStageVecs = 32 * kStageGroups;                 // vectors of one row in a stage
-constexpr int kStageRowBytes = kStageVecs * 16;               // 2 KiB of one row
+// A row is cut into sampling regions of kRegionVecs 16-byte vectors; block r of a cluster of C owns
+// the regions [r*S, (r+1)*S) of every row it works on, S = ceil(regions per row / C).  A stage is
+// kConsumerWarps consecutive regions of the slice, one per consumer warp: 28 KiB of the target row
+// and 28 KiB of the draft row, fetched by one bulk copy each.
+constexpr int kHelperWarps = 4;                               // statistics, resolver, producer, one idle
+constexpr int kConsumerWarps = 28;
+constexpr int kStageVecs = kConsumerWarps * kRegionVecs;      // vectors of one row in a stage
+constexpr int kStageRowBytes = kStageVecs * 16;               // 28 KiB of one row
 constexpr int kStageBytes = 2 * kStageRowBytes;               // target part + draft part
-constexpr int kWarpSlots = 3;                                 // stages a consumer warp has in flight or in use
-constexpr int kRingSlots = kConsumerWarps * kWarpSlots;       // 42 slots, 168 KiB
+constexpr int kRingStages = 3;                                // 168 KiB
 constexpr int kDoneDepth = 4;                                 // units the resolver may lag behind
-constexpr int kStatsWarp = 0, kResolverWarp = 1, kFirstConsumerWarp = 2;
-constexpr int kStreamThreads = (kFirstConsumerWarp + kConsumerWarps) * 32;
+constexpr int kStatsWarp = 0, kResolverWarp = 1, kProducerWarp = 2, kFirstConsumerWarp = kHelperWarps;
+constexpr int kStreamThreads = (kHelperWarps + kConsumerWarps) * 32;
 constexpr int kGenericWarps = 8;
 constexpr int kGenericThreads = kGenericWarps * 32;
 
@@ -110,14 +115,19 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t pa
         : "memory");
     return ok != 0;
 }
-// Bounded wait of one thread.  It gives up after kWaitLimit polls or kWaitCycles clock cycles,
+// Bounded wait of one thread.  It gives up after `limit` polls or kWaitCycles clock cycles,
 // whichever comes first, or as soon as another thread of the block has given up (*abort != 0);
 // the caller then leaves its loop and the kernel returns.  A failed poll is followed by a short
 // sleep (longer for the warps whose waits are long by design).
+struct WaitCtx {
+    volatile int* abort;
+    uint32_t limit;
+};
 template <bool CLUSTER, int SLEEP_NS = 20>
-__device__ __forceinline__ bool mbar_wait_thread(uint64_t* bar, uint32_t parity, volatile int* abort) {
+__device__ __forceinline__ bool mbar_wait_thread(uint64_t* bar, uint32_t parity, const WaitCtx& wc) {
+    volatile int* abort = wc.abort;
     long long t0 = 0;
-    for (uint32_t it = 0; it < kWaitLimit; ++it) {
+    for (uint32_t it = 0; it < wc.limit; ++it) {
         if (CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
         __nanosleep(SLEEP_NS);   // waiting warps leave the issue slots to the working ones
         if ((it & 63u) == 63u) {
@@ -133,15 +143,15 @@ __device__ __forceinline__ bool mbar_wait_thread(uint64_t* bar, uint32_t parity,
 // The same for a whole warp (all 32 lanes call it): every lane observes the barrier itself (a
 // warp whose lanes part ways at a wait is slow to get back together), and all lanes get the same
 // answer.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
-    return __all_sync(0xffffffffu, mbar_wait_thread<false>(bar, parity, abort) ? 1 : 0) != 0;
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const WaitCtx& wc) {
+    return __all_sync(0xffffffffu, mbar_wait_thread<false>(bar, parity, wc) ? 1 : 0) != 0;
 }
-__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, volatile int* abort) {
-    return __all_sync(0xffffffffu, mbar_wait_thread<true, 100>(bar, parity, abort) ? 1 : 0) != 0;
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, const WaitCtx& wc) {
+    return __all_sync(0xffffffffu, mbar_wait_thread<true, 100>(bar, parity, wc) ? 1 : 0) != 0;
 }
 template <int SLEEP_NS>
-__device__ __forceinline__ bool mbar_wait_sleepy(uint64_t* bar, uint32_t parity, volatile int* abort) {
-    return __all_sync(0xffffffffu, mbar_wait_thread<false, SLEEP_NS>(bar, parity, abort) ? 1 : 0) != 0;
+__device__ __forceinline__ bool mbar_wait_sleepy(uint64_t* bar, uint32_t parity, const WaitCtx& wc) {
+    return __all_sync(0xffffffffu, mbar_wait_thread<false, SLEEP_NS>(bar, parity, wc) ? 1 : 0) != 0;
 }
 // 1-D bulk copy global -> shared of this block, completion counted on `bar`, with an L2 eviction
 // policy.  Both addresses 16-byte aligned, bytes a multiple of 16.
@@ -175,31 +185,39 @@ __device__ __forceinline__ void store_streaming(void* p, const uint4& v) {
                  : "memory");
 }
 
-// ---- the two passes over one stage held in shared memory ------------------------------------
-// A stage is kStageGroups vectors per lane and row.  All of them are loaded before any arithmetic; vectors
-// past the end of the row read as -inf, which adds nothing to any sum and is never stored.
+// L2 policy for data nobody will read again (the second pass): first in line for eviction.
+__device__ __forceinline__ uint64_t policy_discard() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
 
-// Pass 1: the stage's softmax sums relative to the warp's integer references (RT, RD), added to
+// ---- the two passes over one region held in registers ----------------------------------------
+// A region is kRegionRows vectors per lane and row.  All of them are loaded from the stage before
+// any arithmetic, and the stage's slot goes back to the producer at once; vectors past the end of
+// the row read as -inf, which adds nothing to any sum and is never stored.
+
+// Pass 1: the region's softmax sums relative to the warp's integer references (RT, RD), added to
 // the running sums.  References need not be the exact maxima: any integers work as long as nothing
 // overflows, and sums under different references are merged exactly later.  So only the first
-// stage of a unit looks for its maxima first; later stages reuse the references, and a stage whose
+// region of a unit looks for its maxima first; later ones reuse the references, and a region whose
 // sums come out too large for comfort (an entry far above everything the warp has seen: rare) is
-// done again by pass1_stage_again after its maxima have raised the references and the running
-// sums have moved with them (exact: powers of two).
+// done again after its maxima have raised the references and the running sums have moved with them
+// (exact: powers of two).
 struct Pass1State {
     float RT, RD;
     LaneSums ls;
 };
 
-// The stage's maxima raise the references; the running sums follow.
+// The region's maxima raise the references; the running sums follow.
 template <int DT, bool BONUS>
-__device__ __forceinline__ void raise_references(const uint4 (&rt)[kStageGroups], const uint4 (&rd)[kStageGroups],
+__device__ __forceinline__ void raise_references(const uint4 (&rt)[kRegionRows], const uint4 (&rd)[kRegionRows],
                                                  float c, Pass1State& s) {
     using E = Elem<DT>;
     constexpr int VEC = E::VEC;
-    float mT[kStageGroups], mD[kStageGroups];
+    float mT[kRegionRows], mD[kRegionRows];
 #pragma unroll
-    for (int g = 0; g < kStageGroups; ++g) {
+    for (int g = 0; g < kRegionRows; ++g) {
         float v[VEC];
         E::unpack(rt[g], v);
         mT[g] = tree_max<VEC>(v);
@@ -208,26 +226,28 @@ __device__ __forceinline__ void raise_references(const uint4 (&rt)[kStageGroups]
             mD[g] = tree_max<VEC>(v);
         }
     }
-    const float nT = fmaxf(s.RT, warp_max_ref(ref_of(tree_max<kStageGroups>(mT), c)));
-    const float nD = BONUS ? kEmptyRef : fmaxf(s.RD, warp_max_ref(ref_of(tree_max<kStageGroups>(mD), c)));
+    const float nT = fmaxf(s.RT, warp_max_ref(ref_of(tree_max<kRegionRows>(mT), c)));
+    const float nD = BONUS ? kEmptyRef : fmaxf(s.RD, warp_max_ref(ref_of(tree_max<kRegionRows>(mD), c)));
     s.ls.rescale(nT - s.RT, nD - s.RD);
     s.RT = nT;
     s.RD = nD;
 }
 
+// The warp's region of a stage (st: where the region starts in the stage's target part; the draft
+// part lies kStageVecs vectors further) into registers; nv = vectors of the region that exist.
 template <int DT, bool BONUS>
-__device__ __forceinline__ void load_stage(const uint4* st, int nv, int lane, uint4 (&rt)[kStageGroups],
-                                           uint4 (&rd)[kStageGroups]) {
+__device__ __forceinline__ void load_region(const uint4* st, int nv, int lane, uint4 (&rt)[kRegionRows],
+                                            uint4 (&rd)[kRegionRows]) {
     using E = Elem<DT>;
-    if (nv == kStageVecs) {
+    if (nv == kRegionVecs) {
 #pragma unroll
-        for (int g = 0; g < kStageGroups; ++g) {
+        for (int g = 0; g < kRegionRows; ++g) {
             rt[g] = st[g * 32 + lane];
             if (!BONUS) rd[g] = st[kStageVecs + g * 32 + lane];
         }
     } else {
 #pragma unroll
-        for (int g = 0; g < kStageGroups; ++g) {
+        for (int g = 0; g < kRegionRows; ++g) {
             const int vi = g * 32 + lane;
             rt[g] = vi < nv ? st[vi] : E::masked();
             if (!BONUS) rd[g] = vi < nv ? st[kStageVecs + vi] : E::masked();
@@ -235,13 +255,13 @@ __device__ __forceinline__ void load_stage(const uint4* st, int nv, int lane, ui
     }
 }
 
-// Returns only when every vector of the stage has arrived in this lane's registers (the value
+// Returns only when every vector of the region has arrived in this lane's registers (the value
 // depends on all of them), so that the stage's slot may be overwritten afterwards.
 template <bool BONUS>
-__device__ __forceinline__ void await_stage_registers(const uint4 (&rt)[kStageGroups], const uint4 (&rd)[kStageGroups]) {
+__device__ __forceinline__ void await_region_registers(const uint4 (&rt)[kRegionRows], const uint4 (&rd)[kRegionRows]) {
     uint32_t dep = 0;
 #pragma unroll
-    for (int g = 0; g < kStageGroups; ++g) {
+    for (int g = 0; g < kRegionRows; ++g) {
         dep ^= rt[g].w;
         if (!BONUS) dep ^= rd[g].w;
     }
@@ -249,13 +269,13 @@ __device__ __forceinline__ void await_stage_registers(const uint4 (&rt)[kStageGr
 }
 
 template <int DT, bool BONUS>
-__device__ __forceinline__ void stage_sums(const uint4 (&rt)[kStageGroups], const uint4 (&rd)[kStageGroups], float c,
-                                           float RT, float RD, float& sT, float& sD, float& sW) {
+__device__ __forceinline__ void region_sums_of(const uint4 (&rt)[kRegionRows], const uint4 (&rd)[kRegionRows], float c,
+                                               float RT, float RD, float& sT, float& sD, float& sW) {
     using E = Elem<DT>;
     constexpr int VEC = E::VEC;
     sT = sD = sW = 0.f;
 #pragma unroll
-    for (int g = 0; g < kStageGroups; ++g) {
+    for (int g = 0; g < kRegionRows; ++g) {
         float tv[VEC];
         E::unpack(rt[g], tv);
         if (!BONUS) {
@@ -272,43 +292,44 @@ __device__ __forceinline__ void stage_sums(const uint4 (&rt)[kStageGroups], cons
 }
 
 // The slow way, out of line: maxima first, then the sums.  By now the stage's slot in the ring
-// has been handed back, so the stage is read once more from global memory (gT, gD: where it
+// has been handed back, so the region is read once more from global memory (gT, gD: where it
 // starts in the two rows).
 template <int DT, bool BONUS>
-__device__ __noinline__ Pass1State pass1_stage_again(const uint4* gT, const uint4* gD, int nv, int lane, float c,
-                                                     Pass1State s) {
+__device__ __noinline__ Pass1State pass1_region_again(const uint4* gT, const uint4* gD, int nv, int lane, float c,
+                                                      Pass1State s) {
     using E = Elem<DT>;
-    uint4 rt[kStageGroups], rd[kStageGroups];
+    uint4 rt[kRegionRows], rd[kRegionRows];
 #pragma unroll
-    for (int g = 0; g < kStageGroups; ++g) {
+    for (int g = 0; g < kRegionRows; ++g) {
         const int vi = g * 32 + lane;
         rt[g] = vi < nv ? __ldg(gT + vi) : E::masked();
         if (!BONUS) rd[g] = vi < nv ? __ldg(gD + vi) : E::masked();
     }
     raise_references<DT, BONUS>(rt, rd, c, s);
     float sT, sD, sW;
-    stage_sums<DT, BONUS>(rt, rd, c, s.RT, s.RD, sT, sD, sW);
+    region_sums_of<DT, BONUS>(rt, rd, c, s.RT, s.RD, sT, sD, sW);
     s.ls.sT += sT;
     s.ls.sD += sD;
     s.ls.w += sW;
     return s;
 }
 
-// `handed_back` is called once the stage is in registers: the caller refills the slot then.
-template <int DT, bool BONUS, class F>
-__device__ __forceinline__ void pass1_stage(const uint4* st, const uint4* gT, const uint4* gD, int nv, int lane, float c,
-                                            bool first, Pass1State& s, F&& handed_back) {
+// `handed_back` is called once the region is in registers: the warp gives up its share of the slot
+// then.  `again(state)` does the region the slow way (pass1_region_again) and returns the new state.
+template <int DT, bool BONUS, class F, class A>
+__device__ __forceinline__ void pass1_region(const uint4* st, int nv, int lane, float c, bool first, Pass1State& s,
+                                             F&& handed_back, A&& again) {
     constexpr float kTooLarge = 1.152921504606846976e18f;   // 2^60
-    uint4 rt[kStageGroups], rd[kStageGroups];
-    load_stage<DT, BONUS>(st, nv, lane, rt, rd);
-    await_stage_registers<BONUS>(rt, rd);
+    uint4 rt[kRegionRows], rd[kRegionRows];
+    load_region<DT, BONUS>(st, nv, lane, rt, rd);
+    await_region_registers<BONUS>(rt, rd);
     handed_back();
     if (first) raise_references<DT, BONUS>(rt, rd, c, s);
     float sT, sD, sW;
-    stage_sums<DT, BONUS>(rt, rd, c, s.RT, s.RD, sT, sD, sW);
+    region_sums_of<DT, BONUS>(rt, rd, c, s.RT, s.RD, sT, sD, sW);
     // (written so that a NaN counts as too large)
     if (!first && __any_sync(0xffffffffu, !(sT < kTooLarge) || !(sD < kTooLarge))) {
-        s = pass1_stage_again<DT, BONUS>(gT, gD, nv, lane, c, s);
+        s = again(s);
         return;
     }
     s.ls.sT += sT;
@@ -316,20 +337,17 @@ __device__ __forceinline__ void pass1_stage(const uint4* st, const uint4* gT, co
     s.ls.w += sW;
 }
 
-// Pass 2: gradient out (gdst = where the stage's part of the gradient row starts, or null) and
-// the stage's mass (sum of max(0,p-q)/tau, or of p on the bonus row), in every lane.
-template <int DT, bool BONUS, class F>
-__device__ __forceinline__ float pass2_stage(const uint4* st, int nv, int lane, float c, const RowConst& rc,
-                                             typename Elem<DT>::type* gdst, F&& handed_back) {
+// Pass 2 of a region held in registers: gradient out (gdst = where the region's part of the
+// gradient row starts, or null) and the region's mass (sum of max(0,p-q)/tau, or of p on the
+// bonus row), in every lane.
+template <int DT, bool BONUS>
+__device__ __forceinline__ float pass2_region(const uint4 (&rt)[kRegionRows], const uint4 (&rd)[kRegionRows], int nv,
+                                              int lane, float c, const RowConst& rc, typename Elem<DT>::type* gdst) {
     using E = Elem<DT>;
     constexpr int VEC = E::VEC;
-    uint4 rt[kStageGroups], rd[kStageGroups];
-    load_stage<DT, BONUS>(st, nv, lane, rt, rd);
-    await_stage_registers<BONUS>(rt, rd);
-    handed_back();
-    float ms[kStageGroups];
+    float ms[kRegionRows];
 #pragma unroll
-    for (int g = 0; g < kStageGroups; ++g) {
+    for (int g = 0; g < kRegionRows; ++g) {
         const int vi = g * 32 + lane;
         float tv[VEC], r[VEC];
         E::unpack(rt[g], tv);
@@ -351,7 +369,7 @@ __device__ __forceinline__ float pass2_stage(const uint4* st, int nv, int lane, 
         }
         ms[g] = tree_sum<VEC>(r);
     }
-    float mass = tree_sum<kStageGroups>(ms);
+    float mass = tree_sum<kRegionRows>(ms);
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) mass += __shfl_xor_sync(0xffffffffu, mass, off);
     return mass;
@@ -359,7 +377,8 @@ __device__ __forceinline__ float pass2_stage(const uint4* st, int nv, int lane, 
 
 // Control block of the fast path; lives in dynamic shared memory after the ring.
 struct StreamShared {
-    uint64_t full[kRingSlots];          // stage filled by the bulk copies        (1 arrival + bytes)
+    uint64_t full[kRingStages];         // stage filled by the bulk copies        (1 arrival + bytes)
+    uint64_t empty[kRingStages];        // stage taken into registers by everyone (consumer warps)
     uint64_t s1_done[2];                // consumers' sums of a unit posted       (consumer warps)
     uint64_t xchg_bar[2];               // partials of every block have arrived   (1 arrival + bytes, remote)
     uint64_t rc_ready[2];               // row constants published                (1)
@@ -380,14 +399,29 @@ __device__ __host__ __forceinline__ void cluster_units(int units, int G, int cid
     u0 = cid * base + (cid < rem ? cid : rem);
 }
 
-// The order in which a consumer warp walks its stages.  The warp has nst stages in every pass.
+// The order in which a block walks the stages of its slice.  There are nst stages in every pass.
 // Pass 2 of a unit needs the row constants, which take an exchange between the blocks of the
-// cluster; so it is scheduled after the first L stages of pass 1 of the next unit:
-//   S1(0)[0,nst)  then for j = 1 .. nu-1:  S1(j)[0,L)  S2(j-1)[0,nst)  S1(j)[L,nst)   then  S2(nu-1)[0,nst)
+// cluster; so it is scheduled after the first L stages of pass 1 of the next unit, and it runs
+// from the last stage to the first (what pass 1 fetched last is what L2 is surest to hold still):
+//   S1(0)[0,nst)  then for j = 1 .. nu-1:  S1(j)[0,L)  S2(j-1)(nst,0]  S1(j)[L,nst)   then  S2(nu-1)(nst,0]
 // The smaller L, the less data lies between the two passes (it has to stay in L2 meanwhile).
+// (Letting the two passes alternate stage by stage was measured too: it doubles that data and is
+// slower on every workload.)  The producer and every consumer warp go through the same list;
+// p1(j, t0, t1, last) stands for the stages [t0,t1) of pass 1 of unit j (last: the pass is over
+// afterwards), p2(j) for pass 2.
+template <class P1, class P2>
+__device__ __forceinline__ void walk_stages(int nu, int nst, int L, P1&& p1, P2&& p2) {
+    for (int j = 0; j < nu; ++j) {
+        const int head = (j == 0) ? nst : L;
+        if (!p1(j, 0, head, head == nst)) return;
+        if (j > 0 && !p2(j - 1)) return;
+        if (head < nst && !p1(j, head, nst, true)) return;
+    }
+    if (nu > 0) p2(nu - 1);
+}
 
 // ---- fast path -----------------------------------------------------------------------------
-// lag_stages: stages (per consumer warp) of pass 1 of the next unit that go before pass 2 of a unit.
+// lag_stages: stages of pass 1 of the next unit that go before pass 2 of a unit.
 // ENS: the units are those of the ensemble feedback (see UnitRef); nothing is verified or drawn.
 // STATS: pass 1 only -- row constants, losses and rejection tests of every row; no gradient, no
 // masses, no draw (the error-position feedback finishes the one row it needs in a kernel of its own).
@@ -397,10 +431,9 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
     using E = Elem<DT>;
     using ET = typename E::type;
     constexpr int VEC = E::VEC;
-    constexpr int R = kRingSlots;
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     unsigned char* ring = dyn_smem;
-    StreamShared& sh = *reinterpret_cast<StreamShared*>(dyn_smem + (size_t)R * kStageBytes);
+    StreamShared& sh = *reinterpret_cast<StreamShared*>(dyn_smem + (size_t)kRingStages * kStageBytes);
 
     cg::cluster_group cluster = cg::this_cluster();
     const int C = (int)cluster.num_blocks();
@@ -424,16 +457,21 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
     }
 
     const int NV = P.V / VEC;                     // vectors per row
-    const int stages_row = (NV + kStageVecs - 1) / kStageVecs;   // = sampling regions per row
-    const int stages_blk = (stages_row + C - 1) / C;
-    const int s0 = rank * stages_blk;             // first stage (region) of this block's slice
-    const int ns = max(0, min(stages_row - s0, stages_blk));     // stages of a pass
-    const int vb0 = s0 * kStageVecs;              // first vector of the slice
-    const int nvb = max(0, min(NV - vb0, ns * kStageVecs));
-    volatile int* abort = &sh.abort;
+    const int regions_row = (NV + kRegionVecs - 1) / kRegionVecs;   // = P.NR
+    const int regions_blk = (regions_row + C - 1) / C;
+    const int r0 = rank * regions_blk;            // first region of this block's slice
+    const int nr = max(0, min(regions_row - r0, regions_blk));      // regions of the slice
+    const int vb0 = r0 * kRegionVecs;             // first vector of the slice
+    const int nvb = max(0, min(NV - vb0, nr * kRegionVecs));        // vectors of the slice
+    const int nst = (nr + kConsumerWarps - 1) / kConsumerWarps;     // stages of a pass
+    const int L = min(max(lag_stages, 0), nst);
+    const WaitCtx wc{&sh.abort, P.wait_polls};
 
     if (tid == 0) {
-        for (int s = 0; s < R; ++s) mbar_init(&sh.full[s], 1);
+        for (int s = 0; s < kRingStages; ++s) {
+            mbar_init(&sh.full[s], 1);
+            mbar_init(&sh.empty[s], kConsumerWarps);
+        }
         for (int s = 0; s < 2; ++s) {
             mbar_init(&sh.s1_done[s], kConsumerWarps);
             mbar_init(&sh.xchg_bar[s], 1);
@@ -459,8 +497,8 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
             const uint32_t ph = (uint32_t)(j >> 1) & 1u;
             const int dslot = j % kDoneDepth;
             if (lane == 0) mbar_expect_tx(&sh.xchg_bar[par], (uint32_t)C * (uint32_t)sizeof(PartialStats));
-            if (!mbar_wait_sleepy<100>(&sh.s1_done[par], ph, abort)) break;
-            // the block's partial from its 16 warp partials, then one copy to every block of the cluster
+            if (!mbar_wait_sleepy<100>(&sh.s1_done[par], ph, wc)) break;
+            // the block's partial from its warps' partials, then one copy to every block of the cluster
             const PartialStats mine = warp_merge_lanes(lane < kConsumerWarps ? sh.wpart[par][lane] : empty_partial());
             if (lane < C) {
                 uint64_t refs;
@@ -470,7 +508,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
                 st_async_remote(&dst->sD, (uint64_t)__double_as_longlong(mine.sD), (uint64_t)__double_as_longlong(mine.w),
                                 &sh.xchg_bar[par], (uint32_t)lane);
             }
-            if (!mbar_wait_cluster(&sh.xchg_bar[par], ph, abort)) break;
+            if (!mbar_wait_cluster(&sh.xchg_bar[par], ph, wc)) break;
             const PartialStats row = warp_merge_lanes(lane < C ? sh.xchg[par][lane] : empty_partial());
             const RowConst rcw = row_constants(P, bonus, row);
             if (lane == 0) {
@@ -479,14 +517,14 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
                 // for the row report by the resolver: wait until it is done with the slot's last use
                 bool ok = true;
                 if (j >= kDoneDepth)
-                    ok = mbar_wait_thread<false>(&sh.res_free[dslot], (uint32_t)(j / kDoneDepth - 1) & 1u, abort);
+                    ok = mbar_wait_thread<false>(&sh.res_free[dslot], (uint32_t)(j / kDoneDepth - 1) & 1u, wc);
                 if (ok) {
                     sh.row[dslot] = row;
                     sh.rc_done[dslot] = rcw;
                     mbar_arrive(&sh.s2_done[dslot]);
                 }
             }
-            if (__any_sync(0xffffffffu, *abort)) break;
+            if (__any_sync(0xffffffffu, sh.abort)) break;
         }
     } else if (warp == kResolverWarp) {
         // ---- resolver: row reports, tickets; the sequence's last tickets draw the token
@@ -496,7 +534,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
             const int dslot = j % kDoneDepth;
             const bool reports = (j % C == rank);   // the blocks of the cluster take turns
             if constexpr (ENS) {
-                if (!mbar_wait_sleepy<500>(&sh.s2_done[dslot], (uint32_t)(j / kDoneDepth) & 1u, abort)) break;
+                if (!mbar_wait_sleepy<500>(&sh.s2_done[dslot], (uint32_t)(j / kDoneDepth) & 1u, wc)) break;
                 if (reports && lane == 0) finish_row_ensemble(P, unit_ref<true>(P, unit), sh.row[dslot]);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.res_free[dslot]);
@@ -507,7 +545,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
             AcceptOperands aop;
             aop.valid = false;
             if (reports && lane == 0 && !bonus) aop = load_accept_operands<DT>(P, b, i);
-            if (!mbar_wait_sleepy<500>(&sh.s2_done[dslot], (uint32_t)(j / kDoneDepth) & 1u, abort)) break;
+            if (!mbar_wait_sleepy<500>(&sh.s2_done[dslot], (uint32_t)(j / kDoneDepth) & 1u, wc)) break;
             if (reports && lane == 0) finish_row(P, b, i, sh.row[dslot], sh.rc_done[dslot], aop);
             __syncwarp();
             if constexpr (STATS) {
@@ -520,186 +558,154 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
                 int last = 0;
                 if (lane == 0) last = take_tickets(P, b, (uint32_t)seg) ? 1 : 0;
                 last = __shfl_sync(0xffffffffu, last, 0);
-                if (last) resolve_sequence<DT>(P, b);
+                if (last) resolve_sequence<DT, true>(P, b);
                 seg = 0;
                 __syncwarp();
             }
             if (lane == 0) mbar_arrive(&sh.res_free[dslot]);
         }
-    } else {
-        // ---- consumers: warp cw owns stages cw, cw+16, ... of every pass; a stage is a sampling
-        // region.  The warp walks its stages of all passes in a fixed order (Walk); stage number n
-        // of that walk goes to slot n % 3 of the warp's own ring, and its copies are issued by the
-        // warp's first lane as soon as stage n-3 has been worked on, whatever pass or unit it is of.
-        const int cw = warp - kFirstConsumerWarp;
-        const int nst = cw < ns ? (ns - cw + kConsumerWarps - 1) / kConsumerWarps : 0;   // my stages per pass
-        if (nst == 0) {
-            // no data of its own (short rows): the warp only keeps the per-unit protocol going
-            for (int j = 0; j < nu; ++j) {
-                if (lane == 0) { sh.wpart[j & 1][cw] = empty_partial(); mbar_arrive(&sh.s1_done[j & 1]); }
-                const int dslot = j % kDoneDepth;
-                if (!mbar_wait(&sh.rc_ready[j & 1], (uint32_t)(j >> 1) & 1u, abort)) break;
-                if (j >= kDoneDepth && !mbar_wait(&sh.res_free[dslot], (uint32_t)(j / kDoneDepth - 1) & 1u, abort)) break;
-                if (lane == 0) mbar_arrive(&sh.s2_done[dslot]);
-            }
-        } else {
-            const int L = min(max(lag_stages, 0), nst);
-            const int n_total = (STATS ? 1 : 2) * nu * nst;
-            unsigned char* myring = ring + (size_t)cw * kWarpSlots * kStageBytes;
-            uint64_t* myfull = &sh.full[cw * kWarpSlots];
-            const uint64_t keep = policy_keep(), normal = policy_normal();
-            // issue cursor (lane 0): the walk S1(0) | S1(j)[0,L) S2(j-1) S1(j)[L,nst) ... | S2(nu-1)
-            // runs of the walk: 0 = S1(0), 1 = head of S1(ji), 2 = S2(ji-1), 3 = rest of S1(ji), 4 = S2(nu-1)
-            int ni = 0, run = 0, ji = 0, ti = 0, endi = nst;   // stage number, run, unit of the run's pass 1, stage, end
-            const ET* Tb = nullptr;       // where the next copy of the run reads from; Db null on a bonus row
-            const ET* Db = nullptr;
-            uint64_t pol = keep;
-            int slot_i = 0;               // ring slot of the next copy
-            constexpr size_t kStride = (size_t)kConsumerWarps * kStageVecs * VEC;   // from one of my stages to the next
-            auto begin_run = [&]() {      // lane 0
-                const UnitRef ur = unit_ref<ENS>(P, u0 + (run == 2 ? ji - 1 : run == 4 ? nu - 1 : ji) * ustep);
-                const size_t off = (size_t)(vb0 + cw * kStageVecs) * VEC + (size_t)ti * kStride;
-                Tb = reinterpret_cast<const ET*>(P.T) + ur.t_row * P.V + off;
-                Db = ur.bonus ? nullptr : reinterpret_cast<const ET*>(ENS ? P.Dn[ur.n] : P.D) + ur.d_row * P.V + off;
-                pol = (run == 2 || run == 4) ? normal : keep;
-            };
-            auto issue_next = [&]() {     // lane 0
-                if (ni >= n_total) return;
-                const uint32_t bytes = (uint32_t)min(kStageVecs, nvb - (cw + ti * kConsumerWarps) * kStageVecs) * 16u;
-                unsigned char* dst = myring + (size_t)slot_i * kStageBytes;
-                mbar_expect_tx(&myfull[slot_i], Db ? 2u * bytes : bytes);
-                bulk_load(dst, Tb, bytes, &myfull[slot_i], pol);
-                if (Db) { bulk_load(dst + kStageRowBytes, Db, bytes, &myfull[slot_i], pol); Db += kStride; }
-                Tb += kStride;
-                if (++slot_i == kWarpSlots) slot_i = 0;
-                ++ni;
-                ++ti;
-                if (ti >= endi) {
-                    while (ti >= endi && run != 5) {
-                        // the next run that is not empty
-                        constexpr int kLast = STATS ? 5 : 4;          // no pass 2 to fetch for in a pass-1-only walk
-                        if (run == 0) { if (nu > 1) { run = 1; ji = 1; } else run = kLast; }
-                        else if (run == 1) run = STATS ? 3 : 2;
-                        else if (run == 2) run = 3;
-                        else if (run == 3) { if (ji + 1 < nu) { run = 1; ++ji; } else run = kLast; }
-                        else run = 5;
-                        if (run == 1) { ti = 0; endi = L; }
-                        else if (run == 3) { ti = L; endi = nst; }
-                        else { ti = 0; endi = nst; }
-                    }
-                    if (run != 5) begin_run();
-                }
-            };
-            if (lane == 0) begin_run();
-            if (lane == 0)
-                for (int t = 0; t < kWarpSlots; ++t) issue_next();
-            int n = 0;                    // consume cursor: stages worked on so far, its slot and parity
-            int slot_c = 0;
-            uint32_t par_c = 0;
+    } else if (warp == kProducerWarp) {
+        // ---- producer: two threads fetch the stages of the walk, in order, into the ring -- the first
+        // arms the stage's barrier and copies the target part, the second copies the draft part (one
+        // thread issuing both copies one after the other gets three quarters of the bytes per clock)
+        if (lane < 2 && nst > 0) {
+            const uint64_t keep = policy_keep(), discard = policy_discard();
+            int ni = 0, slot = 0;                  // stages issued so far; slot of the next one
+            uint32_t epar = 1;                     // parity to wait for on empty[slot]: that of its previous use
             bool ok = true;
-            // The stage is in registers: hand its slot back and fetch stage n+3 of the walk into it.
-            // (Every lane's loads from the slot have returned their values before the copy is issued.)
-            auto recycle = [&]() {
-                __syncwarp();
-                if (lane == 0) issue_next();
-                ++n;
-                if (++slot_c == kWarpSlots) { slot_c = 0; par_c ^= 1u; }
-            };
-            Pass1State ps;
-            ps.RT = ps.RD = kEmptyRef;
-            ps.ls.init();
-            auto run_pass1 = [&](int j, int t0, int t1) {
-                const UnitRef ur = unit_ref<ENS>(P, u0 + j * ustep);
-                const bool bonus = ur.bonus;
-                // the block's slice of the two rows in global memory (for the rare second try of a stage)
-                const ET* Trow = reinterpret_cast<const ET*>(P.T) + ur.t_row * P.V + (size_t)vb0 * VEC;
-                const ET* Drow = reinterpret_cast<const ET*>(ENS ? P.Dn[ur.n] : P.D) + ur.d_row * P.V + (size_t)vb0 * VEC;
-                for (int t = t0; t < t1 && ok; ++t) {
-                    const int slot = slot_c;
-                    if (!mbar_wait(&myfull[slot], par_c, abort)) { ok = false; break; }
-                    const uint4* st = reinterpret_cast<const uint4*>(myring + (size_t)slot * kStageBytes);
-                    const int s = cw + t * kConsumerWarps;
-                    const int nv = min(kStageVecs, nvb - s * kStageVecs);     // vectors of this stage
-                    const uint4* gT = reinterpret_cast<const uint4*>(Trow) + (size_t)s * kStageVecs;
-                    const uint4* gD = reinterpret_cast<const uint4*>(Drow) + (size_t)s * kStageVecs;
-                    if (bonus) pass1_stage<DT, true>(st, gT, gD, nv, lane, P.c, t == 0, ps, recycle);
-                    else       pass1_stage<DT, false>(st, gT, gD, nv, lane, P.c, t == 0, ps, recycle);
+            auto issue = [&](const UnitRef& ur, int t, uint64_t pol) {
+                if (ni >= kRingStages && !mbar_wait_thread<false>(&sh.empty[slot], epar, wc)) { ok = false; return; }
+                const int v0 = t * kStageVecs;     // first vector of the stage within the slice
+                const uint32_t bytes = (uint32_t)min(kStageVecs, nvb - v0) * 16u;
+                const size_t off = (size_t)(vb0 + v0) * VEC;
+                unsigned char* dst = ring + (size_t)slot * kStageBytes;
+                if (lane == 0) {
+                    mbar_expect_tx(&sh.full[slot], ur.bonus ? bytes : 2u * bytes);
+                    bulk_load(dst, reinterpret_cast<const ET*>(P.T) + ur.t_row * P.V + off, bytes, &sh.full[slot], pol);
+                } else if (!ur.bonus) {
+                    // (its bytes may land before the barrier is armed: the count then goes below zero
+                    // for a moment, and the phase cannot end before the first thread's arrival)
+                    bulk_load(dst + kStageRowBytes,
+                              reinterpret_cast<const ET*>(ENS ? P.Dn[ur.n] : P.D) + ur.d_row * P.V + off, bytes,
+                              &sh.full[slot], pol);
                 }
+                ++ni;
+                if (++slot == kRingStages) { slot = 0; epar ^= 1u; }
             };
-            auto run_pass2 = [&](int j) {
-                const int unit = u0 + j * ustep;
-                const UnitRef ur = unit_ref<ENS>(P, unit);
-                const bool bonus = ur.bonus;
-                const int dslot = j % kDoneDepth;
-                if (!mbar_wait(&sh.rc_ready[j & 1], (uint32_t)(j >> 1) & 1u, abort)) { ok = false; return; }
-                const RowConst rc = sh.rc[j & 1];
-                void* const gbase = ENS ? P.Gn[ur.n] : P.grad;
-                ET* Grow = (gbase && !bonus) ? reinterpret_cast<ET*>(gbase) + ur.d_row * P.V + (size_t)vb0 * VEC : nullptr;
-                float* rsum = ENS ? nullptr : P.region_sums + (size_t)unit * P.NR + s0;
-                for (int t = 0; t < nst; ++t) {
-                    const int slot = slot_c;
-                    if (!mbar_wait(&myfull[slot], par_c, abort)) { ok = false; return; }
-                    const uint4* st = reinterpret_cast<const uint4*>(myring + (size_t)slot * kStageBytes);
-                    const int s = cw + t * kConsumerWarps;
-                    const int nv = min(kStageVecs, nvb - s * kStageVecs);
-                    const float mass = bonus ? pass2_stage<DT, true>(st, nv, lane, P.c, rc, nullptr, recycle)
-                                             : pass2_stage<DT, false>(st, nv, lane, P.c, rc,
-                                                                      Grow ? Grow + (size_t)s * kStageVecs * VEC : nullptr,
-                                                                      recycle);
-                    if (!ENS && lane == 0) rsum[s] = mass;
-                }
-                // the resolver's slot of unit j-4 must be free again before this unit is reported done
-                if (j >= kDoneDepth &&
-                    !mbar_wait(&sh.res_free[dslot], (uint32_t)(j / kDoneDepth - 1) & 1u, abort)) { ok = false; return; }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sh.s2_done[dslot]);
-            };
-            // The walk, segment by segment (each pass has one call site, which keeps the hot code small):
-            // unit j contributes  [pass 1 head]  [pass 2 of unit j-1]  [pass 1 rest];  then pass 2 of the last unit.
-            for (int seg = 0; seg <= 3 * nu && ok; ++seg) {
-                const int j = seg / 3, kind = seg - 3 * j;
-                int p1 = -1, p2 = -1, t0 = 0, t1 = 0;
-                const int head = (j == 0) ? nst : L;
-                if (j == nu) p2 = nu - 1;
-                else if (kind == 0) { p1 = j; t0 = 0; t1 = head; }
-                else if (kind == 1) { if (j > 0) p2 = j - 1; }
-                else { p1 = j; t0 = head; t1 = nst; }
-                if (p2 >= 0) {
-                    if constexpr (STATS) {
-                        // nothing to do for the unit but to report it finished -- after its row
-                        // constants are out, as in the full walk: the statistics warp is then done
-                        // with the partials of the unit, whose slots the unit after next reuses
-                        const int dslot = p2 % kDoneDepth;
-                        if (!mbar_wait(&sh.rc_ready[p2 & 1], (uint32_t)(p2 >> 1) & 1u, abort)) { ok = false; break; }
-                        if (p2 >= kDoneDepth &&
-                            !mbar_wait(&sh.res_free[dslot], (uint32_t)(p2 / kDoneDepth - 1) & 1u, abort)) { ok = false; break; }
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&sh.s2_done[dslot]);
-                    } else {
-                        run_pass2(p2);
+            walk_stages(nu, nst, L,
+                [&](int j, int t0, int t1, bool) {
+                    const UnitRef ur = unit_ref<ENS>(P, u0 + j * ustep);
+                    for (int t = t0; t < t1 && ok; ++t) issue(ur, t, STATS ? discard : keep);
+                    return ok;
+                },
+                [&](int j) {
+                    if constexpr (!STATS) {
+                        const UnitRef ur = unit_ref<ENS>(P, u0 + j * ustep);
+                        for (int t = nst - 1; t >= 0 && ok; --t) issue(ur, t, discard);
                     }
-                }
-                if (p1 >= 0) {
-                    run_pass1(p1, t0, t1);
-                    if (ok && kind == 2) {
-                        // pass 1 of the unit is over: the warp's partial for the statistics warp
-                        const PartialStats part = warp_sum_lanes(ps.ls, ps.RT, ps.RD);
-                        if (lane == 0) {
-                            sh.wpart[j & 1][cw] = part;
-                            mbar_arrive(&sh.s1_done[j & 1]);
-                        }
-                        ps.RT = ps.RD = kEmptyRef;
-                        ps.ls.init();
-                    }
-                }
-            }
-            // leaving early: no copy of this warp may still be in flight when the block returns
+                    return ok;
+                });
+            // leaving early: no copy may still be in flight when the block returns (a draft-part copy
+            // whose barrier the first thread never armed has the pause before the block's exit to land)
             if (!ok && lane == 0)
-                for (int t = n; t < ni; ++t) {
-                    const uint32_t par = (uint32_t)(t / kWarpSlots) & 1u;
-                    for (uint32_t it = 0; it < kWaitLimit && !mbar_try_wait(&myfull[t % kWarpSlots], par); ++it) {}
+                for (int i = max(0, ni - kRingStages); i < ni; ++i) {
+                    const uint32_t par = (uint32_t)(i / kRingStages) & 1u;
+                    for (uint32_t it = 0; it < kWaitLimit && !mbar_try_wait(&sh.full[i % kRingStages], par); ++it) {}
                 }
         }
+    } else if (warp >= kFirstConsumerWarp) {
+        // ---- consumers: warp cw owns region cw of every stage; a region is a sampling region.
+        const int cw = warp - kFirstConsumerWarp;
+        const int rv0 = cw * kRegionVecs;          // where my region starts within a stage
+        int slot = 0;                              // ring slot of the next stage and the parity of its full barrier
+        uint32_t fpar = 0;
+        bool ok = true;
+        // The region is in registers: hand the warp's share of the slot back.  (Every lane's loads
+        // from the slot have returned their values before the arrival.)
+        auto hand_back = [&]() {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.empty[slot]);
+            if (++slot == kRingStages) { slot = 0; fpar ^= 1u; }
+        };
+        Pass1State ps;
+        ps.RT = ps.RD = kEmptyRef;
+        ps.ls.init();
+        auto vectors_of = [&](int t) { return max(0, min(kRegionVecs, nvb - t * kStageVecs - rv0)); };   // of my region of stage t
+        auto run_pass1 = [&](int j, int t0, int t1, bool last) {
+            const UnitRef ur = unit_ref<ENS>(P, u0 + j * ustep);
+            const bool bonus = ur.bonus;
+            for (int t = t0; t < t1; ++t) {
+                if (!mbar_wait(&sh.full[slot], fpar, wc)) { ok = false; return false; }
+                const uint4* st = reinterpret_cast<const uint4*>(ring + (size_t)slot * kStageBytes) + rv0;
+                const int nv = vectors_of(t);
+                if (nv == 0) { hand_back(); continue; }
+                // where the region lies in global memory: only the rare second try of a region reads it there
+                auto again = [&](Pass1State s0) {
+                    const size_t voff = (size_t)vb0 + rv0 + (size_t)t * kStageVecs;
+                    const uint4* gT = reinterpret_cast<const uint4*>(reinterpret_cast<const ET*>(P.T) + ur.t_row * P.V) + voff;
+                    const uint4* gD = reinterpret_cast<const uint4*>(reinterpret_cast<const ET*>(ENS ? P.Dn[ur.n] : P.D) + ur.d_row * P.V) + voff;
+                    return bonus ? pass1_region_again<DT, true>(gT, gD, nv, lane, P.c, s0)
+                                 : pass1_region_again<DT, false>(gT, gD, nv, lane, P.c, s0);
+                };
+                if (bonus) pass1_region<DT, true>(st, nv, lane, P.c, t == 0, ps, hand_back, again);
+                else       pass1_region<DT, false>(st, nv, lane, P.c, t == 0, ps, hand_back, again);
+            }
+            if (last) {
+                // pass 1 of the unit is over: the warp's partial for the statistics warp
+                const PartialStats part = warp_sum_lanes(ps.ls, ps.RT, ps.RD);
+                if (lane == 0) {
+                    sh.wpart[j & 1][cw] = part;
+                    mbar_arrive(&sh.s1_done[j & 1]);
+                }
+                ps.RT = ps.RD = kEmptyRef;
+                ps.ls.init();
+                if constexpr (STATS) {
+                    // nothing else to do for the unit but to report it finished -- after its row
+                    // constants are out, as in the full walk: the statistics warp is then done with
+                    // the partials of the unit, whose slots the unit after next reuses
+                    const int dslot = j % kDoneDepth;
+                    if (!mbar_wait(&sh.rc_ready[j & 1], (uint32_t)(j >> 1) & 1u, wc)) { ok = false; return false; }
+                    if (j >= kDoneDepth &&
+                        !mbar_wait(&sh.res_free[dslot], (uint32_t)(j / kDoneDepth - 1) & 1u, wc)) { ok = false; return false; }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sh.s2_done[dslot]);
+                }
+            }
+            return true;
+        };
+        auto run_pass2 = [&](int j) {
+            if constexpr (STATS) return true;
+            const int unit = u0 + j * ustep;
+            const UnitRef ur = unit_ref<ENS>(P, unit);
+            const bool bonus = ur.bonus;
+            const int dslot = j % kDoneDepth;
+            if (!mbar_wait(&sh.rc_ready[j & 1], (uint32_t)(j >> 1) & 1u, wc)) { ok = false; return false; }
+            const RowConst rc = sh.rc[j & 1];
+            void* const gbase = ENS ? P.Gn[ur.n] : P.grad;
+            ET* Grow = (gbase && !bonus) ? reinterpret_cast<ET*>(gbase) + ur.d_row * P.V + (size_t)(vb0 + rv0) * VEC : nullptr;
+            float* rsum = ENS ? nullptr : P.region_sums + (size_t)unit * P.NR + r0 + cw;
+            for (int t = nst - 1; t >= 0; --t) {
+                if (!mbar_wait(&sh.full[slot], fpar, wc)) { ok = false; return false; }
+                const uint4* st = reinterpret_cast<const uint4*>(ring + (size_t)slot * kStageBytes) + rv0;
+                const int nv = vectors_of(t);
+                if (nv == 0) { hand_back(); continue; }
+                uint4 rt[kRegionRows], rd[kRegionRows];
+                if (bonus) { load_region<DT, true>(st, nv, lane, rt, rd); await_region_registers<true>(rt, rd); }
+                else       { load_region<DT, false>(st, nv, lane, rt, rd); await_region_registers<false>(rt, rd); }
+                hand_back();
+                const float mass = bonus ? pass2_region<DT, true>(rt, rd, nv, lane, P.c, rc, nullptr)
+                                         : pass2_region<DT, false>(rt, rd, nv, lane, P.c, rc,
+                                                                   Grow ? Grow + (size_t)t * kStageVecs * VEC : nullptr);
+                if (!ENS && lane == 0) rsum[t * kConsumerWarps] = mass;
+            }
+            // the resolver's slot of unit j-4 must be free again before this unit is reported done
+            if (j >= kDoneDepth &&
+                !mbar_wait(&sh.res_free[dslot], (uint32_t)(j / kDoneDepth - 1) & 1u, wc)) { ok = false; return false; }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.s2_done[dslot]);
+            return true;
+        };
+        walk_stages(nu, nst, L, run_pass1, run_pass2);
     }
 
     __syncthreads();
@@ -709,6 +715,9 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
         if (tid == 0) atomicExch(P.sticky, 1u);
         if (P.status)
             for (int j = tid; j < nu; j += kStreamThreads) atomicOr(P.status + unit_ref<ENS>(P, u0 + j * ustep).b, kStatusTimeout);
+        // whatever another block of the cluster has sent to this one's shared memory meanwhile has
+        // had time to land before the block goes away
+        for (int i = 0; i < 20; ++i) __nanosleep(1000);
     }
     // no block leaves while another may still write to its shared memory
     cluster.sync();
@@ -811,7 +820,7 @@ __global__ void __launch_bounds__(kGenericThreads) sd_generic_kernel(const __gri
     __syncthreads();
     if (tid == 0) sh.last = take_tickets(P, b, 1u) ? 1 : 0;
     __syncthreads();
-    if (sh.last && warp == 0) resolve_sequence<DT>(P, b);
+    if (sh.last && warp == 0) resolve_sequence<DT, false>(P, b);
 }
 
 // ---- online ensemble ---------------------------------------------------------------------
