@@ -308,6 +308,8 @@ int sd_verify_feedback_host(const void* target_logits, const void* draft_logits,
  *   SD_OPT_WAIT_POLLS            env SD_VERIFY_WAIT_POLLS       default 2^21 polls after which a wait
  *                                inside the fast path gives up (the sequences concerned then carry
  *                                SD_STATUS_TIMEOUT); the wait also ends after about a second
+ *   SD_OPT_PREFETCH              env SD_VERIFY_PREFETCH         default 0    non-zero: while a block is in
+ *                                its second pass over a row pair it asks L2 to fetch the next row pair
  * sd_set_option returns SD_OK, or SD_ERR_SHAPE for an unknown option; sd_get_option returns the
  * value in force, or -1 for an unknown option.
  */
@@ -318,7 +320,8 @@ int sd_verify_feedback_host(const void* target_logits, const void* draft_logits,
 #define SD_OPT_FORCE_GENERIC 4
 #define SD_OPT_GREEDY_BLOCKS_PER_SM 5
 #define SD_OPT_WAIT_POLLS 6
-#define SD_OPT_COUNT 7
+#define SD_OPT_PREFETCH 7
+#define SD_OPT_COUNT 8
 int sd_set_option(int option_id, long long value);
 long long sd_get_option(int option_id);
 

@@ -40,6 +40,7 @@ void init_options() {
             {SD_OPT_FORCE_GENERIC, "SD_VERIFY_FORCE_GENERIC", 0},
             {SD_OPT_GREEDY_BLOCKS_PER_SM, "SD_GREEDY_BLOCKS_PER_SM", 4},
             {SD_OPT_WAIT_POLLS, "SD_VERIFY_WAIT_POLLS", (long long)kWaitLimit},
+            {SD_OPT_PREFETCH, "SD_VERIFY_PREFETCH", 0},
         };
         for (const auto& t : table) {
             const char* e = getenv(t.env);
@@ -207,7 +208,8 @@ int launch_stream(DeviceState& d, const Params& P, int C, int G, int lag, cudaSt
         *max_clusters = n;
         return SD_OK;
     }
-    SD_CUDA(cudaLaunchKernelEx(&cfg, kern, P, lag));
+    const int prefetch = option(SD_OPT_PREFETCH) != 0 ? 1 : 0;
+    SD_CUDA(cudaLaunchKernelEx(&cfg, kern, P, lag, prefetch));
     tl_info[0] = 1; tl_info[1] = C; tl_info[2] = kStreamThreads; tl_info[3] = kStreamSmem;
     tl_info[4] = G * C; tl_info[5] = 1;
     return SD_OK;

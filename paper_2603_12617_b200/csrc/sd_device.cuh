@@ -274,14 +274,17 @@ struct LaneSums {
     // The same for one vector, into partial sums of its own (short dependency chains).  Entries are
     // taken two at a time with the packed fp32 instructions of sm_100 (same rounding as the scalar
     // ones); even and odd entries are summed separately and meet at the end.
-    template <int VEC>
+    // MASKED = false leaves out the test for masked target entries (p = 0 exactly, logit -inf):
+    // there eT = 0 meets aT - aD = -inf or NaN and the product is NaN instead of 0, so the caller
+    // must look at pW and do the vector again with MASKED = true when it is NaN.  It saves three
+    // of thirteen instructions per two entries on rows without masked entries, which is most rows.
+    template <int VEC, bool MASKED = true>
     static __device__ __forceinline__ void vector_pair(const float (&t)[VEC], const float (&d)[VEC], float c,
                                                        float negRT, float negRD, float& pT, float& pD, float& pW) {
         static_assert(VEC % 2 == 0, "packed arithmetic takes entries in pairs");
         const float2 c2 = make_float2(c, c), nT2 = make_float2(negRT, negRT), nD2 = make_float2(negRD, negRD);
         const float2 m1 = make_float2(-1.f, -1.f);
-        float2 accT = make_float2(0.f, 0.f), accD = make_float2(0.f, 0.f);
-        float w0 = 0.f, w1 = 0.f;
+        float2 accT = make_float2(0.f, 0.f), accD = make_float2(0.f, 0.f), accW = make_float2(0.f, 0.f);
 #pragma unroll
         for (int e = 0; e < VEC; e += 2) {
             const float2 aT = __ffma2_rn(make_float2(t[e], t[e + 1]), c2, nT2);
@@ -289,14 +292,18 @@ struct LaneSums {
             const float2 eT = make_float2(ex2f(aT.x), ex2f(aT.y));
             const float2 eD = make_float2(ex2f(aD.x), ex2f(aD.y));
             const float2 diff = __ffma2_rn(aD, m1, aT);          // aT - aD
-            if (eT.x > 0.f) w0 = __fmaf_rn(eT.x, diff.x, w0);    // masked target entries (p = 0) add nothing
-            if (eT.y > 0.f) w1 = __fmaf_rn(eT.y, diff.y, w1);
+            if constexpr (MASKED) {
+                if (eT.x > 0.f) accW.x = __fmaf_rn(eT.x, diff.x, accW.x);    // masked target entries (p = 0) add nothing
+                if (eT.y > 0.f) accW.y = __fmaf_rn(eT.y, diff.y, accW.y);
+            } else {
+                accW = __ffma2_rn(eT, diff, accW);               // same products, same order, same rounding
+            }
             accT = __fadd2_rn(accT, eT);
             accD = __fadd2_rn(accD, eD);
         }
         pT = accT.x + accT.y;
         pD = accD.x + accD.y;
-        pW = w0 + w1;
+        pW = accW.x + accW.y;
     }
     template <int VEC>
     static __device__ __forceinline__ float vector_bonus(const float (&t)[VEC], float c, float negRT) {

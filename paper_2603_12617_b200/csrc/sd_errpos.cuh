@@ -14,7 +14,7 @@
 // takes a slice of kErrSliceRegions sampling regions, a warp one region at a time.
 #pragma once
 
-#include "sd_device.cuh"
+#include "sd_kernels.cuh"
 
 namespace sdv {
 
@@ -57,34 +57,21 @@ __global__ void __launch_bounds__(kErrThreads, 4) sd_errpos_kernel(const __grid_
             rt[g] = vi < nv ? __ldcs(Trow + v0 + vi) : E::masked();
             rd[g] = (!bonus && vi < nv) ? __ldcs(Drow + v0 + vi) : E::masked();
         }
-        float ms[kGroups];
+        // the arithmetic of pass 2 of the full step, instruction for instruction
+        float mass;
+        if (!bonus) {
+            mass = pass2_region<DT, false>(rt, rd, nv, lane, P.c, rc,
+                                           Grow ? reinterpret_cast<ET*>(Grow + v0) : nullptr);
+        } else {
+            mass = pass2_region<DT, true>(rt, rd, nv, lane, P.c, rc, nullptr);
+            if (Grow) {
 #pragma unroll
-        for (int g = 0; g < kGroups; ++g) {
-            const int vi = g * 32 + lane;
-            float tv[VEC], rr[VEC];
-            E::unpack(rt[g], tv);
-            if (!bonus) {
-                float dv[VEC], gv[VEC];
-                E::unpack(rd[g], dv);
-#pragma unroll
-                for (int z = 0; z < VEC; z += 2) {
-                    const float2 g2 = grad_elem2(make_float2(tv[z], tv[z + 1]), make_float2(dv[z], dv[z + 1]), P.c, rc);
-                    gv[z] = g2.x;
-                    gv[z + 1] = g2.y;
-                    rr[z] = fmaxf(-g2.x, 0.f);
-                    rr[z + 1] = fmaxf(-g2.y, 0.f);
+                for (int g = 0; g < kGroups; ++g) {
+                    const int vi = g * 32 + lane;
+                    if (vi < nv) __stcs(Grow + v0 + vi, make_uint4(0u, 0u, 0u, 0u));   // no error position: a zero row
                 }
-                if (Grow && vi < nv) __stcs(Grow + v0 + vi, E::pack(gv));
-            } else {
-#pragma unroll
-                for (int z = 0; z < VEC; ++z) rr[z] = prob_elem(tv[z], P.c, rc);
-                if (Grow && vi < nv) __stcs(Grow + v0 + vi, make_uint4(0u, 0u, 0u, 0u));   // no error position: a zero row
             }
-            ms[g] = tree_sum<VEC>(rr);
         }
-        float mass = tree_sum<kGroups>(ms);
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) mass += __shfl_xor_sync(0xffffffffu, mass, off);
         if (lane == 0) rsum[r] = mass;
     }
 

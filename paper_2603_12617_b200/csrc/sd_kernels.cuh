@@ -104,6 +104,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// Non-blocking: has the phase of that parity completed?  (try_wait may suspend the thread for a while.)
+__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.acquire.cta.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -163,6 +175,12 @@ __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, 
         "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
         : "memory");
 }
+// Bulk prefetch global -> L2 (no shared-memory destination, nothing to wait for).  Address 16-byte
+// aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_prefetch_l2(const void* src_gmem, uint32_t bytes, uint64_t policy) {
+    asm volatile("cp.async.bulk.prefetch.L2.global.L2::cache_hint [%0], %1, %2;" ::"l"(src_gmem), "r"(bytes), "l"(policy)
+                 : "memory");
+}
 // L2 policies: keep (a line that will be read again shortly) and the default.
 __device__ __forceinline__ uint64_t policy_keep() {
     uint64_t p;
@@ -203,7 +221,8 @@ __device__ __forceinline__ uint64_t policy_discard() {
 // region of a unit looks for its maxima first; later ones reuse the references, and a region whose
 // sums come out too large for comfort (an entry far above everything the warp has seen: rare) is
 // done again after its maxima have raised the references and the running sums have moved with them
-// (exact: powers of two).
+// (exact: powers of two).  The second try also serves regions with masked target entries (-inf
+// logits), which the first one does not test for.
 struct Pass1State {
     float RT, RD;
     LaneSums ls;
@@ -268,7 +287,7 @@ __device__ __forceinline__ void await_region_registers(const uint4 (&rt)[kRegion
     asm volatile("" ::"r"(dep) : "memory");
 }
 
-template <int DT, bool BONUS>
+template <int DT, bool BONUS, bool MASKED>
 __device__ __forceinline__ void region_sums_of(const uint4 (&rt)[kRegionRows], const uint4 (&rd)[kRegionRows], float c,
                                                float RT, float RD, float& sT, float& sD, float& sW) {
     using E = Elem<DT>;
@@ -281,7 +300,7 @@ __device__ __forceinline__ void region_sums_of(const uint4 (&rt)[kRegionRows], c
         if (!BONUS) {
             float dv[VEC], pT, pD, pW;
             E::unpack(rd[g], dv);
-            LaneSums::vector_pair<VEC>(tv, dv, c, -RT, -RD, pT, pD, pW);
+            LaneSums::vector_pair<VEC, MASKED>(tv, dv, c, -RT, -RD, pT, pD, pW);
             sT += pT;
             sD += pD;
             sW += pW;
@@ -299,15 +318,21 @@ __device__ __noinline__ Pass1State pass1_region_again(const uint4* gT, const uin
                                                       Pass1State s) {
     using E = Elem<DT>;
     uint4 rt[kRegionRows], rd[kRegionRows];
+    if (nv <= 0) return s;
 #pragma unroll
     for (int g = 0; g < kRegionRows; ++g) {
         const int vi = g * 32 + lane;
-        rt[g] = vi < nv ? __ldg(gT + vi) : E::masked();
-        if (!BONUS) rd[g] = vi < nv ? __ldg(gD + vi) : E::masked();
+        const int vc = min(vi, nv - 1);       // every address formed is one of the region's own
+        const uint4 a = __ldg(gT + vc);
+        rt[g] = vi < nv ? a : E::masked();
+        if (!BONUS) {
+            const uint4 b = __ldg(gD + vc);
+            rd[g] = vi < nv ? b : E::masked();
+        }
     }
     raise_references<DT, BONUS>(rt, rd, c, s);
     float sT, sD, sW;
-    region_sums_of<DT, BONUS>(rt, rd, c, s.RT, s.RD, sT, sD, sW);
+    region_sums_of<DT, BONUS, true>(rt, rd, c, s.RT, s.RD, sT, sD, sW);
     s.ls.sT += sT;
     s.ls.sD += sD;
     s.ls.w += sW;
@@ -324,11 +349,20 @@ __device__ __forceinline__ void pass1_region(const uint4* st, int nv, int lane, 
     load_region<DT, BONUS>(st, nv, lane, rt, rd);
     await_region_registers<BONUS>(rt, rd);
     handed_back();
+    // A region cut short by the end of the slice holds -inf in place of the missing vectors, for which
+    // the fast arithmetic has no test: it goes the slow way at once, like (after the vote below) a
+    // region with masked target entries or with entries far above the references.
+    if (nv != kRegionVecs) {
+        s = again(s);
+        return;
+    }
     if (first) raise_references<DT, BONUS>(rt, rd, c, s);
     float sT, sD, sW;
-    region_sums_of<DT, BONUS>(rt, rd, c, s.RT, s.RD, sT, sD, sW);
-    // (written so that a NaN counts as too large)
-    if (!first && __any_sync(0xffffffffu, !(sT < kTooLarge) || !(sD < kTooLarge))) {
+    region_sums_of<DT, BONUS, false>(rt, rd, c, s.RT, s.RD, sT, sD, sW);
+    // Too large (written so that a NaN counts as too large), or a masked target entry has turned
+    // the sum of the products into a NaN: the slow way, which looks for the maxima and tests for
+    // masked entries.
+    if (__any_sync(0xffffffffu, !(sT < kTooLarge) || !(sD < kTooLarge) || sW != sW)) {
         s = again(s);
         return;
     }
@@ -355,19 +389,21 @@ __device__ __forceinline__ float pass2_region(const uint4 (&rt)[kRegionRows], co
             float dv[VEC], gv[VEC];
             E::unpack(rd[g], dv);
 #pragma unroll
+            float2 acc = make_float2(0.f, 0.f);
+#pragma unroll
             for (int z = 0; z < VEC; z += 2) {
                 const float2 g2 = grad_elem2(make_float2(tv[z], tv[z + 1]), make_float2(dv[z], dv[z + 1]), c, rc);
                 gv[z] = g2.x;
                 gv[z + 1] = g2.y;
-                r[z] = fmaxf(-g2.x, 0.f);
-                r[z + 1] = fmaxf(-g2.y, 0.f);
+                acc = __fadd2_rn(acc, make_float2(fmaxf(-g2.x, 0.f), fmaxf(-g2.y, 0.f)));
             }
             if (gdst && vi < nv) store_streaming(gdst + (size_t)vi * VEC, E::pack(gv));
+            ms[g] = acc.x + acc.y;
         } else {
 #pragma unroll
             for (int z = 0; z < VEC; ++z) r[z] = prob_elem(tv[z], c, rc);
+            ms[g] = tree_sum<VEC>(r);
         }
-        ms[g] = tree_sum<VEC>(r);
     }
     float mass = tree_sum<kRegionRows>(ms);
 #pragma unroll
@@ -382,7 +418,8 @@ struct StreamShared {
     uint64_t s1_done[2];                // consumers' sums of a unit posted       (consumer warps)
     uint64_t xchg_bar[2];               // partials of every block have arrived   (1 arrival + bytes, remote)
     uint64_t rc_ready[2];               // row constants published                (1)
-    uint64_t s2_done[kDoneDepth];       // unit finished in this block            (consumer warps + 1)
+    uint64_t row_pub[kDoneDepth];       // statistics of the unit's row published (1)
+    uint64_t s2_done[kDoneDepth];       // unit finished in this block            (consumer warps)
     uint64_t res_free[kDoneDepth];      // resolver is done with the unit         (1)
     PartialStats wpart[2][kConsumerWarps];   // the consumer warps' partials of a unit
     PartialStats xchg[2][kMaxCluster];  // written by every block of the cluster (distributed shared memory)
@@ -422,12 +459,13 @@ __device__ __forceinline__ void walk_stages(int nu, int nst, int L, P1&& p1, P2&
 
 // ---- fast path -----------------------------------------------------------------------------
 // lag_stages: stages of pass 1 of the next unit that go before pass 2 of a unit.
+// prefetch: non-zero lets the producer ask L2 for the next unit's pass-1 stages during pass 2.
 // ENS: the units are those of the ensemble feedback (see UnitRef); nothing is verified or drawn.
 // STATS: pass 1 only -- row constants, losses and rejection tests of every row; no gradient, no
 // masses, no draw (the error-position feedback finishes the one row it needs in a kernel of its own).
 template <int DT, bool ENS, bool STATS = false>
 __global__ void __launch_bounds__(kStreamThreads, 1)
-sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
+sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const int prefetch) {
     using E = Elem<DT>;
     using ET = typename E::type;
     constexpr int VEC = E::VEC;
@@ -478,7 +516,8 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
             mbar_init(&sh.rc_ready[s], 1);
         }
         for (int s = 0; s < kDoneDepth; ++s) {
-            mbar_init(&sh.s2_done[s], kConsumerWarps + 1);
+            mbar_init(&sh.row_pub[s], 1);
+            mbar_init(&sh.s2_done[s], kConsumerWarps);
             mbar_init(&sh.res_free[s], 1);
         }
         sh.abort = 0;
@@ -496,20 +535,23 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
             const int par = j & 1;
             const uint32_t ph = (uint32_t)(j >> 1) & 1u;
             const int dslot = j % kDoneDepth;
-            if (lane == 0) mbar_expect_tx(&sh.xchg_bar[par], (uint32_t)C * (uint32_t)sizeof(PartialStats));
-            if (!mbar_wait_sleepy<100>(&sh.s1_done[par], ph, wc)) break;
-            // the block's partial from its warps' partials, then one copy to every block of the cluster
-            const PartialStats mine = warp_merge_lanes(lane < kConsumerWarps ? sh.wpart[par][lane] : empty_partial());
-            if (lane < C) {
-                uint64_t refs;
-                memcpy(&refs, &mine.RT, 8);
-                PartialStats* dst = &sh.xchg[par][rank];
-                st_async_remote(dst, refs, (uint64_t)__double_as_longlong(mine.sT), &sh.xchg_bar[par], (uint32_t)lane);
-                st_async_remote(&dst->sD, (uint64_t)__double_as_longlong(mine.sD), (uint64_t)__double_as_longlong(mine.w),
-                                &sh.xchg_bar[par], (uint32_t)lane);
+            if (C > 1 && lane == 0) mbar_expect_tx(&sh.xchg_bar[par], (uint32_t)C * (uint32_t)sizeof(PartialStats));
+            if (!mbar_wait(&sh.s1_done[par], ph, wc)) break;
+            // the block's partial from its warps' partials, then (in a cluster of several blocks) one
+            // copy to every block of the cluster
+            PartialStats row = warp_merge_lanes(lane < kConsumerWarps ? sh.wpart[par][lane] : empty_partial());
+            if (C > 1) {
+                if (lane < C) {
+                    uint64_t refs;
+                    memcpy(&refs, &row.RT, 8);
+                    PartialStats* dst = &sh.xchg[par][rank];
+                    st_async_remote(dst, refs, (uint64_t)__double_as_longlong(row.sT), &sh.xchg_bar[par], (uint32_t)lane);
+                    st_async_remote(&dst->sD, (uint64_t)__double_as_longlong(row.sD), (uint64_t)__double_as_longlong(row.w),
+                                    &sh.xchg_bar[par], (uint32_t)lane);
+                }
+                if (!mbar_wait_cluster(&sh.xchg_bar[par], ph, wc)) break;
+                row = warp_merge_lanes(lane < C ? sh.xchg[par][lane] : empty_partial());
             }
-            if (!mbar_wait_cluster(&sh.xchg_bar[par], ph, wc)) break;
-            const PartialStats row = warp_merge_lanes(lane < C ? sh.xchg[par][lane] : empty_partial());
             const RowConst rcw = row_constants(P, bonus, row);
             if (lane == 0) {
                 sh.rc[par] = rcw;
@@ -521,7 +563,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
                 if (ok) {
                     sh.row[dslot] = row;
                     sh.rc_done[dslot] = rcw;
-                    mbar_arrive(&sh.s2_done[dslot]);
+                    mbar_arrive(&sh.row_pub[dslot]);
                 }
             }
             if (__any_sync(0xffffffffu, sh.abort)) break;
@@ -533,9 +575,11 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
             const int unit = u0 + j * ustep;
             const int dslot = j % kDoneDepth;
             const bool reports = (j % C == rank);   // the blocks of the cluster take turns
+            const uint32_t dph = (uint32_t)(j / kDoneDepth) & 1u;
             if constexpr (ENS) {
-                if (!mbar_wait_sleepy<500>(&sh.s2_done[dslot], (uint32_t)(j / kDoneDepth) & 1u, wc)) break;
+                if (!mbar_wait_sleepy<200>(&sh.row_pub[dslot], dph, wc)) break;
                 if (reports && lane == 0) finish_row_ensemble(P, unit_ref<true>(P, unit), sh.row[dslot]);
+                if (!mbar_wait_sleepy<200>(&sh.s2_done[dslot], dph, wc)) break;
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.res_free[dslot]);
                 continue;
@@ -545,8 +589,10 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
             AcceptOperands aop;
             aop.valid = false;
             if (reports && lane == 0 && !bonus) aop = load_accept_operands<DT>(P, b, i);
-            if (!mbar_wait_sleepy<500>(&sh.s2_done[dslot], (uint32_t)(j / kDoneDepth) & 1u, wc)) break;
+            // the row report needs pass 1 only: it runs while the consumers are in pass 2
+            if (!mbar_wait_sleepy<200>(&sh.row_pub[dslot], dph, wc)) break;
             if (reports && lane == 0) finish_row(P, b, i, sh.row[dslot], sh.rc_done[dslot], aop);
+            if (!mbar_wait_sleepy<200>(&sh.s2_done[dslot], dph, wc)) break;
             __syncwarp();
             if constexpr (STATS) {
                 if (lane == 0) mbar_arrive(&sh.res_free[dslot]);
@@ -601,7 +647,25 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
                 [&](int j) {
                     if constexpr (!STATS) {
                         const UnitRef ur = unit_ref<ENS>(P, u0 + j * ustep);
-                        for (int t = nst - 1; t >= 0 && ok; --t) issue(ur, t, discard);
+                        // Optionally each pass-2 stage issued also asks L2 to fetch one stage of pass 1 of
+                        // the next unit, which spreads the HBM reads over the time the consumers spend
+                        // in pass 2 (it pays when the row pairs in flight leave room in L2 for it).
+                        const bool ahead = prefetch != 0 && j + 1 < nu;
+                        UnitRef nx = ur;
+                        if (ahead) nx = unit_ref<ENS>(P, u0 + (j + 1) * ustep);
+                        for (int t = nst - 1; t >= 0 && ok; --t) {
+                            issue(ur, t, discard);
+                            const int tp = L + (nst - 1 - t);
+                            if (ahead && ok && tp < nst) {
+                                const int v0 = tp * kStageVecs;
+                                const uint32_t bytes = (uint32_t)min(kStageVecs, nvb - v0) * 16u;
+                                const size_t off = (size_t)(vb0 + v0) * VEC;
+                                if (lane == 0)
+                                    bulk_prefetch_l2(reinterpret_cast<const ET*>(P.T) + nx.t_row * P.V + off, bytes, keep);
+                                else if (!nx.bonus)
+                                    bulk_prefetch_l2(reinterpret_cast<const ET*>(ENS ? P.Dn[nx.n] : P.D) + nx.d_row * P.V + off, bytes, keep);
+                            }
+                        }
                     }
                     return ok;
                 });
@@ -622,10 +686,19 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
         bool ok = true;
         // The region is in registers: hand the warp's share of the slot back.  (Every lane's loads
         // from the slot have returned their values before the arrival.)
+        // Afterwards a look (no waiting) at the barrier of the next stage: its answer is there long
+        // before the arithmetic on this region is over, and when it says "full" -- the usual case --
+        // the next visit starts without the round trip of a wait.
+        bool next_full = false;
         auto hand_back = [&]() {
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh.empty[slot]);
             if (++slot == kRingStages) { slot = 0; fpar ^= 1u; }
+            next_full = mbar_test(&sh.full[slot], fpar);
+        };
+        auto await_stage = [&]() {
+            if (__all_sync(0xffffffffu, next_full ? 1 : 0)) return true;
+            return mbar_wait(&sh.full[slot], fpar, wc);
         };
         Pass1State ps;
         ps.RT = ps.RD = kEmptyRef;
@@ -635,7 +708,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
             const UnitRef ur = unit_ref<ENS>(P, u0 + j * ustep);
             const bool bonus = ur.bonus;
             for (int t = t0; t < t1; ++t) {
-                if (!mbar_wait(&sh.full[slot], fpar, wc)) { ok = false; return false; }
+                if (!await_stage()) { ok = false; return false; }
                 const uint4* st = reinterpret_cast<const uint4*>(ring + (size_t)slot * kStageBytes) + rv0;
                 const int nv = vectors_of(t);
                 if (nv == 0) { hand_back(); continue; }
@@ -685,7 +758,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages) {
             ET* Grow = (gbase && !bonus) ? reinterpret_cast<ET*>(gbase) + ur.d_row * P.V + (size_t)(vb0 + rv0) * VEC : nullptr;
             float* rsum = ENS ? nullptr : P.region_sums + (size_t)unit * P.NR + r0 + cw;
             for (int t = nst - 1; t >= 0; --t) {
-                if (!mbar_wait(&sh.full[slot], fpar, wc)) { ok = false; return false; }
+                if (!await_stage()) { ok = false; return false; }
                 const uint4* st = reinterpret_cast<const uint4*>(ring + (size_t)slot * kStageBytes) + rv0;
                 const int nv = vectors_of(t);
                 if (nv == 0) { hand_back(); continue; }
