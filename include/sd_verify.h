@@ -42,16 +42,13 @@
  *     logit tensors and for out_grad_draft.  Arithmetic is fp32 per element with fp64 row
  *     scalars in both cases.
  *   - Calls that share a workspace must not overlap on the GPU.
- *   - Side effect on the CUDA context: the first call on a device sets the context's limit
- *     cudaLimitPersistingL2CacheSize to 52 MiB (capped by the device's maximum), because the fast
- *     path fetches with the L2 evict_last policy what its second pass reads again, and that
- *     policy only holds lines inside such a set-aside.  The limit belongs to this process's
- *     context and ends with it; lines kept that way stay until later ones displace them, so a
- *     process whose other kernels want all of L2 may call cudaCtxResetPersistingL2Cache()
- *     between its own phases.  A caller that wants its context left alone calls
- *     sd_set_option(SD_OPT_L2_PERSIST_MIB, 0) before the first call on the device (any other
- *     value chooses another size).  See sd_set_option for the other tuning options; none is ever
- *     needed for correctness.
+ *   - The library changes no setting of the caller's CUDA context unless asked to: with option
+ *     SD_OPT_L2_PERSIST_MIB > 0 (default 0) the first call on a device sets the context's limit
+ *     cudaLimitPersistingL2CacheSize to that many MiB, inside which the lines that the fast path's
+ *     first pass fetches with the L2 evict_last policy are held for its second pass.  Since the second
+ *     pass walks a row pair backwards (last fetched, first re-read) the set-aside no longer pays on the
+ *     workloads measured, and sizes above about 60 MiB cost a third of the throughput.  See
+ *     sd_set_option for the other tuning options; none is ever needed for correctness.
  */
 #ifndef SD_VERIFY_H
 #define SD_VERIFY_H
@@ -294,12 +291,13 @@ int sd_verify_feedback_host(const void* target_logits, const void* draft_logits,
  * at the first use of the library) replaces, and which sd_set_option replaces at any time; a
  * change applies to the calls made after it.  Results never depend on them beyond rounding
  * (sums are taken in another order when the launch shape changes).
- *   SD_OPT_L2_PERSIST_MIB        env SD_VERIFY_L2_PERSIST_MIB   default 52   L2 set-aside requested on the
+ *   SD_OPT_L2_PERSIST_MIB        env SD_VERIFY_L2_PERSIST_MIB   default 0    L2 set-aside requested on the
  *                                first call on a device; 0 = leave the context's limit untouched
  *   SD_OPT_CLUSTER               env SD_VERIFY_CLUSTER          default 0    cluster size of the fast path
  *                                (1..16), 0 = chosen per shape
- *   SD_OPT_LAG                   env SD_VERIFY_LAG              default 1    stages of the next row pair
- *                                that go before the second pass over a row pair
+ *   SD_OPT_LAG                   env SD_VERIFY_LAG              default -1   stages of the next row pair
+ *                                that go before the second pass over a row pair; -1 = all of them when a
+ *                                cluster has at most eight row pairs to work on, none otherwise
  *   SD_OPT_L2_BUDGET_MIB         env SD_VERIFY_L2_MIB           default 80   bytes of row pairs in flight
  *                                between their two passes that the launch shape may assume L2 holds
  *   SD_OPT_FORCE_GENERIC         env SD_VERIFY_FORCE_GENERIC    default 0    non-zero: element-wise path

@@ -19,7 +19,7 @@ constexpr int kMaxDevices = 64;
 constexpr size_t kAlign = 256;
 constexpr int kStreamSmem = kRingStages * kStageBytes + (int)sizeof(StreamShared);
 static_assert(kStreamSmem <= 227 * 1024, "ring does not fit the shared memory of a block");
-constexpr int kL2PersistMiB = 52;
+constexpr int kL2PersistMiB = 0;
 constexpr long long kL2BudgetMiB = 80;             // row pairs in flight between their two passes should fit this
 
 // Tuning options: defaults, overridden once per process by the environment, then by sd_set_option.
@@ -35,7 +35,7 @@ void init_options() {
         static const struct { int id; const char* env; long long dflt; } table[] = {
             {SD_OPT_L2_PERSIST_MIB, "SD_VERIFY_L2_PERSIST_MIB", kL2PersistMiB},
             {SD_OPT_CLUSTER, "SD_VERIFY_CLUSTER", 0},
-            {SD_OPT_LAG, "SD_VERIFY_LAG", 1},
+            {SD_OPT_LAG, "SD_VERIFY_LAG", -1},
             {SD_OPT_L2_BUDGET_MIB, "SD_VERIFY_L2_MIB", kL2BudgetMiB},
             {SD_OPT_FORCE_GENERIC, "SD_VERIFY_FORCE_GENERIC", 0},
             {SD_OPT_GREEDY_BLOCKS_PER_SM, "SD_GREEDY_BLOCKS_PER_SM", 4},
@@ -123,7 +123,7 @@ struct DeviceState {
     bool attr_set[2][3] = {{false, false, false}, {false, false, false}};   // shared-memory / cluster attributes of the fast kernels
     int max_clusters[2][kMaxCluster + 1];   // resident clusters of 1..16 blocks, -1 = not asked yet
     // last launch-shape decision of the fast path
-    int dec_dtype = -1, dec_V = 0, dec_forced = 0, dec_C = 0, dec_G = 0, dec_lag = 0, dec_per = 0;
+    int dec_dtype = -1, dec_V = 0, dec_forced = 0, dec_C = 0, dec_G = 0, dec_lag = 0, dec_use_lag = 0, dec_per = 0;
     long long dec_units = 0;
     double dec_l2 = 0.0;
     // host-memory entry point
@@ -150,11 +150,10 @@ int current_device(int* dev, DeviceState** st) {
         }
         d.cc_major = prop.major;
         d.sm_count = prop.multiProcessorCount;
-        // Part of L2 set aside for lines fetched with the evict_last policy (pass 1 of the fast
-        // path fetches with it what pass 2 reads again): without a set-aside the policy has no
-        // effect and pass 2 of the largest workloads goes back to HBM for most of its lines.  52 MiB
-        // (granted as 58 MB) measured best on the 126 MB L2: larger ones starve everything else.
-        // A limit of this process's context only; option SD_OPT_L2_PERSIST_MIB = 0 leaves it alone.
+        // Optional: part of L2 set aside for lines fetched with the evict_last policy (pass 1 of the
+        // fast path fetches with it what pass 2 reads again).  Off by default: with pass 2 walking a
+        // row pair backwards it measured no better than no set-aside (0.509 ms against 0.511 ms on the
+        // largest workload; 64 MiB and more: 0.67 ms and worse), and the caller's context stays as it was.
         {
             const long long mib = option(SD_OPT_L2_PERSIST_MIB);
             size_t want = (size_t)(mib > 0 ? mib : 0) << 20;
@@ -246,7 +245,7 @@ int choose_stream(DeviceState& d, int V, long long units, int dtype, int* G_out,
         d.dec_l2 == l2_budget && d.dec_lag == lag) {
         *G_out = d.dec_G;
         *per_out = d.dec_per;
-        *lag_out = d.dec_lag;
+        *lag_out = d.dec_use_lag;
         return d.dec_C;
     }
     const int NV = V / vec_elems(dtype);
@@ -279,11 +278,17 @@ int choose_stream(DeviceState& d, int V, long long units, int dtype, int* G_out,
                             (!fits && !best_fits);
         if (better) { best_C = C; best_G = G; best_per = kRegionVecs; best_busy = busy; best_fits = fits; }
     }
+    // Stages of the next row pair that go before the second pass over a row pair: with few row
+    // pairs per cluster every wait for an exchange shows (and the first and the last cannot hide),
+    // so all of the next pair's first pass goes first; with many, the data between the passes is
+    // what costs (L2 holds less of it), and the second pass follows the first at once.
+    int use_lag = lag;
+    if (lag < 0) use_lag = (best_G > 0 && units <= 8LL * best_G) ? 1 << 20 : 0;
     d.dec_dtype = dtype; d.dec_V = V; d.dec_units = units; d.dec_forced = forced; d.dec_l2 = l2_budget;
-    d.dec_C = best_C; d.dec_G = best_G; d.dec_lag = lag; d.dec_per = best_per;
+    d.dec_C = best_C; d.dec_G = best_G; d.dec_lag = lag; d.dec_use_lag = use_lag; d.dec_per = best_per;
     *G_out = best_G;
     *per_out = best_per;
-    *lag_out = lag;
+    *lag_out = use_lag;
     return best_C;
 }
 
