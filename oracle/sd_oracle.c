@@ -426,6 +426,84 @@ int sd_oracle_draw_interval(const void* T, const void* D, int dtype, double tau,
     return 0;
 }
 
+/*
+ * sd_oracle_hint_error -- how far the hint of the optimistic update (Sec. 3.2, Eq. 3: the last
+ * round's gradient, h_t = grad f_{t-1}(w_{t-1})) is from this round's gradient: the summand of the
+ * quantity delta_T that Corollary 2 bounds, sum_t ||h_t - grad f_t(w_t)||_2^2, taken per position
+ * in the space of the draft logits:
+ *     err[b,i] = sum_v ( hint[b,i,v] - (q_{b,i,v} - p_{b,i,v}) / tau )^2.
+ * T [B,k+1,V] (bonus rows unused), D [B,k,V], hint [B,k,V] in `dtype`; out_err [B,k].
+ * Returns 0, or -1 on a bad argument or allocation failure.
+ */
+int sd_oracle_hint_error(const void* T, const void* D, const void* hint, int dtype, double tau, int B,
+                         int k, int V, double* out_err) {
+    if (!T || !D || !hint || !out_err || B < 1 || k < 1 || V < 1) return -1;
+    if (!(tau > 0.0) || !isfinite(tau)) return -1;
+    if (dtype != SD_ORACLE_F32 && dtype != SD_ORACLE_BF16) return -1;
+    double* p = (double*)malloc((size_t)V * sizeof(double));
+    double* q = (double*)malloc((size_t)V * sizeof(double));
+    double* lg = (double*)malloc((size_t)V * sizeof(double));
+    if (!p || !q || !lg) {
+        free(p); free(q); free(lg);
+        return -1;
+    }
+    for (int b = 0; b < B; ++b)
+        for (int i = 0; i < k; ++i) {
+            double S;
+            softmax_row(T, dtype, ((size_t)b * (k + 1) + i) * V, V, tau, p, lg, &S);
+            softmax_row(D, dtype, ((size_t)b * k + i) * V, V, tau, q, lg, &S);
+            double e = 0.0;
+            for (int v = 0; v < V; ++v) {
+                double g = (q[v] - p[v]) / tau;
+                double h = logit_at(hint, dtype, ((size_t)b * k + i) * V + (size_t)v);
+                e += (h - g) * (h - g);
+            }
+            out_err[(size_t)b * k + i] = e;
+        }
+    free(p); free(q); free(lg);
+    return 0;
+}
+
+/*
+ * sd_oracle_lmhead_grad -- the step after the feedback: the gradient of the round's loss with
+ * respect to the weights of the draft model's output layer.  With draft logits D[r,:] = W x_r for
+ * the R = B*k positions of the round (W [V,d], x_r the hidden state the output layer sees at
+ * position r), the chain rule turns the gradient with respect to the logits, g [R,V] (Sec. 3.1:
+ * the feedback gradient, here (q - p)/tau), into
+ *     dW[v,j] = sum_r g[r,v] * x[r,j]                                  (dW = g^T X, [V,d]).
+ * The paper leaves the draft network abstract; a linear output layer is what its draft heads
+ * (Hydra, EAGLE) end in.  g in `dtype_g`, X in `dtype_x` (each SD_ORACLE_F32 or SD_ORACLE_BF16);
+ * only the n entries (vs[e], js[e]) are computed, into out[e]; n < 0 computes all of dW into out
+ * [V,d] (vs, js unused).  Returns 0, or -1 on a bad argument.
+ */
+int sd_oracle_lmhead_grad(const void* g, int dtype_g, const void* X, int dtype_x, int R, int V, int d,
+                          long long n, const int32_t* vs, const int32_t* js, double* out) {
+    if (!g || !X || !out || R < 1 || V < 1 || d < 1) return -1;
+    if ((dtype_g != SD_ORACLE_F32 && dtype_g != SD_ORACLE_BF16) ||
+        (dtype_x != SD_ORACLE_F32 && dtype_x != SD_ORACLE_BF16))
+        return -1;
+    if (n >= 0 && (!vs || !js)) return -1;
+    if (n < 0) {
+        for (int v = 0; v < V; ++v)
+            for (int j = 0; j < d; ++j) {
+                double acc = 0.0;
+                for (int r = 0; r < R; ++r)
+                    acc += logit_at(g, dtype_g, (size_t)r * V + (size_t)v) * logit_at(X, dtype_x, (size_t)r * d + (size_t)j);
+                out[(size_t)v * d + j] = acc;
+            }
+        return 0;
+    }
+    for (long long e = 0; e < n; ++e) {
+        int v = vs[e], j = js[e];
+        if (v < 0 || v >= V || j < 0 || j >= d) return -1;
+        double acc = 0.0;
+        for (int r = 0; r < R; ++r)
+            acc += logit_at(g, dtype_g, (size_t)r * V + (size_t)v) * logit_at(X, dtype_x, (size_t)r * d + (size_t)j);
+        out[e] = acc;
+    }
+    return 0;
+}
+
 /* Threads the build can use: 1 without OpenMP. */
 int sd_oracle_max_threads(void) {
 #ifdef _OPENMP

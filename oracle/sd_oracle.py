@@ -44,6 +44,12 @@ def _load():
         lib.sd_oracle_draw_interval.restype = ctypes.c_int
         lib.sd_oracle_draw_interval.argtypes = [P, P, ctypes.c_int, ctypes.c_double, ctypes.c_int, ctypes.c_int,
                                                 ctypes.c_int, ctypes.c_int, P]
+        lib.sd_oracle_hint_error.restype = ctypes.c_int
+        lib.sd_oracle_hint_error.argtypes = [P, P, P, ctypes.c_int, ctypes.c_double, ctypes.c_int, ctypes.c_int,
+                                             ctypes.c_int, P]
+        lib.sd_oracle_lmhead_grad.restype = ctypes.c_int
+        lib.sd_oracle_lmhead_grad.argtypes = [P, ctypes.c_int, P, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                              ctypes.c_longlong, P, P, P]
         lib.sd_oracle_greedy.restype = ctypes.c_int
         lib.sd_oracle_greedy.argtypes = [P, ctypes.c_int, P, ctypes.c_int, ctypes.c_int, ctypes.c_int, P, P, P]
         lib.sd_oracle_ensemble.restype = ctypes.c_int
@@ -134,6 +140,58 @@ def draw_interval(target_logits: np.ndarray, draft_logits: np.ndarray, temperatu
     if rc != 0:
         raise RuntimeError(f"sd_oracle_draw_interval failed with code {rc}")
     return float(out[0]), float(out[1]), float(out[2])
+
+
+def _code(a: np.ndarray) -> int:
+    if a.dtype == np.float32:
+        return F32
+    if a.dtype == np.uint16:
+        return BF16
+    raise TypeError("arrays must be float32 or uint16 (bf16 bits)")
+
+
+def hint_error(target_logits: np.ndarray, draft_logits: np.ndarray, hint: np.ndarray, temperature: float) -> np.ndarray:
+    """Squared distance, per position, between the hint of the optimistic update (the last round's
+    gradient, Sec. 3.2) and this round's gradient (q - p)/tau with respect to the draft logits:
+    [B,k] float64."""
+    T = np.ascontiguousarray(target_logits)
+    D = np.ascontiguousarray(draft_logits)
+    H = np.ascontiguousarray(hint)
+    if not (T.dtype == D.dtype == H.dtype):
+        raise TypeError("logits and hint must share one dtype")
+    B, k1, V = T.shape
+    k = k1 - 1
+    if D.shape != (B, k, V) or H.shape != (B, k, V):
+        raise ValueError("draft logits and hint must be [B,k,V]")
+    out = np.empty((B, k), np.float64)
+    rc = _load().sd_oracle_hint_error(_ptr(T), _ptr(D), _ptr(H), _code(T), float(temperature), B, k, V, _ptr(out))
+    if rc != 0:
+        raise RuntimeError(f"sd_oracle_hint_error failed with code {rc}")
+    return out
+
+
+def lmhead_grad(grad_logits: np.ndarray, hidden: np.ndarray, vs=None, js=None) -> np.ndarray:
+    """Gradient of the round's loss with respect to the weights of a linear output layer of the draft,
+    dW = g^T X for g [R,V] (gradient w.r.t. the draft logits) and X [R,d] (hidden states): all of it
+    ([V,d] float64) or only the entries (vs[e], js[e])."""
+    g = np.ascontiguousarray(grad_logits)
+    X = np.ascontiguousarray(hidden)
+    if g.ndim != 2 or X.ndim != 2 or g.shape[0] != X.shape[0]:
+        raise ValueError("g must be [R,V] and X [R,d]")
+    R, V = g.shape
+    d = X.shape[1]
+    if vs is None:
+        out = np.empty((V, d), np.float64)
+        rc = _load().sd_oracle_lmhead_grad(_ptr(g), _code(g), _ptr(X), _code(X), R, V, d, -1, None, None, _ptr(out))
+    else:
+        vs = np.ascontiguousarray(vs, dtype=np.int32)
+        js = np.ascontiguousarray(js, dtype=np.int32)
+        out = np.empty(vs.shape[0], np.float64)
+        rc = _load().sd_oracle_lmhead_grad(_ptr(g), _code(g), _ptr(X), _code(X), R, V, d, vs.shape[0], _ptr(vs), _ptr(js),
+                                           _ptr(out))
+    if rc != 0:
+        raise RuntimeError(f"sd_oracle_lmhead_grad failed with code {rc}")
+    return out
 
 
 @dataclass

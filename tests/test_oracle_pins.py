@@ -613,3 +613,95 @@ def test_error_position_feedback_is_a_selection_of_the_full_step():
         assert (res.error_grad[b] == expect).all()
         if n < cfg.k:
             assert abs(res.error_grad[b].sum()) < 1e-12          # a difference of two distributions
+
+
+# ---- the step after the feedback: hint error (Sec. 3.2) and the output layer's gradient (Sec. 3.1) ----
+
+def test_hint_error_hand_values():
+    """p = (1/2,1/2), q = (3/4,1/4), tau = 1: the gradient is q - p = (1/4,-1/4).  Against the hint
+    (1/2, 0) the squared distance is 1/16 + 1/16; against the gradient itself it is 0; at tau = 1/2
+    the gradient doubles."""
+    T = logits_of([[[0.5, 0.5], [0.5, 0.5]]])
+    D = logits_of([[[0.75, 0.25]]])
+    hint = np.array([[[0.5, 0.0]]], np.float32)
+    np.testing.assert_allclose(sd_oracle.hint_error(T, D, hint, 1.0), [[0.125]], rtol=1e-6)
+    np.testing.assert_allclose(sd_oracle.hint_error(T, D, np.array([[[0.25, -0.25]]], np.float32), 1.0), [[0.0]], atol=1e-14)
+    # tau = 1/2 squares the probabilities before normalising: p stays (1/2,1/2), q = (9/10,1/10); g = 2 (q - p)
+    np.testing.assert_allclose(sd_oracle.hint_error(T, D, np.zeros((1, 1, 2), np.float32), 0.5), [[2 * 0.8 ** 2]], rtol=1e-6)
+
+
+def test_hint_error_is_the_squared_distance_to_the_oracles_gradient():
+    rng = np.random.default_rng(31)
+    B, k, V = 3, 2, 41
+    T = rng.normal(0, 2, (B, k + 1, V)).astype(np.float32)
+    D = (T[:, :k] + rng.normal(0, 1, (B, k, V))).astype(np.float32)
+    hint = rng.normal(0, 0.05, (B, k, V)).astype(np.float32)
+    tau = 0.8
+    p = softmax(T[:, :k].astype(np.float64) / tau, axis=-1)
+    q = softmax(D.astype(np.float64) / tau, axis=-1)
+    want = ((hint.astype(np.float64) - (q - p) / tau) ** 2).sum(-1)
+    np.testing.assert_allclose(sd_oracle.hint_error(T, D, hint, tau), want, rtol=1e-11)
+    # bf16 inputs are widened exactly
+    Tb, Db, hb = (synth.f32_to_bf16_bits(a) for a in (T, D, hint))
+    p = softmax(synth.bf16_bits_to_f32(Tb)[:, :k].astype(np.float64) / tau, axis=-1)
+    q = softmax(synth.bf16_bits_to_f32(Db).astype(np.float64) / tau, axis=-1)
+    want = ((synth.bf16_bits_to_f32(hb).astype(np.float64) - (q - p) / tau) ** 2).sum(-1)
+    np.testing.assert_allclose(sd_oracle.hint_error(Tb, Db, hb, tau), want, rtol=1e-11)
+
+
+def test_lmhead_gradient_hand_case_and_numpy():
+    """R = 2 positions, V = 2, d = 2: g = [[1,2],[3,4]], X = [[5,6],[7,8]]:
+    dW = g^T X = [[1*5+3*7, 1*6+3*8], [2*5+4*7, 2*6+4*8]] = [[26,30],[38,44]]."""
+    g = np.array([[1, 2], [3, 4]], np.float32)
+    X = np.array([[5, 6], [7, 8]], np.float32)
+    np.testing.assert_array_equal(sd_oracle.lmhead_grad(g, X), [[26, 30], [38, 44]])
+    # not the transposed product, and not X^T g
+    assert not np.array_equal(sd_oracle.lmhead_grad(g, X), g @ X)
+    rng = np.random.default_rng(32)
+    g = rng.normal(0, 1, (7, 13)).astype(np.float32)
+    X = rng.normal(0, 1, (7, 5)).astype(np.float32)
+    full = sd_oracle.lmhead_grad(g, X)
+    np.testing.assert_allclose(full, g.astype(np.float64).T @ X.astype(np.float64), rtol=1e-12, atol=1e-14)
+    # sampled entries equal the full result; linear in X
+    vs, js = np.array([0, 12, 5, 5]), np.array([4, 0, 2, 3])
+    np.testing.assert_array_equal(sd_oracle.lmhead_grad(g, X, vs, js), full[vs, js])
+    np.testing.assert_allclose(sd_oracle.lmhead_grad(g, (2 * X).astype(np.float32)), 2 * full, rtol=1e-12)
+    # bf16 operands are widened exactly
+    gb, Xb = synth.f32_to_bf16_bits(g), synth.f32_to_bf16_bits(X)
+    want = synth.bf16_bits_to_f32(gb).astype(np.float64).T @ synth.bf16_bits_to_f32(Xb).astype(np.float64)
+    np.testing.assert_allclose(sd_oracle.lmhead_grad(gb, Xb), want, rtol=1e-12, atol=1e-14)
+
+
+def test_lmhead_gradient_is_the_derivative_of_the_loss_in_the_output_layers_weights():
+    """Draft logits D = X W^T for a small linear output layer: central finite differences of the
+    oracle's summed loss in every entry of W equal g^T X with the oracle's own gradient g."""
+    rng = np.random.default_rng(33)
+    B, k, V, d = 2, 2, 6, 3
+    tau = 0.9
+    T = rng.normal(0, 1.5, (B, k + 1, V)).astype(np.float32)
+    X = rng.normal(0, 1, (B * k, d))
+    W = rng.normal(0, 1, (V, d))
+    x = np.zeros((B, k), np.int32)
+    u = np.zeros((B, k + 1), np.float32)
+
+    def loss_of(Wm):
+        # the oracle takes float32 logits: keep the perturbation visible by working at a coarse step
+        D = (X @ Wm.T).reshape(B, k, V)
+        Tq = T.astype(np.float64)
+        p = softmax(Tq[:, :k] / tau, axis=-1)
+        q = softmax(D / tau, axis=-1)
+        return rel_entr(p, q).sum()
+
+    D32 = (X @ W.T).reshape(B, k, V).astype(np.float32)
+    res = sd_oracle.verify_feedback(T, D32, x, u, tau)
+    # the oracle's loss is the KL that loss_of restates with scipy (pinned elsewhere); its gradient feeds g^T X
+    dW = sd_oracle.lmhead_grad(res.grad.reshape(B * k, V).astype(np.float32), X.astype(np.float32))
+    h = 1e-5
+    fd = np.zeros_like(W)
+    for v in range(V):
+        for j in range(d):
+            Wp, Wm = W.copy(), W.copy()
+            Wp[v, j] += h
+            Wm[v, j] -= h
+            fd[v, j] = (loss_of(Wp) - loss_of(Wm)) / (2 * h)
+    np.testing.assert_allclose(dW, fd, rtol=2e-4, atol=2e-6)      # float32 logits and operands
