@@ -93,23 +93,23 @@ __device__ __forceinline__ void st_async_remote(void* dst, uint64_t a, uint64_t 
         "r"(smem_u32(bar)), "l"(a), "l"(b), "r"(rank)
         : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cta.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
 // Non-blocking: has the phase of that parity completed?  (try_wait may suspend the thread for a while.)
 __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.test_wait.parity.acquire.cta.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cta.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(smem_u32(bar)), "r"(parity)
@@ -139,8 +139,13 @@ template <bool CLUSTER, int SLEEP_NS = 20>
 __device__ __forceinline__ bool mbar_wait_thread(uint64_t* bar, uint32_t parity, const WaitCtx& wc) {
     volatile int* abort = wc.abort;
     long long t0 = 0;
+    // (A limit of a few polls is a caller asking for waits that give up at once: those polls only
+    // look, where the usual ones let the hardware suspend the thread until the phase ends or a
+    // time limit of its own runs out.)
+    const bool look_only = wc.limit < 64u;
     for (uint32_t it = 0; it < wc.limit; ++it) {
-        if (CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
+        if (look_only ? mbar_test(bar, parity)
+                      : (CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity))) return true;
         __nanosleep(SLEEP_NS);   // waiting warps leave the issue slots to the working ones
         if ((it & 63u) == 63u) {
             if (*abort) return false;
@@ -620,7 +625,12 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const i
             uint32_t epar = 1;                     // parity to wait for on empty[slot]: that of its previous use
             bool ok = true;
             auto issue = [&](const UnitRef& ur, int t, uint64_t pol) {
-                if (ni >= kRingStages && !mbar_wait_thread<false>(&sh.empty[slot], epar, wc)) { ok = false; return; }
+                // the first thread waits for the slot and decides for both, so that a stage is
+                // either fetched whole or not at all
+                int go = 1;
+                if (ni >= kRingStages && lane == 0) go = mbar_wait_thread<false>(&sh.empty[slot], epar, wc) ? 1 : 0;
+                go = __shfl_sync(0x3u, go, 0);
+                if (!go) { ok = false; return; }
                 const int v0 = t * kStageVecs;     // first vector of the stage within the slice
                 const uint32_t bytes = (uint32_t)min(kStageVecs, nvb - v0) * 16u;
                 const size_t off = (size_t)(vb0 + v0) * VEC;
@@ -669,13 +679,15 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const i
                     }
                     return ok;
                 });
-            // leaving early: no copy may still be in flight when the block returns (a draft-part copy
-            // whose barrier the first thread never armed has the pause before the block's exit to land)
-            if (!ok && lane == 0)
+            // leaving early: no copy may still be in flight when the block returns
+            if (!ok && lane == 0) {
+                const long long t0 = clock64();
                 for (int i = max(0, ni - kRingStages); i < ni; ++i) {
                     const uint32_t par = (uint32_t)(i / kRingStages) & 1u;
-                    for (uint32_t it = 0; it < kWaitLimit && !mbar_try_wait(&sh.full[i % kRingStages], par); ++it) {}
+                    for (uint32_t it = 0; it < kWaitLimit && !mbar_try_wait(&sh.full[i % kRingStages], par); ++it)
+                        if (clock64() - t0 > kWaitCycles) break;
                 }
+            }
         }
     } else if (warp >= kFirstConsumerWarp) {
         // ---- consumers: warp cw owns region cw of every stage; a region is a sampling region.

@@ -596,6 +596,39 @@ def test_non_default_stream_and_changing_shapes(binding):
         check(inp, out, oracle_of(inp), max_band_frac=1.0)
 
 
+def test_a_wait_that_runs_out_is_reported_and_leaves_the_library_usable(binding, options):
+    """Every wait inside the fast path is bounded.  With the bound set to a few polls (an option
+    that exists for this purpose) the first wait for data gives up long before the data can be
+    there: the kernel must come back on its own, flag the sequences with SD_STATUS_TIMEOUT, and
+    the next call with the usual bound must be exact again.  Nothing is made to hang: the waits
+    simply run out."""
+    cfg = synth.custom_config(B=6, k=3, V=40000, dtype="f32", index=68)
+    inp = synth.make_inputs(cfg)
+    T, D, x, u = to_device(inp)
+    options(binding.SD_OPT_WAIT_POLLS, 4)
+    out = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
+    torch.cuda.synchronize()                                  # the kernel returned
+    assert binding.sd_launch_info()["path"] == 1
+    st = out.status.cpu().numpy().astype(np.uint32)
+    assert (st & np.uint32(binding.SD_STATUS_TIMEOUT)).all(), st
+    # the error-position and ensemble entry points share the waits
+    err = binding.sd_verify_error_feedback(T, D, x, u, inp.tau)
+    ens = binding.sd_ensemble_feedback(T, [D, D], inp.tau, 10.0, want_status=True)
+    torch.cuda.synchronize()
+    assert (err.status.cpu().numpy().astype(np.uint32) & np.uint32(binding.SD_STATUS_TIMEOUT)).all()
+    assert (ens.status.cpu().numpy().astype(np.uint32) & np.uint32(binding.SD_STATUS_TIMEOUT)).all()
+    # back to the usual bound: exact again, on caller scratch and on the library's own
+    options(binding.SD_OPT_WAIT_POLLS, 1 << 21)
+    binding.sd_release_cached_buffers()
+    out = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
+    torch.cuda.synchronize()
+    ref = oracle_of(inp)
+    check(inp, out, ref, max_band_frac=1.0)
+    out2 = binding.sd_verify_feedback(T, D, x, u, inp.tau)
+    torch.cuda.synchronize()
+    check(inp, out2, ref, max_band_frac=1.0)
+
+
 @pytest.mark.parametrize("name", ["cfg2", "cfg3"])
 def test_host_entry_point_matches_device_entry_point(binding, name):
     cfg = synth.CONFIGS[name]
