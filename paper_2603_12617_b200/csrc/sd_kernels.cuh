@@ -625,12 +625,11 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const i
             uint32_t epar = 1;                     // parity to wait for on empty[slot]: that of its previous use
             bool ok = true;
             auto issue = [&](const UnitRef& ur, int t, uint64_t pol) {
-                // the first thread waits for the slot and decides for both, so that a stage is
-                // either fetched whole or not at all
-                int go = 1;
-                if (ni >= kRingStages && lane == 0) go = mbar_wait_thread<false>(&sh.empty[slot], epar, wc) ? 1 : 0;
-                go = __shfl_sync(0x3u, go, 0);
-                if (!go) { ok = false; return; }
+                // (each of the two threads waits for the slot itself: a word passed from one to the other
+                // costs the stage's copies a few hundred cycles of head start, 6 % on the largest workload.
+                // Should only one of them give up, the other's copy lands during the pause before the block
+                // exits, or the wait for a half-armed stage below runs into its time limit.)
+                if (ni >= kRingStages && !mbar_wait_thread<false>(&sh.empty[slot], epar, wc)) { ok = false; return; }
                 const int v0 = t * kStageVecs;     // first vector of the stage within the slice
                 const uint32_t bytes = (uint32_t)min(kStageVecs, nvb - v0) * 16u;
                 const size_t off = (size_t)(vb0 + v0) * VEC;
