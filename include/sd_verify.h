@@ -273,6 +273,29 @@ int sd_verify_error_feedback(const void* target_logits, const void* draft_logits
                              size_t workspace_bytes, void* stream);
 
 /*
+ * sd_lmhead_grad -- the step after the feedback: the gradient of the round's loss with respect to
+ * the weights W [V,d] of the draft model's linear output layer.  The feedback gradient of Sec. 3.1
+ * ("nabla f_t(w_t)") reaches the parameters through the chain rule; with draft logits
+ * D[r,:] = W x_r for the R = B*k positions of the round, and g = out_grad_draft of the step viewed
+ * as [R,V],
+ *     dW[v,j] = sum_r g[r,v] * x[r,j]                      (dW = g^T X).
+ * (The paper leaves the draft network abstract; a linear output layer is what its draft heads end in.)
+ * A dense contraction over the positions: tensor cores (tcgen05.mma, bf16 x bf16 -> fp32).
+ *
+ *   grad_logits  [R, V]   in   device, bfloat16 bit patterns: out_grad_draft of sd_verify_feedback_bf16
+ *   hidden       [R, d]   in   device, bfloat16 bit patterns
+ *   out_dW       [V, d]   out  device, fp32
+ *   out_status   [1]      out  device uint32, or NULL: non-zero if a bounded wait inside the kernel gave
+ *                              up (out_dW is then invalid)
+ *   stream                in   cudaStream_t
+ * V and d must be multiples of 8 and every pointer 16-byte aligned (SD_ERR_ALIGN otherwise); all
+ * three tensors must be memory of the current GPU.  Returns SD_OK or a negative SD_ERR_* code
+ * (nothing enqueued).
+ */
+int sd_lmhead_grad(const uint16_t* grad_logits, const uint16_t* hidden, int R, int V, int d, float* out_dW,
+                   uint32_t* out_status, void* stream);
+
+/*
  * sd_verify_feedback_host -- the same step for callers whose tensors live in HOST memory.
  * Every pointer is a HOST pointer (pinned memory gives asynchronous copies, pageable memory
  * works too).  The call copies the inputs to device buffers the library keeps per device
@@ -325,7 +348,7 @@ long long sd_get_option(int option_id);
 
 /*
  * sd_launch_info -- HOST out-parameters describing how the last successful device call on this
- * thread was launched: path (0 = generic, 1 = stream fast path, 2 = greedy verification, 3 = ensemble feedback, 4 = error-position feedback), cluster size, threads per
+ * thread was launched: path (0 = generic, 1 = stream fast path, 2 = greedy verification, 3 = ensemble feedback, 4 = error-position feedback, 5 = output-layer gradient), cluster size, threads per
  * block, dynamic shared memory per block, blocks launched, kernels launched.  Any pointer may
  * be NULL.  Diagnostic only.
  */

@@ -67,6 +67,8 @@ def _load() -> ctypes.CDLL:
     lib.sd_ensemble_feedback.restype = I
     lib.sd_ensemble_feedback.argtypes = [P, P, I, ctypes.c_float, ctypes.c_float, I, I, I, I, P, P, P, P, P, P, P,
                                          P, Z, P]
+    lib.sd_lmhead_grad.restype = I
+    lib.sd_lmhead_grad.argtypes = [P, P, I, I, I, P, P, P]
     lib.sd_verify_feedback_host.restype = I
     lib.sd_verify_feedback_host.argtypes = [P, P, P, P, F, I, I, I, I, P, P, P, P, P, P]
     lib.sd_workspace_bytes.restype = Z
@@ -346,6 +348,32 @@ def sd_ensemble_feedback(target_logits: torch.Tensor, draft_logits, temperature:
                                        _stream_ptr(stream))
     if rc != 0:
         raise SdVerifyError(rc, "sd_ensemble_feedback")
+    return out
+
+
+def sd_lmhead_grad(grad_logits: torch.Tensor, hidden: torch.Tensor, *, out: Optional[torch.Tensor] = None,
+                   status: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """``sd_lmhead_grad``: dW = g^T X for g [R,V] (or [B,k,V]) and X [R,d], both bfloat16 on the device;
+    returns dW [V,d] float32."""
+    if grad_logits.dim() == 3:
+        grad_logits = grad_logits.reshape(-1, grad_logits.shape[-1])
+    if grad_logits.dim() != 2 or hidden.dim() != 2 or grad_logits.shape[0] != hidden.shape[0]:
+        raise ValueError("grad_logits must be [R,V] and hidden [R,d]")
+    if grad_logits.dtype != torch.bfloat16 or hidden.dtype != torch.bfloat16:
+        raise TypeError("both operands must be bfloat16")
+    if not grad_logits.is_contiguous() or not hidden.is_contiguous():
+        raise ValueError("operands must be contiguous")
+    dev = grad_logits.device
+    if dev.type != "cuda" or hidden.device != dev:
+        raise ValueError("device tensors on one GPU required")
+    R, V = grad_logits.shape
+    d = hidden.shape[1]
+    if out is None:
+        out = torch.empty((V, d), dtype=torch.float32, device=dev)
+    with torch.cuda.device(dev):
+        rc = _lib.sd_lmhead_grad(_ptr(grad_logits), _ptr(hidden), R, V, d, _ptr(out), _ptr(status), _stream_ptr(stream))
+    if rc != 0:
+        raise SdVerifyError(rc, "sd_lmhead_grad")
     return out
 
 

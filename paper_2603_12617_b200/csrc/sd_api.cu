@@ -10,6 +10,7 @@
 #include "sd_kernels.cuh"
 #include "sd_greedy.cuh"
 #include "sd_errpos.cuh"
+#include "sd_lmhead.cuh"
 
 namespace {
 
@@ -126,6 +127,9 @@ struct DeviceState {
     int dec_dtype = -1, dec_V = 0, dec_forced = 0, dec_C = 0, dec_G = 0, dec_lag = 0, dec_use_lag = 0, dec_per = 0;
     long long dec_units = 0;
     double dec_l2 = 0.0;
+    // output-layer gradient
+    uint32_t* gemm_error = nullptr;
+    bool gemm_attr = false;
     // host-memory entry point
     StageSet stage[2];
     cudaStream_t s_h2d = nullptr, s_comp = nullptr, s_d2h = nullptr;
@@ -418,6 +422,48 @@ int static_scratch(int dev, unsigned char** out) {
         g_static_ptr[dev] = static_cast<unsigned char*>(ptr);
     }
     *out = g_static_ptr[dev];
+    return SD_OK;
+}
+
+// ---- tensor maps for the output-layer gradient ---------------------------------------------
+// cuTensorMapEncodeTiled lives in the driver; its address comes from the runtime, so the library
+// links against nothing but the CUDA runtime.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        else
+            (void)cudaGetLastError();
+    });
+    return fn;
+}
+// Map of a row-major bf16 matrix [rows, cols] (device memory of this GPU) for boxes of
+// box_rows x 64 columns in the 128-byte swizzle; entries outside the matrix read as zero.
+int bf16_matrix_map(CUtensorMap* map, const void* base, int rows, int cols, int box_rows) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) {
+        snprintf(tl_cuda_error, sizeof tl_cuda_error, "cuTensorMapEncodeTiled is not available from this driver");
+        return SD_ERR_CUDA;
+    }
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kGemmChunk, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(tl_cuda_error, sizeof tl_cuda_error, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+        return SD_ERR_CUDA;
+    }
     return SD_OK;
 }
 
@@ -831,6 +877,44 @@ int sd_verify_feedback_host(const void* target_logits, const void* draft_logits,
     return SD_OK;
 }
 
+// ---- the output layer's gradient ----------------------------------------------------------------
+int sd_lmhead_grad(const uint16_t* grad_logits, const uint16_t* hidden, int R, int V, int d, float* out_dW,
+                   uint32_t* out_status, void* stream) {
+    if (!grad_logits || !hidden || !out_dW) return SD_ERR_NULL;
+    if (R < 1 || V < 1 || d < 1 || (long double)V * d >= 4.0e18L) return SD_ERR_SHAPE;
+    if (V % 8 != 0 || d % 8 != 0) return SD_ERR_ALIGN;            // rows of whole 16-byte vectors (TMA strides)
+    if (!aligned(grad_logits, 16) || !aligned(hidden, 16) || !aligned(out_dW, 16) || (out_status && !aligned(out_status, 4)))
+        return SD_ERR_ALIGN;
+    int dev;
+    DeviceState* ds = nullptr;
+    int rc = current_device(&dev, &ds);
+    if (rc != SD_OK) return rc;
+    std::lock_guard<std::mutex> lock(ds->mu);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!ds->gemm_error) SD_CUDA(cudaMalloc(reinterpret_cast<void**>(&ds->gemm_error), 256));
+    uint32_t* err = out_status ? out_status : ds->gemm_error;
+    SD_CUDA(cudaMemsetAsync(err, 0, 4, st));
+    CUtensorMap map_g, map_x;
+    rc = bf16_matrix_map(&map_g, grad_logits, R, V, kGemmBK);
+    if (rc != SD_OK) return rc;
+    rc = bf16_matrix_map(&map_x, hidden, R, d, kGemmBK);
+    if (rc != SD_OK) return rc;
+    if (!ds->gemm_attr) {
+        SD_CUDA(cudaFuncSetAttribute(sd_lmhead_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem));
+        ds->gemm_attr = true;
+    }
+    GemmParams P;
+    P.R = R; P.V = V; P.d = d;
+    P.out = out_dW;
+    P.error = err;
+    const long long tiles = (long long)((V + kGemmBM - 1) / kGemmBM) * ((d + kGemmBN - 1) / kGemmBN);
+    const unsigned grid = (unsigned)(tiles < ds->sm_count ? tiles : ds->sm_count);
+    sd_lmhead_kernel<<<grid, kGemmThreads, kGemmSmem, st>>>(map_g, map_x, P);
+    SD_CUDA(cudaGetLastError());
+    tl_info[0] = 5; tl_info[1] = 1; tl_info[2] = kGemmThreads; tl_info[3] = kGemmSmem; tl_info[4] = (int)grid; tl_info[5] = 1;
+    return SD_OK;
+}
+
 int sd_set_option(int option_id, long long value) {
     if (option_id < 0 || option_id >= SD_OPT_COUNT) return SD_ERR_SHAPE;
     init_options();
@@ -857,12 +941,13 @@ void sd_release_cached_buffers(void) {
     for (int i = 0; i < kMaxDevices; ++i) {
         DeviceState& d = g_dev[i];
         std::lock_guard<std::mutex> lock(d.mu);
-        if (!d.probed || (!d.ws && !d.stage[0].base && !d.stage[1].base)) continue;
+        if (!d.probed || (!d.ws && !d.gemm_error && !d.stage[0].base && !d.stage[1].base)) continue;
         int prev = -1;
         if (cudaGetDevice(&prev) != cudaSuccess) continue;
         if (cudaSetDevice(i) != cudaSuccess) continue;
         cudaDeviceSynchronize();
         if (d.ws) { cudaFree(d.ws); d.ws = nullptr; d.ws_bytes = 0; d.ws_zero_bytes = 0; }
+        if (d.gemm_error) { cudaFree(d.gemm_error); d.gemm_error = nullptr; }
         for (StageSet& st : d.stage)
             if (st.base) { cudaFree(st.base); st.base = nullptr; st.bytes = 0; }
         cudaSetDevice(prev);
