@@ -10,29 +10,32 @@ draw, KL loss and its gradient) over one batch.  Prints ONE JSON line (rank 0).
              on the launching stream over exactly K steps, max over ranks
   roofline   algorithmic bytes (read (2k+1)*V*B logits, write k*V*B gradient entries) per launch
              over the mean kernel duration, against the measured HBM copy bandwidth
-  e2e        the same metric through the host-memory entry point: pinned host buffers in, host
-             buffers out, every copy inside the timed region
+  e2e        the same metric through host buffers: pinned host memory in, host buffers out, every
+             copy inside the timed region (the headline path: sd_verify_feedback_host)
   cpu_baseline  the CPU oracle, as it stands, on a bounded sample of the same workload
+  parity     the timed outputs against the oracle on that sample: sequences compared, rows inside the
+             two threshold bands, mismatches inside and outside them, mean accept length, mean sum min(p,q)
   --impl reference  times the CPU oracle on the host cores (there is no other implementation of
              this path to run); rank 0 only
 
-With N > 1 (launched by torch.distributed.run) every rank runs the full batch of its own
-(weak scaling: sequences are independent, no collective on the path).
+With N > 1 every rank runs the full batch of its own (weak scaling: sequences are independent, no
+collective on the path).  Started without torch.distributed.run, `--gpus N` starts its own ranks.
 
-  --path greedy   times greedy verification instead (Algorithm 1 in the limit tau -> 0, the decoding
-             mode of the paper's experiments): only the target logits are read, (k+1)*V*B entries per
-             launch; the line has the same keys, with "path": "greedy" in config.  Not the headline.
-  --path ensemble  times the feedback of an online ensemble of --learners N draft models (Sec. 3.3):
-             (k + N*k)*V*B logits in, N*k*V*B gradient entries out per launch; value counts the B*k
-             positions of the round (each served for all N learners).  Not the headline.
-  --path errors   times the step with the feedback restricted to the error position (what OSD
-             collects, Sec. 3.1): (2k+1)*V*B logits in, B*V gradient entries out.  Not the headline.
+  --path greedy    greedy verification (Algorithm 1 in the limit tau -> 0): (k+1)*V*B entries read
+  --path ensemble  feedback of an online ensemble of --learners N draft models (Sec. 3.3)
+  --path errors    feedback restricted to the error position (what OSD collects, Sec. 3.1)
+  --path lmhead    the step after the path: the output layer's gradient dW = g^T X on the tensor cores,
+                   R = B*k positions of the workload, --features d; roofline in TFLOP/s
+Each prints the same keys with "path" in config; none of them is the headline.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
+import socket
+import subprocess
 import sys
 import threading
 import time
@@ -48,21 +51,46 @@ from paper_2603_12617_b200 import synth  # noqa: E402
 METRIC = "verified draft positions/sec"
 UNIT = "positions/s"
 L2_BYTES = 126 * 1024 * 1024
-# dram__bytes_read.sum + dram__bytes_write.sum per launch at full size, from the ncu captures
-# summarised under profiles/ (bytes; a workload that is not listed has not been captured)
-NCU_TRAFFIC_ENSEMBLE = {("cfg5", 3): 3388811776 + 2325275904}
-NCU_TRAFFIC_ERRORS = {"cfg5": 1707537664 + 3327232 + 251808256 + 99995904}   # both kernels of the step
-NCU_TRAFFIC_GREEDY = {"cfg5": 919481088 + 244224}
-NCU_TRAFFIC_BYTES = {"cfg5": 2078492160 + 758877952, "cfg3": 155482368 + 36729856, "cfg4": 179505152 + 50643456}
+TOL = {"f32": 1e-5, "bf16": 2e-2}
 
 
-def measured_peak_gbs():
-    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+def measured_peaks():
     try:
-        with open(path) as fh:
-            return float(json.load(fh)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
+            d = json.load(fh)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d["bf16_tflops_sustained"]), "source": "measured (MEASURED_PEAKS.json)"}
     except Exception:
-        return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+        return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
+                "source": "fallback (6.65 TB/s, 1.59 PFLOP/s burst, 1.4 sustained)"}
+
+
+def kernel_source_hash() -> str:
+    """Identifies the kernels a DRAM-traffic capture belongs to: the CUDA sources, hashed."""
+    h = hashlib.sha256()
+    src = os.path.join(ROOT, "paper_2603_12617_b200", "csrc")
+    for name in sorted(os.listdir(src)):
+        with open(os.path.join(src, name), "rb") as fh:
+            h.update(name.encode())
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def captured_traffic(path: str, cfg_name: str, extra: str = "-"):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised in
+    profiles/dram_traffic.txt -- only if the kernels have not changed since it was taken."""
+    fname = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    try:
+        with open(fname) as fh:
+            rows = [ln.split() for ln in fh if ln.strip() and not ln.startswith("#")]
+    except OSError:
+        return None, "no capture on file"
+    for row in rows:
+        if len(row) >= 6 and row[0] == path and row[1] == cfg_name and row[2] == extra:
+            if row[5] != kernel_source_hash():
+                return None, "the kernels have changed since the capture in profiles/dram_traffic.txt"
+            return int(row[3]) + int(row[4]), "ncu capture summarised in profiles/dram_traffic.txt (same kernel sources)"
+    return None, "this workload has not been captured"
 
 
 class ClockSampler:
@@ -89,24 +117,32 @@ class ClockSampler:
         except Exception as exc:  # NVML missing: report that, do not fail the run
             self._nv, self._err = None, repr(exc)
 
-    def _run(self):
+    def _sample(self):
         nv = self._nv
+        try:
+            self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+            mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+            for bit, name in self.REASONS.items():
+                if mask & bit:
+                    self.reasons.add(name)
+        except Exception:
+            pass
+
+    def _run(self):
         while not self._stop.is_set():
-            try:
-                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
-                mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
-                for bit, name in self.REASONS.items():
-                    if mask & bit:
-                        self.reasons.add(name)
-            except Exception:
-                pass
-            time.sleep(0.004)
+            self._sample()
+            time.sleep(0.002)
 
     def __enter__(self):
         if self._nv is not None:
             self._thread = threading.Thread(target=self._run, daemon=True)
             self._thread.start()
         return self
+
+    def sample_now(self):
+        """One more sample from the calling thread (the GPU is still under load when this is called)."""
+        if self._nv is not None:
+            self._sample()
 
     def __exit__(self, *a):
         self._stop.set()
@@ -120,36 +156,59 @@ class ClockSampler:
                 "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
-def time_oracle(inp, seqs, nthreads):
+# ------------------------------------------------------------------------------------------
+# the oracle legs
+
+def run_oracle(inp, seqs, nthreads, want_grad=True):
     from oracle import sd_oracle
     sl = np.asarray(seqs)
     t0 = time.perf_counter()
-    sd_oracle.verify_feedback(inp.target_logits[sl], inp.draft_logits[sl], inp.draft_tokens[sl],
-                              inp.uniforms[sl], inp.tau, nthreads=nthreads)
-    return time.perf_counter() - t0
+    res = sd_oracle.verify_feedback(inp.target_logits[sl], inp.draft_logits[sl], inp.draft_tokens[sl],
+                                    inp.uniforms[sl], inp.tau, want_grad=want_grad, nthreads=nthreads)
+    return time.perf_counter() - t0, res
 
 
 def cpu_baseline(cfg, inp, target_seconds=12.0):
-    """The oracle on the host cores over a bounded sample of the workload's sequences."""
+    """The oracle on the host cores over a bounded sample of the workload's sequences; also returns
+    the sequences and the oracle's result for them (the parity counts of the line come from it)."""
     from oracle import sd_oracle
     cores = min(sd_oracle.max_threads(), os.cpu_count() or 1)
     n = min(cfg.B, cores)
-    t = time_oracle(inp, range(n), cores)
+    t, res = run_oracle(inp, range(n), cores)
     if t < target_seconds / 2 and n < cfg.B:
         n2 = int(min(cfg.B, max(n, n * target_seconds / max(t, 1e-3))))
         n2 = max(cores, n2 // cores * cores)
         if n2 > n:
-            n, t = n2, time_oracle(inp, range(n2), cores)
-    return {"value": n * cfg.k / t, "unit": UNIT, "cores": cores, "kind": "oracle",
+            n = n2
+            t, res = run_oracle(inp, range(n2), cores)
+    base = {"value": n * cfg.k / t, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"{n} of {cfg.B} sequences of {cfg.name} (k={cfg.k}, V={cfg.V}, {cfg.dtype}), "
                       f"one call, {t:.2f} s",
             "gb_per_s": n * cfg.algorithmic_bytes / cfg.B / t / 1e9}
+    return base, np.arange(n), res
+
+
+def parity_counts(cfg, ref, seqs, accept_len, tokens, loss):
+    """The timed outputs against the oracle on `seqs`: rows in the two threshold bands, mismatches
+    inside and outside them, and whether the losses hold the tolerance."""
+    n_gpu, tok_gpu = accept_len[seqs], tokens[seqs]
+    accept_band = ref.accept_band.sum(1) > 0
+    sample_band = ref.cdf_margin <= 1e-6
+    band = accept_band | sample_band
+    mismatch = (n_gpu != ref.accept_len) | (tok_gpu != ref.tokens).any(axis=1)
+    out = {"sequences_compared": int(len(seqs)), "accept_band_rows": int(ref.accept_band.sum()),
+           "sample_band_rows": int(sample_band.sum()), "mismatches_inside_the_bands": int((mismatch & band).sum()),
+           "mismatches_outside_the_bands": int((mismatch & ~band).sum()),
+           "mean_accept_len": float(accept_len.mean()), "mean_acc_prob_oracle": float(ref.acc_prob.mean())}
+    if loss is not None:
+        err = np.abs(loss[seqs].astype(np.float64) - ref.loss)
+        out["loss_within_tolerance"] = bool((err <= TOL[cfg.dtype] * np.maximum(np.abs(ref.loss), 1e-6)).all())
+    return out
 
 
 def run_reference(args, cfg):
     """--impl reference: the CPU oracle timed on the host cores, bounded sample per step."""
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    if int(os.environ.get("RANK", "0")) != 0:
         return
     from oracle import sd_oracle
     sd_oracle.build()
@@ -157,17 +216,17 @@ def run_reference(args, cfg):
     # a step is the oracle on n sequences; n is sized so the run ends within about two minutes
     probe_cfg = cfg.with_batch(min(cfg.B, cores))
     inp = synth.make_inputs(probe_cfg)
-    t_probe = time_oracle(inp, range(probe_cfg.B), cores)
+    t_probe, _ = run_oracle(inp, range(probe_cfg.B), cores)
     budget = 120.0 / max(1, args.steps + args.warmup)
     n = probe_cfg.B
     if t_probe > budget:
         n = max(1, int(probe_cfg.B * budget / t_probe))
     threads = min(cores, n)
     for _ in range(args.warmup):
-        time_oracle(inp, range(n), threads)
+        run_oracle(inp, range(n), threads)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        time_oracle(inp, range(n), threads)
+        run_oracle(inp, range(n), threads)
     dt = time.perf_counter() - t0
     value = args.steps * n * cfg.k / dt
     sample = f"{n} of {cfg.B} sequences of {cfg.name} per step, {threads} threads"
@@ -189,6 +248,317 @@ def workload_config(cfg, **extra):
     return d
 
 
+# ------------------------------------------------------------------------------------------
+# the paths: each describes one entry point to the common timing loop
+
+def as_torch(a):
+    import torch
+    t = torch.from_numpy(a)
+    return t.view(torch.bfloat16) if a.dtype == np.uint16 else t
+
+
+def rotating_sets(host_tensors, dev):
+    """Device copies of the inputs: one set if it is larger than L2 by itself, else enough rotating
+    sets that every step reads from HBM."""
+    in_bytes = sum(t.numel() * t.element_size() for t in host_tensors)
+    nsets = 1 if in_bytes > 2 * L2_BYTES else int(min(64, -(-3 * L2_BYTES // in_bytes)))
+    return [[t.to(dev) for t in host_tensors] for _ in range(nsets)], in_bytes, nsets
+
+
+class SamplePath:
+    """The headline: sd_verify_feedback (library scratch), e2e through sd_verify_feedback_host."""
+    name, kernel, traffic_path = "sample", "sd_stream_kernel", "sample"
+
+    def __init__(self, args, cfg, dev, rank, binding):
+        import torch
+        self.b, self.cfg, self.torch = binding, cfg, torch
+        self.inp = inp = synth.make_inputs(cfg, seed=synth.BASE_SEED + 1000 * rank)
+        self.host = [as_torch(inp.target_logits).pin_memory(), as_torch(inp.draft_logits).pin_memory(),
+                     torch.from_numpy(inp.draft_tokens).pin_memory(), torch.from_numpy(inp.uniforms).pin_memory()]
+        self.sets, self.in_bytes, self.nsets = rotating_sets(self.host, dev)
+        tdt = self.host[0].dtype
+        self.out = binding.StepOutputs(
+            accept_len=torch.empty(cfg.B, dtype=torch.int32, device=dev),
+            tokens=torch.empty((cfg.B, cfg.k + 1), dtype=torch.int32, device=dev),
+            loss=torch.empty((cfg.B, cfg.k), dtype=torch.float32, device=dev),
+            grad_draft=torch.empty((cfg.B, cfg.k, cfg.V), dtype=tdt, device=dev))
+        self.algorithmic = cfg.algorithmic_bytes
+        self.positions = cfg.B * cfg.k
+        self.dtype = "f32" if cfg.dtype == "f32" else "f32 (bf16 storage)"
+        self.extra = {}
+        self.e2e_entry = "sd_verify_feedback_host"
+
+    def step(self, i):
+        T, D, x, u = self.sets[i % self.nsets]
+        self.b.sd_verify_feedback(T, D, x, u, self.inp.tau, out=self.out)
+
+    def e2e_prepare(self):
+        torch, cfg = self.torch, self.cfg
+        self.hout = self.b.StepOutputs(
+            accept_len=torch.empty(cfg.B, dtype=torch.int32).pin_memory(),
+            tokens=torch.empty((cfg.B, cfg.k + 1), dtype=torch.int32).pin_memory(),
+            loss=torch.empty((cfg.B, cfg.k), dtype=torch.float32).pin_memory(),
+            grad_draft=torch.empty((cfg.B, cfg.k, cfg.V), dtype=self.host[0].dtype).pin_memory())
+        self.h2d = self.in_bytes
+        self.d2h = sum(t.numel() * t.element_size() for t in (self.hout.accept_len, self.hout.tokens, self.hout.loss, self.hout.grad_draft))
+
+    def e2e_step(self):
+        self.b.sd_verify_feedback_host(*self.host, self.inp.tau, out=self.hout)
+
+    def finish(self, args):
+        """CPU baseline and parity of the timed outputs (rank 0)."""
+        torch, cfg = self.torch, self.cfg
+        T, D, x, u = self.sets[0]
+        chk = self.b.sd_verify_feedback(T, D, x, u, self.inp.tau)
+        torch.cuda.synchronize()
+        if args.no_cpu_baseline:
+            seqs = np.asarray(sorted({0, cfg.B // 2, cfg.B - 1}))
+            base, (_, ref) = None, run_oracle(self.inp, seqs, len(seqs), want_grad=False)
+        else:
+            base, seqs, ref = cpu_baseline(cfg, self.inp)
+        parity = parity_counts(cfg, ref, seqs, chk.accept_len.cpu().numpy(), chk.tokens.cpu().numpy(), chk.loss.cpu().numpy())
+        verified = parity["mismatches_outside_the_bands"] == 0 and parity.get("loss_within_tolerance", True)
+        return base, parity, bool(verified)
+
+
+class GreedyPath:
+    name, kernel, traffic_path = "greedy", "sd_greedy_kernel", "greedy"
+
+    def __init__(self, args, cfg, dev, rank, binding):
+        import torch
+        self.b, self.cfg, self.torch = binding, cfg, torch
+        self.inp = inp = synth.make_inputs(cfg, seed=synth.BASE_SEED + 1000 * rank)
+        # greedy drafting proposes the draft's argmax; the inputs carry sampled tokens, which serves as well:
+        # the work does not depend on the tokens
+        self.host = [as_torch(inp.target_logits).pin_memory(), torch.from_numpy(inp.draft_tokens).pin_memory()]
+        self.sets, self.in_bytes, self.nsets = rotating_sets(self.host, dev)
+        self.out = binding.sd_verify_greedy(*self.sets[0])
+        self.algorithmic = (cfg.k + 1) * cfg.V * cfg.B * cfg.elem_bytes
+        self.positions = cfg.B * cfg.k
+        self.dtype = "f32 comparisons" if cfg.dtype == "f32" else "bf16 comparisons"
+        self.extra = {}
+        self.e2e_entry = "sd_verify_greedy between pinned-memory copies"
+
+    def step(self, i):
+        self.b.sd_verify_greedy(*self.sets[i % self.nsets], out=self.out)
+
+    def e2e_prepare(self):
+        torch, cfg = self.torch, self.cfg
+        self.dbuf = [torch.empty_like(t) for t in self.sets[0]]
+        self.h_n = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
+        self.h_tok = torch.empty((cfg.B, cfg.k + 1), dtype=torch.int32).pin_memory()
+        self.h2d = self.in_bytes
+        self.d2h = self.h_n.numel() * 4 + self.h_tok.numel() * 4
+
+    def e2e_step(self):
+        for a, b in zip(self.dbuf, self.host):
+            a.copy_(b, non_blocking=True)
+        self.b.sd_verify_greedy(*self.dbuf, out=self.out)
+        self.h_n.copy_(self.out.accept_len, non_blocking=True)
+        self.h_tok.copy_(self.out.tokens, non_blocking=True)
+        self.torch.cuda.synchronize()
+
+    def finish(self, args):
+        from oracle import sd_oracle
+        cfg = self.cfg
+        t0 = time.perf_counter()
+        ref = sd_oracle.verify_greedy(self.inp.target_logits, self.inp.draft_tokens)
+        t_cpu = time.perf_counter() - t0
+        verified = bool((self.h_n.numpy() == ref.accept_len).all() and (self.h_tok.numpy() == ref.tokens).all()
+                        and (self.out.argmax.cpu().numpy() == ref.argmax).all())
+        base = {"value": cfg.B * cfg.k / t_cpu, "unit": UNIT, "cores": 1, "kind": "oracle",
+                "sample": f"all {cfg.B} sequences of {cfg.name}, one call, {t_cpu:.2f} s"}
+        parity = {"sequences_compared": cfg.B, "mismatches_outside_the_bands": 0 if verified else None,
+                  "mean_accept_len": float(self.h_n.float().mean())}
+        return base, parity, verified
+
+
+class ErrorsPath:
+    name, kernel, traffic_path = "errors", "sd_stream_kernel<pass 1 only> + sd_errpos_kernel", "errors"
+
+    def __init__(self, args, cfg, dev, rank, binding):
+        import torch
+        self.b, self.cfg, self.torch = binding, cfg, torch
+        self.inp = inp = synth.make_inputs(cfg, seed=synth.BASE_SEED + 1000 * rank)
+        self.host = [as_torch(inp.target_logits).pin_memory(), as_torch(inp.draft_logits).pin_memory(),
+                     torch.from_numpy(inp.draft_tokens).pin_memory(), torch.from_numpy(inp.uniforms).pin_memory()]
+        self.sets, self.in_bytes, self.nsets = rotating_sets(self.host, dev)
+        self.out = binding.sd_verify_error_feedback(*self.sets[0], inp.tau)
+        self.algorithmic = ((2 * cfg.k + 1) + 1) * cfg.V * cfg.B * cfg.elem_bytes
+        self.positions = cfg.B * cfg.k
+        self.dtype = "f32" if cfg.dtype == "f32" else "f32 (bf16 storage)"
+        self.extra = {}
+        self.e2e_entry = "sd_verify_error_feedback between pinned-memory copies"
+
+    def step(self, i):
+        self.b.sd_verify_error_feedback(*self.sets[i % self.nsets], self.inp.tau, out=self.out)
+
+    def e2e_prepare(self):
+        torch, cfg = self.torch, self.cfg
+        self.dbuf = [torch.empty_like(t) for t in self.sets[0]]
+        self.h_n = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
+        self.h_tok = torch.empty((cfg.B, cfg.k + 1), dtype=torch.int32).pin_memory()
+        self.h_loss = torch.empty((cfg.B, cfg.k), dtype=torch.float32).pin_memory()
+        self.h_g = torch.empty((cfg.B, cfg.V), dtype=self.host[0].dtype).pin_memory()
+        self.h2d = self.in_bytes
+        self.d2h = self.h_n.numel() * 4 + self.h_tok.numel() * 4 + self.h_loss.numel() * 4 + self.h_g.numel() * self.h_g.element_size()
+
+    def e2e_step(self):
+        for a, b in zip(self.dbuf, self.host):
+            a.copy_(b, non_blocking=True)
+        self.b.sd_verify_error_feedback(*self.dbuf, self.inp.tau, out=self.out)
+        self.h_n.copy_(self.out.accept_len, non_blocking=True)
+        self.h_tok.copy_(self.out.tokens, non_blocking=True)
+        self.h_loss.copy_(self.out.loss, non_blocking=True)
+        self.h_g.copy_(self.out.error_grad, non_blocking=True)
+        self.torch.cuda.synchronize()
+
+    def finish(self, args):
+        from oracle import sd_oracle
+        cfg, inp = self.cfg, self.inp
+        cores = min(sd_oracle.max_threads(), os.cpu_count() or 1)
+        nseq = min(cfg.B, cores)
+        sl = np.arange(nseq)
+        t0 = time.perf_counter()
+        ref = sd_oracle.error_position_feedback(inp.target_logits[sl], inp.draft_logits[sl], inp.draft_tokens[sl],
+                                                inp.uniforms[sl], inp.tau, nthreads=cores)
+        t_cpu = time.perf_counter() - t0
+        parity = parity_counts(cfg, ref.full, sl, self.h_n.numpy(), self.h_tok.numpy(), self.h_loss.numpy())
+        safe = (ref.full.accept_band.sum(1) == 0) & (ref.full.cdf_margin > 1e-6)
+        g = self.h_g[:nseq].float().numpy().astype(np.float64)
+        tol = TOL[cfg.dtype]
+        grads_ok = all(np.abs(g[b] - ref.error_grad[b]).max() <= tol * np.abs(ref.error_grad[b]).max() + 1e-6
+                       for b in range(nseq) if safe[b])
+        verified = bool(parity["mismatches_outside_the_bands"] == 0 and parity["loss_within_tolerance"] and grads_ok)
+        base = {"value": nseq * cfg.k / t_cpu, "unit": UNIT, "cores": cores, "kind": "oracle",
+                "sample": f"{nseq} of {cfg.B} sequences of {cfg.name}, one call, {t_cpu:.2f} s"}
+        return base, parity, verified
+
+
+class EnsemblePath:
+    name, kernel, traffic_path = "ensemble", "sd_stream_kernel<ensemble> + sd_hedge_kernel", "ensemble"
+    EPS = 10.0
+
+    def __init__(self, args, cfg, dev, rank, binding):
+        import torch
+        self.b, self.cfg, self.torch = binding, cfg, torch
+        self.N = N = args.learners
+        self.inp = inp = synth.make_inputs(cfg, seed=synth.BASE_SEED + 1000 * rank)
+        self.drafts = synth.ensemble_drafts(inp, N, seed=synth.BASE_SEED + 1000 * rank)
+        self.host = [as_torch(inp.target_logits).pin_memory()] + [as_torch(d).pin_memory() for d in self.drafts]
+        self.sets, self.in_bytes, self.nsets = rotating_sets(self.host, dev)
+        self.out = binding.sd_ensemble_feedback(self.sets[0][0], self.sets[0][1:], inp.tau, self.EPS)
+        self.cum = torch.zeros(N, dtype=torch.float64, device=dev)
+        self.algorithmic = ((cfg.k + N * cfg.k) + N * cfg.k) * cfg.V * cfg.B * cfg.elem_bytes
+        self.positions = cfg.B * cfg.k
+        self.dtype = "f32" if cfg.dtype == "f32" else "f32 (bf16 storage)"
+        self.extra = {"learners": N, "epsilon": self.EPS}
+        self.traffic_extra = str(N)
+        self.e2e_entry = "sd_ensemble_feedback between pinned-memory copies"
+
+    def step(self, i):
+        s = self.sets[i % self.nsets]
+        self.b.sd_ensemble_feedback(s[0], s[1:], self.inp.tau, self.EPS, cum_loss=self.cum, out=self.out)
+
+    def e2e_prepare(self):
+        torch, cfg, N = self.torch, self.cfg, self.N
+        self.dbuf = [torch.empty_like(t) for t in self.sets[0]]
+        self.h_loss = torch.empty((N, cfg.B, cfg.k), dtype=torch.float32).pin_memory()
+        self.h_w = torch.empty(N, dtype=torch.float32).pin_memory()
+        self.h_grad = [torch.empty_like(d).pin_memory() for d in self.host[1:]]
+        self.h2d = self.in_bytes
+        self.d2h = self.h_loss.numel() * 4 + self.h_w.numel() * 4 + sum(g.numel() * g.element_size() for g in self.h_grad)
+
+    def e2e_step(self):
+        for a, b in zip(self.dbuf, self.host):
+            a.copy_(b, non_blocking=True)
+        self.b.sd_ensemble_feedback(self.dbuf[0], self.dbuf[1:], self.inp.tau, self.EPS, cum_loss=self.cum, out=self.out)
+        self.h_loss.copy_(self.out.loss, non_blocking=True)
+        self.h_w.copy_(self.out.weights, non_blocking=True)
+        for a, b in zip(self.h_grad, self.out.grad):
+            a.copy_(b, non_blocking=True)
+        self.torch.cuda.synchronize()
+
+    def finish(self, args):
+        from oracle import sd_oracle
+        cfg, inp, N = self.cfg, self.inp, self.N
+        cores = min(sd_oracle.max_threads(), os.cpu_count() or 1)
+        nseq = min(cfg.B, max(1, cores // cfg.k))
+        sl = np.arange(nseq)
+        t0 = time.perf_counter()
+        ref = sd_oracle.ensemble_feedback(inp.target_logits[sl], [d[sl] for d in self.drafts], inp.tau, self.EPS,
+                                          want_grad=False, nthreads=cores)
+        t_cpu = time.perf_counter() - t0
+        loss = self.h_loss.numpy()[:, :nseq].astype(np.float64)
+        ok = bool((np.abs(loss - ref.loss) <= TOL[cfg.dtype] * np.maximum(np.abs(ref.loss), 1e-6)).all()
+                  and abs(float(self.h_w.sum()) - 1.0) < 1e-5)
+        base = {"value": nseq * cfg.k / t_cpu, "unit": UNIT, "cores": cores, "kind": "oracle",
+                "sample": f"{nseq} of {cfg.B} sequences of {cfg.name}, {N} learners, no gradients, one call, {t_cpu:.2f} s"}
+        parity = {"sequences_compared": int(nseq), "loss_within_tolerance": ok}
+        return base, parity, ok
+
+
+class LmHeadPath:
+    """The step after the path: dW = g^T X for the R = B*k positions of the workload."""
+    name, kernel, traffic_path = "lmhead", "sd_lmhead_kernel", "lmhead"
+
+    def __init__(self, args, cfg, dev, rank, binding):
+        import torch
+        self.b, self.cfg, self.torch = binding, cfg, torch
+        self.R, self.V, self.d = cfg.B * cfg.k, cfg.V, args.features
+        gb, Xb = synth.lmhead_operands(self.R, self.V, self.d, seed=synth.BASE_SEED + 1000 * rank)
+        self.gb, self.Xb = gb, Xb
+        self.host = [as_torch(gb).pin_memory(), as_torch(Xb).pin_memory()]
+        self.sets, self.in_bytes, self.nsets = rotating_sets(self.host, dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.out = torch.empty((self.V, self.d), dtype=torch.float32, device=dev)
+        self.algorithmic = 2 * self.R * self.V * self.d         # flops
+        self.positions = self.R
+        self.dtype = "bf16 operands, f32 accumulation"
+        self.extra = {"features": self.d, "positions": self.R}
+        self.e2e_entry = "sd_lmhead_grad between pinned-memory copies"
+        self.bound = "tensor"
+
+    def step(self, i):
+        g, X = self.sets[i % self.nsets]
+        self.b.sd_lmhead_grad(g, X, out=self.out, status=self.status)
+
+    def e2e_prepare(self):
+        torch = self.torch
+        self.dbuf = [torch.empty_like(t) for t in self.sets[0]]
+        self.h_out = torch.empty((self.V, self.d), dtype=torch.float32).pin_memory()
+        self.h2d = self.in_bytes
+        self.d2h = self.h_out.numel() * 4
+
+    def e2e_step(self):
+        for a, b in zip(self.dbuf, self.host):
+            a.copy_(b, non_blocking=True)
+        self.b.sd_lmhead_grad(*self.dbuf, out=self.out, status=self.status)
+        self.h_out.copy_(self.out, non_blocking=True)
+        self.torch.cuda.synchronize()
+
+    def finish(self, args):
+        from oracle import sd_oracle
+        rng = np.random.default_rng(11)
+        n = 4000
+        vs, js = rng.integers(0, self.V, n), rng.integers(0, self.d, n)
+        t0 = time.perf_counter()
+        ref = sd_oracle.lmhead_grad(self.gb, self.Xb, vs, js)
+        t_cpu = time.perf_counter() - t0
+        got = self.h_out.numpy()[vs, js].astype(np.float64)
+        g = np.abs(synth.bf16_bits_to_f32(self.gb).astype(np.float64))
+        X = np.abs(synth.bf16_bits_to_f32(self.Xb).astype(np.float64))
+        bound = 2e-5 * np.einsum("re,re->e", g[:, vs], X[:, js]) + 1e-30
+        ok = bool((np.abs(got - ref) <= bound).all() and int(self.status.item()) == 0)
+        full_s = t_cpu * (self.V * self.d / n)
+        base = {"value": self.R / full_s, "unit": UNIT, "cores": 1, "kind": "oracle",
+                "sample": f"{n} of {self.V * self.d} entries of dW, {t_cpu:.2f} s, scaled to all of dW"}
+        return base, {"entries_compared": n, "within_tolerance": ok}, ok
+
+
+PATHS = {"sample": SamplePath, "greedy": GreedyPath, "errors": ErrorsPath, "ensemble": EnsemblePath, "lmhead": LmHeadPath}
+
+
 def run_ours(args, cfg):
     import torch
     import torch.distributed as dist
@@ -200,39 +570,13 @@ def run_ours(args, cfg):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
-    if world != args.gpus:
-        if world == 1 and args.gpus > 1:
-            raise SystemExit("launch with torch.distributed.run for --gpus > 1")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    # every rank verifies a full batch of its own (different seed per rank): weak scaling
-    inp = synth.make_inputs(cfg, seed=synth.BASE_SEED + 1000 * rank)
-    tdt = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
-
-    def as_torch(a):
-        t = torch.from_numpy(a)
-        return t.view(torch.bfloat16) if a.dtype == np.uint16 else t
-
-    hT, hD = as_torch(inp.target_logits).pin_memory(), as_torch(inp.draft_logits).pin_memory()
-    hx, hu = torch.from_numpy(inp.draft_tokens).pin_memory(), torch.from_numpy(inp.uniforms).pin_memory()
-    in_bytes = hT.numel() * hT.element_size() + hD.numel() * hD.element_size()
-    # inputs larger than L2, or enough rotating copies that every step reads from HBM
-    nsets = 1 if in_bytes > 2 * L2_BYTES else int(min(64, -(-3 * L2_BYTES // in_bytes)))
-    sets = []
-    for _ in range(nsets):
-        sets.append((hT.to(dev), hD.to(dev), hx.to(dev), hu.to(dev)))
-    out = binding.StepOutputs(
-        accept_len=torch.empty(cfg.B, dtype=torch.int32, device=dev),
-        tokens=torch.empty((cfg.B, cfg.k + 1), dtype=torch.int32, device=dev),
-        loss=torch.empty((cfg.B, cfg.k), dtype=torch.float32, device=dev),
-        grad_draft=torch.empty((cfg.B, cfg.k, cfg.V), dtype=tdt, device=dev))
-
-    def step(i):
-        T, D, x, u = sets[i % nsets]
-        binding.sd_verify_feedback(T, D, x, u, inp.tau, out=out)
+    # every rank works on a full batch of its own (different seed per rank): weak scaling
+    path = PATHS[args.path](args, cfg, dev, rank, binding)
 
     def barrier():
         torch.cuda.synchronize()
@@ -240,8 +584,9 @@ def run_ours(args, cfg):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(max(3, args.warmup)):
-        step(i)
+    warmup = max(3, args.warmup)
+    for i in range(warmup):
+        path.step(i)
     info = binding.sd_launch_info()
     barrier()
     starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
@@ -251,473 +596,92 @@ def run_ours(args, cfg):
         t_begin.record()
         for i in range(args.steps):
             starts[i].record()
-            step(i)
+            path.step(i)
             ends[i].record()
+            if (i & 15) == 15:
+                clocks.sample_now()           # the queue is full of work: the GPU is under load here
         t_end.record()
+        clocks.sample_now()
         barrier()
-    total_ms = shard.max_over_ranks(t_begin.elapsed_time(t_end), device=str(dev) if world > 1 else "cpu")
+    dev_arg = str(dev) if world > 1 else "cpu"
+    total_ms = shard.max_over_ranks(t_begin.elapsed_time(t_end), device=dev_arg)
     kernel_ms = [s.elapsed_time(e) for s, e in zip(starts, ends)]
     mean_kernel_ms = float(np.mean(kernel_ms))
     if args.times_out and rank == 0:
         with open(args.times_out, "w") as fh:
             json.dump(kernel_ms, fh)
-    positions = cfg.B * cfg.k * world
+    positions = path.positions * world
     value = positions * args.steps / (total_ms * 1e-3)
 
-    # sanity: the timed outputs are the real ones (checked against the oracle on a few sequences)
-    check_seqs = [0, cfg.B // 2, cfg.B - 1] if cfg.B > 2 else list(range(cfg.B))
-    verified = None
-    if rank == 0:
-        from oracle import sd_oracle
-        sl = np.asarray(sorted(set(check_seqs)))
-        ref = sd_oracle.verify_feedback(inp.target_logits[sl], inp.draft_logits[sl], inp.draft_tokens[sl],
-                                        inp.uniforms[sl], inp.tau, want_grad=False, nthreads=len(sl))
-        T, D, x, u = sets[0]
-        chk = binding.sd_verify_feedback(T, D, x, u, inp.tau)
-        torch.cuda.synchronize()
-        safe = (ref.accept_band.sum(1) == 0) & (ref.cdf_margin > 1e-6)
-        verified = bool((chk.accept_len.cpu().numpy()[sl][safe] == ref.accept_len[safe]).all()
-                        and (chk.tokens.cpu().numpy()[sl][safe] == ref.tokens[safe]).all()
-                        and np.allclose(chk.loss.cpu().numpy()[sl], ref.loss, rtol=2e-2 if cfg.dtype == "bf16" else 1e-5, atol=4e-7))
-
-    # end to end through the host-memory entry point: pinned host buffers, copies inside the region
-    e2e_steps = max(1, min(args.steps, 10))
-    hout = binding.StepOutputs(
-        accept_len=torch.empty(cfg.B, dtype=torch.int32).pin_memory(),
-        tokens=torch.empty((cfg.B, cfg.k + 1), dtype=torch.int32).pin_memory(),
-        loss=torch.empty((cfg.B, cfg.k), dtype=torch.float32).pin_memory(),
-        grad_draft=torch.empty((cfg.B, cfg.k, cfg.V), dtype=tdt).pin_memory())
+    # end to end: pinned host buffers in, host buffers out, every copy inside the timed region
+    e2e_steps = max(1, min(args.steps, 3 if args.path == "lmhead" else 10))
+    path.e2e_prepare()
     for _ in range(2):
-        binding.sd_verify_feedback_host(hT, hD, hx, hu, inp.tau, out=hout)
+        path.e2e_step()
     barrier()
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
-        binding.sd_verify_feedback_host(hT, hD, hx, hu, inp.tau, out=hout)
+        path.e2e_step()
     barrier()
-    e2e_s = shard.max_over_ranks(time.perf_counter() - t0, device=str(dev) if world > 1 else "cpu")
-    h2d = in_bytes + hx.numel() * 4 + hu.numel() * 4
-    d2h = sum(t.numel() * t.element_size() for t in (hout.accept_len, hout.tokens, hout.loss, hout.grad_draft))
-    e2e = {"value": positions * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
-           "d2h_bytes_per_step": int(d2h), "steps": e2e_steps, "ms_per_step": e2e_s / e2e_steps * 1e3,
-           "entry_point": "sd_verify_feedback_host"}
+    e2e_s = shard.max_over_ranks(time.perf_counter() - t0, device=dev_arg)
+    e2e = {"value": positions * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": int(path.h2d),
+           "d2h_bytes_per_step": int(path.d2h), "steps": e2e_steps, "ms_per_step": e2e_s / e2e_steps * 1e3,
+           "entry_point": path.e2e_entry}
 
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    peak, peak_src = measured_peak_gbs()
-    achieved = cfg.algorithmic_bytes / (mean_kernel_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": NCU_TRAFFIC_BYTES.get(cfg.name) if not args.batch else None, "peak_source": peak_src,
-                "algorithmic_bytes_per_launch": cfg.algorithmic_bytes, "kernel_ms_mean": mean_kernel_ms,
-                "kernel_ms_min": float(np.min(kernel_ms)), "kernel": "sd_stream_kernel" if info["path"] == 1 else "sd_generic_kernel",
-                "frac_of_nominal_8000_GBps": achieved / 8000.0}
-    # second ceiling: the special-function units (4 ex2 per entry pair and 2 per bonus entry; 16 results per
-    # clock and SM, 148 SMs at the maximum SM clock): what binds when entries are 2 bytes
-    ex2 = (4 * cfg.k + 2) * cfg.V * cfg.B
-    sfu_peak = 148 * 16 * 1.965e9
-    roofline["sfu"] = {"ex2_per_launch": ex2, "achieved_per_s": ex2 / (mean_kernel_ms * 1e-3), "peak_per_s": sfu_peak,
-                       "frac": ex2 / (mean_kernel_ms * 1e-3) / sfu_peak,
-                       "peak_source": "148 SMs x 16 ex2/clk x 1965 MHz (nominal unit count and maximum clock)"}
-    base = cpu_baseline(cfg, inp) if not args.no_cpu_baseline else None
+    peaks = measured_peaks()
+    if getattr(path, "bound", "hbm") == "tensor":
+        achieved = path.algorithmic / (mean_kernel_ms * 1e-3) / 1e12
+        long_run = args.steps * mean_kernel_ms > 2000.0
+        peak = peaks["bf16_tflops_sustained"] if long_run else peaks["bf16_tflops"]
+        roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                    "traffic": None, "peak_source": peaks["source"] + (", sustained figure (timed region over 2 s)" if long_run else ", burst figure"),
+                    "flops_per_launch": path.algorithmic, "kernel_ms_mean": mean_kernel_ms,
+                    "kernel_ms_min": float(np.min(kernel_ms)), "kernel": path.kernel}
+    else:
+        achieved = path.algorithmic / (mean_kernel_ms * 1e-3) / 1e9
+        traffic, traffic_source = (None, "not the full-size workload") if args.batch else \
+            captured_traffic(path.traffic_path, cfg.name, getattr(path, "traffic_extra", "-"))
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / peaks["hbm_gbs"], "traffic": traffic, "traffic_source": traffic_source,
+                    "peak_source": peaks["source"], "algorithmic_bytes_per_launch": path.algorithmic,
+                    "kernel_ms_mean": mean_kernel_ms, "kernel_ms_min": float(np.min(kernel_ms)),
+                    "kernel": path.kernel if info["path"] != 0 else "sd_generic_kernel",
+                    "frac_of_nominal_8000_GBps": achieved / 8000.0}
+    base, parity, verified = path.finish(args)
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(3, args.warmup), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32" if cfg.dtype == "f32" else "f32 (bf16 storage)",
-            "data": "synthetic",
-            "config": workload_config(cfg, l2="inputs larger than L2" if nsets == 1 else f"{nsets} rotating input sets larger than L2 together",
+            "warmup": warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": path.dtype, "data": "synthetic",
+            "config": workload_config(cfg, path=args.path,
+                                      l2="inputs larger than L2" if path.nsets == 1 else f"{path.nsets} rotating input sets larger than L2 together",
                                       parallelism=f"replicas x{world}, sequences independent, no collective",
-                                      launch=info),
+                                      launch=info, **path.extra),
             "roofline": roofline, "cpu_baseline": base, "e2e": e2e, "gpu_launches": args.steps * info["kernels"],
-            "clocks": clocks.summary(), "outputs_verified_against_oracle": verified}
+            "clocks": clocks.summary(), "parity": parity, "outputs_verified_against_oracle": verified}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
 
 
-def run_greedy(args, cfg):
-    """--path greedy: sd_verify_greedy on the target logits of the workload, one GPU per rank."""
-    import torch
-    import torch.distributed as dist
-
-    import __graft_entry__ as entry
-    entry.build()
-    from paper_2603_12617_b200 import binding, shard
-
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-    inp = synth.make_inputs(cfg, seed=synth.BASE_SEED + 1000 * rank)
-    hT = torch.from_numpy(inp.target_logits)
-    if inp.target_logits.dtype == np.uint16:
-        hT = hT.view(torch.bfloat16)
-    hT = hT.pin_memory()
-    # greedy drafting proposes the draft's argmax; the inputs carry sampled tokens, which serves as well:
-    # the work does not depend on the tokens
-    hx = torch.from_numpy(inp.draft_tokens).pin_memory()
-    in_bytes = hT.numel() * hT.element_size()
-    nsets = 1 if in_bytes > 2 * L2_BYTES else int(min(64, -(-3 * L2_BYTES // in_bytes)))
-    sets = [(hT.to(dev), hx.to(dev)) for _ in range(nsets)]
-    out = binding.sd_verify_greedy(*sets[0])
-
-    def barrier():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    for i in range(max(3, args.warmup)):
-        binding.sd_verify_greedy(*sets[i % nsets], out=out)
-    info = binding.sd_launch_info()
-    barrier()
-    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with ClockSampler(local) as clocks:
-        t_begin.record()
-        for i in range(args.steps):
-            starts[i].record()
-            binding.sd_verify_greedy(*sets[i % nsets], out=out)
-            ends[i].record()
-        t_end.record()
-        barrier()
-    total_ms = shard.max_over_ranks(t_begin.elapsed_time(t_end), device=str(dev) if world > 1 else "cpu")
-    kernel_ms = [s.elapsed_time(e) for s, e in zip(starts, ends)]
-    mean_kernel_ms = float(np.mean(kernel_ms))
-    positions = cfg.B * cfg.k * world
-    value = positions * args.steps / (total_ms * 1e-3)
-
-    # end to end: pinned host logits in, results back to the host, every copy inside the region
-    e2e_steps = max(1, min(args.steps, 10))
-    dT, dx = torch.empty_like(sets[0][0]), torch.empty_like(sets[0][1])
-    h_n = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
-    h_tok = torch.empty((cfg.B, cfg.k + 1), dtype=torch.int32).pin_memory()
-
-    def e2e_step():
-        dT.copy_(hT, non_blocking=True)
-        dx.copy_(hx, non_blocking=True)
-        binding.sd_verify_greedy(dT, dx, out=out)
-        h_n.copy_(out.accept_len, non_blocking=True)
-        h_tok.copy_(out.tokens, non_blocking=True)
-        torch.cuda.synchronize()
-
-    e2e_step()
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        e2e_step()
-    barrier()
-    e2e_s = shard.max_over_ranks(time.perf_counter() - t0, device=str(dev) if world > 1 else "cpu")
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
-
-    from oracle import sd_oracle
-    t0 = time.perf_counter()
-    ref = sd_oracle.verify_greedy(inp.target_logits, inp.draft_tokens)
-    t_cpu = time.perf_counter() - t0
-    verified = bool((h_n.numpy() == ref.accept_len).all() and (h_tok.numpy() == ref.tokens).all()
-                    and (out.argmax.cpu().numpy() == ref.argmax).all())
-    algo = (cfg.k + 1) * cfg.V * cfg.B * cfg.elem_bytes
-    peak, peak_src = measured_peak_gbs()
-    achieved = algo / (mean_kernel_ms * 1e-3) / 1e9
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(3, args.warmup), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32 comparisons" if cfg.dtype == "f32" else "bf16 comparisons",
-            "data": "synthetic",
-            "config": workload_config(cfg, path="greedy", l2="inputs larger than L2" if nsets == 1 else f"{nsets} rotating input sets larger than L2 together",
-                                      parallelism=f"replicas x{world}, sequences independent, no collective", launch=info),
-            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": NCU_TRAFFIC_GREEDY.get(cfg.name) if not args.batch else None,
-                         "peak_source": peak_src, "algorithmic_bytes_per_launch": algo,
-                         "kernel_ms_mean": mean_kernel_ms, "kernel_ms_min": float(np.min(kernel_ms)),
-                         "kernel": "sd_greedy_kernel"},
-            "cpu_baseline": {"value": cfg.B * cfg.k / t_cpu, "unit": UNIT, "cores": 1, "kind": "oracle",
-                             "sample": f"all {cfg.B} sequences of {cfg.name}, one call, {t_cpu:.2f} s"},
-            "e2e": {"value": positions * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": int(in_bytes + hx.numel() * 4),
-                    "d2h_bytes_per_step": int(h_n.numel() * 4 + h_tok.numel() * 4), "steps": e2e_steps,
-                    "ms_per_step": e2e_s / e2e_steps * 1e3, "entry_point": "sd_verify_greedy between pinned-memory copies"},
-            "gpu_launches": args.steps * info["kernels"], "clocks": clocks.summary(),
-            "outputs_verified_against_oracle": verified}
-    print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+# ------------------------------------------------------------------------------------------
+def free_port() -> int:
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
 
 
-def run_errors(args, cfg):
-    """--path errors: sd_verify_error_feedback on the workload, one GPU per rank."""
-    import torch
-    import torch.distributed as dist
-
-    import __graft_entry__ as entry
-    entry.build()
-    from paper_2603_12617_b200 import binding, shard
-
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-    inp = synth.make_inputs(cfg, seed=synth.BASE_SEED + 1000 * rank)
-
-    def as_torch(a):
-        t = torch.from_numpy(a)
-        return t.view(torch.bfloat16) if a.dtype == np.uint16 else t
-
-    hT, hD = as_torch(inp.target_logits).pin_memory(), as_torch(inp.draft_logits).pin_memory()
-    hx, hu = torch.from_numpy(inp.draft_tokens).pin_memory(), torch.from_numpy(inp.uniforms).pin_memory()
-    in_bytes = hT.numel() * hT.element_size() + hD.numel() * hD.element_size()
-    nsets = 1 if in_bytes > 2 * L2_BYTES else int(min(64, -(-3 * L2_BYTES // in_bytes)))
-    sets = [(hT.to(dev), hD.to(dev), hx.to(dev), hu.to(dev)) for _ in range(nsets)]
-    out = binding.sd_verify_error_feedback(*sets[0], inp.tau)
-
-    def barrier():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    for i in range(max(3, args.warmup)):
-        binding.sd_verify_error_feedback(*sets[i % nsets], inp.tau, out=out)
-    info = binding.sd_launch_info()
-    barrier()
-    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with ClockSampler(local) as clocks:
-        t_begin.record()
-        for i in range(args.steps):
-            starts[i].record()
-            binding.sd_verify_error_feedback(*sets[i % nsets], inp.tau, out=out)
-            ends[i].record()
-        t_end.record()
-        barrier()
-    total_ms = shard.max_over_ranks(t_begin.elapsed_time(t_end), device=str(dev) if world > 1 else "cpu")
-    kernel_ms = [s.elapsed_time(e) for s, e in zip(starts, ends)]
-    mean_kernel_ms = float(np.mean(kernel_ms))
-    positions = cfg.B * cfg.k * world
-    value = positions * args.steps / (total_ms * 1e-3)
-
-    # end to end: pinned host logits in, results and the gradient rows back to the host
-    e2e_steps = max(1, min(args.steps, 10))
-    dbuf = [torch.empty_like(t) for t in sets[0]]
-    h_n = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
-    h_tok = torch.empty((cfg.B, cfg.k + 1), dtype=torch.int32).pin_memory()
-    h_loss = torch.empty((cfg.B, cfg.k), dtype=torch.float32).pin_memory()
-    h_g = torch.empty((cfg.B, cfg.V), dtype=hT.dtype).pin_memory()
-
-    def e2e_step():
-        for a, b in zip(dbuf, (hT, hD, hx, hu)):
-            a.copy_(b, non_blocking=True)
-        binding.sd_verify_error_feedback(*dbuf, inp.tau, out=out)
-        h_n.copy_(out.accept_len, non_blocking=True)
-        h_tok.copy_(out.tokens, non_blocking=True)
-        h_loss.copy_(out.loss, non_blocking=True)
-        h_g.copy_(out.error_grad, non_blocking=True)
-        torch.cuda.synchronize()
-
-    e2e_step()
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        e2e_step()
-    barrier()
-    e2e_s = shard.max_over_ranks(time.perf_counter() - t0, device=str(dev) if world > 1 else "cpu")
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
-
-    from oracle import sd_oracle
-    cores = min(sd_oracle.max_threads(), os.cpu_count() or 1)
-    nseq = min(cfg.B, cores)
-    sl = np.arange(nseq)
-    t0 = time.perf_counter()
-    ref = sd_oracle.error_position_feedback(inp.target_logits[sl], inp.draft_logits[sl], inp.draft_tokens[sl],
-                                            inp.uniforms[sl], inp.tau, nthreads=cores)
-    t_cpu = time.perf_counter() - t0
-    safe = (ref.full.accept_band.sum(1) == 0) & (ref.full.cdf_margin > 1e-6)
-    g = h_g[:nseq].float().numpy().astype(np.float64)
-    tol = 2e-2 if cfg.dtype == "bf16" else 1e-5
-    verified = bool((h_n.numpy()[sl][safe] == ref.full.accept_len[safe]).all()
-                    and (h_tok.numpy()[sl][safe] == ref.full.tokens[safe]).all()
-                    and np.allclose(h_loss.numpy()[sl], ref.full.loss, rtol=tol, atol=4e-7)
-                    and all(np.abs(g[b] - ref.error_grad[b]).max() <= tol * np.abs(ref.error_grad[b]).max() + 1e-6
-                            for b in range(nseq) if safe[b]))
-    s = cfg.elem_bytes
-    algo = ((2 * cfg.k + 1) + 1) * cfg.V * cfg.B * s
-    peak, peak_src = measured_peak_gbs()
-    achieved = algo / (mean_kernel_ms * 1e-3) / 1e9
-    d2h = h_n.numel() * 4 + h_tok.numel() * 4 + h_loss.numel() * 4 + h_g.numel() * h_g.element_size()
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(3, args.warmup), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32" if cfg.dtype == "f32" else "f32 (bf16 storage)",
-            "data": "synthetic",
-            "config": workload_config(cfg, path="errors", mean_accept_len=float(h_n.float().mean()),
-                                      l2="inputs larger than L2" if nsets == 1 else f"{nsets} rotating input sets larger than L2 together",
-                                      parallelism=f"replicas x{world}, sequences independent, no collective", launch=info),
-            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": NCU_TRAFFIC_ERRORS.get(cfg.name) if not args.batch else None,
-                         "peak_source": peak_src, "algorithmic_bytes_per_launch": algo,
-                         "kernel_ms_mean": mean_kernel_ms, "kernel_ms_min": float(np.min(kernel_ms)),
-                         "kernel": "sd_stream_kernel<pass 1 only> + sd_errpos_kernel"},
-            "cpu_baseline": {"value": nseq * cfg.k / t_cpu, "unit": UNIT, "cores": cores, "kind": "oracle",
-                             "sample": f"{nseq} of {cfg.B} sequences of {cfg.name}, one call, {t_cpu:.2f} s"},
-            "e2e": {"value": positions * e2e_steps / e2e_s, "unit": UNIT,
-                    "h2d_bytes_per_step": int(in_bytes + hx.numel() * 4 + hu.numel() * 4), "d2h_bytes_per_step": int(d2h),
-                    "steps": e2e_steps, "ms_per_step": e2e_s / e2e_steps * 1e3,
-                    "entry_point": "sd_verify_error_feedback between pinned-memory copies"},
-            "gpu_launches": args.steps * info["kernels"], "clocks": clocks.summary(),
-            "outputs_verified_against_oracle": verified}
-    print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+def launcher_command(argv, gpus: int, port: int):
+    """The command that starts one rank per GPU on this node for `python bench.py <argv>`."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={gpus}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
 
 
-def run_ensemble(args, cfg):
-    """--path ensemble: sd_ensemble_feedback with N learners on the workload, one GPU per rank."""
-    import torch
-    import torch.distributed as dist
-
-    import __graft_entry__ as entry
-    entry.build()
-    from paper_2603_12617_b200 import binding, shard
-
-    N = args.learners
-    eps = 10.0
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-    inp = synth.make_inputs(cfg, seed=synth.BASE_SEED + 1000 * rank)
-    drafts = synth.ensemble_drafts(inp, N, seed=synth.BASE_SEED + 1000 * rank)
-
-    def as_torch(a):
-        t = torch.from_numpy(a)
-        return t.view(torch.bfloat16) if a.dtype == np.uint16 else t
-
-    hT = as_torch(inp.target_logits).pin_memory()
-    hD = [as_torch(d).pin_memory() for d in drafts]
-    in_bytes = hT.numel() * hT.element_size() + sum(d.numel() * d.element_size() for d in hD)
-    nsets = 1 if in_bytes > 2 * L2_BYTES else int(min(64, -(-3 * L2_BYTES // in_bytes)))
-    sets = [(hT.to(dev), [d.to(dev) for d in hD]) for _ in range(nsets)]
-    out = binding.sd_ensemble_feedback(sets[0][0], sets[0][1], inp.tau, eps)
-    cum = torch.zeros(N, dtype=torch.float64, device=dev)
-
-    def step(i):
-        T, Ds = sets[i % nsets]
-        binding.sd_ensemble_feedback(T, Ds, inp.tau, eps, cum_loss=cum, out=out)
-
-    def barrier():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    for i in range(max(3, args.warmup)):
-        step(i)
-    info = binding.sd_launch_info()
-    barrier()
-    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with ClockSampler(local) as clocks:
-        t_begin.record()
-        for i in range(args.steps):
-            starts[i].record()
-            step(i)
-            ends[i].record()
-        t_end.record()
-        barrier()
-    total_ms = shard.max_over_ranks(t_begin.elapsed_time(t_end), device=str(dev) if world > 1 else "cpu")
-    kernel_ms = [s.elapsed_time(e) for s, e in zip(starts, ends)]
-    mean_kernel_ms = float(np.mean(kernel_ms))
-    positions = cfg.B * cfg.k * world
-    value = positions * args.steps / (total_ms * 1e-3)
-
-    # end to end: pinned host logits in, losses, weights and gradients back to the host
-    e2e_steps = max(1, min(args.steps, 5))
-    dT, dD = torch.empty_like(sets[0][0]), [torch.empty_like(d) for d in sets[0][1]]
-    h_loss = torch.empty((N, cfg.B, cfg.k), dtype=torch.float32).pin_memory()
-    h_w = torch.empty(N, dtype=torch.float32).pin_memory()
-    h_grad = [torch.empty_like(d).pin_memory() for d in hD]
-
-    def e2e_step():
-        dT.copy_(hT, non_blocking=True)
-        for a, b in zip(dD, hD):
-            a.copy_(b, non_blocking=True)
-        binding.sd_ensemble_feedback(dT, dD, inp.tau, eps, cum_loss=cum, out=out)
-        h_loss.copy_(out.loss, non_blocking=True)
-        h_w.copy_(out.weights, non_blocking=True)
-        for a, b in zip(h_grad, out.grad):
-            a.copy_(b, non_blocking=True)
-        torch.cuda.synchronize()
-
-    e2e_step()
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        e2e_step()
-    barrier()
-    e2e_s = shard.max_over_ranks(time.perf_counter() - t0, device=str(dev) if world > 1 else "cpu")
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
-
-    # the timed outputs against the oracle on a few sequences, and the oracle's own speed
-    from oracle import sd_oracle
-    cores = min(sd_oracle.max_threads(), os.cpu_count() or 1)
-    nseq = min(cfg.B, max(1, cores // cfg.k))
-    sl = np.arange(nseq)
-    t0 = time.perf_counter()
-    ref = sd_oracle.ensemble_feedback(inp.target_logits[sl], [d[sl] for d in drafts], inp.tau, eps, want_grad=False,
-                                      nthreads=cores)
-    t_cpu = time.perf_counter() - t0
-    loss = h_loss.numpy()[:, :nseq].astype(np.float64)
-    verified = bool(np.allclose(loss, ref.loss, rtol=2e-2 if cfg.dtype == "bf16" else 1e-5, atol=4e-7)
-                    and abs(float(h_w.sum()) - 1.0) < 1e-5)
-    s = cfg.elem_bytes
-    algo = ((cfg.k + N * cfg.k) + N * cfg.k) * cfg.V * cfg.B * s
-    d2h = h_loss.numel() * 4 + h_w.numel() * 4 + sum(g.numel() * g.element_size() for g in h_grad)
-    peak, peak_src = measured_peak_gbs()
-    achieved = algo / (mean_kernel_ms * 1e-3) / 1e9
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(3, args.warmup), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32" if cfg.dtype == "f32" else "f32 (bf16 storage)",
-            "data": "synthetic",
-            "config": workload_config(cfg, path="ensemble", learners=N, epsilon=eps,
-                                      l2="inputs larger than L2" if nsets == 1 else f"{nsets} rotating input sets larger than L2 together",
-                                      parallelism=f"replicas x{world}, sequences independent, no collective", launch=info),
-            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": NCU_TRAFFIC_ENSEMBLE.get((cfg.name, N)) if not args.batch else None,
-                         "peak_source": peak_src, "algorithmic_bytes_per_launch": algo,
-                         "kernel_ms_mean": mean_kernel_ms, "kernel_ms_min": float(np.min(kernel_ms)),
-                         "kernel": "sd_stream_kernel<ensemble> + sd_hedge_kernel"},
-            "cpu_baseline": {"value": nseq * cfg.k / t_cpu, "unit": UNIT, "cores": cores, "kind": "oracle",
-                             "sample": f"{nseq} of {cfg.B} sequences of {cfg.name}, {N} learners, no gradients, "
-                                       f"one call, {t_cpu:.2f} s"},
-            "e2e": {"value": positions * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": int(in_bytes),
-                    "d2h_bytes_per_step": int(d2h), "steps": e2e_steps, "ms_per_step": e2e_s / e2e_steps * 1e3,
-                    "entry_point": "sd_ensemble_feedback between pinned-memory copies"},
-            "gpu_launches": args.steps * info["kernels"], "clocks": clocks.summary(),
-            "outputs_verified_against_oracle": verified}
-    print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
-
-
-def main():
+def main(argv=None):
+    argv = sys.argv[1:] if argv is None else argv
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
@@ -726,23 +690,22 @@ def main():
     ap.add_argument("--config", default="cfg5", choices=sorted(synth.CONFIGS))
     ap.add_argument("--batch", type=int, default=0, help="override B (profiling on a smaller case)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--path", choices=["sample", "greedy", "ensemble", "errors"], default="sample",
-                    help="sample: the verify-and-feedback step (the headline); greedy: greedy verification; "
-                         "ensemble: feedback of an online ensemble of draft models; errors: feedback at the error position only")
+    ap.add_argument("--path", choices=sorted(PATHS), default="sample",
+                    help="sample: the verify-and-feedback step (the headline); the others: see the module text")
     ap.add_argument("--learners", type=int, default=3, help="draft models of --path ensemble")
-    ap.add_argument("--times-out", default="", help="write the per-step device times (ms) of the headline path here")
-    args = ap.parse_args()
+    ap.add_argument("--features", type=int, default=4096, help="width d of the output layer of --path lmhead")
+    ap.add_argument("--times-out", default="", help="write the per-step device times (ms) here")
+    args = ap.parse_args(argv)
     cfg = synth.CONFIGS[args.config]
     if args.batch:
         cfg = cfg.with_batch(args.batch)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # not started by torch.distributed.run: start one rank per GPU ourselves (the ranks print; rank 0 the line)
+        env = dict(os.environ)
+        env.setdefault("NCCL_DEBUG", "INFO")      # the communicator's rank count shows in the log (stderr)
+        raise SystemExit(subprocess.call(launcher_command(argv, args.gpus, free_port()), env=env))
     if args.impl == "reference":
         run_reference(args, cfg)
-    elif args.path == "greedy":
-        run_greedy(args, cfg)
-    elif args.path == "ensemble":
-        run_ensemble(args, cfg)
-    elif args.path == "errors":
-        run_errors(args, cfg)
     else:
         run_ours(args, cfg)
 

@@ -194,3 +194,14 @@ def ensemble_drafts(inp: Inputs, n_learners: int, seed: int = BASE_SEED) -> list
         D = Tf + noise
         out.append(f32_to_bf16_bits(D) if cfg.dtype == "bf16" else D.astype(np.float32))
     return out
+
+
+def lmhead_operands(R: int, V: int, d: int, seed: int = BASE_SEED):
+    """Operands of the output layer's gradient dW = g^T X as bf16 bit patterns: g [R,V] shaped like a
+    gradient with respect to logits (most entries tiny, a few large per row), X [R,d] ~ N(0,1)."""
+    rng = np.random.Generator(np.random.Philox(key=[seed & (2**64 - 1), 77]))
+    g = rng.standard_normal((R, V), dtype=np.float32) * np.float32(1e-3)
+    hot = rng.integers(0, V, (R, 3))
+    g[np.arange(R)[:, None], hot] += rng.standard_normal((R, 3), dtype=np.float32) * np.float32(0.3)
+    X = rng.standard_normal((R, d), dtype=np.float32)
+    return f32_to_bf16_bits(g), f32_to_bf16_bits(X)
