@@ -273,6 +273,52 @@ int sd_verify_error_feedback(const void* target_logits, const void* draft_logits
                              size_t workspace_bytes, void* stream);
 
 /*
+ * Vocabulary-parallel step -- the step of sd_verify_feedback for logits that are sharded along the
+ * vocabulary, as a tensor-parallel output layer leaves them (the paper's deployment spreads a model
+ * over four GPUs, Sec. 4.1 "Implementation Details").  Rank g of G holds the columns
+ * [v_offset, v_offset + V_shard) of every row of both logit tensors; draft tokens, uniforms and
+ * temperature are the same on every rank.  A softmax needs every column, so the step is three local
+ * calls with an exchange after each; the library makes no collective call itself -- the caller
+ * gathers with NCCL (or, on one GPU, by concatenation: no call waits for another rank).
+ *
+ *   sd_vp_partial   phase 1: per row the shard's softmax sums and, where the shard holds it, the
+ *                   logits of the drafted token: out_records [B*(k+1)] records of SD_VP_RECORD_BYTES.
+ *   exchange        all-gather the records: all_records [G][B*(k+1)], in rank order.
+ *   sd_vp_finish    phase 2: merges the records (same bits on every rank), then out_accept_len [B],
+ *                   out_loss [B,k] (or NULL), out_status [B] (or NULL) -- identical on every rank --,
+ *                   the shard's columns of the gradient out_grad_shard [B,k,V_shard] (or NULL), and
+ *                   out_local_mass [B][2] (double): the shard's share of the mass of the distribution the
+ *                   extra token is drawn from (residual of row n_b, or the bonus row), and of the mass of
+ *                   p_{n_b} (what a residual without mass falls back to).
+ *   exchange        all-gather the shares: all_masses [G][B][2], in rank order.
+ *   sd_vp_draw      phase 3: out_tokens [B,k+1]: the accepted draft tokens, then the extra token if this
+ *                   rank's shard holds it (global index) and -1 otherwise, then -1 padding.
+ *   exchange        element-wise maximum of out_tokens over the ranks.
+ *
+ * The same workspace (sd_vp_workspace_bytes, 256-byte aligned) must be passed to all three calls of
+ * a round; it carries the row constants and region masses from phase 2 to phase 3.  Cuts must fall on
+ * 16-byte boundaries (V_shard * element size a multiple of 16, shards 16-byte aligned): SD_ERR_ALIGN
+ * otherwise.  Shards may differ in width.  A rejection whose residual has no mass on any rank (only a
+ * forced rejection with q = p produces one) sets SD_STATUS_ZERO_RESIDUAL and draws from p_{n_b} instead,
+ * as sd_verify_feedback does.
+ * Every logit is read from HBM twice (once per phase).
+ */
+#define SD_VP_RECORD_BYTES 48
+size_t sd_vp_workspace_bytes(int B, int k, int V_shard, int dtype);
+int sd_vp_partial(const void* target_shard, const void* draft_shard, const int32_t* draft_tokens, float temperature,
+                  int B, int k, int V_shard, int v_offset, int V_total, int dtype, void* out_records, void* workspace,
+                  size_t workspace_bytes, void* stream);
+int sd_vp_finish(const void* target_shard, const void* draft_shard, const int32_t* draft_tokens, const float* uniforms,
+                 float temperature, int B, int k, int V_shard, int v_offset, int V_total, int dtype,
+                 const void* all_records, int n_ranks, int rank, int32_t* out_accept_len, float* out_loss,
+                 void* out_grad_shard, double* out_local_mass, uint32_t* out_status, void* workspace,
+                 size_t workspace_bytes, void* stream);
+int sd_vp_draw(const void* target_shard, const void* draft_shard, const int32_t* draft_tokens, const float* uniforms,
+               float temperature, int B, int k, int V_shard, int v_offset, int V_total, int dtype,
+               const int32_t* accept_len, const double* all_masses, int n_ranks, int rank, int32_t* out_tokens,
+               uint32_t* out_status, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * sd_lmhead_grad -- the step after the feedback: the gradient of the round's loss with respect to
  * the weights W [V,d] of the draft model's linear output layer.  The feedback gradient of Sec. 3.1
  * ("nabla f_t(w_t)") reaches the parameters through the chain rule; with draft logits
@@ -348,7 +394,7 @@ long long sd_get_option(int option_id);
 
 /*
  * sd_launch_info -- HOST out-parameters describing how the last successful device call on this
- * thread was launched: path (0 = generic, 1 = stream fast path, 2 = greedy verification, 3 = ensemble feedback, 4 = error-position feedback, 5 = output-layer gradient), cluster size, threads per
+ * thread was launched: path (0 = generic, 1 = stream fast path, 2 = greedy verification, 3 = ensemble feedback, 4 = error-position feedback, 5 = output-layer gradient, 6 = vocabulary-parallel step), cluster size, threads per
  * block, dynamic shared memory per block, blocks launched, kernels launched.  Any pointer may
  * be NULL.  Diagnostic only.
  */

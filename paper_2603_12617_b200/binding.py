@@ -69,6 +69,14 @@ def _load() -> ctypes.CDLL:
                                          P, Z, P]
     lib.sd_lmhead_grad.restype = I
     lib.sd_lmhead_grad.argtypes = [P, P, I, I, I, P, P, P]
+    lib.sd_vp_workspace_bytes.restype = Z
+    lib.sd_vp_workspace_bytes.argtypes = [I, I, I, I]
+    lib.sd_vp_partial.restype = I
+    lib.sd_vp_partial.argtypes = [P, P, P, F, I, I, I, I, I, I, P, P, Z, P]
+    lib.sd_vp_finish.restype = I
+    lib.sd_vp_finish.argtypes = [P, P, P, P, F, I, I, I, I, I, I, P, I, I, P, P, P, P, P, P, Z, P]
+    lib.sd_vp_draw.restype = I
+    lib.sd_vp_draw.argtypes = [P, P, P, P, F, I, I, I, I, I, I, P, P, I, I, P, P, P, Z, P]
     lib.sd_verify_feedback_host.restype = I
     lib.sd_verify_feedback_host.argtypes = [P, P, P, P, F, I, I, I, I, P, P, P, P, P, P]
     lib.sd_workspace_bytes.restype = Z
@@ -378,6 +386,94 @@ def sd_lmhead_grad(grad_logits: torch.Tensor, hidden: torch.Tensor, *, out: Opti
 
 
 SD_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
+
+
+SD_VP_RECORD_BYTES = 48
+
+
+def sd_vp_workspace_bytes(B: int, k: int, V_shard: int, dtype: int) -> int:
+    return int(_lib.sd_vp_workspace_bytes(B, k, V_shard, dtype))
+
+
+def _vp_shapes(target_shard, draft_shard, draft_tokens):
+    if target_shard.dim() != 3 or draft_shard.dim() != 3:
+        raise ValueError("shards must be [B,k+1,V_shard] and [B,k,V_shard]")
+    B, k1, Vs = target_shard.shape
+    k = k1 - 1
+    if tuple(draft_shard.shape) != (B, k, Vs) or tuple(draft_tokens.shape) != (B, k):
+        raise ValueError("shape mismatch between the shards and the draft tokens")
+    if target_shard.dtype != draft_shard.dtype:
+        raise TypeError("target and draft shards must have the same dtype")
+    for t in (target_shard, draft_shard, draft_tokens):
+        if not t.is_cuda or not t.is_contiguous():
+            raise ValueError("device-resident contiguous tensors expected")
+    return B, k, Vs
+
+
+def sd_vp_partial(target_shard: torch.Tensor, draft_shard: torch.Tensor, draft_tokens: torch.Tensor,
+                  temperature: float, v_offset: int, V_total: int, workspace: torch.Tensor, *,
+                  out_records: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """Phase 1 of the vocabulary-parallel step: this shard's record of every row, [B*(k+1), 48] bytes."""
+    B, k, Vs = _vp_shapes(target_shard, draft_shard, draft_tokens)
+    if out_records is None:
+        out_records = torch.empty((B * (k + 1), SD_VP_RECORD_BYTES), dtype=torch.uint8, device=target_shard.device)
+    rc = _lib.sd_vp_partial(_ptr(target_shard), _ptr(draft_shard), _ptr(draft_tokens), float(temperature), B, k, Vs,
+                            int(v_offset), int(V_total), _dtype_code(target_shard), _ptr(out_records), _ptr(workspace),
+                            workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    if rc != 0:
+        raise SdVerifyError(rc, "sd_vp_partial")
+    return out_records
+
+
+@dataclass
+class VpFinishOutputs:
+    accept_len: torch.Tensor            # [B] int32, the same on every rank
+    loss: Optional[torch.Tensor]        # [B,k] float32, the same on every rank
+    grad_shard: Optional[torch.Tensor]  # [B,k,V_shard]
+    local_mass: torch.Tensor            # [B,2] float64
+    status: torch.Tensor                # [B] int32 view of the status words
+
+
+def sd_vp_finish(target_shard: torch.Tensor, draft_shard: torch.Tensor, draft_tokens: torch.Tensor,
+                 uniforms: torch.Tensor, temperature: float, v_offset: int, V_total: int, all_records: torch.Tensor,
+                 n_ranks: int, rank: int, workspace: torch.Tensor, *, want_loss: bool = True, want_grad: bool = True,
+                 stream: Optional[torch.cuda.Stream] = None) -> VpFinishOutputs:
+    """Phase 2: ``all_records`` is the rank-ordered gather [n_ranks, B*(k+1), 48] of phase 1's records."""
+    B, k, Vs = _vp_shapes(target_shard, draft_shard, draft_tokens)
+    if all_records.numel() * all_records.element_size() != n_ranks * B * (k + 1) * SD_VP_RECORD_BYTES:
+        raise ValueError("all_records must hold n_ranks * B * (k+1) records")
+    dev = target_shard.device
+    accept_len = torch.empty((B,), dtype=torch.int32, device=dev)
+    loss = torch.empty((B, k), dtype=torch.float32, device=dev) if want_loss else None
+    grad = torch.empty_like(draft_shard) if want_grad else None
+    mass = torch.empty((B, 2), dtype=torch.float64, device=dev)
+    status = torch.empty((B,), dtype=torch.int32, device=dev)
+    rc = _lib.sd_vp_finish(_ptr(target_shard), _ptr(draft_shard), _ptr(draft_tokens), _ptr(uniforms), float(temperature),
+                           B, k, Vs, int(v_offset), int(V_total), _dtype_code(target_shard), _ptr(all_records),
+                           int(n_ranks), int(rank), _ptr(accept_len), _ptr(loss), _ptr(grad), _ptr(mass), _ptr(status),
+                           _ptr(workspace), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    if rc != 0:
+        raise SdVerifyError(rc, "sd_vp_finish")
+    return VpFinishOutputs(accept_len, loss, grad, mass, status)
+
+
+def sd_vp_draw(target_shard: torch.Tensor, draft_shard: torch.Tensor, draft_tokens: torch.Tensor,
+               uniforms: torch.Tensor, temperature: float, v_offset: int, V_total: int, accept_len: torch.Tensor,
+               all_masses: torch.Tensor, n_ranks: int, rank: int, status: torch.Tensor, workspace: torch.Tensor, *,
+               stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """Phase 3: ``all_masses`` is the rank-ordered gather [n_ranks, B, 2] of phase 2's shares.  Returns
+    tokens [B,k+1] with -1 where another rank's shard holds the extra token."""
+    B, k, Vs = _vp_shapes(target_shard, draft_shard, draft_tokens)
+    if all_masses.dtype != torch.float64 or all_masses.numel() != n_ranks * B * 2:
+        raise ValueError("all_masses must be float64 [n_ranks, B, 2]")
+    tokens = torch.empty((B, k + 1), dtype=torch.int32, device=target_shard.device)
+    rc = _lib.sd_vp_draw(_ptr(target_shard), _ptr(draft_shard), _ptr(draft_tokens), _ptr(uniforms), float(temperature),
+                         B, k, Vs, int(v_offset), int(V_total), _dtype_code(target_shard), _ptr(accept_len),
+                         _ptr(all_masses), int(n_ranks), int(rank), _ptr(tokens), _ptr(status), _ptr(workspace),
+                         workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    if rc != 0:
+        raise SdVerifyError(rc, "sd_vp_draw")
+    return tokens
 
 
 def sd_verify_feedback_static(target_logits: torch.Tensor, draft_logits: torch.Tensor,

@@ -11,6 +11,7 @@
 #include "sd_greedy.cuh"
 #include "sd_errpos.cuh"
 #include "sd_lmhead.cuh"
+#include "sd_vocab_parallel.cuh"
 
 namespace {
 
@@ -874,6 +875,143 @@ int sd_verify_feedback_host(const void* target_logits, const void* draft_logits,
     if (e2 != cudaSuccess) return cuda_fail(e2, "cudaStreamSynchronize(compute)");
     if (e3 != cudaSuccess) return cuda_fail(e3, "cudaStreamSynchronize(d2h)");
     tl_info[5] = kernels;
+    return SD_OK;
+}
+
+// ---- vocabulary-parallel step ------------------------------------------------------------------
+namespace {
+struct VpLayout { size_t rowc, region_sums, total; int NR; };
+VpLayout vp_layout(int B, int k, int Vs, int dtype) {
+    VpLayout L;
+    const int NV = Vs / vec_elems(dtype);
+    L.NR = (NV + kRegionVecs - 1) / kRegionVecs;
+    size_t off = 0;
+    L.rowc = off;        off = align_up(off + (size_t)B * (k + 1) * sizeof(RowConst), kAlign);
+    L.region_sums = off; off = align_up(off + (size_t)B * 2 * L.NR * 4, kAlign);
+    L.total = off;
+    return L;
+}
+int vp_check(const void* T, const void* D, const int32_t* x, float tau, int B, int k, int Vs, int v_offset, int V_total,
+             int dtype, const void* ws, size_t ws_bytes) {
+    if (dtype != SD_DTYPE_F32 && dtype != SD_DTYPE_BF16) return SD_ERR_DTYPE;
+    if (!T || !D || !x) return SD_ERR_NULL;
+    if (!shape_ok(B, k, Vs) || V_total < Vs || v_offset < 0 || v_offset > V_total - Vs) return SD_ERR_SHAPE;
+    if (!(tau > 0.f) || !isfinite(tau)) return SD_ERR_TEMPERATURE;
+    if (((size_t)Vs * elem_bytes(dtype)) % 16 != 0 || !aligned(T, 16) || !aligned(D, 16) || !aligned(x, 4)) return SD_ERR_ALIGN;
+    if (!ws || !aligned(ws, kAlign) || ws_bytes < vp_layout(B, k, Vs, dtype).total) return SD_ERR_WORKSPACE;
+    return SD_OK;
+}
+VpParams vp_params(const void* T, const void* D, const int32_t* x, const float* u, float tau, int B, int k, int Vs,
+                   int v_offset, int V_total, int dtype, int G, int rank, unsigned char* ws) {
+    VpParams P;
+    memset(&P, 0, sizeof P);
+    const VpLayout L = vp_layout(B, k, Vs, dtype);
+    P.T = T; P.D = D; P.x = x; P.u = u;
+    P.B = B; P.k = k; P.Vs = Vs; P.v_offset = v_offset; P.V_total = V_total;
+    P.G = G; P.rank = rank;
+    P.c = (float)(1.4426950408889634 / (double)tau);
+    P.tau = tau;
+    P.inv_tau = 1.0 / (double)tau;
+    P.NR = L.NR;
+    P.rowc = reinterpret_cast<RowConst*>(ws + L.rowc);
+    P.region_sums = reinterpret_cast<float*>(ws + L.region_sums);
+    return P;
+}
+}  // namespace
+
+size_t sd_vp_workspace_bytes(int B, int k, int V_shard, int dtype) {
+    if ((dtype != SD_DTYPE_F32 && dtype != SD_DTYPE_BF16) || !shape_ok(B, k, V_shard)) return 0;
+    return vp_layout(B, k, V_shard, dtype).total;
+}
+
+int sd_vp_partial(const void* target_shard, const void* draft_shard, const int32_t* draft_tokens, float temperature,
+                  int B, int k, int V_shard, int v_offset, int V_total, int dtype, void* out_records, void* workspace,
+                  size_t workspace_bytes, void* stream) {
+    int rc = vp_check(target_shard, draft_shard, draft_tokens, temperature, B, k, V_shard, v_offset, V_total, dtype,
+                      workspace, workspace_bytes);
+    if (rc != SD_OK) return rc;
+    if (!out_records) return SD_ERR_NULL;
+    if (!aligned(out_records, 16)) return SD_ERR_ALIGN;
+    int dev;
+    DeviceState* ds = nullptr;
+    rc = current_device(&dev, &ds);
+    if (rc != SD_OK) return rc;
+    VpParams P = vp_params(target_shard, draft_shard, draft_tokens, nullptr, temperature, B, k, V_shard, v_offset, V_total,
+                           dtype, 1, 0, static_cast<unsigned char*>(workspace));
+    P.records = static_cast<VpRecord*>(out_records);
+    const unsigned units = (unsigned)B * (unsigned)(k + 1);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (dtype == SD_DTYPE_F32) sd_vp_stats_kernel<SD_DTYPE_F32><<<units, kVpThreads, 0, st>>>(P);
+    else                       sd_vp_stats_kernel<SD_DTYPE_BF16><<<units, kVpThreads, 0, st>>>(P);
+    SD_CUDA(cudaGetLastError());
+    tl_info[0] = 6; tl_info[1] = 1; tl_info[2] = kVpThreads; tl_info[3] = 0; tl_info[4] = (int)units; tl_info[5] = 1;
+    return SD_OK;
+}
+
+int sd_vp_finish(const void* target_shard, const void* draft_shard, const int32_t* draft_tokens, const float* uniforms,
+                 float temperature, int B, int k, int V_shard, int v_offset, int V_total, int dtype,
+                 const void* all_records, int n_ranks, int rank, int32_t* out_accept_len, float* out_loss,
+                 void* out_grad_shard, double* out_local_mass, uint32_t* out_status, void* workspace,
+                 size_t workspace_bytes, void* stream) {
+    int rc = vp_check(target_shard, draft_shard, draft_tokens, temperature, B, k, V_shard, v_offset, V_total, dtype,
+                      workspace, workspace_bytes);
+    if (rc != SD_OK) return rc;
+    if (!uniforms || !all_records || !out_accept_len || !out_local_mass) return SD_ERR_NULL;
+    if (n_ranks < 1 || rank < 0 || rank >= n_ranks) return SD_ERR_SHAPE;
+    if (!aligned(all_records, 16) || !aligned(uniforms, 4) || !aligned(out_accept_len, 4) || !aligned(out_local_mass, 8) ||
+        (out_loss && !aligned(out_loss, 4)) || (out_grad_shard && !aligned(out_grad_shard, 16)) ||
+        (out_status && !aligned(out_status, 4)))
+        return SD_ERR_ALIGN;
+    int dev;
+    DeviceState* ds = nullptr;
+    rc = current_device(&dev, &ds);
+    if (rc != SD_OK) return rc;
+    VpParams P = vp_params(target_shard, draft_shard, draft_tokens, uniforms, temperature, B, k, V_shard, v_offset, V_total,
+                           dtype, n_ranks, rank, static_cast<unsigned char*>(workspace));
+    P.all = static_cast<const VpRecord*>(all_records);
+    P.accept_len = out_accept_len;
+    P.loss = out_loss;
+    P.grad = out_grad_shard;
+    P.status = out_status;
+    P.local_mass = out_local_mass;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    sd_vp_rows_kernel<<<(unsigned)B, 96, 0, st>>>(P);
+    const int slices = (P.NR + kVpSliceRegions - 1) / kVpSliceRegions;
+    const unsigned grid = (unsigned)B * (unsigned)(k + 1) * (unsigned)slices;
+    if (dtype == SD_DTYPE_F32) sd_vp_grad_kernel<SD_DTYPE_F32><<<grid, kVpThreads, 0, st>>>(P, slices);
+    else                       sd_vp_grad_kernel<SD_DTYPE_BF16><<<grid, kVpThreads, 0, st>>>(P, slices);
+    sd_vp_mass_kernel<<<(unsigned)B, 32, 0, st>>>(P);
+    SD_CUDA(cudaGetLastError());
+    tl_info[0] = 6; tl_info[1] = 1; tl_info[2] = kVpThreads; tl_info[3] = 0; tl_info[4] = (int)grid; tl_info[5] = 3;
+    return SD_OK;
+}
+
+int sd_vp_draw(const void* target_shard, const void* draft_shard, const int32_t* draft_tokens, const float* uniforms,
+               float temperature, int B, int k, int V_shard, int v_offset, int V_total, int dtype,
+               const int32_t* accept_len, const double* all_masses, int n_ranks, int rank, int32_t* out_tokens,
+               uint32_t* out_status, void* workspace, size_t workspace_bytes, void* stream) {
+    int rc = vp_check(target_shard, draft_shard, draft_tokens, temperature, B, k, V_shard, v_offset, V_total, dtype,
+                      workspace, workspace_bytes);
+    if (rc != SD_OK) return rc;
+    if (!uniforms || !accept_len || !all_masses || !out_tokens) return SD_ERR_NULL;
+    if (n_ranks < 1 || rank < 0 || rank >= n_ranks) return SD_ERR_SHAPE;
+    if (!aligned(all_masses, 8) || !aligned(out_tokens, 4) || !aligned(accept_len, 4) || (out_status && !aligned(out_status, 4)))
+        return SD_ERR_ALIGN;
+    int dev;
+    DeviceState* ds = nullptr;
+    rc = current_device(&dev, &ds);
+    if (rc != SD_OK) return rc;
+    VpParams P = vp_params(target_shard, draft_shard, draft_tokens, uniforms, temperature, B, k, V_shard, v_offset, V_total,
+                           dtype, n_ranks, rank, static_cast<unsigned char*>(workspace));
+    P.accept_len = const_cast<int32_t*>(accept_len);
+    P.all_mass = all_masses;
+    P.tokens = out_tokens;
+    P.status = out_status;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (dtype == SD_DTYPE_F32) sd_vp_draw_kernel<SD_DTYPE_F32><<<(unsigned)B, 32, 0, st>>>(P);
+    else                       sd_vp_draw_kernel<SD_DTYPE_BF16><<<(unsigned)B, 32, 0, st>>>(P);
+    SD_CUDA(cudaGetLastError());
+    tl_info[0] = 6; tl_info[5] = 1;
     return SD_OK;
 }
 

@@ -415,13 +415,16 @@ __device__ __forceinline__ PartialStats warp_sum_lanes(const LaneSums& ls, float
 
 // ------------------------------------------------------------------------------------------
 // Constants of a finished row for the second sweep and the inverse-CDF search.
-__device__ __forceinline__ RowConst row_constants(const Params& P, bool bonus, const PartialStats& st) {
+__device__ __forceinline__ RowConst row_constants_of(double inv_tau, bool bonus, const PartialStats& st) {
     RowConst rc;
     rc.negRT = -st.RT;
     rc.negRD = bonus ? 0.f : -st.RD;
-    rc.kT = (float)((bonus ? 1.0 : P.inv_tau) / st.sT);
-    rc.kD = bonus ? 0.f : (float)(P.inv_tau / st.sD);
+    rc.kT = (float)((bonus ? 1.0 : inv_tau) / st.sT);
+    rc.kD = bonus ? 0.f : (float)(inv_tau / st.sD);
     return rc;
+}
+__device__ __forceinline__ RowConst row_constants(const Params& P, bool bonus, const PartialStats& st) {
+    return row_constants_of(P.inv_tau, bonus, st);
 }
 
 // What the accept test of one pair row needs from global memory; loaded early by the thread that
