@@ -321,6 +321,68 @@ class SamplePath:
         return base, parity, bool(verified)
 
 
+class HintPath(SamplePath):
+    """sd_verify_feedback_hint: the step plus the hint error of the optimistic update, the gradient
+    written over the hint in place.  One more read of B*k*V entries per step than the headline."""
+    name, kernel, traffic_path = "hint", "sd_stream_kernel", "hint"
+
+    def __init__(self, args, cfg, dev, rank, binding):
+        super().__init__(args, cfg, dev, rank, binding)
+        torch = self.torch
+        code = binding.SD_DTYPE_F32 if cfg.dtype == "f32" else binding.SD_DTYPE_BF16
+        self.ws = torch.empty(binding.sd_hint_workspace_bytes(cfg.B, cfg.k, cfg.V, code), dtype=torch.uint8, device=dev)
+        # the buffer that holds the last round's gradient on entry and this round's on return
+        self.hint = self.out.grad_draft
+        self.hint.zero_()
+        self.algorithmic = cfg.algorithmic_bytes + cfg.B * cfg.k * cfg.V * (4 if cfg.dtype == "f32" else 2)
+        self.extra = {"hint": "the gradient of the step before, replaced in place"}
+
+    def step(self, i):
+        T, D, x, u = self.sets[i % self.nsets]
+        self.res = self.b.sd_verify_feedback_hint(T, D, x, u, self.inp.tau, self.hint, grad_out=self.hint,
+                                                  workspace=self.ws)
+
+    def e2e_prepare(self):
+        torch, cfg = self.torch, self.cfg
+        self.dbuf = [torch.empty_like(t) for t in self.sets[0]]
+        self.h_hint = torch.zeros((cfg.B, cfg.k, cfg.V), dtype=self.host[0].dtype).pin_memory()
+        self.h_small = [torch.empty(cfg.B, dtype=torch.int32).pin_memory(),
+                        torch.empty((cfg.B, cfg.k + 1), dtype=torch.int32).pin_memory(),
+                        torch.empty((cfg.B, cfg.k), dtype=torch.float32).pin_memory(),
+                        torch.empty((cfg.B, cfg.k), dtype=torch.float32).pin_memory()]
+        nbytes = lambda ts: sum(t.numel() * t.element_size() for t in ts)
+        self.h2d = self.in_bytes + nbytes([self.h_hint])
+        self.d2h = nbytes(self.h_small) + nbytes([self.h_hint])
+        self.e2e_entry = "sd_verify_feedback_hint between pinned-memory copies"
+
+    def e2e_step(self):
+        for a, b in zip(self.dbuf, self.host):
+            a.copy_(b, non_blocking=True)
+        self.hint.copy_(self.h_hint, non_blocking=True)
+        r = self.b.sd_verify_feedback_hint(*self.dbuf, self.inp.tau, self.hint, grad_out=self.hint, workspace=self.ws)
+        for h, d in zip(self.h_small, (r.accept_len, r.tokens, r.loss, r.hint_err)):
+            h.copy_(d, non_blocking=True)
+        self.h_hint.copy_(self.hint, non_blocking=True)
+        self.torch.cuda.synchronize()
+
+    def finish(self, args):
+        base, parity, verified = super().finish(args)
+        # the hint error of one more step against the oracle on a few sequences (hint = the gradient in place)
+        from oracle import sd_oracle
+        torch, cfg = self.torch, self.cfg
+        seqs = sorted({0, cfg.B // 2, cfg.B - 1})
+        T, D, x, u = self.sets[0]
+        before = self.hint[seqs].cpu()
+        res = self.b.sd_verify_feedback_hint(T, D, x, u, self.inp.tau, self.hint, grad_out=self.hint, workspace=self.ws)
+        torch.cuda.synchronize()
+        hb = before.view(torch.uint16).numpy() if cfg.dtype == "bf16" else before.numpy()
+        want = sd_oracle.hint_error(self.inp.target_logits[seqs], self.inp.draft_logits[seqs], hb, self.inp.tau)
+        got = res.hint_err[seqs].cpu().numpy().astype(np.float64)
+        ok = bool((np.abs(got - want) <= 1e-3 * want + 1e-12).all())
+        parity["hint_error_within_tolerance"] = ok
+        return base, parity, bool(verified and ok)
+
+
 class GreedyPath:
     name, kernel, traffic_path = "greedy", "sd_greedy_kernel", "greedy"
 
@@ -556,7 +618,7 @@ class LmHeadPath:
         return base, {"entries_compared": n, "within_tolerance": ok}, ok
 
 
-PATHS = {"sample": SamplePath, "greedy": GreedyPath, "errors": ErrorsPath, "ensemble": EnsemblePath, "lmhead": LmHeadPath}
+PATHS = {"sample": SamplePath, "hint": HintPath, "greedy": GreedyPath, "errors": ErrorsPath, "ensemble": EnsemblePath, "lmhead": LmHeadPath}
 
 
 def run_ours(args, cfg):

@@ -137,6 +137,29 @@ int sd_verify_feedback_ex(const void* target_logits, const void* draft_logits,
                           size_t workspace_bytes, void* stream);
 
 /*
+ * sd_verify_feedback_hint -- sd_verify_feedback_ex plus the hint error of the optimistic online
+ * update (Sec. 3.2, Eq. 3: the update looks ahead with a hint h_t, taken to be the last round's
+ * gradient; Corollary 2 bounds the regret by the sum over rounds of ||h_t - grad f_t(w_t)||^2).
+ * In the space of the draft logits, per position:
+ *     out_hint_err[b,i] = sum_v ( hint[b,i,v] - (q_{b,i,v} - p_{b,i,v}) / tau )^2,
+ * summed while the gradient is written: the hint is the only additional read (B*k*V entries).
+ *   hint           in   [B,k,V] in `dtype`, the gradient a previous call wrote (or any tensor of that
+ *                       shape); may be the same buffer as out_grad_draft -- every entry is read
+ *                       before it is overwritten
+ *   out_hint_err   out  [B,k] float; the difference is taken against the fp32 gradient before it is
+ *                       rounded to `dtype`; partial sums in fp32 per warp, then fp64 in a fixed order
+ *   workspace           at least sd_hint_workspace_bytes(B,k,V,dtype) bytes, 256-byte aligned
+ * Everything else -- arguments, results, status bits, error codes -- as sd_verify_feedback_ex
+ * (without out_acc_prob).  SD_ERR_NULL if hint or out_hint_err is NULL.
+ */
+size_t sd_hint_workspace_bytes(int B, int k, int V, int dtype);
+int sd_verify_feedback_hint(const void* target_logits, const void* draft_logits, const int32_t* draft_tokens,
+                            const float* uniforms, float temperature, int B, int k, int V, int dtype, const void* hint,
+                            int32_t* out_accept_len, int32_t* out_tokens, float* out_loss, void* out_grad_draft,
+                            float* out_hint_err, uint32_t* out_status, void* workspace, size_t workspace_bytes,
+                            void* stream);
+
+/*
  * sd_verify_feedback_static -- the same computation as sd_verify_feedback_ex for callers that
  * cannot allocate device memory.  (The paper has no counterpart of this entry point; it exists
  * for the way the library is embedded.)

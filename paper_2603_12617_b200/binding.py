@@ -69,6 +69,10 @@ def _load() -> ctypes.CDLL:
                                          P, Z, P]
     lib.sd_lmhead_grad.restype = I
     lib.sd_lmhead_grad.argtypes = [P, P, I, I, I, P, P, P]
+    lib.sd_hint_workspace_bytes.restype = Z
+    lib.sd_hint_workspace_bytes.argtypes = [I, I, I, I]
+    lib.sd_verify_feedback_hint.restype = I
+    lib.sd_verify_feedback_hint.argtypes = [P, P, P, P, F, I, I, I, I, P, P, P, P, P, P, P, P, Z, P]
     lib.sd_vp_workspace_bytes.restype = Z
     lib.sd_vp_workspace_bytes.argtypes = [I, I, I, I]
     lib.sd_vp_partial.restype = I
@@ -109,6 +113,7 @@ class StepOutputs:
     grad_draft: Optional[torch.Tensor]  # [B,k,V], dtype of the logits
     acc_prob: Optional[torch.Tensor] = None   # [B,k] float32
     status: Optional[torch.Tensor] = None     # [B] int32 view of the uint32 status words
+    hint_err: Optional[torch.Tensor] = None   # [B,k] float32, sd_verify_feedback_hint only
 
 
 def _dtype_code(t: torch.Tensor) -> int:
@@ -231,6 +236,41 @@ def sd_verify_feedback_ex(target_logits: torch.Tensor, draft_logits: torch.Tenso
             _stream_ptr(stream))
     if rc != 0:
         raise SdVerifyError(rc, "sd_verify_feedback_ex")
+    return out
+
+
+def sd_hint_workspace_bytes(B: int, k: int, V: int, dtype: int) -> int:
+    return int(_lib.sd_hint_workspace_bytes(B, k, V, dtype))
+
+
+def sd_verify_feedback_hint(target_logits: torch.Tensor, draft_logits: torch.Tensor, draft_tokens: torch.Tensor,
+                            uniforms: torch.Tensor, temperature: float, hint: torch.Tensor, *,
+                            grad_out: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                            stream: Optional[torch.cuda.Stream] = None) -> StepOutputs:
+    """``sd_verify_feedback_hint``: the step plus sum_v (hint - gradient)^2 per position.  ``grad_out``
+    may be ``hint`` itself (the gradient then replaces the hint in place)."""
+    B, k, V = _shapes(target_logits, draft_logits, draft_tokens, uniforms)
+    if tuple(hint.shape) != (B, k, V) or hint.dtype != draft_logits.dtype or not hint.is_contiguous():
+        raise ValueError("hint must be a contiguous [B,k,V] tensor of the logits' dtype")
+    dev = target_logits.device
+    code = _dtype_code(target_logits)
+    if workspace is None:
+        workspace = torch.empty(sd_hint_workspace_bytes(B, k, V, code), dtype=torch.uint8, device=dev)
+    out = StepOutputs(
+        accept_len=torch.empty(B, dtype=torch.int32, device=dev),
+        tokens=torch.empty((B, k + 1), dtype=torch.int32, device=dev),
+        loss=torch.empty((B, k), dtype=torch.float32, device=dev),
+        grad_draft=grad_out if grad_out is not None else torch.empty_like(draft_logits),
+        status=torch.empty(B, dtype=torch.int32, device=dev),
+        hint_err=torch.empty((B, k), dtype=torch.float32, device=dev))
+    with torch.cuda.device(dev):
+        rc = _lib.sd_verify_feedback_hint(
+            _ptr(target_logits), _ptr(draft_logits), _ptr(draft_tokens), _ptr(uniforms), float(temperature),
+            B, k, V, code, _ptr(hint), _ptr(out.accept_len), _ptr(out.tokens), _ptr(out.loss), _ptr(out.grad_draft),
+            _ptr(out.hint_err), _ptr(out.status), _ptr(workspace), workspace.numel() * workspace.element_size(),
+            _stream_ptr(stream))
+    if rc != 0:
+        raise SdVerifyError(rc, "sd_verify_feedback_hint")
     return out
 
 

@@ -74,7 +74,7 @@ int elem_bytes(int dtype) { return dtype == SD_DTYPE_F32 ? 4 : 2; }
 int vec_elems(int dtype) { return 16 / elem_bytes(dtype); }
 
 struct WorkspaceLayout {
-    size_t ticket, wstatus, sticky, accept, rowc, region_sums, total;
+    size_t ticket, wstatus, sticky, accept, rowc, region_sums, hint_part, total;
     int NRmax;   // room for region sums per row: enough for either path at any cluster size
 };
 
@@ -84,7 +84,7 @@ bool shape_ok(int B, int k, int V) {
     return n < 4.0e18L && (long double)B * (k + 1) < 2.0e9L;
 }
 
-WorkspaceLayout workspace_layout(int B, int k, int V, int dtype) {
+WorkspaceLayout workspace_layout(int B, int k, int V, int dtype, bool with_hint = false) {
     WorkspaceLayout L;
     // room for region sums per row: enough for either path (the fast path's regions are 64 vectors,
     // 256 fp32 or 512 bf16 entries; the generic path's 512 entries)
@@ -98,6 +98,8 @@ WorkspaceLayout workspace_layout(int B, int k, int V, int dtype) {
     L.accept = off;      off = align_up(off + (size_t)B * k, kAlign);
     L.rowc = off;        off = align_up(off + (size_t)B * (k + 1) * sizeof(RowConst), kAlign);
     L.region_sums = off; off = align_up(off + (size_t)B * (k + 1) * L.NRmax * 4, kAlign);
+    L.hint_part = off;
+    if (with_hint) off = align_up(off + (size_t)B * (k + 1) * kMaxCluster * 8, kAlign);
     L.total = off;
     return L;
 }
@@ -122,7 +124,7 @@ struct DeviceState {
     // writes whatever it likes behind it -- and where the head ends depends on the shape.  So a call
     // whose head is longer than this clears it first, and afterwards its own head is what is known.
     size_t ws_zero_bytes = 0;
-    bool attr_set[2][3] = {{false, false, false}, {false, false, false}};   // shared-memory / cluster attributes of the fast kernels
+    bool attr_set[2][4] = {};   // shared-memory / cluster attributes of the fast kernels
     int max_clusters[2][kMaxCluster + 1];   // resident clusters of 1..16 blocks, -1 = not asked yet
     // last launch-shape decision of the fast path
     int dec_dtype = -1, dec_V = 0, dec_forced = 0, dec_C = 0, dec_G = 0, dec_lag = 0, dec_use_lag = 0, dec_per = 0;
@@ -179,11 +181,11 @@ int current_device(int* dev, DeviceState** st) {
 
 // Launches the fast path with G clusters of C blocks, or (query_only) asks how many such
 // clusters the device can hold at once.
-template <int DT, bool ENS = false, bool STATS = false>
+template <int DT, bool ENS = false, bool STATS = false, bool HINT = false>
 int launch_stream(DeviceState& d, const Params& P, int C, int G, int lag, cudaStream_t stream, bool query_only,
                   int* max_clusters) {
-    auto kern = sd_stream_kernel<DT, ENS, STATS>;
-    constexpr int kVariant = ENS ? 1 : STATS ? 2 : 0;
+    auto kern = sd_stream_kernel<DT, ENS, STATS, HINT>;
+    constexpr int kVariant = ENS ? 1 : STATS ? 2 : HINT ? 3 : 0;
     if (!d.attr_set[DT][kVariant]) {
         SD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmem));
         SD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
@@ -323,7 +325,7 @@ int check_args(const void* T, const void* D, const int32_t* x, const float* u, f
 int run_device(DeviceState& d, const void* T, const void* D, const int32_t* x, const float* u, float tau, int B,
                int k, int V, int dtype, int32_t* accept_len, int32_t* tokens, float* loss, void* grad,
                float* acc_prob, uint32_t* status, unsigned char* ws, const WorkspaceLayout& L, bool clean,
-               cudaStream_t stream) {
+               cudaStream_t stream, const void* hint = nullptr, float* hint_err = nullptr) {
     Params P;
     memset(&P, 0, sizeof P);
     P.T = T; P.D = D; P.x = x; P.u = u;
@@ -340,13 +342,16 @@ int run_device(DeviceState& d, const void* T, const void* D, const int32_t* x, c
     P.rowc = reinterpret_cast<RowConst*>(ws + L.rowc);
     P.region_sums = reinterpret_cast<float*>(ws + L.region_sums);
     P.wait_polls = wait_polls();
+    P.hint = hint;
+    P.hint_err = hint_err;
+    P.hint_part = hint ? reinterpret_cast<double*>(ws + L.hint_part) : nullptr;
 
     if (!clean) SD_CUDA(cudaMemsetAsync(ws, 0, L.accept, stream));   // tickets, status words, sticky flag
     if (status) SD_CUDA(cudaMemsetAsync(status, 0, (size_t)B * 4, stream));   // bits are ORed in on the device
 
     const size_t row_bytes = (size_t)V * elem_bytes(dtype);
     const bool fast = (row_bytes % 16 == 0) && aligned(T, 16) && aligned(D, 16) && (!grad || aligned(grad, 16)) &&
-                      option(SD_OPT_FORCE_GENERIC) == 0;
+                      (!hint || aligned(hint, 16)) && option(SD_OPT_FORCE_GENERIC) == 0;
     int C = 0, G = 0, lag = 0, per = 0;
     if (fast) C = choose_stream(d, V, (long long)B * (k + 1), dtype, &G, &per, &lag);
     int rc;
@@ -354,8 +359,12 @@ int run_device(DeviceState& d, const void* T, const void* D, const int32_t* x, c
         P.blocks_per_unit = C;
         P.RE = per * vec_elems(dtype);
         P.NR = (V + P.RE - 1) / P.RE;
-        rc = dtype == SD_DTYPE_F32 ? launch_stream<SD_DTYPE_F32>(d, P, C, G, lag, stream, false, nullptr)
-                                   : launch_stream<SD_DTYPE_BF16>(d, P, C, G, lag, stream, false, nullptr);
+        if (hint)
+            rc = dtype == SD_DTYPE_F32 ? launch_stream<SD_DTYPE_F32, false, false, true>(d, P, C, G, lag, stream, false, nullptr)
+                                       : launch_stream<SD_DTYPE_BF16, false, false, true>(d, P, C, G, lag, stream, false, nullptr);
+        else
+            rc = dtype == SD_DTYPE_F32 ? launch_stream<SD_DTYPE_F32>(d, P, C, G, lag, stream, false, nullptr)
+                                       : launch_stream<SD_DTYPE_BF16>(d, P, C, G, lag, stream, false, nullptr);
     } else {
         P.blocks_per_unit = 1;
         P.RE = kGenericRegionElems;
@@ -510,6 +519,34 @@ int sd_verify_feedback_ex(const void* target_logits, const void* draft_logits, c
     return run_device(*d, target_logits, draft_logits, draft_tokens, uniforms, temperature, B, k, V, dtype,
                       out_accept_len, out_tokens, out_loss, out_grad_draft, out_acc_prob, out_status,
                       static_cast<unsigned char*>(workspace), L, false, static_cast<cudaStream_t>(stream));
+}
+
+size_t sd_hint_workspace_bytes(int B, int k, int V, int dtype) {
+    if ((dtype != SD_DTYPE_F32 && dtype != SD_DTYPE_BF16) || !shape_ok(B, k, V)) return 0;
+    return workspace_layout(B, k, V, dtype, true).total;
+}
+
+int sd_verify_feedback_hint(const void* target_logits, const void* draft_logits, const int32_t* draft_tokens,
+                            const float* uniforms, float temperature, int B, int k, int V, int dtype, const void* hint,
+                            int32_t* out_accept_len, int32_t* out_tokens, float* out_loss, void* out_grad_draft,
+                            float* out_hint_err, uint32_t* out_status, void* workspace, size_t workspace_bytes,
+                            void* stream) {
+    int rc = check_args(target_logits, draft_logits, draft_tokens, uniforms, temperature, B, k, V, dtype,
+                        out_accept_len, out_tokens, out_loss, out_grad_draft, nullptr, out_status);
+    if (rc != SD_OK) return rc;
+    if (!hint || !out_hint_err) return SD_ERR_NULL;
+    if (!aligned(hint, (size_t)elem_bytes(dtype)) || !aligned(out_hint_err, 4)) return SD_ERR_ALIGN;
+    const WorkspaceLayout L = workspace_layout(B, k, V, dtype, true);
+    if (!workspace || !aligned(workspace, kAlign) || workspace_bytes < L.total) return SD_ERR_WORKSPACE;
+    int dev;
+    DeviceState* d = nullptr;
+    rc = current_device(&dev, &d);
+    if (rc != SD_OK) return rc;
+    std::lock_guard<std::mutex> lock(d->mu);
+    return run_device(*d, target_logits, draft_logits, draft_tokens, uniforms, temperature, B, k, V, dtype,
+                      out_accept_len, out_tokens, out_loss, out_grad_draft, nullptr, out_status,
+                      static_cast<unsigned char*>(workspace), L, false, static_cast<cudaStream_t>(stream), hint,
+                      out_hint_err);
 }
 
 int sd_verify_feedback_static(const void* target_logits, const void* draft_logits, const int32_t* draft_tokens,

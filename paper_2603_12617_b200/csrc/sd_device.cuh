@@ -77,6 +77,10 @@ struct Params {
     float* region_sums;      // [B*(k+1)*NR] mass of each sampling region of each row
     int blocks_per_unit;     // blocks that take a ticket per (sequence, row)
     uint32_t wait_polls;     // polls after which a bounded wait gives up (kWaitLimit unless a caller asks otherwise)
+    // hint error of the optimistic update (null: not asked for)
+    const void* hint;        // [B,k,V] the last round's gradient, in the dtype of the logits
+    float* hint_err;         // [B,k] sum_v (hint - this round's gradient)^2
+    double* hint_part;       // workspace [B*(k+1)][kMaxCluster]: each block's share of a row's sum
     // online ensemble: feedback of `learners` draft models against one target (0: the plain step).
     // Then loss is [learners,B,k], D and grad above are unused, and nothing is verified or drawn.
     int learners;
@@ -635,6 +639,16 @@ __device__ __noinline__ void resolve_sequence(const Params& P, int b) {
         if (m) { n = i0 + __ffs(m) - 1; break; }
     }
     uint32_t flags = 0;
+
+    // hint error per position: the shares of the blocks that worked on the row, in their order
+    if (P.hint_err) {
+        for (int i = lane; i < k; i += 32) {
+            const double* hp = P.hint_part + (size_t)(b * (k + 1) + i) * kMaxCluster;
+            double e = 0.0;
+            for (int r = 0; r < P.blocks_per_unit; ++r) e += __ldcg(hp + r);
+            P.hint_err[b * k + i] = (float)e;
+        }
+    }
 
     // diagnostic: acceptance probability 1 - sum max(0,p-q) per position (Eq. 1)
     if (P.acc_prob) {

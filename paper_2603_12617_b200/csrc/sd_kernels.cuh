@@ -378,10 +378,12 @@ __device__ __forceinline__ void pass1_region(const uint4* st, int nv, int lane, 
 
 // Pass 2 of a region held in registers: gradient out (gdst = where the region's part of the
 // gradient row starts, or null) and the region's mass (sum of max(0,p-q)/tau, or of p on the
-// bonus row), in every lane.
-template <int DT, bool BONUS>
-__device__ __forceinline__ float pass2_region(const uint4 (&rt)[kRegionRows], const uint4 (&rd)[kRegionRows], int nv,
-                                              int lane, float c, const RowConst& rc, typename Elem<DT>::type* gdst) {
+// bonus row), in every lane.  HINT: hq holds the region of the hint (the last round's gradient), and
+// this lane's sum of squared differences between hint and gradient is added to herr.
+template <int DT, bool BONUS, bool HINT>
+__device__ __forceinline__ float pass2_region_impl(const uint4 (&rt)[kRegionRows], const uint4 (&rd)[kRegionRows], int nv,
+                                                   int lane, float c, const RowConst& rc, typename Elem<DT>::type* gdst,
+                                                   const uint4 (&hq)[kRegionRows], float& herr) {
     using E = Elem<DT>;
     constexpr int VEC = E::VEC;
     float ms[kRegionRows];
@@ -393,7 +395,6 @@ __device__ __forceinline__ float pass2_region(const uint4 (&rt)[kRegionRows], co
         if (!BONUS) {
             float dv[VEC], gv[VEC];
             E::unpack(rd[g], dv);
-#pragma unroll
             float2 acc = make_float2(0.f, 0.f);
 #pragma unroll
             for (int z = 0; z < VEC; z += 2) {
@@ -403,6 +404,18 @@ __device__ __forceinline__ float pass2_region(const uint4 (&rt)[kRegionRows], co
                 acc = __fadd2_rn(acc, make_float2(fmaxf(-g2.x, 0.f), fmaxf(-g2.y, 0.f)));
             }
             if (gdst && vi < nv) store_streaming(gdst + (size_t)vi * VEC, E::pack(gv));
+            if constexpr (HINT) {
+                // distance to the hint, against the gradient before it is rounded to the output type
+                if (vi < nv) {
+                    float hv[VEC];
+                    E::unpack(hq[g], hv);
+#pragma unroll
+                    for (int z = 0; z < VEC; ++z) {
+                        const float dlt = hv[z] - gv[z];
+                        herr = fmaf(dlt, dlt, herr);
+                    }
+                }
+            }
             ms[g] = acc.x + acc.y;
         } else {
 #pragma unroll
@@ -414,6 +427,12 @@ __device__ __forceinline__ float pass2_region(const uint4 (&rt)[kRegionRows], co
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) mass += __shfl_xor_sync(0xffffffffu, mass, off);
     return mass;
+}
+template <int DT, bool BONUS>
+__device__ __forceinline__ float pass2_region(const uint4 (&rt)[kRegionRows], const uint4 (&rd)[kRegionRows], int nv,
+                                              int lane, float c, const RowConst& rc, typename Elem<DT>::type* gdst) {
+    float unused = 0.f;
+    return pass2_region_impl<DT, BONUS, false>(rt, rd, nv, lane, c, rc, gdst, rt, unused);
 }
 
 // Control block of the fast path; lives in dynamic shared memory after the ring.
@@ -431,6 +450,7 @@ struct StreamShared {
     PartialStats row[kDoneDepth];       // statistics of the whole row, for the row report
     RowConst rc[2];
     RowConst rc_done[kDoneDepth];       // the same, kept for the row report
+    float hpart[kDoneDepth][kConsumerWarps];   // the consumer warps' shares of a unit's hint error
     int abort;                          // a bounded wait gave up somewhere in this block
 };
 
@@ -468,7 +488,9 @@ __device__ __forceinline__ void walk_stages(int nu, int nst, int L, P1&& p1, P2&
 // ENS: the units are those of the ensemble feedback (see UnitRef); nothing is verified or drawn.
 // STATS: pass 1 only -- row constants, losses and rejection tests of every row; no gradient, no
 // masses, no draw (the error-position feedback finishes the one row it needs in a kernel of its own).
-template <int DT, bool ENS, bool STATS = false>
+// HINT: pass 2 also reads the hint of the optimistic update (the last round's gradient) and sums its
+// squared distance to this round's gradient per row.
+template <int DT, bool ENS, bool STATS = false, bool HINT = false>
 __global__ void __launch_bounds__(kStreamThreads, 1)
 sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const int prefetch) {
     using E = Elem<DT>;
@@ -602,6 +624,12 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const i
             if constexpr (STATS) {
                 if (lane == 0) mbar_arrive(&sh.res_free[dslot]);
                 continue;
+            }
+            if constexpr (HINT) {
+                // this block's share of the row's hint error: the warps' shares in their order, in fp64
+                double hp = (lane < kConsumerWarps) ? (double)sh.hpart[dslot][lane] : 0.0;
+                hp = warp_sum(hp);
+                if (lane == 0 && !bonus) P.hint_part[(size_t)unit * kMaxCluster + rank] = hp;
             }
             ++seg;
             const bool leaves = (i == P.k) || (j == nu - 1);   // last unit of the sequence in this cluster
@@ -768,25 +796,53 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const i
             void* const gbase = ENS ? P.Gn[ur.n] : P.grad;
             ET* Grow = (gbase && !bonus) ? reinterpret_cast<ET*>(gbase) + ur.d_row * P.V + (size_t)(vb0 + rv0) * VEC : nullptr;
             float* rsum = ENS ? nullptr : P.region_sums + (size_t)unit * P.NR + r0 + cw;
+            const uint4* Hrow = nullptr;
+            if constexpr (HINT)
+                Hrow = reinterpret_cast<const uint4*>(reinterpret_cast<const ET*>(P.hint) + ur.d_row * P.V) + vb0 + rv0;
+            float herr = 0.f;
             for (int t = nst - 1; t >= 0; --t) {
+                const int nv = vectors_of(t);
+                // the hint does not go through the ring: each lane asks for its vectors before it waits
+                // for the stage, and they are there when the gradient is
+                uint4 hq[kRegionRows];
+                if constexpr (HINT) {
+#pragma unroll
+                    for (int g = 0; g < kRegionRows; ++g)
+                        hq[g] = (!bonus && g * 32 + lane < nv) ? __ldcs(Hrow + (size_t)t * kStageVecs + g * 32 + lane)
+                                                               : make_uint4(0u, 0u, 0u, 0u);
+                }
                 if (!await_stage()) { ok = false; return false; }
                 const uint4* st = reinterpret_cast<const uint4*>(ring + (size_t)slot * kStageBytes) + rv0;
-                const int nv = vectors_of(t);
                 if (nv == 0) { hand_back(); continue; }
                 uint4 rt[kRegionRows], rd[kRegionRows];
                 if (bonus) { load_region<DT, true>(st, nv, lane, rt, rd); await_region_registers<true>(rt, rd); }
                 else       { load_region<DT, false>(st, nv, lane, rt, rd); await_region_registers<false>(rt, rd); }
                 hand_back();
-                const float mass = bonus ? pass2_region<DT, true>(rt, rd, nv, lane, P.c, rc, nullptr)
-                                         : pass2_region<DT, false>(rt, rd, nv, lane, P.c, rc,
-                                                                   Grow ? Grow + (size_t)t * kStageVecs * VEC : nullptr);
+                float mass;
+                if constexpr (HINT) {
+                    mass = bonus ? pass2_region<DT, true>(rt, rd, nv, lane, P.c, rc, nullptr)
+                                 : pass2_region_impl<DT, false, true>(rt, rd, nv, lane, P.c, rc,
+                                                                      Grow ? Grow + (size_t)t * kStageVecs * VEC : nullptr,
+                                                                      hq, herr);
+                } else {
+                    mass = bonus ? pass2_region<DT, true>(rt, rd, nv, lane, P.c, rc, nullptr)
+                                 : pass2_region<DT, false>(rt, rd, nv, lane, P.c, rc,
+                                                           Grow ? Grow + (size_t)t * kStageVecs * VEC : nullptr);
+                }
                 if (!ENS && lane == 0) rsum[t * kConsumerWarps] = mass;
+            }
+            if constexpr (HINT) {
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) herr += __shfl_xor_sync(0xffffffffu, herr, off);
             }
             // the resolver's slot of unit j-4 must be free again before this unit is reported done
             if (j >= kDoneDepth &&
                 !mbar_wait(&sh.res_free[dslot], (uint32_t)(j / kDoneDepth - 1) & 1u, wc)) { ok = false; return false; }
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sh.s2_done[dslot]);
+            if (lane == 0) {
+                if constexpr (HINT) sh.hpart[dslot][cw] = herr;
+                mbar_arrive(&sh.s2_done[dslot]);
+            }
             return true;
         };
         walk_stages(nu, nst, L, run_pass1, run_pass2);
@@ -810,6 +866,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const i
 // ---- generic path --------------------------------------------------------------------------
 struct GenericShared {
     PartialStats warp_part[kGenericWarps];
+    float hpart[kGenericWarps];
     RowConst rc;
     int last;
 };
@@ -877,6 +934,7 @@ __global__ void __launch_bounds__(kGenericThreads) sd_generic_kernel(const __gri
 
     // sweep 2: gradient and region sums, one sampling region per warp at a time
     float* rsum = P.region_sums + (size_t)unit * P.NR;
+    float herr = 0.f;
     for (int q = warp; q < P.NR; q += kGenericWarps) {
         const int ebase = q * P.RE;
         float mass = 0.f;
@@ -889,6 +947,10 @@ __global__ void __launch_bounds__(kGenericThreads) sd_generic_kernel(const __gri
                     const float d = E::load(P.D, offD + v);
                     const float g = grad_elem(t, d, P.c, rc);
                     mass += fmaxf(-g, 0.f);
+                    if (P.hint) {
+                        const float dlt = E::load(P.hint, offD + v) - g;
+                        herr = fmaf(dlt, dlt, herr);
+                    }
                     if (P.grad) E::store(P.grad, offD + v, g);
                 } else {
                     mass += prob_elem(t, P.c, rc);
@@ -900,8 +962,18 @@ __global__ void __launch_bounds__(kGenericThreads) sd_generic_kernel(const __gri
         if (lane == 0) rsum[q] = mass;
     }
 
+    if (P.hint) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) herr += __shfl_xor_sync(0xffffffffu, herr, off);
+        if (lane == 0) sh.hpart[warp] = herr;
+    }
     // the block that takes the sequence's last ticket resolves it
     __syncthreads();
+    if (tid == 0 && P.hint && !bonus) {
+        double e = 0.0;
+        for (int w = 0; w < kGenericWarps; ++w) e += (double)sh.hpart[w];
+        P.hint_part[(size_t)unit * kMaxCluster] = e;
+    }
     if (tid == 0) sh.last = take_tickets(P, b, 1u) ? 1 : 0;
     __syncthreads();
     if (sh.last && warp == 0) resolve_sequence<DT, false>(P, b);

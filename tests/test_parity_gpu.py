@@ -678,3 +678,110 @@ def test_pinsker_ties_acceptance_probability_to_the_loss_on_every_row(binding, n
     assert ((acc >= -1e-6) & (acc <= 1 + 1e-6)).all()
     assert ((1.0 - acc) <= np.sqrt(loss / 2.0) + 1e-5).all()
     assert (out.status.cpu().numpy() == 0).all()
+
+
+# ------------------------------------------------------------------ hint error of the optimistic update
+def hint_of(inp, seed):
+    """A stand-in for the last round's gradient: this round's oracle gradient of other inputs, i.e. a
+    tensor with the scale and structure of a gradient (rows that sum to zero, most mass on few entries)."""
+    other = synth.make_inputs(inp.cfg, seed)
+    ref = sd_oracle.verify_feedback(other.target_logits, other.draft_logits, other.draft_tokens, other.uniforms,
+                                    other.tau, want_grad=True, nthreads=min(8, sd_oracle.max_threads()))
+    g = ref.grad.astype(np.float32)
+    return synth.f32_to_bf16_bits(g) if inp.cfg.dtype == "bf16" else g
+
+
+def check_hint_error(inp, hint_bits, got, tol):
+    want = sd_oracle.hint_error(inp.target_logits, inp.draft_logits, hint_bits, inp.tau)
+    err = np.abs(got.astype(np.float64) - want)
+    assert (err <= tol * want + 1e-12).all(), f"hint error: worst ratio {np.max(err / (tol * want + 1e-12)):.3g}"
+
+
+@pytest.mark.parametrize("dtype,B,k,V", [("f32", 5, 3, 32000), ("bf16", 5, 3, 32000), ("f32", 20, 4, 128256),
+                                         ("bf16", 33, 2, 151936), ("f32", 3, 2, 1001), ("bf16", 2, 1, 777)])
+def test_hint_error_matches_the_oracle(binding, dtype, B, k, V):
+    """Sec. 3.2: sum_v (h - grad)^2 per position, h a gradient-like tensor; every other output is the
+    plain step's.  The difference is taken against the fp32 gradient before it is rounded to the output
+    type, so bf16 logits cost no accuracy here: every entry of that gradient carries a relative error of
+    a few 2^-22 of max(p,q)/tau, and the fp32 partial sums of a warp add about as much again.  Bars:
+    2e-4 (fp32 logits) and 1e-3 (bf16 logits, whose hint is itself coarse) of the exact value."""
+    cfg = synth.custom_config(B, k, V, dtype=dtype, tau=0.9, index=80)
+    inp = synth.make_inputs(cfg)
+    hint_bits = hint_of(inp, synth.BASE_SEED + 7)
+    T, D, x, u = to_device(inp)
+    H = torch.from_numpy(hint_bits).cuda()
+    if dtype == "bf16":
+        H = H.view(torch.bfloat16)
+    out = binding.sd_verify_feedback_hint(T, D, x, u, inp.tau, H)
+    torch.cuda.synchronize()
+    ref = oracle_of(inp)
+    check(inp, out, ref, max_band_frac=0.5)
+    check_hint_error(inp, hint_bits, out.hint_err.cpu().numpy(), 2e-4 if dtype == "f32" else 1e-3)
+    plain = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
+    torch.cuda.synchronize()
+    assert torch.equal(plain.grad_draft.view(torch.uint8), out.grad_draft.view(torch.uint8))
+    assert torch.equal(plain.tokens, out.tokens) and torch.equal(plain.loss, out.loss)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_hint_error_in_place_and_special_hints(binding, dtype):
+    """The gradient may replace the hint in its own buffer; a hint equal to the gradient the step writes
+    gives the rounding of the output type only (zero for fp32), a zero hint gives the gradient's norm."""
+    cfg = synth.custom_config(6, 3, 50000, dtype=dtype, tau=1.1, index=81)
+    inp = synth.make_inputs(cfg)
+    T, D, x, u = to_device(inp)
+    first = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
+    torch.cuda.synchronize()
+    same = binding.sd_verify_feedback_hint(T, D, x, u, inp.tau, first.grad_draft)
+    torch.cuda.synchronize()
+    g = first.grad_draft.float().cpu().numpy().astype(np.float64)
+    norm2 = (g * g).sum(-1)
+    if dtype == "f32":
+        assert (same.hint_err.cpu().numpy() == 0).all()
+    else:
+        assert (same.hint_err.cpu().numpy() <= 2.0 ** -16 * norm2).all()      # (2^-8 relative per entry)^2
+    zero = binding.sd_verify_feedback_hint(T, D, x, u, inp.tau, torch.zeros_like(D))
+    torch.cuda.synchronize()
+    ref = oracle_of(inp)
+    want = (ref.grad * ref.grad).sum(-1)
+    assert np.abs(zero.hint_err.cpu().numpy() - want).max() <= 1e-4 * want.max()
+    # in place: the hint's buffer receives the gradient
+    hint_bits = hint_of(inp, synth.BASE_SEED + 9)
+    H = torch.from_numpy(hint_bits).cuda()
+    if dtype == "bf16":
+        H = H.view(torch.bfloat16)
+    inplace = binding.sd_verify_feedback_hint(T, D, x, u, inp.tau, H, grad_out=H)
+    torch.cuda.synchronize()
+    assert torch.equal(H.view(torch.uint8), first.grad_draft.view(torch.uint8))
+    check_hint_error(inp, hint_bits, inplace.hint_err.cpu().numpy(), 2e-4 if dtype == "f32" else 1e-3)
+
+
+def test_hint_error_every_cluster_size_and_the_generic_path(binding, options):
+    cfg = synth.custom_config(7, 2, 65536, dtype="bf16", tau=0.8, index=82)
+    inp = synth.make_inputs(cfg)
+    hint_bits = hint_of(inp, synth.BASE_SEED + 11)
+    T, D, x, u = to_device(inp)
+    H = torch.from_numpy(hint_bits).cuda().view(torch.bfloat16)
+    for cluster in (1, 2, 3, 8, 16):
+        options(binding.SD_OPT_CLUSTER, cluster)
+        out = binding.sd_verify_feedback_hint(T, D, x, u, inp.tau, H)
+        torch.cuda.synchronize()
+        assert binding.sd_launch_info()["cluster_size"] == cluster
+        check_hint_error(inp, hint_bits, out.hint_err.cpu().numpy(), 1e-3)
+    options(binding.SD_OPT_CLUSTER, 0)
+    options(binding.SD_OPT_FORCE_GENERIC, 1)
+    out = binding.sd_verify_feedback_hint(T, D, x, u, inp.tau, H)
+    torch.cuda.synchronize()
+    assert binding.sd_launch_info()["path"] == 0
+    check_hint_error(inp, hint_bits, out.hint_err.cpu().numpy(), 1e-3)
+
+
+def test_hint_entry_refusals(binding):
+    cfg = synth.custom_config(2, 2, 4096, dtype="f32", index=83)
+    inp = synth.make_inputs(cfg)
+    T, D, x, u = to_device(inp)
+    with pytest.raises(ValueError):
+        binding.sd_verify_feedback_hint(T, D, x, u, inp.tau, torch.zeros((2, 2, 4000), device="cuda"))
+    with pytest.raises(binding.SdVerifyError):
+        binding.sd_verify_feedback_hint(T, D, x, u, inp.tau, torch.zeros_like(D),
+                                        workspace=torch.empty(256, dtype=torch.uint8, device="cuda"))
