@@ -290,7 +290,7 @@ int choose_stream(DeviceState& d, int V, long long units, int dtype, int* G_out,
     // so all of the next pair's first pass goes first; with many, the data between the passes is
     // what costs (L2 holds less of it), and the second pass follows the first at once.
     int use_lag = lag;
-    if (lag < 0) use_lag = (best_G > 0 && units <= 8LL * best_G) ? 1 << 20 : 0;
+    if (lag == -1) use_lag = (best_G > 0 && units <= 8LL * best_G) ? 1 << 20 : 0;
     d.dec_dtype = dtype; d.dec_V = V; d.dec_units = units; d.dec_forced = forced; d.dec_l2 = l2_budget;
     d.dec_C = best_C; d.dec_G = best_G; d.dec_lag = lag; d.dec_use_lag = use_lag; d.dec_per = best_per;
     *G_out = best_G;

@@ -630,6 +630,17 @@ __device__ __noinline__ void resolve_sequence(const Params& P, int b) {
     const int lane = threadIdx.x & 31;
     const int k = P.k, NR = P.NR;
 
+    // The warp that resolves a sequence is the last thing between the kernel and its end, and almost
+    // all of its time is memory round trips: everything that does not depend on the accept length is
+    // asked for here, in one go, together with the rejection flags.
+    const float uk_f = P.u[b * (k + 1) + k];
+    const int32_t x_first = (lane < k) ? P.x[b * k + lane] : -1;
+    uint32_t st_word = 0, sticky_word = 0;
+    if (lane == 0) {
+        st_word = __ldcg(P.wstatus + b);
+        sticky_word = __ldcg(P.sticky);
+    }
+
     // accept length: first rejected position
     int n = k;
     for (int i0 = 0; i0 < k; i0 += 32) {
@@ -674,19 +685,26 @@ __device__ __noinline__ void resolve_sequence(const Params& P, int b) {
     const RowConst rc{rcv.x, rcv.y, rcv.z, rcv.w};
     const size_t offT = (size_t)unit * P.V;
     const size_t offD = (size_t)(b * k + (bonus ? 0 : n)) * P.V;
-    const double uk = (double)P.u[b * (k + 1) + k];
+    const double uk = (double)uk_f;
 
-    // prefix over the region sums: each lane owns a contiguous run of regions, which it reads eight
-    // at a time (all eight loads in flight together) and adds up in index order
+    // prefix over the region sums: each lane owns a contiguous run of regions, which it reads sixteen
+    // at a time (all sixteen loads in flight together) and adds up in index order; the first sixteen
+    // stay in registers for the search below
+    constexpr int kHeld = 16;
     const int per = (NR + 31) / 32;
     const int j0 = min(NR, lane * per), j1 = min(NR, j0 + per);
+    float held[kHeld];
+#pragma unroll
+    for (int q = 0; q < kHeld; ++q) held[q] = (j0 + q < j1) ? __ldcg(rs + j0 + q) : 0.f;
     double mine = 0.0;
-    for (int c = j0; c < j1; c += 8) {
-        float v[8];
 #pragma unroll
-        for (int q = 0; q < 8; ++q) v[q] = (c + q < j1) ? __ldcg(rs + c + q) : 0.f;
+    for (int q = 0; q < kHeld; ++q) mine += (double)held[q];
+    for (int c = j0 + kHeld; c < j1; c += kHeld) {
+        float v[kHeld];
 #pragma unroll
-        for (int q = 0; q < 8; ++q) mine += (double)v[q];
+        for (int q = 0; q < kHeld; ++q) v[q] = (c + q < j1) ? __ldcg(rs + c + q) : 0.f;
+#pragma unroll
+        for (int q = 0; q < kHeld; ++q) mine += (double)v[q];
     }
     const double incl = warp_inclusive_scan(mine);
     const double before = incl - mine;
@@ -707,12 +725,20 @@ __device__ __noinline__ void resolve_sequence(const Params& P, int b) {
         double cand_prefix = 0.0;
         if (before + mine > t) {                  // the crossing can only be in a lane whose run reaches t
             double run = before;
-            for (int c = j0; c < j1 && cand == 0x7fffffff; c += 8) {
-                float v[8];
 #pragma unroll
-                for (int q = 0; q < 8; ++q) v[q] = (c + q < j1) ? __ldcg(rs + c + q) : 0.f;
+            for (int q = 0; q < kHeld; ++q) {
+                if (cand == 0x7fffffff && j0 + q < j1) {
+                    const double next = run + (double)held[q];
+                    if (next > t) { cand = j0 + q; cand_prefix = run; }
+                    else run = next;
+                }
+            }
+            for (int c = j0 + kHeld; c < j1 && cand == 0x7fffffff; c += kHeld) {
+                float v[kHeld];
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {
+                for (int q = 0; q < kHeld; ++q) v[q] = (c + q < j1) ? __ldcg(rs + c + q) : 0.f;
+#pragma unroll
+                for (int q = 0; q < kHeld; ++q) {
                     if (cand == 0x7fffffff && c + q < j1) {
                         const double next = run + (double)v[q];
                         if (next > t) { cand = c + q; cand_prefix = run; }
@@ -750,15 +776,17 @@ __device__ __noinline__ void resolve_sequence(const Params& P, int b) {
 
     if (lane == 0) {
         P.accept_len[b] = n;
-        uint32_t st = __ldcg(P.wstatus + b) | flags;
-        if (__ldcg(P.sticky) != 0) st |= kStatusTimeout;
+        uint32_t st = st_word | flags;
+        if (sticky_word != 0) st |= kStatusTimeout;
         if (P.status && st) atomicOr(P.status + b, st);   // zero on entry; a block that gave up may have set its bit already
         // leave the workspace ready for the next call
         P.wstatus[b] = 0;
         P.ticket[b] = 0;
     }
-    for (int i = lane; i <= k; i += 32)
-        P.tokens[b * (k + 1) + i] = (i < n) ? P.x[b * k + i] : (i == n ? y : -1);
+    for (int i = lane; i <= k; i += 32) {
+        const int32_t xi = (i == lane) ? x_first : ((i < k) ? P.x[b * k + i] : -1);
+        P.tokens[b * (k + 1) + i] = (i < n) ? xi : (i == n ? y : -1);
+    }
 }
 
 // Tickets of one block for sequence b: `n` of the (k+1) * blocks_per_unit tickets of the

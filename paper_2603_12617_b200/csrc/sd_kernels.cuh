@@ -529,7 +529,9 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const i
     const int vb0 = r0 * kRegionVecs;             // first vector of the slice
     const int nvb = max(0, min(NV - vb0, nr * kRegionVecs));        // vectors of the slice
     const int nst = (nr + kConsumerWarps - 1) / kConsumerWarps;     // stages of a pass
-    const int L = min(max(lag_stages, 0), nst);
+    // lag_stages = -2: every other cluster takes all of the next unit's pass 1 first, the rest none of it,
+    // so that half of the GPU reads from HBM while the other half works from L2
+    const int L = lag_stages == -2 ? ((cid & 1) ? nst : 0) : min(max(lag_stages, 0), nst);
     const WaitCtx wc{&sh.abort, P.wait_polls};
 
     if (tid == 0) {
