@@ -25,7 +25,7 @@ namespace sdv {
 
 namespace cg = cooperative_groups;
 
-constexpr int kMaxCluster = 16;
+constexpr int kMaxCluster = 8;
 constexpr int kMaxLearners = 8;                  // draft models of an online ensemble
 constexpr int kGenericRegionElems = 512;         // sampling region of the generic path
 constexpr int kRegionRows = 2;                   // fast path: 16-byte vectors per lane and row in a sampling region

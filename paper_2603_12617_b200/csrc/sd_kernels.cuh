@@ -50,8 +50,8 @@ constexpr int kConsumerWarps = 28;
 constexpr int kStageVecs = kConsumerWarps * kRegionVecs;      // vectors of one row in a stage
 constexpr int kStageRowBytes = kStageVecs * 16;               // 28 KiB of one row
 constexpr int kStageBytes = 2 * kStageRowBytes;               // target part + draft part
-constexpr int kRingStages = 3;                                // 168 KiB
-constexpr int kDoneDepth = 4;                                 // units the resolver may lag behind
+constexpr int kRingStages = 4;                                // 224 KiB
+constexpr int kDoneDepth = 3;                                 // units the resolver may lag behind
 constexpr int kStatsWarp = 0, kResolverWarp = 1, kProducerWarp = 2, kFirstConsumerWarp = kHelperWarps;
 constexpr int kStreamThreads = (kHelperWarps + kConsumerWarps) * 32;
 constexpr int kGenericWarps = 8;
@@ -492,7 +492,7 @@ __device__ __forceinline__ void walk_stages(int nu, int nst, int L, P1&& p1, P2&
 // squared distance to this round's gradient per row.
 template <int DT, bool ENS, bool STATS = false, bool HINT = false>
 __global__ void __launch_bounds__(kStreamThreads, 1)
-sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const int prefetch) {
+sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const int prefetch, const int resident_arg) {
     using E = Elem<DT>;
     using ET = typename E::type;
     constexpr int VEC = E::VEC;
@@ -531,7 +531,13 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const i
     const int nst = (nr + kConsumerWarps - 1) / kConsumerWarps;     // stages of a pass
     // lag_stages = -2: every other cluster takes all of the next unit's pass 1 first, the rest none of it,
     // so that half of the GPU reads from HBM while the other half works from L2
-    const int L = lag_stages == -2 ? ((cid & 1) ? nst : 0) : min(max(lag_stages, 0), nst);
+    // Resident walk: the slice of a unit (at most kRingStages - 1 stages) stays in the ring between its
+    // two passes, so every logit enters the SM once; a stage is released by pass 2, and the producer
+    // runs ahead into the next unit as far as the free slots reach.  Pass 1 of the next unit can go
+    // before pass 2 of a unit only as far as the producer can get without a release.
+    const bool resident = !STATS && resident_arg != 0 && nst < kRingStages;
+    const int Lreq = lag_stages == -2 ? ((cid & 1) ? nst : 0) : min(max(lag_stages, 0), nst);
+    const int L = resident ? min(Lreq, kRingStages - nst) : Lreq;
     const WaitCtx wc{&sh.abort, P.wait_polls};
 
     if (tid == 0) {
@@ -677,6 +683,13 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const i
                 ++ni;
                 if (++slot == kRingStages) { slot = 0; epar ^= 1u; }
             };
+            if (resident) {
+                // every stage once, in order; nobody reads it from L2 again
+                for (int j = 0; j < nu && ok; ++j) {
+                    const UnitRef ur = unit_ref<ENS>(P, u0 + j * ustep);
+                    for (int t = 0; t < nst && ok; ++t) issue(ur, t, discard);
+                }
+            } else
             walk_stages(nu, nst, L,
                 [&](int j, int t0, int t1, bool) {
                     const UnitRef ur = unit_ref<ENS>(P, u0 + j * ustep);
@@ -731,11 +744,21 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const i
         // before the arithmetic on this region is over, and when it says "full" -- the usual case --
         // the next visit starts without the round trip of a wait.
         bool next_full = false;
-        auto hand_back = [&]() {
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sh.empty[slot]);
+        int rslot = 0;                             // resident walk: slot of the next stage that pass 2 releases
+        auto advance = [&]() {
             if (++slot == kRingStages) { slot = 0; fpar ^= 1u; }
             next_full = mbar_test(&sh.full[slot], fpar);
+        };
+        auto hand_back = [&]() {
+            if (resident) { advance(); return; }   // pass 1 of the resident walk keeps the stage
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.empty[slot]);
+            advance();
+        };
+        auto release = [&]() {                     // pass 2 of the resident walk: the stage goes back
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.empty[rslot]);
+            if (++rslot == kRingStages) rslot = 0;
         };
         auto await_stage = [&]() {
             if (__all_sync(0xffffffffu, next_full ? 1 : 0)) return true;
@@ -802,7 +825,8 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const i
             if constexpr (HINT)
                 Hrow = reinterpret_cast<const uint4*>(reinterpret_cast<const ET*>(P.hint) + ur.d_row * P.V) + vb0 + rv0;
             float herr = 0.f;
-            for (int t = nst - 1; t >= 0; --t) {
+            for (int s = 0; s < nst; ++s) {
+                const int t = resident ? s : nst - 1 - s;   // (the streaming walk finds the last stages still in L2)
                 const int nv = vectors_of(t);
                 // the hint does not go through the ring: each lane asks for its vectors before it waits
                 // for the stage, and they are there when the gradient is
@@ -813,13 +837,16 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const i
                         hq[g] = (!bonus && g * 32 + lane < nv) ? __ldcs(Hrow + (size_t)t * kStageVecs + g * 32 + lane)
                                                                : make_uint4(0u, 0u, 0u, 0u);
                 }
-                if (!await_stage()) { ok = false; return false; }
-                const uint4* st = reinterpret_cast<const uint4*>(ring + (size_t)slot * kStageBytes) + rv0;
-                if (nv == 0) { hand_back(); continue; }
+                if (!resident && !await_stage()) { ok = false; return false; }
+                const uint4* st = reinterpret_cast<const uint4*>(ring + (size_t)(resident ? rslot : slot) * kStageBytes) + rv0;
+                if (nv == 0) {
+                    if (resident) release(); else hand_back();
+                    continue;
+                }
                 uint4 rt[kRegionRows], rd[kRegionRows];
                 if (bonus) { load_region<DT, true>(st, nv, lane, rt, rd); await_region_registers<true>(rt, rd); }
                 else       { load_region<DT, false>(st, nv, lane, rt, rd); await_region_registers<false>(rt, rd); }
-                hand_back();
+                if (resident) release(); else hand_back();
                 float mass;
                 if constexpr (HINT) {
                     mass = bonus ? pass2_region<DT, true>(rt, rd, nv, lane, P.c, rc, nullptr)
