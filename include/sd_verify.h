@@ -388,10 +388,9 @@ int sd_verify_feedback_host(const void* target_logits, const void* draft_logits,
  *   SD_OPT_CLUSTER               env SD_VERIFY_CLUSTER          default 0    cluster size of the fast path
  *                                (1..8), 0 = chosen per shape
  *   SD_OPT_LAG                   env SD_VERIFY_LAG              default -1   stages of the next row pair
- *                                that go before the second pass over a row pair; -1 = chosen per shape
- *                                (resident walk: as many as the ring has room for; streaming walk: all
- *                                when a cluster has at most eight row pairs to work on, none otherwise);
- *                                -2 = all in every other cluster, none in the rest
+ *                                that go before the second pass over a row pair; -1 = all of them when a
+ *                                cluster has at most eight row pairs to work on, none otherwise; -2 = all
+ *                                in every other cluster, none in the rest
  *   SD_OPT_L2_BUDGET_MIB         env SD_VERIFY_L2_MIB           default 80   bytes of row pairs in flight
  *                                between their two passes that the launch shape may assume L2 holds
  *   SD_OPT_FORCE_GENERIC         env SD_VERIFY_FORCE_GENERIC    default 0    non-zero: element-wise path
@@ -402,10 +401,6 @@ int sd_verify_feedback_host(const void* target_logits, const void* draft_logits,
  *                                SD_STATUS_TIMEOUT); the wait also ends after about a second
  *   SD_OPT_PREFETCH              env SD_VERIFY_PREFETCH         default 0    non-zero: while a block is in
  *                                its second pass over a row pair it asks L2 to fetch the next row pair
- *                                (streaming walk only)
- *   SD_OPT_RESIDENT              env SD_VERIFY_RESIDENT         default 0    non-zero: a block keeps its slice
- *                                of a row pair in shared memory between the two passes when the slice is
- *                                at most three stages (84 regions) long, instead of fetching it twice
  * sd_set_option returns SD_OK, or SD_ERR_SHAPE for an unknown option; sd_get_option returns the
  * value in force, or -1 for an unknown option.
  */
@@ -417,8 +412,7 @@ int sd_verify_feedback_host(const void* target_logits, const void* draft_logits,
 #define SD_OPT_GREEDY_BLOCKS_PER_SM 5
 #define SD_OPT_WAIT_POLLS 6
 #define SD_OPT_PREFETCH 7
-#define SD_OPT_RESIDENT 8
-#define SD_OPT_COUNT 9
+#define SD_OPT_COUNT 8
 int sd_set_option(int option_id, long long value);
 long long sd_get_option(int option_id);
 

@@ -25,7 +25,6 @@ SD_OPT_FORCE_GENERIC = 4
 SD_OPT_GREEDY_BLOCKS_PER_SM = 5
 SD_OPT_WAIT_POLLS = 6
 SD_OPT_PREFETCH = 7
-SD_OPT_RESIDENT = 8
 
 SD_STATUS_BAD_TOKEN = 1
 SD_STATUS_BAD_ROW = 2

@@ -19,9 +19,9 @@ using namespace sdv;
 
 constexpr int kMaxDevices = 64;
 constexpr size_t kAlign = 256;
+template <int DT> constexpr int stream_smem() { return RingStages<DT>::value * kStageBytes + (int)sizeof(StreamShared); }
 constexpr int kStreamSmem = kRingStages * kStageBytes + (int)sizeof(StreamShared);
 static_assert(kStreamSmem <= 227 * 1024, "ring does not fit the shared memory of a block");
-static_assert(kMaxCluster <= 8, "cluster sizes above 8 are not portable");
 constexpr int kL2PersistMiB = 0;
 constexpr long long kL2BudgetMiB = 80;             // row pairs in flight between their two passes should fit this
 
@@ -44,7 +44,6 @@ void init_options() {
             {SD_OPT_GREEDY_BLOCKS_PER_SM, "SD_GREEDY_BLOCKS_PER_SM", 4},
             {SD_OPT_WAIT_POLLS, "SD_VERIFY_WAIT_POLLS", (long long)kWaitLimit},
             {SD_OPT_PREFETCH, "SD_VERIFY_PREFETCH", 0},
-            {SD_OPT_RESIDENT, "SD_VERIFY_RESIDENT", 0},
         };
         for (const auto& t : table) {
             const char* e = getenv(t.env);
@@ -127,10 +126,9 @@ struct DeviceState {
     // whose head is longer than this clears it first, and afterwards its own head is what is known.
     size_t ws_zero_bytes = 0;
     bool attr_set[2][4] = {};   // shared-memory / cluster attributes of the fast kernels
-    int max_clusters[2][kMaxCluster + 1];   // resident clusters of 1..16 blocks, -1 = not asked yet
+    int max_clusters[2][kMaxCluster + 1];   // resident clusters of 1..8 blocks, -1 = not asked yet
     // last launch-shape decision of the fast path
     int dec_dtype = -1, dec_V = 0, dec_forced = 0, dec_C = 0, dec_G = 0, dec_lag = 0, dec_use_lag = 0, dec_per = 0;
-    int dec_allow_resident = -1, dec_resident = 0;
     long long dec_units = 0;
     double dec_l2 = 0.0;
     // output-layer gradient
@@ -186,11 +184,11 @@ int current_device(int* dev, DeviceState** st) {
 // clusters the device can hold at once.
 template <int DT, bool ENS = false, bool STATS = false, bool HINT = false>
 int launch_stream(DeviceState& d, const Params& P, int C, int G, int lag, cudaStream_t stream, bool query_only,
-                  int* max_clusters, int resident = 0) {
+                  int* max_clusters) {
     auto kern = sd_stream_kernel<DT, ENS, STATS, HINT>;
     constexpr int kVariant = ENS ? 1 : STATS ? 2 : HINT ? 3 : 0;
     if (!d.attr_set[DT][kVariant]) {
-        SD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamSmem));
+        SD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, stream_smem<DT>()));
         SD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
         d.attr_set[DT][kVariant] = true;
     }
@@ -198,7 +196,7 @@ int launch_stream(DeviceState& d, const Params& P, int C, int G, int lag, cudaSt
     memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3((unsigned)(G * C), 1, 1);
     cfg.blockDim = dim3(kStreamThreads, 1, 1);
-    cfg.dynamicSmemBytes = (size_t)kStreamSmem;
+    cfg.dynamicSmemBytes = (size_t)stream_smem<DT>();
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -218,8 +216,8 @@ int launch_stream(DeviceState& d, const Params& P, int C, int G, int lag, cudaSt
         return SD_OK;
     }
     const int prefetch = option(SD_OPT_PREFETCH) != 0 ? 1 : 0;
-    SD_CUDA(cudaLaunchKernelEx(&cfg, kern, P, lag, prefetch, resident));
-    tl_info[0] = 1; tl_info[1] = C; tl_info[2] = kStreamThreads; tl_info[3] = kStreamSmem;
+    SD_CUDA(cudaLaunchKernelEx(&cfg, kern, P, lag, prefetch));
+    tl_info[0] = 1; tl_info[1] = C; tl_info[2] = kStreamThreads; tl_info[3] = stream_smem<DT>();
     tl_info[4] = G * C; tl_info[5] = 1;
     return SD_OK;
 }
@@ -235,11 +233,8 @@ int launch_generic(const Params& P, cudaStream_t stream) {
 }
 
 // Launch shape of the fast path: cluster size C (0 if the fast path cannot run), number of
-// clusters G, vectors per sampling region, how many stages of pass 1 of the next unit a consumer
-// warp takes before pass 2 of a unit, and whether the blocks keep their slice of a row pair in
-// shared memory between the two passes (only on request, and only when the slice is at most
-// kRingStages - 1 stages: measured, the clusters large enough for that lose more to their many
-// short row pairs -- every one costs an exchange and a row report -- than the second fetch costs).
+// clusters G, vectors per sampling region, and how many stages of pass 1 of the next unit a
+// consumer warp takes before pass 2 of a unit.
 //
 // A row is cut into stages and block r of a cluster of C takes every C-th share of them.  A
 // block's slice lives in L2 between its two passes, so the row pairs the resident clusters work on
@@ -250,18 +245,15 @@ int launch_generic(const Params& P, cudaStream_t stream) {
 // costs (exchange, row report) over more bytes and small clusters pack the GPU best (resident
 // blocks: 148 for C = 1 and 2, 135 for 3, 132 for 4 and 6, 130 for 5, 112 for 7, 120 for 8).  If none fits, the
 // largest cluster.
-int choose_stream(DeviceState& d, int V, long long units, int dtype, int* G_out, int* per_out, int* lag_out,
-                  int* resident_out) {
+int choose_stream(DeviceState& d, int V, long long units, int dtype, int* G_out, int* per_out, int* lag_out) {
     const int forced = (int)option(SD_OPT_CLUSTER);
     const double l2_budget = (double)option(SD_OPT_L2_BUDGET_MIB) * 1048576.0;
     const int lag = (int)option(SD_OPT_LAG);       // stages of the next unit before pass 2 of a unit
-    const int allow_resident = (int)option(SD_OPT_RESIDENT);
     if (d.dec_dtype == dtype && d.dec_V == V && d.dec_units == units && d.dec_forced == forced &&
-        d.dec_l2 == l2_budget && d.dec_lag == lag && d.dec_allow_resident == allow_resident) {
+        d.dec_l2 == l2_budget && d.dec_lag == lag) {
         *G_out = d.dec_G;
         *per_out = d.dec_per;
         *lag_out = d.dec_use_lag;
-        *resident_out = d.dec_resident;
         return d.dec_C;
     }
     const int NV = V / vec_elems(dtype);
@@ -298,16 +290,8 @@ int choose_stream(DeviceState& d, int V, long long units, int dtype, int* G_out,
     // pairs per cluster every wait for an exchange shows (and the first and the last cannot hide),
     // so all of the next pair's first pass goes first; with many, the data between the passes is
     // what costs (L2 holds less of it), and the second pass follows the first at once.
-    int best_res = 0;
-    if (best_C > 0 && allow_resident != 0) {
-        const int regions_row = (NV + kRegionVecs - 1) / kRegionVecs;
-        const int regions_blk = (regions_row + best_C - 1) / best_C;
-        best_res = (regions_blk + kConsumerWarps - 1) / kConsumerWarps < kRingStages ? 1 : 0;
-    }
     int use_lag = lag;
-    if (lag == -1) use_lag = (best_res || (best_G > 0 && units <= 8LL * best_G)) ? 1 << 20 : 0;
-    d.dec_allow_resident = allow_resident; d.dec_resident = best_res;
-    *resident_out = best_res;
+    if (lag == -1) use_lag = (best_G > 0 && units <= 8LL * best_G) ? 1 << 20 : 0;
     d.dec_dtype = dtype; d.dec_V = V; d.dec_units = units; d.dec_forced = forced; d.dec_l2 = l2_budget;
     d.dec_C = best_C; d.dec_G = best_G; d.dec_lag = lag; d.dec_use_lag = use_lag; d.dec_per = best_per;
     *G_out = best_G;
@@ -369,19 +353,19 @@ int run_device(DeviceState& d, const void* T, const void* D, const int32_t* x, c
     const size_t row_bytes = (size_t)V * elem_bytes(dtype);
     const bool fast = (row_bytes % 16 == 0) && aligned(T, 16) && aligned(D, 16) && (!grad || aligned(grad, 16)) &&
                       (!hint || aligned(hint, 16)) && option(SD_OPT_FORCE_GENERIC) == 0;
-    int C = 0, G = 0, lag = 0, per = 0, res = 0;
-    if (fast) C = choose_stream(d, V, (long long)B * (k + 1), dtype, &G, &per, &lag, &res);
+    int C = 0, G = 0, lag = 0, per = 0;
+    if (fast) C = choose_stream(d, V, (long long)B * (k + 1), dtype, &G, &per, &lag);
     int rc;
     if (C > 0) {
         P.blocks_per_unit = C;
         P.RE = per * vec_elems(dtype);
         P.NR = (V + P.RE - 1) / P.RE;
         if (hint)
-            rc = dtype == SD_DTYPE_F32 ? launch_stream<SD_DTYPE_F32, false, false, true>(d, P, C, G, lag, stream, false, nullptr, res)
-                                       : launch_stream<SD_DTYPE_BF16, false, false, true>(d, P, C, G, lag, stream, false, nullptr, res);
+            rc = dtype == SD_DTYPE_F32 ? launch_stream<SD_DTYPE_F32, false, false, true>(d, P, C, G, lag, stream, false, nullptr)
+                                       : launch_stream<SD_DTYPE_BF16, false, false, true>(d, P, C, G, lag, stream, false, nullptr);
         else
-            rc = dtype == SD_DTYPE_F32 ? launch_stream<SD_DTYPE_F32>(d, P, C, G, lag, stream, false, nullptr, res)
-                                       : launch_stream<SD_DTYPE_BF16>(d, P, C, G, lag, stream, false, nullptr, res);
+            rc = dtype == SD_DTYPE_F32 ? launch_stream<SD_DTYPE_F32>(d, P, C, G, lag, stream, false, nullptr)
+                                       : launch_stream<SD_DTYPE_BF16>(d, P, C, G, lag, stream, false, nullptr);
     } else {
         P.blocks_per_unit = 1;
         P.RE = kGenericRegionElems;
@@ -654,14 +638,14 @@ int sd_ensemble_feedback(const void* target_logits, const void* const* draft_log
         P.Dn[n] = draft_logits[n];
         P.Gn[n] = out_grad ? out_grad[n] : nullptr;
     }
-    int G = 0, lag = 0, per = 0, res = 0;
-    const int C = choose_stream(*d, V, (long long)B * k * n_learners, dtype, &G, &per, &lag, &res);
+    int G = 0, lag = 0, per = 0;
+    const int C = choose_stream(*d, V, (long long)B * k * n_learners, dtype, &G, &per, &lag);
     if (C <= 0) return SD_ERR_CUDA;
     P.blocks_per_unit = C;
     P.RE = per * vec_elems(dtype);
     P.NR = (V + P.RE - 1) / P.RE;
-    rc = dtype == SD_DTYPE_F32 ? launch_stream<SD_DTYPE_F32, true>(*d, P, C, G, lag, st, false, nullptr, res)
-                               : launch_stream<SD_DTYPE_BF16, true>(*d, P, C, G, lag, st, false, nullptr, res);
+    rc = dtype == SD_DTYPE_F32 ? launch_stream<SD_DTYPE_F32, true>(*d, P, C, G, lag, st, false, nullptr)
+                               : launch_stream<SD_DTYPE_BF16, true>(*d, P, C, G, lag, st, false, nullptr);
     if (rc != SD_OK) return rc;
     sd_hedge_kernel<<<1, 256, 0, st>>>(out_loss, n_learners, (long long)B * k, (double)epsilon, cum_loss_in,
                                        out_round_loss, out_cum_loss, out_weights, P.sticky, out_status, B);
@@ -725,8 +709,8 @@ int sd_verify_error_feedback(const void* target_logits, const void* draft_logits
     P.wait_polls = wait_polls();
     SD_CUDA(cudaMemsetAsync(ws, 0, L.accept, st));   // tickets, status words, sticky flag
     if (out_status) SD_CUDA(cudaMemsetAsync(out_status, 0, (size_t)B * 4, st));   // bits are ORed in on the device
-    int G = 0, lag = 0, per = 0, res = 0;
-    const int C = choose_stream(*d, V, (long long)B * (k + 1), dtype, &G, &per, &lag, &res);   // (pass 1 only: always streams)
+    int G = 0, lag = 0, per = 0;
+    const int C = choose_stream(*d, V, (long long)B * (k + 1), dtype, &G, &per, &lag);
     if (C <= 0) return SD_ERR_CUDA;
     P.blocks_per_unit = C;
     P.RE = per * vec_elems(dtype);

@@ -50,7 +50,10 @@ constexpr int kConsumerWarps = 28;
 constexpr int kStageVecs = kConsumerWarps * kRegionVecs;      // vectors of one row in a stage
 constexpr int kStageRowBytes = kStageVecs * 16;               // 28 KiB of one row
 constexpr int kStageBytes = 2 * kStageRowBytes;               // target part + draft part
-constexpr int kRingStages = 4;                                // 224 KiB
+constexpr int kRingStages = 4;                                // most stages a ring has (224 KiB)
+// Stages of the ring by element type: measured, the fourth stage gains 4 % on the largest fp32 workload
+// and loses 3 % on the bf16 ones.
+template <int DT> struct RingStages { static constexpr int value = DT == SD_DTYPE_F32 ? 4 : 3; };
 constexpr int kDoneDepth = 3;                                 // units the resolver may lag behind
 constexpr int kStatsWarp = 0, kResolverWarp = 1, kProducerWarp = 2, kFirstConsumerWarp = kHelperWarps;
 constexpr int kStreamThreads = (kHelperWarps + kConsumerWarps) * 32;
@@ -492,13 +495,14 @@ __device__ __forceinline__ void walk_stages(int nu, int nst, int L, P1&& p1, P2&
 // squared distance to this round's gradient per row.
 template <int DT, bool ENS, bool STATS = false, bool HINT = false>
 __global__ void __launch_bounds__(kStreamThreads, 1)
-sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const int prefetch, const int resident_arg) {
+sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const int prefetch) {
     using E = Elem<DT>;
     using ET = typename E::type;
     constexpr int VEC = E::VEC;
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     unsigned char* ring = dyn_smem;
-    StreamShared& sh = *reinterpret_cast<StreamShared*>(dyn_smem + (size_t)kRingStages * kStageBytes);
+    constexpr int kRing = RingStages<DT>::value;
+    StreamShared& sh = *reinterpret_cast<StreamShared*>(dyn_smem + (size_t)kRing * kStageBytes);
 
     cg::cluster_group cluster = cg::this_cluster();
     const int C = (int)cluster.num_blocks();
@@ -531,17 +535,11 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const i
     const int nst = (nr + kConsumerWarps - 1) / kConsumerWarps;     // stages of a pass
     // lag_stages = -2: every other cluster takes all of the next unit's pass 1 first, the rest none of it,
     // so that half of the GPU reads from HBM while the other half works from L2
-    // Resident walk: the slice of a unit (at most kRingStages - 1 stages) stays in the ring between its
-    // two passes, so every logit enters the SM once; a stage is released by pass 2, and the producer
-    // runs ahead into the next unit as far as the free slots reach.  Pass 1 of the next unit can go
-    // before pass 2 of a unit only as far as the producer can get without a release.
-    const bool resident = !STATS && resident_arg != 0 && nst < kRingStages;
-    const int Lreq = lag_stages == -2 ? ((cid & 1) ? nst : 0) : min(max(lag_stages, 0), nst);
-    const int L = resident ? min(Lreq, kRingStages - nst) : Lreq;
+    const int L = lag_stages == -2 ? ((cid & 1) ? nst : 0) : min(max(lag_stages, 0), nst);
     const WaitCtx wc{&sh.abort, P.wait_polls};
 
     if (tid == 0) {
-        for (int s = 0; s < kRingStages; ++s) {
+        for (int s = 0; s < kRing; ++s) {
             mbar_init(&sh.full[s], 1);
             mbar_init(&sh.empty[s], kConsumerWarps);
         }
@@ -665,7 +663,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const i
                 // costs the stage's copies a few hundred cycles of head start, 6 % on the largest workload.
                 // Should only one of them give up, the other's copy lands during the pause before the block
                 // exits, or the wait for a half-armed stage below runs into its time limit.)
-                if (ni >= kRingStages && !mbar_wait_thread<false>(&sh.empty[slot], epar, wc)) { ok = false; return; }
+                if (ni >= kRing && !mbar_wait_thread<false>(&sh.empty[slot], epar, wc)) { ok = false; return; }
                 const int v0 = t * kStageVecs;     // first vector of the stage within the slice
                 const uint32_t bytes = (uint32_t)min(kStageVecs, nvb - v0) * 16u;
                 const size_t off = (size_t)(vb0 + v0) * VEC;
@@ -681,15 +679,8 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const i
                               &sh.full[slot], pol);
                 }
                 ++ni;
-                if (++slot == kRingStages) { slot = 0; epar ^= 1u; }
+                if (++slot == kRing) { slot = 0; epar ^= 1u; }
             };
-            if (resident) {
-                // every stage once, in order; nobody reads it from L2 again
-                for (int j = 0; j < nu && ok; ++j) {
-                    const UnitRef ur = unit_ref<ENS>(P, u0 + j * ustep);
-                    for (int t = 0; t < nst && ok; ++t) issue(ur, t, discard);
-                }
-            } else
             walk_stages(nu, nst, L,
                 [&](int j, int t0, int t1, bool) {
                     const UnitRef ur = unit_ref<ENS>(P, u0 + j * ustep);
@@ -724,9 +715,9 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const i
             // leaving early: no copy may still be in flight when the block returns
             if (!ok && lane == 0) {
                 const long long t0 = clock64();
-                for (int i = max(0, ni - kRingStages); i < ni; ++i) {
-                    const uint32_t par = (uint32_t)(i / kRingStages) & 1u;
-                    for (uint32_t it = 0; it < kWaitLimit && !mbar_try_wait(&sh.full[i % kRingStages], par); ++it)
+                for (int i = max(0, ni - kRing); i < ni; ++i) {
+                    const uint32_t par = (uint32_t)(i / kRing) & 1u;
+                    for (uint32_t it = 0; it < kWaitLimit && !mbar_try_wait(&sh.full[i % kRing], par); ++it)
                         if (clock64() - t0 > kWaitCycles) break;
                 }
             }
@@ -744,21 +735,11 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const i
         // before the arithmetic on this region is over, and when it says "full" -- the usual case --
         // the next visit starts without the round trip of a wait.
         bool next_full = false;
-        int rslot = 0;                             // resident walk: slot of the next stage that pass 2 releases
-        auto advance = [&]() {
-            if (++slot == kRingStages) { slot = 0; fpar ^= 1u; }
-            next_full = mbar_test(&sh.full[slot], fpar);
-        };
         auto hand_back = [&]() {
-            if (resident) { advance(); return; }   // pass 1 of the resident walk keeps the stage
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh.empty[slot]);
-            advance();
-        };
-        auto release = [&]() {                     // pass 2 of the resident walk: the stage goes back
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sh.empty[rslot]);
-            if (++rslot == kRingStages) rslot = 0;
+            if (++slot == kRing) { slot = 0; fpar ^= 1u; }
+            next_full = mbar_test(&sh.full[slot], fpar);
         };
         auto await_stage = [&]() {
             if (__all_sync(0xffffffffu, next_full ? 1 : 0)) return true;
@@ -825,8 +806,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const i
             if constexpr (HINT)
                 Hrow = reinterpret_cast<const uint4*>(reinterpret_cast<const ET*>(P.hint) + ur.d_row * P.V) + vb0 + rv0;
             float herr = 0.f;
-            for (int s = 0; s < nst; ++s) {
-                const int t = resident ? s : nst - 1 - s;   // (the streaming walk finds the last stages still in L2)
+            for (int t = nst - 1; t >= 0; --t) {
                 const int nv = vectors_of(t);
                 // the hint does not go through the ring: each lane asks for its vectors before it waits
                 // for the stage, and they are there when the gradient is
@@ -837,16 +817,13 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const i
                         hq[g] = (!bonus && g * 32 + lane < nv) ? __ldcs(Hrow + (size_t)t * kStageVecs + g * 32 + lane)
                                                                : make_uint4(0u, 0u, 0u, 0u);
                 }
-                if (!resident && !await_stage()) { ok = false; return false; }
-                const uint4* st = reinterpret_cast<const uint4*>(ring + (size_t)(resident ? rslot : slot) * kStageBytes) + rv0;
-                if (nv == 0) {
-                    if (resident) release(); else hand_back();
-                    continue;
-                }
+                if (!await_stage()) { ok = false; return false; }
+                const uint4* st = reinterpret_cast<const uint4*>(ring + (size_t)slot * kStageBytes) + rv0;
+                if (nv == 0) { hand_back(); continue; }
                 uint4 rt[kRegionRows], rd[kRegionRows];
                 if (bonus) { load_region<DT, true>(st, nv, lane, rt, rd); await_region_registers<true>(rt, rd); }
                 else       { load_region<DT, false>(st, nv, lane, rt, rd); await_region_registers<false>(rt, rd); }
-                if (resident) release(); else hand_back();
+                hand_back();
                 float mass;
                 if constexpr (HINT) {
                     mass = bonus ? pass2_region<DT, true>(rt, rd, nv, lane, P.c, rc, nullptr)

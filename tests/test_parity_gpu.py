@@ -240,13 +240,9 @@ def test_largest_k(binding):
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("cluster", [1, 2, 3, 4, 5, 6, 7, 8])
-@pytest.mark.parametrize("resident", [0, 1])
-def test_every_cluster_size_gives_the_same_answer(binding, dtype, cluster, resident, options):
-    """Slices of 1 to 4 stages: the larger clusters keep theirs in shared memory between the passes
-    when that is allowed, the smaller ones fetch it twice."""
+def test_every_cluster_size_gives_the_same_answer(binding, dtype, cluster, options):
     cfg = synth.custom_config(B=3, k=3, V=24000 if dtype == "f32" else 48000, dtype=dtype, tau=1.2, index=52)
     options(binding.SD_OPT_CLUSTER, cluster)
-    options(binding.SD_OPT_RESIDENT, resident)
     inp, out, ref, _ = run_and_check(binding, cfg, ex=True, max_band_frac=1.0)
     info = binding.sd_launch_info()
     assert info["path"] == 1 and info["cluster_size"] == cluster
@@ -254,15 +250,12 @@ def test_every_cluster_size_gives_the_same_answer(binding, dtype, cluster, resid
 
 @pytest.mark.parametrize("lag", [0, 1, 2, 100, -2])
 @pytest.mark.parametrize("cluster", [1, 3, 4, 8])
-@pytest.mark.parametrize("resident", [0, 1])
-def test_every_order_of_the_two_passes_gives_the_same_answer(binding, lag, cluster, resident, options):
+def test_every_order_of_the_two_passes_gives_the_same_answer(binding, lag, cluster, options):
     """Pass 2 of a unit may come 0, 1, 2 ... stages (per warp) into pass 1 of the next unit, or after
-    all of it (or both, cluster by cluster); the slice may stay in shared memory between the passes
-    (clusters of 3 and more here: 3, 2 and 1 stages) or be fetched twice; several units per cluster."""
+    all of it (or both, cluster by cluster); several units per cluster, slices of 1 to 7 stages."""
     cfg = synth.custom_config(B=40, k=3, V=100000, dtype="bf16", tau=1.1, index=65)
     options(binding.SD_OPT_CLUSTER, cluster)
     options(binding.SD_OPT_LAG, lag)
-    options(binding.SD_OPT_RESIDENT, resident)
     inp = synth.make_inputs(cfg)
     T, D, x, u = to_device(inp)
     out = binding.sd_verify_feedback_ex(T, D, x, u, inp.tau)
