@@ -66,13 +66,18 @@ def measured_peaks():
 
 
 def kernel_source_hash() -> str:
-    """Identifies the kernels a DRAM-traffic capture belongs to: the CUDA sources, hashed."""
+    """Identifies the kernels a DRAM-traffic capture belongs to: the CUDA sources without their
+    comments and blank space, hashed (a reworded comment does not change a kernel)."""
+    import re
     h = hashlib.sha256()
     src = os.path.join(ROOT, "paper_2603_12617_b200", "csrc")
     for name in sorted(os.listdir(src)):
-        with open(os.path.join(src, name), "rb") as fh:
-            h.update(name.encode())
-            h.update(fh.read())
+        with open(os.path.join(src, name), "r", encoding="utf-8") as fh:
+            text = fh.read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        text = re.sub(r"//[^\n]*", "", text)
+        h.update(name.encode())
+        h.update("".join(text.split()).encode())
     return h.hexdigest()[:16]
 
 

@@ -1,24 +1,24 @@
 // The two kernels of the verify-and-feedback step.
 //
-//   sd_stream_kernel   fast path.  A persistent kernel of thread-block clusters.  A cluster takes a
-//                      contiguous range of (sequence, row) units, one after the other; each block
-//                      of the cluster owns a contiguous slice of the vocabulary, cut into sampling
-//                      regions of 64 16-byte vectors (1 KiB of a row) and into stages of 28 regions.
-//                      A slice is read twice: pass 1 (softmax sums relative to integer references)
-//                      streams it from HBM through a ring of three shared-memory stages, pass 2
-//                      (gradient out, residual mass) reads it again a few microseconds later with
-//                      plain 16-byte loads, last stage first, when it is still in L2, so HBM sees
-//                      each logit once.  (One SM takes in about 48 bytes per clock through bulk
-//                      copies of this size and about as much again through plain loads; the two
-//                      passes together need 30 at the HBM roofline, so they use one path each.)
-//                      Inside a block the warps are specialised:
-//                        producer   one thread fetches the pass-1 stages of unit after unit, each
-//                                   with two bulk asynchronous copies (cp.async.bulk + mbarrier),
-//                                   as soon as the consumers have handed the slot back;
-//                        consumers  28 warps; warp w takes region w of every stage into registers
-//                                   (pass 1: from the ring, handing the slot back at once; pass 2:
-//                                   from global memory, one region ahead) and works from registers;
-//                                   warps meet only through the ring's barriers and once per unit and pass;
+//   sd_stream_kernel   fast path.  A persistent kernel of thread-block clusters, one block of 32
+//                      warps per SM.  A cluster takes a contiguous range of (sequence, row) units,
+//                      one after the other; each block of the cluster owns a contiguous slice of
+//                      the vocabulary, cut into sampling regions of 64 16-byte vectors (1 KiB of a
+//                      row) and into stages of 28 regions (28 KiB of the target row and 28 KiB of
+//                      the draft row).  A slice goes through a ring of shared-memory stages twice:
+//                      pass 1 (softmax sums relative to integer references) brings it from HBM and
+//                      asks L2 to hold on to it, pass 2 (gradient out, residual mass) fetches it
+//                      again a few microseconds later, last stage first, when it is still in L2,
+//                      so HBM sees each logit once.  Inside a block the warps are specialised:
+//                        producer   two threads fetch the stages of the walk, in order, with bulk
+//                                   asynchronous copies (cp.async.bulk + mbarrier): the first arms
+//                                   the stage's barrier and copies the target part, the second
+//                                   copies the draft part, each as soon as the consumers have
+//                                   handed the slot back;
+//                        consumers  28 warps; warp w takes region w of every stage into registers,
+//                                   hands its share of the slot back at once and works from
+//                                   registers; warps meet only through the ring's barriers and
+//                                   once per unit and pass;
 //                        statistics adds up the consumers' sums, exchanges the block's partial
 //                                   with the other blocks of the cluster through distributed
 //                                   shared memory (remote stores + remote mbarrier arrivals, no
