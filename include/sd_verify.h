@@ -342,6 +342,16 @@ int sd_vp_draw(const void* target_shard, const void* draft_shard, const int32_t*
                uint32_t* out_status, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * sd_bounds_report -- for the checked build of the library (compiled with -DSD_BOUNDS_CHECK: every index
+ * the kernels form into global memory is tested against its extent before the access, an access that
+ * fails is skipped and counted).  Waits for the current device, then fills out4 (host memory) with: the
+ * number of violations since the last report, and the site code, index and limit of the first; the
+ * counters go back to zero.  The regular build has no checks and reports out4[0] = 2^64 - 1.
+ * Returns SD_OK, SD_ERR_NULL or SD_ERR_CUDA.
+ */
+int sd_bounds_report(unsigned long long* out4);
+
+/*
  * sd_lmhead_grad -- the step after the feedback: the gradient of the round's loss with respect to
  * the weights W [V,d] of the draft model's linear output layer.  The feedback gradient of Sec. 3.1
  * ("nabla f_t(w_t)") reaches the parameters through the chain rule; with draft logits

@@ -32,7 +32,8 @@ SD_STATUS_ZERO_RESIDUAL = 4
 SD_STATUS_TIMEOUT = 0x80000000
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "lib", "libsd_verify.so")
+# SD_VERIFY_LIBRARY selects another build of the same library (the range-checked one); there is still no fallback.
+LIB_PATH = os.environ.get("SD_VERIFY_LIBRARY") or os.path.join(_HERE, "lib", "libsd_verify.so")
 
 
 class SdVerifyError(RuntimeError):
@@ -99,6 +100,8 @@ def _load() -> ctypes.CDLL:
     lib.sd_last_cuda_error.argtypes = []
     lib.sd_version.restype = I
     lib.sd_version.argtypes = []
+    lib.sd_bounds_report.restype = I
+    lib.sd_bounds_report.argtypes = [P]
     return lib
 
 
@@ -154,6 +157,17 @@ def _stream_ptr(stream: Optional[torch.cuda.Stream]):
 
 def sd_version() -> int:
     return int(_lib.sd_version())
+
+
+def sd_bounds_report() -> Optional[dict]:
+    """Violations the range-checked build has counted since the last report (None: this build has no checks)."""
+    out = (ctypes.c_ulonglong * 4)()
+    rc = _lib.sd_bounds_report(out)
+    if rc != 0:
+        raise SdVerifyError(rc, "sd_bounds_report")
+    if out[0] == 2 ** 64 - 1:
+        return None
+    return {"violations": int(out[0]), "site": int(out[1]), "index": int(out[2]), "limit": int(out[3])}
 
 
 def sd_workspace_bytes(B: int, k: int, V: int, dtype: int) -> int:

@@ -1147,6 +1147,25 @@ const char* sd_strerror(int code) {
 
 const char* sd_last_cuda_error(void) { return tl_cuda_error; }
 
+int sd_bounds_report(unsigned long long* out4) {
+    if (!out4) return SD_ERR_NULL;
+#ifdef SD_BOUNDS_CHECK
+    int dev;
+    DeviceState* ds = nullptr;
+    int rc = current_device(&dev, &ds);
+    if (rc != SD_OK) return rc;
+    SD_CUDA(cudaDeviceSynchronize());
+    SD_CUDA(cudaMemcpyFromSymbol(out4, g_sd_bounds, 4 * sizeof(unsigned long long)));
+    const unsigned long long zero[4] = {0, 0, 0, 0};
+    SD_CUDA(cudaMemcpyToSymbol(g_sd_bounds, zero, sizeof zero));
+    return SD_OK;
+#else
+    out4[0] = ~0ull;
+    out4[1] = out4[2] = out4[3] = 0;
+    return SD_OK;
+#endif
+}
+
 int sd_version(void) { return SD_VERSION; }
 
 }  // extern "C"

@@ -48,6 +48,34 @@ struct __align__(16) PartialStats {
     double sT, sD;     // sum of eT = 2^aT, aT = t*c - RT; sum of eD likewise
     double w;          // sum of eT*(aT - aD)
 };
+// ---- range checks of the checked build ------------------------------------------------------
+// With -DSD_BOUNDS_CHECK every index the kernels form into global memory is tested against its
+// extent before the access: SD_IN(index, limit, site) is false for an index outside [0, limit), the
+// access is then skipped, and the first violation (site, index, limit) and their number are kept
+// for sd_bounds_report.  Without the flag SD_IN is the constant true and costs nothing.
+#ifdef SD_BOUNDS_CHECK
+__device__ unsigned long long g_sd_bounds[4];    // violations; site of the first; its index; its limit
+__device__ __noinline__ void sd_bounds_record(long long idx, long long limit, int site) {
+    if (atomicAdd(&g_sd_bounds[0], 1ull) == 0ull) {
+        g_sd_bounds[1] = (unsigned long long)site;
+        g_sd_bounds[2] = (unsigned long long)idx;
+        g_sd_bounds[3] = (unsigned long long)limit;
+    }
+}
+__device__ __forceinline__ bool sd_in(long long idx, long long limit, int site) {
+    if (idx >= 0 && idx < limit) return true;
+    sd_bounds_record(idx, limit, site);
+    return false;
+}
+#define SD_IN(idx, limit, site) (::sdv::sd_in((long long)(idx), (long long)(limit), (site)))
+#else
+#define SD_IN(idx, limit, site) (true)
+#endif
+// Sites: 1x fast path (10 target copy, 11 draft copy, 12 gradient store, 13 region mass, 14 second try,
+// 15 hint), 2x row report and resolver (20 row constants, 21 loss, 22 accept flag, 23 region masses,
+// 24 region searched, 25 tokens), 3x element-wise path, 4x greedy, 5x error-position kernel,
+// 6x vocabulary-parallel kernels.
+
 constexpr float kEmptyRef = -1073741824.f;       // reference of a part without a finite entry (-2^30)
 
 struct Params {
@@ -462,12 +490,12 @@ __device__ inline void finish_row(const Params& P, int b, int i, const PartialSt
     const bool okT = (st.sT > 0.0) && isfinite(st.sT);
     const bool okD = bonus || ((st.sD > 0.0) && isfinite(st.sD));
     if (!okT || !okD) flags |= SD_STATUS_BAD_ROW;
-    P.rowc[unit] = rc;
+    if (SD_IN(unit, P.B * (P.k + 1), 20)) P.rowc[unit] = rc;
     if (!bonus) {
         // log2 p_v = aT_v - log2 S_T and log2 q_v = aD_v - log2 S_D, so
         // KL(p||q) = ln2 * [ E_p(aT - aD) - log2 S_T + log2 S_D ]
         const double l2ST = log2(st.sT), l2SD = log2(st.sD);
-        if (P.loss) {
+        if (P.loss && SD_IN(b * P.k + i, P.B * P.k, 21)) {
             const double kl = 0.6931471805599453 * (st.w / st.sT - l2ST + l2SD);
             P.loss[b * P.k + i] = (float)kl;
         }
@@ -488,7 +516,7 @@ __device__ inline void finish_row(const Params& P, int b, int i, const PartialSt
             const double thr = rho < 1.0 ? rho : 1.0;
             acc = (double)op.u < thr;
         }
-        P.accept[b * P.k + i] = acc ? 1 : 0;
+        if (SD_IN(b * P.k + i, P.B * P.k, 22)) P.accept[b * P.k + i] = acc ? 1 : 0;
     }
     if (flags) atomicOr(&P.wstatus[b], flags);
 }
@@ -533,7 +561,7 @@ __device__ __forceinline__ void lane_masses(const Params& P, const RowConst& rc,
         uint4 qt[PER / VEC], qd[PER / VEC];
 #pragma unroll
         for (int g = 0; g < PER / VEC; ++g) {
-            const bool in = v0 + g * VEC < P.V;
+            const bool in = v0 + g * VEC < P.V && SD_IN(v0 + g * VEC + VEC - 1, P.V, 24);
             qt[g] = in ? __ldg(pT + g) : E::masked();
             qd[g] = (in && mode == 0) ? __ldg(pD + g) : E::masked();
         }
@@ -680,6 +708,7 @@ __device__ __noinline__ void resolve_sequence(const Params& P, int b) {
 
     const bool bonus = (n == k);
     const int unit = b * (k + 1) + n;
+    if (!SD_IN(unit, P.B * (k + 1), 23) || !SD_IN(n, k + 1, 23)) return;
     const float* rs = P.region_sums + (size_t)unit * NR;
     const float4 rcv = __ldcg(reinterpret_cast<const float4*>(P.rowc + unit));
     const RowConst rc{rcv.x, rcv.y, rcv.z, rcv.w};
@@ -765,7 +794,7 @@ __device__ __noinline__ void resolve_sequence(const Params& P, int b) {
             for (int off = 16; off > 0; off >>= 1) lastr = max(lastr, __shfl_xor_sync(0xffffffffu, lastr, off));
             region = lastr;
         }
-        if (region >= 0) {
+        if (region >= 0 && SD_IN(region, NR, 24)) {
             double rtot;
             y = search_region<DT, PER, FAST>(P, rc, bonus ? 1 : 0, offT, offD, region, prefix, t, past_end, &rtot);
             // region sum and re-summed entries may disagree in the last bits: last entry with mass
@@ -785,7 +814,7 @@ __device__ __noinline__ void resolve_sequence(const Params& P, int b) {
     }
     for (int i = lane; i <= k; i += 32) {
         const int32_t xi = (i == lane) ? x_first : ((i < k) ? P.x[b * k + i] : -1);
-        P.tokens[b * (k + 1) + i] = (i < n) ? xi : (i == n ? y : -1);
+        if (SD_IN(b * (k + 1) + i, P.B * (k + 1), 25)) P.tokens[b * (k + 1) + i] = (i < n) ? xi : (i == n ? y : -1);
     }
 }
 

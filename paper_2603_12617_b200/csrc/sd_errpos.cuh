@@ -50,6 +50,7 @@ __global__ void __launch_bounds__(kErrThreads, 4) sd_errpos_kernel(const __grid_
     for (int r = r0 + warp; r < r1; r += kErrThreads / 32) {
         const int v0 = r * RV;
         const int nv = min(RV, NV - v0);
+        if (!SD_IN(r, P.NR, 50) || !SD_IN((long long)(v0 + nv) * VEC - 1, P.V, 51) || !SD_IN(unit, P.B * (k + 1), 52)) continue;
         uint4 rt[kGroups], rd[kGroups];
 #pragma unroll
         for (int g = 0; g < kGroups; ++g) {

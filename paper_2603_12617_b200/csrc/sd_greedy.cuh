@@ -59,6 +59,7 @@ __global__ void __launch_bounds__(kGreedyThreads) sd_greedy_kernel(const GreedyP
         const int piece = (int)(it - (long long)row * P.items_per_row);
         const int e0 = piece * item_elems;
         const int n = min(item_elems, P.V - e0);           // entries of this item
+        if (!SD_IN(row, (long long)P.B * K1, 40) || !SD_IN(e0 + n - 1, P.V, 41)) continue;
         float best = -INFINITY;
         int besti = 0x7fffffff;
         if (P.vectorised) {

@@ -71,6 +71,12 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
                  : "memory");
 }
+// Counts `bytes` as transferred on the barrier without a copy (the checked build's stand-in for a
+// copy that it refused to issue).
+__device__ __forceinline__ void mbar_complete_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.complete_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
@@ -668,6 +674,17 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const i
                 const uint32_t bytes = (uint32_t)min(kStageVecs, nvb - v0) * 16u;
                 const size_t off = (size_t)(vb0 + v0) * VEC;
                 unsigned char* dst = ring + (size_t)slot * kStageBytes;
+#ifdef SD_BOUNDS_CHECK
+                // a copy that fails its check is not issued; its bytes are counted on the stage's barrier
+                // by hand instead, so that nobody waits for them (the stage then holds what it held before)
+                const long long rowsT = (long long)P.B * (P.k + 1), rowsD = (long long)P.B * P.k;
+                const bool okc = SD_IN(off + bytes / sizeof(ET) - 1, P.V, lane == 0 ? 10 : 11) &&
+                                 (lane == 0 ? SD_IN(ur.t_row, rowsT, 10) : SD_IN(ur.d_row, rowsD, 11));
+                if (!okc) {
+                    if (lane == 0) mbar_expect_tx(&sh.full[slot], ur.bonus ? bytes : 2u * bytes);
+                    if (lane == 0 || !ur.bonus) mbar_complete_tx(&sh.full[slot], bytes);
+                } else
+#endif
                 if (lane == 0) {
                     mbar_expect_tx(&sh.full[slot], ur.bonus ? bytes : 2u * bytes);
                     bulk_load(dst, reinterpret_cast<const ET*>(P.T) + ur.t_row * P.V + off, bytes, &sh.full[slot], pol);
@@ -760,6 +777,7 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const i
                 // where the region lies in global memory: only the rare second try of a region reads it there
                 auto again = [&](Pass1State s0) {
                     const size_t voff = (size_t)vb0 + rv0 + (size_t)t * kStageVecs;
+                    if (!SD_IN((voff + nv) * VEC - 1, P.V, 14)) return s0;
                     const uint4* gT = reinterpret_cast<const uint4*>(reinterpret_cast<const ET*>(P.T) + ur.t_row * P.V) + voff;
                     const uint4* gD = reinterpret_cast<const uint4*>(reinterpret_cast<const ET*>(ENS ? P.Dn[ur.n] : P.D) + ur.d_row * P.V) + voff;
                     return bonus ? pass1_region_again<DT, true>(gT, gD, nv, lane, P.c, s0)
@@ -810,11 +828,17 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const i
                 const int nv = vectors_of(t);
                 // the hint does not go through the ring: each lane asks for its vectors before it waits
                 // for the stage, and they are there when the gradient is
+#ifdef SD_BOUNDS_CHECK
+                const size_t vfirst = (size_t)vb0 + rv0 + (size_t)t * kStageVecs;   // first vector of my region in the row
+                const bool in_row = nv == 0 || SD_IN((vfirst + nv) * VEC - 1, P.V, 12);
+#else
+                constexpr bool in_row = true;
+#endif
                 uint4 hq[kRegionRows];
                 if constexpr (HINT) {
 #pragma unroll
                     for (int g = 0; g < kRegionRows; ++g)
-                        hq[g] = (!bonus && g * 32 + lane < nv) ? __ldcs(Hrow + (size_t)t * kStageVecs + g * 32 + lane)
+                        hq[g] = (!bonus && in_row && g * 32 + lane < nv) ? __ldcs(Hrow + (size_t)t * kStageVecs + g * 32 + lane)
                                                                : make_uint4(0u, 0u, 0u, 0u);
                 }
                 if (!await_stage()) { ok = false; return false; }
@@ -828,14 +852,14 @@ sd_stream_kernel(const __grid_constant__ Params P, const int lag_stages, const i
                 if constexpr (HINT) {
                     mass = bonus ? pass2_region<DT, true>(rt, rd, nv, lane, P.c, rc, nullptr)
                                  : pass2_region_impl<DT, false, true>(rt, rd, nv, lane, P.c, rc,
-                                                                      Grow ? Grow + (size_t)t * kStageVecs * VEC : nullptr,
+                                                                      (Grow && in_row) ? Grow + (size_t)t * kStageVecs * VEC : nullptr,
                                                                       hq, herr);
                 } else {
                     mass = bonus ? pass2_region<DT, true>(rt, rd, nv, lane, P.c, rc, nullptr)
                                  : pass2_region<DT, false>(rt, rd, nv, lane, P.c, rc,
-                                                           Grow ? Grow + (size_t)t * kStageVecs * VEC : nullptr);
+                                                           (Grow && in_row) ? Grow + (size_t)t * kStageVecs * VEC : nullptr);
                 }
-                if (!ENS && lane == 0) rsum[t * kConsumerWarps] = mass;
+                if (!ENS && lane == 0 && SD_IN(r0 + cw + t * kConsumerWarps, P.NR, 13)) rsum[t * kConsumerWarps] = mass;
             }
             if constexpr (HINT) {
 #pragma unroll
@@ -957,7 +981,7 @@ __global__ void __launch_bounds__(kGenericThreads) sd_generic_kernel(const __gri
                         const float dlt = E::load(P.hint, offD + v) - g;
                         herr = fmaf(dlt, dlt, herr);
                     }
-                    if (P.grad) E::store(P.grad, offD + v, g);
+                    if (P.grad && SD_IN(offD + v, (long long)P.B * P.k * P.V, 31)) E::store(P.grad, offD + v, g);
                 } else {
                     mass += prob_elem(t, P.c, rc);
                 }
@@ -965,7 +989,7 @@ __global__ void __launch_bounds__(kGenericThreads) sd_generic_kernel(const __gri
         }
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) mass += __shfl_xor_sync(0xffffffffu, mass, off);
-        if (lane == 0) rsum[q] = mass;
+        if (lane == 0 && SD_IN((long long)unit * P.NR + q, (long long)P.B * (P.k + 1) * P.NR, 32)) rsum[q] = mass;
     }
 
     if (P.hint) {

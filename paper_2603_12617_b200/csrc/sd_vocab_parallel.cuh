@@ -80,6 +80,7 @@ __global__ void __launch_bounds__(kVpThreads) sd_vp_stats_kernel(const VpParams 
     const int b = unit / K1, i = unit - b * K1;
     const bool bonus = (i == P.k);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (!SD_IN(unit, P.B * K1, 60)) return;
     const uint4* Trow = reinterpret_cast<const uint4*>(reinterpret_cast<const ET*>(P.T) + (size_t)unit * P.Vs);
     const uint4* Drow = reinterpret_cast<const uint4*>(reinterpret_cast<const ET*>(P.D) + (size_t)(b * P.k + (bonus ? 0 : i)) * P.Vs);
     const int NV = P.Vs / VEC;
@@ -242,6 +243,7 @@ __global__ void __launch_bounds__(kVpThreads, 4) sd_vp_grad_kernel(const VpParam
     for (int r = r0 + warp; r < r1; r += kVpWarps) {
         const int v0 = r * kRegionVecs;
         const int nv = min(kRegionVecs, NV - v0);
+        if (!SD_IN((long long)(v0 + nv) * VEC - 1, P.Vs, 61) || !SD_IN(unit, P.B * K1, 62)) continue;
         uint4 rt[kRegionRows], rd[kRegionRows];
 #pragma unroll
         for (int g = 0; g < kRegionRows; ++g) {
