@@ -388,6 +388,93 @@ class HintPath(SamplePath):
         return base, parity, bool(verified and ok)
 
 
+class VocabParallelPath(SamplePath):
+    """One rank of the vocabulary-parallel step on this GPU: the workload's logits cut into --shards column
+    shards, this rank's three local calls timed on its own shard with the other ranks' records and masses
+    already in place (the gathers of a real deployment are not part of the timed region: one GPU here)."""
+    name, kernel, traffic_path = "vp", "sd_vp_stats_kernel + sd_vp_rows_kernel + sd_vp_grad_kernel + sd_vp_mass_kernel + sd_vp_draw_kernel", "vp"
+
+    def __init__(self, args, cfg, dev, rank, binding):
+        import torch
+        from paper_2603_12617_b200 import shard
+        self.b, self.cfg, self.torch = binding, cfg, torch
+        self.inp = inp = synth.make_inputs(cfg, seed=synth.BASE_SEED + 1000 * rank)
+        G = self.G = max(1, args.shards)
+        es = cfg.elem_bytes
+        self.cuts = cuts = shard.vocab_cuts(cfg.V, G, es)
+        code = binding.SD_DTYPE_F32 if cfg.dtype == "f32" else binding.SD_DTYPE_BF16
+        T, D = as_torch(inp.target_logits), as_torch(inp.draft_logits)
+        x, u = torch.from_numpy(inp.draft_tokens).to(dev), torch.from_numpy(inp.uniforms).to(dev)
+        self.x, self.u = x, u
+        recs, fins, shards, wss = [], [], [], []
+        for r, (a, c) in enumerate(cuts):          # every rank's phases once: what the gathers would deliver
+            Ts, Ds = T[:, :, a:c].contiguous().to(dev), D[:, :, a:c].contiguous().to(dev)
+            ws = torch.empty(max(256, binding.sd_vp_workspace_bytes(cfg.B, cfg.k, c - a, code)), dtype=torch.uint8, device=dev)
+            recs.append(binding.sd_vp_partial(Ts, Ds, x, inp.tau, a, cfg.V, ws))
+            shards.append((Ts, Ds)); wss.append(ws)
+        self.all_records = torch.stack(recs, 0).contiguous()
+        for r, (a, c) in enumerate(cuts):
+            fins.append(binding.sd_vp_finish(*shards[r], x, u, inp.tau, a, cfg.V, self.all_records, G, r, wss[r]))
+        self.all_masses = torch.stack([f.local_mass for f in fins], 0).contiguous()
+        toks = [binding.sd_vp_draw(*shards[r], x, u, inp.tau, cuts[r][0], cfg.V, fins[r].accept_len, self.all_masses,
+                                   G, r, fins[r].status, wss[r]) for r in range(G)]
+        torch.cuda.synchronize()
+        self.check_accept = fins[0].accept_len.cpu().numpy()
+        self.check_tokens = torch.stack(toks, 0).max(0).values.cpu().numpy()
+        self.check_loss = fins[0].loss.cpu().numpy()
+        # the timed rank: rank 0's shard, rotating copies if it is not larger than L2 by itself
+        self.host = [shards[0][0].cpu().pin_memory(), shards[0][1].cpu().pin_memory()]
+        self.sets, self.in_bytes, self.nsets = rotating_sets(self.host, dev)
+        self.ws = wss[0]
+        del shards, wss
+        Vs = cuts[0][1] - cuts[0][0]
+        self.Vs = Vs
+        self.algorithmic = (2 * (2 * cfg.k + 1) + cfg.k) * Vs * cfg.B * es
+        self.positions = cfg.B * cfg.k
+        self.dtype = "f32" if cfg.dtype == "f32" else "f32 (bf16 storage)"
+        self.extra = {"shards": G, "timed": f"the three local calls of rank 0 (columns 0..{Vs - 1}); the two gathers and the "
+                                           "token maximum of a real deployment are not in the timed region",
+                      "kernels_per_step": 5}
+        self.e2e_entry = "sd_vp_partial + sd_vp_finish + sd_vp_draw of one rank between pinned-memory copies of its shard"
+
+    def step(self, i):
+        Ts, Ds = self.sets[i % self.nsets]
+        b, c = self.b, self.cfg
+        b.sd_vp_partial(Ts, Ds, self.x, self.inp.tau, 0, c.V, self.ws)
+        self.fin = b.sd_vp_finish(Ts, Ds, self.x, self.u, self.inp.tau, 0, c.V, self.all_records, self.G, 0, self.ws)
+        self.tok = b.sd_vp_draw(Ts, Ds, self.x, self.u, self.inp.tau, 0, c.V, self.fin.accept_len, self.all_masses, self.G, 0,
+                                self.fin.status, self.ws)
+
+    def e2e_prepare(self):
+        torch = self.torch
+        self.dbuf = [torch.empty_like(t) for t in self.sets[0]]
+        self.h_g = torch.empty(self.sets[0][1].shape, dtype=self.host[0].dtype).pin_memory()
+        self.h_tok = torch.empty((self.cfg.B, self.cfg.k + 1), dtype=torch.int32).pin_memory()
+        self.h2d = self.in_bytes
+        self.d2h = self.h_g.numel() * self.h_g.element_size() + self.h_tok.numel() * 4
+
+    def e2e_step(self):
+        for a, h in zip(self.dbuf, self.host):
+            a.copy_(h, non_blocking=True)
+        keep, self.sets, self.nsets = (self.sets, self.nsets), [self.dbuf], 1
+        self.step(0)
+        self.sets, self.nsets = keep
+        self.h_g.copy_(self.fin.grad_shard, non_blocking=True)
+        self.h_tok.copy_(self.tok, non_blocking=True)
+        self.torch.cuda.synchronize()
+
+    def finish(self, args):
+        cfg = self.cfg
+        if args.no_cpu_baseline:
+            seqs = np.asarray(sorted({0, cfg.B // 2, cfg.B - 1}))
+            base, (_, ref) = None, run_oracle(self.inp, seqs, len(seqs), want_grad=False)
+        else:
+            base, seqs, ref = cpu_baseline(cfg, self.inp)
+        parity = parity_counts(cfg, ref, seqs, self.check_accept, self.check_tokens, self.check_loss)
+        verified = parity["mismatches_outside_the_bands"] == 0 and parity.get("loss_within_tolerance", True)
+        return base, parity, bool(verified)
+
+
 class GreedyPath:
     name, kernel, traffic_path = "greedy", "sd_greedy_kernel", "greedy"
 
@@ -623,7 +710,7 @@ class LmHeadPath:
         return base, {"entries_compared": n, "within_tolerance": ok}, ok
 
 
-PATHS = {"sample": SamplePath, "hint": HintPath, "greedy": GreedyPath, "errors": ErrorsPath, "ensemble": EnsemblePath, "lmhead": LmHeadPath}
+PATHS = {"sample": SamplePath, "hint": HintPath, "vp": VocabParallelPath, "greedy": GreedyPath, "errors": ErrorsPath, "ensemble": EnsemblePath, "lmhead": LmHeadPath}
 
 
 def run_ours(args, cfg):
@@ -733,7 +820,8 @@ def run_ours(args, cfg):
                                       l2="inputs larger than L2" if path.nsets == 1 else f"{path.nsets} rotating input sets larger than L2 together",
                                       parallelism=f"replicas x{world}, sequences independent, no collective",
                                       launch=info, **path.extra),
-            "roofline": roofline, "cpu_baseline": base, "e2e": e2e, "gpu_launches": args.steps * info["kernels"],
+            "roofline": roofline, "cpu_baseline": base, "e2e": e2e,
+            "gpu_launches": args.steps * int(path.extra.get("kernels_per_step", info["kernels"])),
             "clocks": clocks.summary(), "parity": parity, "outputs_verified_against_oracle": verified}
     print(json.dumps(line), flush=True)
     if world > 1:
@@ -766,6 +854,7 @@ def main(argv=None):
     ap.add_argument("--path", choices=sorted(PATHS), default="sample",
                     help="sample: the verify-and-feedback step (the headline); the others: see the module text")
     ap.add_argument("--learners", type=int, default=3, help="draft models of --path ensemble")
+    ap.add_argument("--shards", type=int, default=4, help="column shards of --path vp (one rank of them is timed)")
     ap.add_argument("--features", type=int, default=4096, help="width d of the output layer of --path lmhead")
     ap.add_argument("--times-out", default="", help="write the per-step device times (ms) here")
     args = ap.parse_args(argv)
