@@ -180,7 +180,8 @@ int sd_verify_feedback_hint(const void* target_logits, const void* draft_logits,
  *
  *   - Shapes whose sd_workspace_bytes(B,k,V,dtype) exceeds SD_STATIC_SCRATCH_BYTES are refused
  *     with SD_ERR_WORKSPACE (sd_last_cuda_error() says how many bytes were needed); nothing is
- *     enqueued.  4 MiB covers, for instance, B*(k+1) up to about 3900 rows at V <= 131072.
+ *     enqueued.  4 MiB covers, for instance, B*(k+1) up to about 1900 rows of fp32 logits (3800 of
+ *     bf16) at V <= 131072.
  *   - The first call on each device looks up the device address of the array
  *     (cudaGetSymbolAddress, with that device current).  Make that first call outside any stream
  *     capture; later calls only enqueue a small memset and the kernel.
