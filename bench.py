@@ -106,6 +106,7 @@ class ClockSampler:
 
     def __init__(self, device_index: int):
         self.samples, self.reasons = [], set()
+        self.mem_samples, self.power_samples = [], []
         self.max_mhz = None
         self._stop = threading.Event()
         self._thread = None
@@ -126,6 +127,8 @@ class ClockSampler:
         nv = self._nv
         try:
             self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+            self.mem_samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_MEM)))
+            self.power_samples.append(nv.nvmlDeviceGetPowerUsage(self._h) / 1000.0)
             mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
             for bit, name in self.REASONS.items():
                 if mask & bit:
@@ -158,7 +161,11 @@ class ClockSampler:
         if self._nv is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvml unavailable: " + self._err]}
         return {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
-                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples),
+                "sm_mhz_min": float(min(self.samples)) if self.samples else None,
+                "mem_mhz": float(np.median(self.mem_samples)) if self.mem_samples else None,
+                "mem_mhz_min": float(min(self.mem_samples)) if self.mem_samples else None,
+                "power_w_max": float(max(self.power_samples)) if self.power_samples else None}
 
 
 # ------------------------------------------------------------------------------------------
